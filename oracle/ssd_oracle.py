@@ -1,0 +1,452 @@
+"""CPU oracle for Self Speculative Decoding (SSD) on a masked-diffusion LM.
+
+TEST INFRASTRUCTURE.  Plain, slow, fp64 numpy.  Only the test-suite, the
+smoke check and the benchmark's cpu-baseline leg may import this file; the
+CUDA library shares no code with it and never calls it.
+
+What is defined here, and from where:
+
+* the model f_theta of Eq. 2 (a bidirectional transformer; the paper gives no
+  architecture, the shapes and the pre-norm RMSNorm/RoPE/SwiGLU layout are the
+  workload's) -> ``Oracle.forward_rows``;
+* semi-autoregressive blocks, Eq. 3 -> ``block_ranges``;
+* stepwise decoding (one token per forward, the highest-confidence masked
+  position of the current block takes its argmax token; Fig. 2 and the
+  baseline of Section 4.1) -> ``Oracle.decode_block_stepwise``;
+* SSD: self-drafting (Eq. 4), greedy candidate selection (Section 3.2.2), the
+  greedy verification chain of N+1 nodes (Section 3.2.3), batch verification
+  (Eq. 5), parent-prediction-vs-child-draft traversal (Section 3.2.4) and the
+  loop of Algorithm 1 -> ``select_candidates``, ``build_chain``,
+  ``node_predictions``, ``accept_length``, ``Oracle.decode_block_ssd``.
+
+Readings where the paper is silent (each also listed in the design notes):
+the forward of a block attends to the cached prefix plus the block itself; a
+finished block enters the cache through one more forward over its final
+tokens; confidence is the maximum softmax probability with the mask token
+excluded; ties go to the lower token id / lower position; a draft "matches"
+only if position AND token agree; the next drafts are the last valid node's
+own predictions from the same forward.
+
+Precision: everything is fp64.  ``operand_rounding`` optionally rounds the
+operands of every contraction (matmul inputs, attention Q/K/V/P) to bfloat16,
+which is the arithmetic type the accelerated path is specified to use (bf16
+operands, wide accumulation); with ``None`` nothing is rounded.
+
+Pins: see tests/test_oracle_*.py.  The accept-count VALUES on random-init
+models have no value printed in the paper to compare with: parity unpinned by
+the paper for those (they are pinned by brute force against the stepwise
+continuation instead).
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Callable, Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------------------
+# configuration and small helpers
+# --------------------------------------------------------------------------------------
+@dataclasses.dataclass(frozen=True)
+class ModelConfig:
+    n_layers: int
+    d_model: int
+    n_heads: int
+    n_kv_heads: int
+    head_dim: int
+    d_ffn: int
+    vocab: int
+    mask_id: int
+    rope_theta: float
+    rms_eps: float
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest bfloat16 (ties to even); returns fp64 holding bf16 values."""
+    f = np.ascontiguousarray(x, dtype=np.float32)
+    b = f.view(np.uint32).astype(np.uint64)
+    b = (b + 0x7FFF + ((b >> 16) & 1)) & 0xFFFF0000
+    return b.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
+def block_ranges(gen_len: int, block_len: int) -> List[Tuple[int, int]]:
+    """Eq. 3: generation offsets [j*B, min((j+1)*B, L)) for j = 0 .. ceil(L/B)-1."""
+    n_blocks = -(-gen_len // block_len)
+    return [(j * block_len, min((j + 1) * block_len, gen_len)) for j in range(n_blocks)]
+
+
+# --------------------------------------------------------------------------------------
+# model primitives (each is its textbook definition)
+# --------------------------------------------------------------------------------------
+def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * gain over the last axis."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * gain
+
+
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary embedding, "rotate-half" pairing: feature i is paired with i + hd/2.
+
+    x [T, H, hd], pos [T] absolute positions.  Pair (a, b) at frequency
+    theta^(-2i/hd) is rotated by angle pos * frequency.
+    """
+    hd = x.shape[-1]
+    half = hd // 2
+    inv_freq = theta ** (-(np.arange(half, dtype=np.float64) * 2.0) / hd)
+    ang = pos.astype(np.float64)[:, None] * inv_freq[None, :]
+    c = np.cos(ang)[:, None, :]
+    s = np.sin(ang)[:, None, :]
+    a, b = x[..., :half], x[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, rnd: Callable[[np.ndarray], np.ndarray]) -> np.ndarray:
+    """Bidirectional (unmasked) softmax attention with grouped KV heads.
+
+    q [T, H, hd]; k, v [S, Hkv, hd]; query head h reads KV head h // (H/Hkv);
+    scale 1/sqrt(hd).  ``rnd`` rounds the probability operand of P.V (the
+    normaliser is the unrounded sum).  Returns [T, H*hd].
+    """
+    T, H, hd = q.shape
+    group = H // k.shape[1]
+    out = np.empty((T, H, hd), dtype=np.float64)
+    for h in range(H):
+        g = h // group
+        s = (q[:, h, :] @ k[:, g, :].T) / np.sqrt(float(hd))
+        p = np.exp(s - s.max(axis=-1, keepdims=True))
+        out[:, h, :] = (rnd(p) @ v[:, g, :]) / p.sum(axis=-1, keepdims=True)
+    return out.reshape(T, H * hd)
+
+
+def token_and_confidence(logits: np.ndarray, mask_id: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. 2 + Eq. 4 for rows of logits [T, V]: draft token = argmax of the softmax with
+    the mask token excluded (lowest id on ties), confidence = that maximum probability."""
+    l = np.array(logits, dtype=np.float64, copy=True)
+    l[:, mask_id] = -np.inf
+    tok = np.argmax(l, axis=-1)
+    m = l.max(axis=-1, keepdims=True)
+    conf = 1.0 / np.exp(l - m).sum(axis=-1)
+    return tok.astype(np.int64), conf
+
+
+def top2_gap(logits: np.ndarray, mask_id: int) -> np.ndarray:
+    """Softmax probability of the best token minus that of the runner-up, per row."""
+    l = np.array(logits, dtype=np.float64, copy=True)
+    l[:, mask_id] = -np.inf
+    m = l.max(axis=-1, keepdims=True)
+    p = np.exp(l - m)
+    z = p.sum(axis=-1)
+    part = np.partition(p, -2, axis=-1)
+    return (part[:, -1] - part[:, -2]) / z
+
+
+# --------------------------------------------------------------------------------------
+# SSD logic that does not touch the model (Section 3.2.2 - 3.2.4)
+# --------------------------------------------------------------------------------------
+def best_masked_position(conf: np.ndarray, masked: np.ndarray) -> int:
+    """Highest-confidence masked position; the lower position wins ties."""
+    best, best_c = -1, -1.0
+    for p in range(len(conf)):
+        if masked[p] and conf[p] > best_c:
+            best, best_c = p, conf[p]
+    return best
+
+
+def select_candidates(draft_tok: np.ndarray, draft_conf: np.ndarray, masked: np.ndarray,
+                      max_drafts: int) -> List[Tuple[int, int]]:
+    """Greedy selection: the N = min(max_drafts, r-1) masked positions of the current block
+    with the highest draft confidence, in descending confidence (lower position first on
+    ties).  r-1 because every node of the chain must keep one masked position to predict."""
+    pos = [p for p in range(len(masked)) if masked[p]]
+    n = max(0, min(max_drafts, len(pos) - 1))
+    order = sorted(pos, key=lambda p: (-draft_conf[p], p))
+    return [(p, int(draft_tok[p])) for p in order[:n]]
+
+
+def build_chain(ids: np.ndarray, masked: np.ndarray, cand: Sequence[Tuple[int, int]], mask_id: int
+                ) -> Tuple[np.ndarray, np.ndarray]:
+    """Greedy verification chain: node i = current state with candidates 1..i written in
+    (N+1 nodes for N candidates).  Returns node ids [N+1, B] and masked flags [N+1, B]."""
+    n = len(cand) + 1
+    node_ids = np.tile(np.where(masked, mask_id, ids), (n, 1)).astype(np.int64)
+    node_masked = np.tile(masked.astype(bool), (n, 1))
+    for i in range(1, n):
+        for (p, t) in cand[:i]:
+            node_ids[i, p] = t
+            node_masked[i, p] = False
+    return node_ids, node_masked
+
+
+def node_predictions(tok: np.ndarray, conf: np.ndarray, node_masked: np.ndarray) -> List[Tuple[int, int]]:
+    """Per node: the (position, token) that a stepwise step from that node's state would write."""
+    out = []
+    for i in range(node_masked.shape[0]):
+        q = best_masked_position(conf[i], node_masked[i])
+        out.append((q, int(tok[i, q])))
+    return out
+
+
+def accept_length(pred: Sequence[Tuple[int, int]], cand: Sequence[Tuple[int, int]]) -> int:
+    """Walk the chain from the root: node i's prediction must equal (position and token) the
+    draft that node i+1 assumed; stop at the first mismatch.  Returns a = index of the last
+    valid node, so a+1 tokens are accepted."""
+    a = 0
+    while a < len(cand) and pred[a] == cand[a]:
+        a += 1
+    return a
+
+
+# --------------------------------------------------------------------------------------
+# the model and the decode loops
+# --------------------------------------------------------------------------------------
+class Cache:
+    """Per-layer prefix K (post-RoPE) and V, each [S, Hkv, hd]."""
+
+    def __init__(self, cfg: ModelConfig):
+        self.k = [np.zeros((0, cfg.n_kv_heads, cfg.head_dim)) for _ in range(cfg.n_layers)]
+        self.v = [np.zeros((0, cfg.n_kv_heads, cfg.head_dim)) for _ in range(cfg.n_layers)]
+
+    @property
+    def length(self) -> int:
+        return self.k[0].shape[0]
+
+    def append(self, new_k: List[np.ndarray], new_v: List[np.ndarray]) -> None:
+        for l in range(len(self.k)):
+            self.k[l] = np.concatenate([self.k[l], new_k[l]], axis=0)
+            self.v[l] = np.concatenate([self.v[l], new_v[l]], axis=0)
+
+
+@dataclasses.dataclass
+class ForwardRecord:
+    """Everything about one verification forward (for teacher-forced comparisons)."""
+    block: int
+    cache_len: int
+    ids_before: np.ndarray          # [B] tokens (mask_id where masked)
+    masked_before: np.ndarray       # [B] bool
+    draft_tok: Optional[np.ndarray]  # [B] stale drafts used to build the chain (None: no drafts yet)
+    draft_conf: Optional[np.ndarray]
+    cand: List[Tuple[int, int]]
+    node_ids: np.ndarray            # [n, B]
+    node_masked: np.ndarray         # [n, B]
+    tok: np.ndarray                 # [n, B] argmax token per row
+    conf: np.ndarray                # [n, B] confidence per row
+    gap: np.ndarray                 # [n, B] top-1 minus top-2 probability per row
+    pred: List[Tuple[int, int]]
+    accepted: int                   # a+1
+
+
+class Oracle:
+    """f_theta plus the two decode loops.
+
+    ``weights`` maps names to arrays: embed [V,d], lm_head [V,d], norm_final [d] and per
+    layer l ``layers.l.{wq,wk,wv,wo,w_gate,w_up,w_down,norm_attn,norm_ffn}`` with matmul
+    weights stored [out_features, in_features].  It may be a dict or any object with
+    ``__getitem__`` (so that large models can materialise one tensor at a time).
+    """
+
+    def __init__(self, cfg: ModelConfig, weights, operand_rounding: Optional[str] = None):
+        assert operand_rounding in (None, "bf16")
+        self.cfg = cfg
+        self.w = weights
+        self.rnd = bf16_round if operand_rounding == "bf16" else (lambda a: a)
+
+    def _W(self, name: str) -> np.ndarray:
+        return np.asarray(self.w[name], dtype=np.float64)
+
+    # ---- one transformer layer over independent row groups --------------------------
+    def layer(self, l: int, groups: List[np.ndarray], positions: List[np.ndarray],
+              prefix_k: np.ndarray, prefix_v: np.ndarray) -> Tuple[List[np.ndarray], List[np.ndarray], List[np.ndarray]]:
+        """Apply layer l to every group (a group = the rows of one node, [T, d]).  Each group
+        attends to [prefix ; its own rows].  Returns (new hidden, post-RoPE K, V) per group."""
+        c = self.cfg
+        rnd = self.rnd
+        p = f"layers.{l}."
+        wq, wk, wv, wo = self._W(p + "wq"), self._W(p + "wk"), self._W(p + "wv"), self._W(p + "wo")
+        wg, wu, wd = self._W(p + "w_gate"), self._W(p + "w_up"), self._W(p + "w_down")
+        g1, g2 = self._W(p + "norm_attn"), self._W(p + "norm_ffn")
+        outs, ks, vs = [], [], []
+        for h, pos in zip(groups, positions):
+            T = h.shape[0]
+            u = rnd(rmsnorm(h, g1, c.rms_eps))
+            q = rope((u @ wq.T).reshape(T, c.n_heads, c.head_dim), pos, c.rope_theta)
+            k = rope((u @ wk.T).reshape(T, c.n_kv_heads, c.head_dim), pos, c.rope_theta)
+            v = (u @ wv.T).reshape(T, c.n_kv_heads, c.head_dim)
+            q, k, v = rnd(q), rnd(k), rnd(v)
+            keys = np.concatenate([prefix_k, k], axis=0)
+            vals = np.concatenate([prefix_v, v], axis=0)
+            att = rnd(attention(q, keys, vals, rnd))
+            h = h + att @ wo.T
+            u = rnd(rmsnorm(h, g2, c.rms_eps))
+            act = rnd(silu(u @ wg.T) * (u @ wu.T))
+            h = h + act @ wd.T
+            outs.append(h)
+            ks.append(k)
+            vs.append(v)
+        return outs, ks, vs
+
+    def forward_rows(self, ids: np.ndarray, pos0: int, cache: Cache, want_logits: bool = True,
+                     logit_rows: Optional[np.ndarray] = None):
+        """f_theta on one or several nodes.  ids [n, T] (or [T]); all nodes sit at absolute
+        positions pos0 .. pos0+T-1 and each attends to the cache plus its own T rows.
+        Returns (logits [n, T, V] or None, K list per layer [n,T,Hkv,hd], V list)."""
+        c = self.cfg
+        ids = np.atleast_2d(np.asarray(ids))
+        n, T = ids.shape
+        emb = self._W("embed")
+        groups = [emb[ids[i]].copy() for i in range(n)]
+        pos = [np.arange(pos0, pos0 + T) for _ in range(n)]
+        all_k, all_v = [], []
+        for l in range(c.n_layers):
+            groups, ks, vs = self.layer(l, groups, pos, cache.k[l], cache.v[l])
+            all_k.append(np.stack(ks))
+            all_v.append(np.stack(vs))
+        logits = None
+        if want_logits:
+            gf, wlm = self._W("norm_final"), self._W("lm_head")
+            logits = np.stack([self.rnd(rmsnorm(h, gf, c.rms_eps)) @ wlm.T for h in groups])
+        return logits, all_k, all_v
+
+    # ---- cache maintenance ----------------------------------------------------------
+    def prefill(self, prompt: np.ndarray) -> Cache:
+        """The prompt attends to the prompt only; its K/V become the prefix cache."""
+        cache = Cache(self.cfg)
+        _, ks, vs = self.forward_rows(prompt, 0, cache, want_logits=False)
+        cache.append([k[0] for k in ks], [v[0] for v in vs])
+        return cache
+
+    def commit_block(self, ids: np.ndarray, cache: Cache) -> None:
+        """One forward over the finished block appends its K/V to the prefix cache."""
+        _, ks, vs = self.forward_rows(ids, cache.length, cache, want_logits=False)
+        cache.append([k[0] for k in ks], [v[0] for v in vs])
+
+    # ---- one verification forward ---------------------------------------------------
+    def verify(self, node_ids: np.ndarray, node_masked: np.ndarray, cache: Cache):
+        """Eq. 5: all nodes through the model at once; per row (token, confidence, gap)."""
+        logits, _, _ = self.forward_rows(node_ids, cache.length, cache)
+        n, T, V = logits.shape
+        tok, conf = token_and_confidence(logits.reshape(n * T, V), self.cfg.mask_id)
+        gap = top2_gap(logits.reshape(n * T, V), self.cfg.mask_id)
+        return tok.reshape(n, T), conf.reshape(n, T), gap.reshape(n, T), logits
+
+    # ---- decode loops ---------------------------------------------------------------
+    def decode_block_stepwise(self, block_len: int, cache: Cache, block_index: int = 0,
+                              trace: Optional[List[ForwardRecord]] = None):
+        """One token per forward.  Returns (ids [B], accept counts = [1]*B)."""
+        mid = self.cfg.mask_id
+        ids = np.full(block_len, mid, dtype=np.int64)
+        masked = np.ones(block_len, dtype=bool)
+        counts = []
+        while masked.any():
+            node_ids, node_masked = build_chain(ids, masked, [], mid)
+            tok, conf, gap, _ = self.verify(node_ids, node_masked, cache)
+            pred = node_predictions(tok, conf, node_masked)
+            if trace is not None:
+                trace.append(ForwardRecord(block_index, cache.length, ids.copy(), masked.copy(), None, None, [],
+                                           node_ids, node_masked, tok, conf, gap, pred, 1))
+            q, t = pred[0]
+            ids[q] = t
+            masked[q] = False
+            counts.append(1)
+        return ids, counts
+
+    def decode_block_ssd(self, block_len: int, cache: Cache, max_drafts: int, block_index: int = 0,
+                         trace: Optional[List[ForwardRecord]] = None,
+                         draft_override: Optional[Callable] = None):
+        """Algorithm 1 restricted to one block.  Returns (ids [B], accept counts per forward).
+
+        ``draft_override(ids, masked, draft_tok, draft_conf) -> (draft_tok, draft_conf)``
+        lets a test replace the drafts (perfect or adversarial) to pin the accept logic
+        independently of the model.
+        """
+        mid = self.cfg.mask_id
+        ids = np.full(block_len, mid, dtype=np.int64)
+        masked = np.ones(block_len, dtype=bool)
+        draft_tok: Optional[np.ndarray] = None
+        draft_conf: Optional[np.ndarray] = None
+        counts = []
+        while masked.any():
+            if draft_tok is None:
+                cand: List[Tuple[int, int]] = []          # no drafts yet: root-only forward
+            else:
+                dt, dc = draft_tok, draft_conf
+                if draft_override is not None:
+                    dt, dc = draft_override(ids.copy(), masked.copy(), dt.copy(), dc.copy())
+                cand = select_candidates(dt, dc, masked, max_drafts)
+            node_ids, node_masked = build_chain(ids, masked, cand, mid)
+            tok, conf, gap, _ = self.verify(node_ids, node_masked, cache)
+            pred = node_predictions(tok, conf, node_masked)
+            a = accept_length(pred, cand)
+            if trace is not None:
+                trace.append(ForwardRecord(block_index, cache.length, ids.copy(), masked.copy(),
+                                           None if draft_tok is None else draft_tok.copy(),
+                                           None if draft_conf is None else draft_conf.copy(),
+                                           list(cand), node_ids, node_masked, tok, conf, gap, pred, a + 1))
+            for (p, t) in cand[:a]:
+                ids[p] = t
+                masked[p] = False
+            q, t = pred[a]
+            ids[q] = t
+            masked[q] = False
+            # next drafts: the last valid node's own predictions on what is still masked
+            draft_tok = np.where(masked, tok[a], 0).astype(np.int64)
+            draft_conf = np.where(masked, conf[a], 0.0)
+            counts.append(a + 1)
+        return ids, counts
+
+    def generate(self, prompt: np.ndarray, gen_len: int, block_len: int, mode: str = "ssd",
+                 max_drafts: int = 0, trace: Optional[List[ForwardRecord]] = None,
+                 draft_override: Optional[Callable] = None):
+        """Semi-autoregressive generation of gen_len tokens after the prompt.
+        Returns (tokens [gen_len], accept counts per block (list of lists), cache)."""
+        cache = self.prefill(np.asarray(prompt))
+        out, all_counts = [], []
+        for j, (lo, hi) in enumerate(block_ranges(gen_len, block_len)):
+            if mode == "stepwise":
+                ids, counts = self.decode_block_stepwise(hi - lo, cache, j, trace)
+            else:
+                ids, counts = self.decode_block_ssd(hi - lo, cache, max_drafts, j, trace, draft_override)
+            self.commit_block(ids, cache)
+            out.append(ids)
+            all_counts.append(counts)
+        return np.concatenate(out), all_counts, cache
+
+    # ---- the uncached definition used to pin the cache semantics --------------------
+    def uncached_block_causal(self, tokens: np.ndarray, segment_lengths: Sequence[int]):
+        """Forward over the whole sequence with NO cache: position t attends to every
+        position of its own segment and of all earlier segments (prompt = first segment).
+        Returns (logits [T,V], K list [T,Hkv,hd], V list).  Written as a plain masked
+        attention over the full sequence, independently of ``layer``'s cache handling."""
+        c = self.cfg
+        T = len(tokens)
+        seg = np.repeat(np.arange(len(segment_lengths)), segment_lengths)
+        assert len(seg) == T
+        allow = seg[None, :] <= seg[:, None]            # [query, key]
+        pos = np.arange(T)
+        h = self._W("embed")[np.asarray(tokens)].copy()
+        rnd = self.rnd
+        Ks, Vs = [], []
+        for l in range(c.n_layers):
+            p = f"layers.{l}."
+            u = rnd(rmsnorm(h, self._W(p + "norm_attn"), c.rms_eps))
+            q = rnd(rope((u @ self._W(p + "wq").T).reshape(T, c.n_heads, c.head_dim), pos, c.rope_theta))
+            k = rnd(rope((u @ self._W(p + "wk").T).reshape(T, c.n_kv_heads, c.head_dim), pos, c.rope_theta))
+            v = rnd((u @ self._W(p + "wv").T).reshape(T, c.n_kv_heads, c.head_dim))
+            group = c.n_heads // c.n_kv_heads
+            att = np.empty((T, c.n_heads, c.head_dim))
+            for hh in range(c.n_heads):
+                s = (q[:, hh, :] @ k[:, hh // group, :].T) / np.sqrt(float(c.head_dim))
+                s = np.where(allow, s, -np.inf)
+                pr = np.exp(s - s.max(axis=-1, keepdims=True))
+                att[:, hh, :] = (rnd(pr) @ v[:, hh // group, :]) / pr.sum(axis=-1, keepdims=True)
+            h = h + rnd(att.reshape(T, -1)) @ self._W(p + "wo").T
+            u = rnd(rmsnorm(h, self._W(p + "norm_ffn"), c.rms_eps))
+            h = h + rnd(silu(u @ self._W(p + "w_gate").T) * (u @ self._W(p + "w_up").T)) @ self._W(p + "w_down").T
+            Ks.append(k)
+            Vs.append(v)
+        logits = rnd(rmsnorm(h, self._W("norm_final"), c.rms_eps)) @ self._W("lm_head").T
+        return logits, Ks, Vs

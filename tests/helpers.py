@@ -1,0 +1,38 @@
+"""Glue used by the tests: turns a seeded workload into oracle inputs.
+
+Holds no arithmetic of the method: it only converts tensors and builds configs.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle.ssd_oracle import ModelConfig, Oracle, bf16_round
+from paper_2510_04147_b200 import workloads as wl
+
+
+def oracle_config(w: wl.Workload) -> ModelConfig:
+    return ModelConfig(n_layers=w.n_layers, d_model=w.d_model, n_heads=w.n_heads, n_kv_heads=w.n_kv_heads,
+                       head_dim=w.head_dim, d_ffn=w.d_ffn, vocab=w.vocab, mask_id=w.mask_id,
+                       rope_theta=w.rope_theta, rms_eps=w.rms_eps)
+
+
+def oracle_weights(w: wl.Workload, as_bf16: bool) -> dict:
+    """All tensors of a (small) workload as fp64 numpy arrays.  ``as_bf16`` rounds the matrices
+    to bfloat16 values first (what a bf16-only accelerator sees of fp32-drawn weights)."""
+    out = {}
+    for name, t in wl.iter_tensors(w, "cpu"):
+        a = t.to(torch.float32).numpy().astype(np.float64)
+        if as_bf16 and a.ndim == 2:
+            a = bf16_round(a)
+        out[name] = a
+    return out
+
+
+def make_oracle(w: wl.Workload, as_bf16: bool = False, operand_rounding=None) -> Oracle:
+    return Oracle(oracle_config(w), oracle_weights(w, as_bf16), operand_rounding)
+
+
+SMALL = wl.TINY.replace(name="small", d_model=64, n_heads=2, n_kv_heads=2, head_dim=32, d_ffn=96,
+                        vocab=96, prompt_len=6, gen_len=12, block_len=6, seed=11)
+SMALL_GQA = SMALL.replace(name="small_gqa", n_heads=4, n_kv_heads=2, head_dim=16, seed=12)

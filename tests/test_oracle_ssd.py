@@ -1,0 +1,294 @@
+"""Pins for the oracle's decoding logic: what the paper fixes about SSD.
+
+* output identical to stepwise decoding (abstract, Section 4.2, Conclusion);
+* N+1 nodes for draft length N, between 1 and N+1 tokens per forward (Sections 3.2.3-3.2.4,
+  Appendix A) and the node counts 4/5/6 printed in Table 3;
+* the forward-pass reduction bound N/(N+1) printed in Table 2;
+* a child is valid only if its parent's prediction equals the stepwise result, and a draft with
+  the right tokens in another order fails (Section 5.1);
+* block order (Section 3.1): nothing of block j+1 before block j is complete.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import ssd_oracle as so
+from tests.helpers import SMALL, SMALL_GQA, make_oracle
+from paper_2510_04147_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                a, b = line.split()
+                rows.append((int(a), float(b)))
+    return rows
+
+
+# ---------------------------------------------------------------------------------------
+# model-free pins: a scripted verifier replaces f_theta
+# ---------------------------------------------------------------------------------------
+class ScriptedOracle(so.Oracle):
+    """verify() answers from a script instead of a transformer.
+
+    ``rule(node_ids_row, node_masked_row) -> (tok[B], conf[B])`` plays the model for one node.
+    """
+
+    def __init__(self, vocab, rule):
+        cfg = so.ModelConfig(0, 0, 0, 0, 0, 0, vocab, vocab - 1, 1.0, 0.0)
+        super().__init__(cfg, {})
+        self.rule = rule
+        self.n_forwards = 0
+        self.nodes_per_forward = []
+
+    def verify(self, node_ids, node_masked, cache):
+        self.n_forwards += 1
+        self.nodes_per_forward.append(node_ids.shape[0])
+        out = [self.rule(node_ids[i], node_masked[i]) for i in range(node_ids.shape[0])]
+        tok = np.stack([o[0] for o in out])
+        conf = np.stack([o[1] for o in out])
+        return tok, conf, np.ones_like(conf), None
+
+
+class NoCache:
+    length = 0
+
+
+def _context_free_rule(B):
+    """Predictions depend on the position only: drafts never go stale."""
+    tok = (np.arange(B) * 7 + 3) % 50
+    conf = np.linspace(0.9, 0.1, B)
+    return lambda ids, masked: (tok.copy(), conf.copy())
+
+
+@pytest.mark.parametrize("N,pct", _golden("step_reduction_upper_bound.txt"))
+def test_upper_bound_of_step_reduction(N, pct):
+    """With drafts that are always right every forward after the first accepts N+1 tokens, so
+    the reduction of forward passes tends to N/(N+1): 75.0 / 80.0 / 83.3 % (Table 2)."""
+    B = 12000
+    o = ScriptedOracle(64, _context_free_rule(B))
+    ids, counts = o.decode_block_ssd(B, NoCache(), max_drafts=N)
+    assert np.array_equal(ids, (np.arange(B) * 7 + 3) % 50)
+    assert counts[0] == 1 and all(c == N + 1 for c in counts[1:-1]) and sum(counts) == B
+    assert len(counts) == 1 + -(-(B - 1) // (N + 1))
+    assert round(100.0 * (1 - len(counts) / B), 1) == pct
+    assert abs((1 - len(counts) / B) - N / (N + 1)) < 1e-3
+
+
+@pytest.mark.parametrize("N,nodes", _golden("greedy_verification_batch.txt"))
+def test_chain_has_n_plus_one_nodes(N, nodes):
+    B = 16
+    o = ScriptedOracle(64, _context_free_rule(B))
+    o.decode_block_ssd(B, NoCache(), max_drafts=N)
+    # first forward is root-only; while at least N+1 positions are masked the chain has N+1 nodes
+    assert o.nodes_per_forward[0] == 1
+    assert o.nodes_per_forward[1] == int(nodes) == N + 1
+    assert max(o.nodes_per_forward) == N + 1
+
+
+def test_build_chain_contents():
+    ids = np.array([5, 63, 63, 9, 63, 63])
+    masked = np.array([0, 1, 1, 0, 1, 1], dtype=bool)
+    cand = [(4, 11), (1, 12), (5, 13)]
+    node_ids, node_masked = so.build_chain(ids, masked, cand, 63)
+    assert node_ids.shape == (4, 6)
+    assert node_ids.tolist() == [[5, 63, 63, 9, 63, 63], [5, 63, 63, 9, 11, 63],
+                                 [5, 12, 63, 9, 11, 63], [5, 12, 63, 9, 11, 13]]
+    assert node_masked.sum(axis=1).tolist() == [4, 3, 2, 1]
+    assert node_masked[3].tolist() == [False, False, True, False, False, False]
+
+
+def test_select_candidates_order_and_cap():
+    tok = np.array([10, 11, 12, 13, 14, 15])
+    conf = np.array([0.2, 0.9, 0.5, 0.9, 0.1, 0.7])
+    masked = np.array([1, 1, 0, 1, 1, 1], dtype=bool)
+    # descending confidence, lower position first on the 0.9 tie, unmasked position 2 never chosen
+    assert so.select_candidates(tok, conf, masked, 10) == [(1, 11), (3, 13), (5, 15), (0, 10)]
+    assert so.select_candidates(tok, conf, masked, 2) == [(1, 11), (3, 13)]
+    assert so.select_candidates(tok, conf, masked, 0) == []
+    one = np.array([0, 0, 0, 0, 1, 0], dtype=bool)
+    assert so.select_candidates(tok, conf, one, 5) == []     # r = 1 -> plain stepwise step
+
+
+def test_accept_length_walk():
+    cand = [(4, 11), (1, 12), (5, 13)]
+    assert so.accept_length([(4, 11), (1, 12), (5, 13), (2, 7)], cand) == 3
+    assert so.accept_length([(4, 11), (1, 99), (5, 13), (2, 7)], cand) == 1     # wrong token
+    assert so.accept_length([(4, 11), (5, 13), (1, 12), (2, 7)], cand) == 1     # right tokens, other order
+    assert so.accept_length([(0, 11), (1, 12), (5, 13), (2, 7)], cand) == 0     # right token, wrong position
+    assert so.accept_length([(3, 3)], []) == 0
+
+
+def test_wrong_drafts_accept_exactly_one_and_keep_tokens():
+    """Adversarial drafts (wrong token / swapped order) cost nothing but speed."""
+    B = 24
+    base = ScriptedOracle(64, _context_free_rule(B))
+    want, _ = base.decode_block_stepwise(B, NoCache())
+
+    def wrong_token(ids, masked, dt, dc):
+        return (dt + 1) % 50, dc
+
+    def swapped_order(ids, masked, dt, dc):
+        return dt, 1.0 - dc         # same tokens, reversed priority
+
+    for override in (wrong_token, swapped_order):
+        o = ScriptedOracle(64, _context_free_rule(B))
+        ids, counts = o.decode_block_ssd(B, NoCache(), max_drafts=4, draft_override=override)
+        assert np.array_equal(ids, want)
+        if override is wrong_token:
+            assert counts == [1] * B
+        else:
+            # reversed priority: the first candidate is never the stepwise choice
+            # (except when a single masked position is left)
+            assert all(c == 1 for c in counts)
+
+
+def test_context_dependent_script_matches_bruteforce():
+    """A scripted model whose predictions change with the context (so drafts do go stale):
+    accepted count per forward == 1 + longest common prefix of the draft chain with the true
+    stepwise continuation from the same state, capped at N+1."""
+    B, V = 14, 40
+    table_rng = np.random.default_rng(5)
+    tok_tab = table_rng.integers(0, V - 1, (B + 1, B))
+    conf_tab = table_rng.random((B + 1, B))
+
+    def rule(ids, masked):
+        r = int(masked.sum())           # context = how many positions are still masked
+        return tok_tab[r].copy(), conf_tab[r].copy()
+
+    ref = ScriptedOracle(V, rule)
+    want, _ = ref.decode_block_stepwise(B, NoCache())
+    # stepwise order of (position, token)
+    order = []
+    ids = np.full(B, V - 1)
+    masked = np.ones(B, dtype=bool)
+    while masked.any():
+        t, c = rule(ids, masked)
+        q = so.best_masked_position(c, masked)
+        order.append((q, int(t[q])))
+        ids[q] = t[q]
+        masked[q] = False
+    for N in (1, 3, 5, B):
+        trace = []
+        o = ScriptedOracle(V, rule)
+        got, counts = o.decode_block_ssd(B, NoCache(), max_drafts=N, trace=trace)
+        assert np.array_equal(got, want)
+        done = 0
+        for rec in trace:
+            cont = order[done:]
+            lcp = 0
+            while lcp < len(rec.cand) and rec.cand[lcp] == cont[lcp]:
+                lcp += 1
+            assert rec.accepted == lcp + 1
+            assert 1 <= rec.accepted <= len(rec.cand) + 1 <= N + 1
+            done += rec.accepted
+        assert done == B
+
+
+# ---------------------------------------------------------------------------------------
+# pins that use the real model
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("w", [SMALL, SMALL_GQA], ids=lambda w: w.name)
+@pytest.mark.parametrize("max_drafts", [0, 1, 3, 5, 64])
+def test_ssd_equals_stepwise_small(w, max_drafts):
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    want, c0, _ = o.generate(prompt, w.gen_len, w.block_len, mode="stepwise")
+    got, c1, _ = o.generate(prompt, w.gen_len, w.block_len, mode="ssd", max_drafts=max_drafts)
+    assert np.array_equal(got, want)
+    for blk in c1:
+        assert sum(blk) == w.block_len and all(1 <= c <= max_drafts + 1 for c in blk)
+    if max_drafts == 0:
+        assert c1 == c0            # no drafts -> exactly the stepwise forward count
+
+
+def test_ssd_equals_stepwise_ragged_last_block():
+    w = SMALL.replace(gen_len=10, block_len=4)
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    want, _, cache0 = o.generate(prompt, w.gen_len, w.block_len, mode="stepwise")
+    got, counts, cache1 = o.generate(prompt, w.gen_len, w.block_len, mode="ssd", max_drafts=3)
+    assert np.array_equal(got, want) and len(got) == 10
+    assert [sum(c) for c in counts] == [4, 4, 2]
+    assert cache0.length == cache1.length == w.prompt_len + 10
+
+
+@pytest.mark.parametrize("peaked", [1.0, 8.0])
+def test_ssd_equals_stepwise_tiny_config(peaked):
+    """Config 1 (tiny model, prompt 32, L 64, B 16), plain and the 'peaked' LM-head variant."""
+    w = wl.TINY.replace(lm_head_scale=peaked)
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    want, _, _ = o.generate(prompt, w.gen_len, w.block_len, mode="stepwise")
+    trace = []
+    got, counts, _ = o.generate(prompt, w.gen_len, w.block_len, mode="ssd", max_drafts=w.block_len, trace=trace)
+    assert np.array_equal(got, want)
+    assert all(sum(c) == w.block_len for c in counts)
+    assert w.mask_id not in got
+    # every record: accepted = 1 + LCP(draft chain, stepwise continuation from that state)
+    o2 = make_oracle(w)
+    for rec in trace[:12]:
+        cache = _cache_at(o2, prompt, want, rec.block, w.block_len)
+        ids, masked = rec.ids_before.copy(), rec.masked_before.copy()
+        cont = []
+        while masked.any() and len(cont) <= len(rec.cand):
+            tok, conf, _, _ = o2.verify(*so.build_chain(ids, masked, [], w.mask_id), cache)
+            q = so.best_masked_position(conf[0], masked)
+            cont.append((q, int(tok[0, q])))
+            ids[q] = tok[0, q]
+            masked[q] = False
+        lcp = 0
+        while lcp < len(rec.cand) and lcp < len(cont) and rec.cand[lcp] == cont[lcp]:
+            lcp += 1
+        assert rec.accepted == lcp + 1
+
+
+def _cache_at(o, prompt, tokens, block, B):
+    cache = o.prefill(prompt)
+    for j in range(block):
+        o.commit_block(tokens[j * B:(j + 1) * B], cache)
+    return cache
+
+
+def test_block_length_one_is_stepwise():
+    w = SMALL.replace(gen_len=5, block_len=1)
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    a, ca, _ = o.generate(prompt, 5, 1, mode="stepwise")
+    b, cb, _ = o.generate(prompt, 5, 1, mode="ssd", max_drafts=4)
+    assert np.array_equal(a, b) and ca == cb == [[1]] * 5
+
+
+def test_context_free_model_accepts_everything():
+    """One layer with Wo = 0 and Wd = 0: a row's logits depend on its own token only, so a masked
+    row always predicts the same thing, drafts never go stale and every verify accepts N+1."""
+    w = SMALL.replace(n_layers=1, gen_len=12, block_len=12)
+    from tests.helpers import oracle_config, oracle_weights
+    W = oracle_weights(w, as_bf16=False)
+    W["layers.0.wo"] = np.zeros_like(W["layers.0.wo"])
+    W["layers.0.w_down"] = np.zeros_like(W["layers.0.w_down"])
+    o = so.Oracle(oracle_config(w), W)
+    prompt = wl.make_prompts(w)[0].numpy()
+    # all masked rows are identical -> equal confidences -> lowest position first
+    got, counts, _ = o.generate(prompt, 12, 12, mode="ssd", max_drafts=3)
+    assert counts == [[1, 4, 4, 3]]
+    assert len(set(got.tolist())) == 1
+
+
+def test_block_order_constraint():
+    """Nothing of block j+1 exists while block j is decoded: the trace of block j never touches
+    positions beyond it, and the cache grows by exactly one block per commit."""
+    w = SMALL
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    trace = []
+    o.generate(prompt, w.gen_len, w.block_len, mode="ssd", max_drafts=3, trace=trace)
+    for rec in trace:
+        assert rec.cache_len == w.prompt_len + rec.block * w.block_len
+        assert rec.node_ids.shape[1] == w.block_len
+        assert all(0 <= p < w.block_len for p, _ in rec.cand)
