@@ -1,0 +1,171 @@
+/*
+ * ssd.h - C ABI of the B200 (sm_100a) Self Speculative Decoding library.
+ *
+ * The library runs the hot path of SSD for masked-diffusion language models: per block of
+ * the semi-autoregressive schedule (Eq. 3) it turns the model's own drafts for the masked
+ * positions (Eq. 4) into the greedy verification chain of N+1 nodes (Section 3.2.3), runs all
+ * nodes through the model in ONE forward against the cached prefix K/V (Eq. 5), and accepts
+ * the longest draft prefix that one-token-per-step decoding would also have produced
+ * (Section 3.2.4, Algorithm 1).  The tokens it returns are those of stepwise decoding.
+ *
+ * General rules
+ *  - Every function returns SSD_OK (0) or a negative SSD_ERR_* code; ssd_last_error() gives a
+ *    message.  Nothing aborts, traps or throws across this boundary.  Arguments are checked on
+ *    the host before any kernel is launched.
+ *  - "host" pointers are ordinary host memory owned by the caller and only used during the
+ *    call.  "device" pointers are CUDA device memory of the current device.
+ *  - All device work is enqueued on the stream given to ssd_create().  Calls that return
+ *    results in host memory synchronise that stream before returning.
+ *  - A context is not thread-safe; use one per host thread / GPU.
+ *  - There is no CPU fallback: without a CUDA device ssd_create() fails with SSD_ERR_CUDA.
+ */
+#ifndef SSD_B200_H_
+#define SSD_B200_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SSD_OK                0
+#define SSD_ERR_INVALID_ARG  (-1)   /* null pointer, negative size, unknown name or enum          */
+#define SSD_ERR_SHAPE        (-2)   /* a shape the kernels do not support, or a mismatching one   */
+#define SSD_ERR_OOM          (-3)   /* device or host allocation failed                           */
+#define SSD_ERR_CUDA         (-4)   /* a CUDA runtime / driver call failed                        */
+#define SSD_ERR_OVERFLOW     (-5)   /* cached length + block would exceed max_seq, batch too big  */
+#define SSD_ERR_TIMEOUT      (-6)   /* a bounded device-side wait expired (kernel bailed out)     */
+#define SSD_ERR_STATE        (-7)   /* call out of order (weights missing, no prefill, ...)       */
+#define SSD_ERR_NONFINITE    (-8)   /* a confidence came out NaN/Inf (non-finite weights?)        */
+
+#define SSD_DTYPE_BF16 0
+#define SSD_DTYPE_F32  1
+
+#define SSD_MODE_STEPWISE 0   /* one token per forward (the lossless reference behaviour, Fig. 2)  */
+#define SSD_MODE_SSD      1   /* self speculative decoding, greedy chain                           */
+
+typedef struct ssd_ctx ssd_ctx;   /* opaque: owns weights copy, KV cache, workspaces, decode state */
+
+/* Model f_theta (Eq. 2: a bidirectional transformer; pre-norm RMSNorm, rotary embedding with the
+ * rotate-half pairing, grouped-query attention without mask, SwiGLU, untied LM head, no biases)
+ * and decode limits. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  int32_t mask_id;          /* id of the mask token m_i of Eq. 1; never predicted                  */
+  float   rope_theta, rms_eps;
+  int32_t max_batch;        /* sequences decoded in lockstep, each with its own tree               */
+  int32_t max_seq;          /* P + L of Eq. 1: capacity of the KV cache per sequence               */
+  int32_t block_len;        /* B of Eq. 3                                                          */
+  int32_t max_drafts;       /* cap on the draft length N (Section 3.2.2); >= block_len-1 means the
+                               chain may cover the whole block; 0 makes SSD mode equal stepwise    */
+} ssd_config;
+
+/* Supported shapes: head_dim 64 or 128; d_model, d_ffn, n_heads*head_dim multiples of 8;
+ * n_heads a multiple of n_kv_heads; block_len <= 256.  `cuda_stream` is a cudaStream_t (NULL =
+ * legacy default stream).  Allocates everything the context will ever need. */
+int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out);
+void ssd_destroy(ssd_ctx* ctx);
+const char* ssd_last_error(const ssd_ctx* ctx);   /* ctx may be NULL: message of a failed create */
+
+/* Copy one weight tensor into the context (the library keeps its own bf16, re-laid-out copy; the
+ * caller may free `dev_ptr` afterwards).  `dev_ptr` is DEVICE memory, row-major, `shape[ndim]`,
+ * of type SSD_DTYPE_BF16 or SSD_DTYPE_F32 (fp32 matrices are rounded to bf16, the arithmetic
+ * type of every contraction here; norm gains stay fp32).  Names: "embed" [V,d], "lm_head" [V,d],
+ * "norm_final" [d], and for layer l "layers.l.wq" [H*hd,d], ".wk"/".wv" [Hkv*hd,d], ".wo"
+ * [d,H*hd], ".w_gate"/".w_up" [ffn,d], ".w_down" [d,ffn], ".norm_attn"/".norm_ffn" [d]
+ * (matrices are [out_features, in_features]).  Synchronises the stream. */
+int ssd_load_weights(ssd_ctx* ctx, const char* tensor_name, const void* dev_ptr, int32_t dtype,
+                     const int64_t* shape, int32_t ndim);
+
+/* Eq. 1 initial state: forward of the prompts (each prompt attends to itself only) that fills
+ * the prefix K/V cache.  `prompt_ids` HOST [batch, prompt_len], ids in [0, vocab), no mask id
+ * required.  Resets the decode position to prompt_len.  1 <= batch <= max_batch. */
+int ssd_prefill(ssd_ctx* ctx, int32_t batch, int32_t prompt_len, const int32_t* prompt_ids);
+/* Same with `prompt_ids` in DEVICE memory (no host->device copy of inputs). */
+int ssd_prefill_dev(ssd_ctx* ctx, int32_t batch, int32_t prompt_len, const int32_t* prompt_ids_dev);
+
+/* Decode the next block B_j (Eq. 3) for every sequence of the batch (Algorithm 1 restricted to
+ * one block, or stepwise decoding), then append the block's K/V to the cache.
+ *   mode           SSD_MODE_STEPWISE or SSD_MODE_SSD
+ *   block_tokens   number of positions in this block: block_len, or less for a ragged last block
+ *   out_tokens         HOST [batch, block_tokens]   decoded ids
+ *   out_accept_counts  HOST [batch, block_tokens]   tokens accepted by forward 0,1,2,... of each
+ *                      sequence, 0-terminated list; each entry in [1, N+1], sum = block_tokens
+ *   out_n_forwards     HOST [batch]                 verification forwards the sequence took part in
+ * Any out pointer may be NULL.  Errors: SSD_ERR_STATE before prefill, SSD_ERR_OVERFLOW if the
+ * cache would exceed max_seq. */
+int ssd_decode_block(ssd_ctx* ctx, int32_t mode, int32_t block_tokens, int32_t* out_tokens,
+                     int32_t* out_accept_counts, int32_t* out_n_forwards);
+
+/* ---- the same block, one step at a time (used by ssd_decode_block; exposed so that every
+ * ---- forward can be checked against a reference with the state forced to the reference's) --- */
+
+/* Start block B_j: all `block_tokens` positions masked, no drafts. */
+int ssd_block_begin(ssd_ctx* ctx, int32_t block_tokens);
+/* Overwrite the state of the current block.  HOST arrays [batch, block_tokens]: ids (value
+ * ignored where masked), masked (0/1), and either both draft_tok/draft_conf (drafts for the
+ * masked positions, Eq. 4) or both NULL (no drafts: next forward is root-only). */
+int ssd_set_block_state(ssd_ctx* ctx, const int32_t* ids, const uint8_t* masked,
+                        const int32_t* draft_tok, const float* draft_conf);
+/* Read the state back; any pointer may be NULL.  draft arrays are zero where not masked. */
+int ssd_get_block_state(ssd_ctx* ctx, int32_t* ids, uint8_t* masked, int32_t* draft_tok, float* draft_conf);
+/* One iteration of Algorithm 1's loop for every unfinished sequence: candidate selection with
+ * draft length N = min(max_drafts, masked-1) (0 if there are no drafts), chain of N+1 nodes,
+ * one batched forward, traversal, state and draft update.  `max_drafts` < 0 uses the config's;
+ * 0 gives a stepwise step.  accepted HOST [batch] (0 for finished sequences), n_nodes HOST
+ * [batch]; both may be NULL. */
+int ssd_block_step(ssd_ctx* ctx, int32_t max_drafts, int32_t* accepted, int32_t* n_nodes);
+/* Forward over the (fully unmasked) block that appends its K/V to the prefix cache. */
+int ssd_block_commit(ssd_ctx* ctx);
+
+/* The verification forward alone (Eq. 5) on caller-given node rows, against the current cache;
+ * the decode state is not touched.  HOST arrays: node_ids [batch, n_nodes, block_tokens],
+ * node_masked same shape (1 = this row's prediction is wanted); out_tok / out_conf same shape
+ * (token = argmax with the mask id excluded, lowest id on ties; conf = its softmax probability;
+ * -1 / 0 on rows not masked); out_logits [batch, n_nodes, block_tokens, vocab] fp32 or NULL
+ * (debug: materialises the logits, which the normal path never does). */
+int ssd_verify_forward(ssd_ctx* ctx, int32_t batch, int32_t n_nodes, int32_t block_tokens,
+                       const int32_t* node_ids, const uint8_t* node_masked,
+                       int32_t* out_tok, float* out_conf, float* out_logits);
+
+/* Read cached K (post-rotary) and V of one layer and sequence: HOST fp32
+ * [length, n_kv_heads, head_dim] each, positions [0, length).  Test hook for cache semantics. */
+int ssd_read_cache(ssd_ctx* ctx, int32_t layer, int32_t seq, int32_t length, float* out_k, float* out_v);
+
+/* Cached prefix length S (prompt + committed blocks), or a negative error. */
+int ssd_cache_length(const ssd_ctx* ctx);
+
+/* The skinny projection kernel alone: out[r][n] = sum_k x[r][k] * w[n][k] with bf16 operands and
+ * fp32 accumulation, split over `split_k` K ranges that are summed in order.  DEVICE pointers:
+ * x [rows, k] bf16, w [n, k] bf16, out [rows, n] fp32.  k a multiple of 8.  Test / tuning hook. */
+int ssd_gemm_bf16(ssd_ctx* ctx, const void* x_dev, const void* w_dev, float* out_dev,
+                  int32_t rows, int32_t n, int32_t k, int32_t split_k);
+
+/* ---- measurement ---------------------------------------------------------------------------- */
+
+/* Kernel launches issued by this context since creation (all streams of the context). */
+int64_t ssd_launch_count(const ssd_ctx* ctx);
+
+/* Per-kernel-family device time.  When enabled, every launch is bracketed by CUDA events on the
+ * context's stream (this serialises launches; do not time throughput in this mode).
+ * ssd_profile_read fills, for family f in [0, SSD_PROF_FAMILIES): launches[f], milliseconds[f],
+ * algorithmic bytes[f] (operand bytes that must cross HBM once), and resets the counters. */
+#define SSD_PROF_GEMM      0   /* QKV / O / gate-up / down projections                         */
+#define SSD_PROF_LMHEAD    1   /* LM head fused with softmax statistics                        */
+#define SSD_PROF_ATTN      2   /* shared-prefix attention (+ split merge)                      */
+#define SSD_PROF_ELEMWISE  3   /* embedding, norms, residuals, rotary, reductions              */
+#define SSD_PROF_TREE      4   /* tree build, acceptance                                       */
+#define SSD_PROF_FAMILIES  5
+int ssd_profile_enable(ssd_ctx* ctx, int32_t on);
+int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, double* bytes);
+
+/* Tuning knobs (set before prefill).  key: "split_k_qkv", "split_k_o", "split_k_down" (1..8),
+ * "kv_split" (prefix keys per attention split, multiple of 64; 0 = automatic from the prefix
+ * length), "gemm_impl" (1 = TMA + tcgen05 kernel, the default; 0 = the plain CUDA-core bring-up
+ * kernel, for cross-checks only).  Unknown key: SSD_ERR_INVALID_ARG. */
+int ssd_set_option(ssd_ctx* ctx, const char* key, int32_t value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* SSD_B200_H_ */

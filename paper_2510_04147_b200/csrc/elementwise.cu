@@ -1,0 +1,278 @@
+// Small memory-bound kernels around the projections: embedding gather, RMSNorm + residual with
+// split-K reduction, QKV finalisation with rotary embedding, SwiGLU, softmax statistics.
+// Every reduction has a fixed order that depends on the row alone, so a row's result does not
+// depend on how many other rows share the launch.
+#include "kernels.h"
+
+#include <math.h>
+
+namespace ssd {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// Deterministic block-wide sum (xor butterfly inside warps, then warp partials in warp order).
+__device__ __forceinline__ float block_sum(float v, float* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  __syncthreads();
+  if (l == 0) red[w] = v;
+  __syncthreads();
+  float t = 0.f;
+  const int nw = blockDim.x >> 5;
+  for (int i = 0; i < nw; ++i) t += red[i];
+  return t;
+}
+
+__global__ void convert_rows_kernel(const void* src, int src_is_f32, bf16* dst, int rows, int cols, int dst_pitch,
+                                    int group, int group_stride, int group_offset) {
+  const size_t total = (size_t)rows * cols;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int j = (int)(i / cols), c = (int)(i % cols);
+    const float v = src_is_f32 ? ((const float*)src)[i] : __bfloat162float(((const bf16*)src)[i]);
+    const size_t dr = (size_t)(j / group) * group_stride + group_offset + (j % group);
+    dst[dr * dst_pitch + c] = __float2bfloat16_rn(v);
+  }
+}
+
+__global__ void copy_f32_kernel(const void* src, int src_is_f32, float* dst, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src_is_f32 ? ((const float*)src)[i] : __bfloat162float(((const bf16*)src)[i]);
+}
+
+__device__ __forceinline__ void write_norm_row(const float* hrow, const float* gain, float inv, bf16* xrow, int d) {
+  for (int c = threadIdx.x * 4; c < d; c += kThreads * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(hrow + c);
+    const float4 g = *reinterpret_cast<const float4*>(gain + c);
+    __nv_bfloat162 a = __floats2bfloat162_rn(v.x * inv * g.x, v.y * inv * g.y);
+    __nv_bfloat162 b = __floats2bfloat162_rn(v.z * inv * g.z, v.w * inv * g.w);
+    *reinterpret_cast<__nv_bfloat162*>(xrow + c) = a;
+    *reinterpret_cast<__nv_bfloat162*>(xrow + c + 2) = b;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) embed_rmsnorm_kernel(const int* ids, const bf16* embed, const float* gain,
+                                                                 float eps, float* h, bf16* xn, int d) {
+  __shared__ float red[kThreads / 32];
+  const int r = blockIdx.x;
+  const bf16* e = embed + (size_t)ids[r] * d;
+  float* hrow = h + (size_t)r * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x * 4; c < d; c += kThreads * 4) {
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(e + c);
+    const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(e + c + 2);
+    float4 v = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
+    *reinterpret_cast<float4*>(hrow + c) = v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = block_sum(ss, red);
+  const float inv = rsqrtf(ss / (float)d + eps);
+  write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
+}
+
+__global__ void __launch_bounds__(kThreads) residual_rmsnorm_kernel(const float* partial, int splits, size_t split_stride,
+                                                                    const float* gain, float eps, float* h, bf16* xn,
+                                                                    int d) {
+  __shared__ float red[kThreads / 32];
+  const int r = blockIdx.x;
+  float* hrow = h + (size_t)r * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x * 4; c < d; c += kThreads * 4) {
+    float4 v = *reinterpret_cast<const float4*>(hrow + c);
+    for (int s = 0; s < splits; ++s) {
+      const float4 p = *reinterpret_cast<const float4*>(partial + s * split_stride + (size_t)r * d + c);
+      v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+    }
+    *reinterpret_cast<float4*>(hrow + c) = v;
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  if (gain == nullptr) return;
+  ss = block_sum(ss, red);
+  const float inv = rsqrtf(ss / (float)d + eps);
+  write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
+}
+
+__global__ void __launch_bounds__(kThreads) qkv_rope_kernel(const float* partial, int splits, size_t split_stride, int H,
+                                                            int Hkv, int hd, const float2* rope_table, RowMap map,
+                                                            bf16* q, bf16* k_dst, bf16* v_dst, int kv_to_cache,
+                                                            size_t cache_seq_stride) {
+  const int r = blockIdx.x;
+  const int half = hd >> 1;
+  const int nqkv = (H + 2 * Hkv) * hd;
+  const int slot = r / map.rows_per_seq;
+  const int t = r % map.T;
+  const int pos = map.pos0 + t;
+  const int seq = map.seq_map ? map.seq_map[slot] : map.seq_base + slot;
+  const float* prow = partial + (size_t)r * nqkv;
+  const size_t kv_row = kv_to_cache ? ((size_t)seq * cache_seq_stride + (size_t)pos * Hkv * hd) : (size_t)r * Hkv * hd;
+  const float2* rt = rope_table + (size_t)pos * half;
+  for (int p = threadIdx.x; p < (H + Hkv) * half; p += kThreads) {
+    const int head = p / half, i = p % half;
+    const int c1 = head * hd + i, c2 = c1 + half;
+    float x1 = 0.f, x2 = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      x1 += prow[s * split_stride + c1];
+      x2 += prow[s * split_stride + c2];
+    }
+    const float2 cs = rt[i];
+    const float y1 = x1 * cs.x - x2 * cs.y;
+    const float y2 = x2 * cs.x + x1 * cs.y;
+    if (head < H) {
+      bf16* dst = q + ((size_t)r * H + head) * hd;
+      dst[i] = __float2bfloat16_rn(y1);
+      dst[i + half] = __float2bfloat16_rn(y2);
+    } else {
+      bf16* dst = k_dst + kv_row + (size_t)(head - H) * hd;
+      dst[i] = __float2bfloat16_rn(y1);
+      dst[i + half] = __float2bfloat16_rn(y2);
+    }
+  }
+  const int voff = (H + Hkv) * hd;
+  for (int e = threadIdx.x; e < Hkv * hd; e += kThreads) {
+    float x = 0.f;
+    for (int s = 0; s < splits; ++s) x += prow[s * split_stride + voff + e];
+    v_dst[kv_row + e] = __float2bfloat16_rn(x);
+  }
+}
+
+__global__ void swiglu_kernel(const float* gu, bf16* act, int R, int ffn_pad) {
+  const size_t total = (size_t)R * ffn_pad;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / ffn_pad), f = (int)(i % ffn_pad);
+    const float* row = gu + (size_t)r * 2 * ffn_pad + (size_t)(f >> 6) * 128 + (f & 63);
+    const float g = row[0], u = row[64];
+    act[i] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) lm_stats_from_logits_kernel(const float* logits, int V, int mask_id,
+                                                                        const uint8_t* row_wanted, int* tok,
+                                                                        float* conf) {
+  __shared__ float red[kThreads / 32];
+  __shared__ float s_m[kThreads / 32];
+  __shared__ int s_a[kThreads / 32];
+  const int r = blockIdx.x;
+  if (row_wanted && !row_wanted[r]) {
+    if (threadIdx.x == 0) { tok[r] = -1; conf[r] = 0.f; }
+    return;
+  }
+  const float* l = logits + (size_t)r * V;
+  float m = -INFINITY;
+  int a = 0x7fffffff;
+  for (int v = threadIdx.x; v < V; v += kThreads) {
+    const float x = (v == mask_id) ? -INFINITY : l[v];
+    if (x > m) { m = x; a = v; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o);
+    const int oa = __shfl_xor_sync(0xffffffffu, a, o);
+    if (om > m || (om == m && oa < a)) { m = om; a = oa; }
+  }
+  if ((threadIdx.x & 31) == 0) { s_m[threadIdx.x >> 5] = m; s_a[threadIdx.x >> 5] = a; }
+  __syncthreads();
+  m = s_m[0]; a = s_a[0];
+  for (int i = 1; i < kThreads / 32; ++i)
+    if (s_m[i] > m || (s_m[i] == m && s_a[i] < a)) { m = s_m[i]; a = s_a[i]; }
+  float s = 0.f;
+  for (int v = threadIdx.x; v < V; v += kThreads)
+    if (v != mask_id) s += expf(l[v] - m);
+  s = block_sum(s, red);
+  if (threadIdx.x == 0) { tok[r] = a; conf[r] = 1.f / s; }
+}
+
+// One warp per row; lanes stride over the vocabulary tiles, then a fixed butterfly merge.
+__global__ void __launch_bounds__(kThreads) lm_merge_kernel(const float* tile_max, const float* tile_sum,
+                                                            const int* tile_arg, int tiles, int R,
+                                                            const uint8_t* row_wanted, int* tok, float* conf) {
+  const int r = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (r >= R) return;
+  if (row_wanted && !row_wanted[r]) {
+    if (lane == 0) { tok[r] = -1; conf[r] = 0.f; }
+    return;
+  }
+  float m = -INFINITY, s = 0.f;
+  int a = 0x7fffffff;
+  for (int t = lane; t < tiles; t += 32) {
+    const float tm = tile_max[(size_t)t * R + r];
+    if (tm == -INFINITY) continue;
+    const float ts = tile_sum[(size_t)t * R + r];
+    const int ta = tile_arg[(size_t)t * R + r];
+    if (tm > m) { s = s * expf(m - tm) + ts; m = tm; a = ta; }   // expf(-inf) = 0 on the first hit
+    else { s += ts * expf(tm - m); if (tm == m && ta < a) a = ta; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o);
+    const float os = __shfl_xor_sync(0xffffffffu, s, o);
+    const int oa = __shfl_xor_sync(0xffffffffu, a, o);
+    const float nm = fmaxf(m, om);
+    if (nm == -INFINITY) continue;
+    // symmetric in (self, other) so that both partners compute bit-identical results
+    const float lo_m = fminf(m, om);
+    const float hi_s = (m >= om) ? s : os;
+    const float lo_s = (m >= om) ? os : s;
+    const float ns = (m == om) ? (s + os) : (hi_s + lo_s * expf(lo_m - nm));
+    int na;
+    if (m == om) na = min(a, oa); else na = (m > om) ? a : oa;
+    m = nm; s = ns; a = na;
+  }
+  if (lane == 0) { tok[r] = a; conf[r] = 1.f / s; }
+}
+
+}  // namespace
+
+void launch_convert_rows(cudaStream_t st, const void* src, int src_is_f32, bf16* dst, int rows, int cols, int dst_pitch,
+                         int group, int group_stride, int group_offset) {
+  const size_t total = (size_t)rows * cols;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  convert_rows_kernel<<<blocks, 256, 0, st>>>(src, src_is_f32, dst, rows, cols, dst_pitch, group, group_stride,
+                                              group_offset);
+}
+
+void launch_copy_f32(cudaStream_t st, const void* src, int src_is_f32, float* dst, int n) {
+  copy_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(src, src_is_f32, dst, n);
+}
+
+void launch_embed_rmsnorm(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float eps, float* h,
+                          bf16* xn, int R, int d) {
+  embed_rmsnorm_kernel<<<R, kThreads, 0, st>>>(ids, embed, gain, eps, h, xn, d);
+}
+
+void launch_residual_rmsnorm(cudaStream_t st, const float* partial, int splits, size_t split_stride, const float* gain,
+                             float eps, float* h, bf16* xn, int R, int d) {
+  residual_rmsnorm_kernel<<<R, kThreads, 0, st>>>(partial, splits, split_stride, gain, eps, h, xn, d);
+}
+
+void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H, int Hkv,
+                     int hd, const float2* rope_table, RowMap map, bf16* q, bf16* k_dst, bf16* v_dst, int kv_to_cache,
+                     size_t cache_seq_stride) {
+  qkv_rope_kernel<<<R, kThreads, 0, st>>>(partial, splits, split_stride, H, Hkv, hd, rope_table, map, q, k_dst, v_dst,
+                                          kv_to_cache, cache_seq_stride);
+}
+
+void launch_swiglu(cudaStream_t st, const float* gu, bf16* act, int R, int ffn_pad) {
+  const size_t total = (size_t)R * ffn_pad;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  swiglu_kernel<<<blocks, 256, 0, st>>>(gu, act, R, ffn_pad);
+}
+
+void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, int V, int mask_id,
+                                 const uint8_t* row_wanted, int* tok, float* conf) {
+  lm_stats_from_logits_kernel<<<R, kThreads, 0, st>>>(logits, V, mask_id, row_wanted, tok, conf);
+}
+
+void launch_lm_merge(cudaStream_t st, const float* tile_max, const float* tile_sum, const int* tile_arg, int tiles,
+                     int R, const uint8_t* row_wanted, int* tok, float* conf) {
+  const int rows_per_block = kThreads / 32;
+  lm_merge_kernel<<<(R + rows_per_block - 1) / rows_per_block, kThreads, 0, st>>>(tile_max, tile_sum, tile_arg, tiles,
+                                                                                  R, row_wanted, tok, conf);
+}
+
+}  // namespace ssd

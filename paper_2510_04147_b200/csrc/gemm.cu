@@ -1,0 +1,478 @@
+// Weight-streaming skinny GEMM for the projections of the verification forward:
+//     out[r][n] = sum_k x[r][k] * w[n][k]      (bf16 operands, fp32 accumulation)
+// with r = rows of ALL tree nodes (tens to a few hundred) and n = output features (thousands).
+// The weight matrix is the big operand and is read from HBM exactly once per forward; the
+// activations are small and stay in L2.
+//
+// Tensor-core kernel (sm_100a): "swap-AB" mapping.  A CTA owns 128 output features: the weight
+// tile [128 x 64] is the M x K operand of tcgen05.mma, the activation tile [rows x 64] is the
+// N x K operand, the fp32 accumulator [128 lanes x rows columns] lives in tensor memory.  Both
+// tiles are staged by TMA (128-byte swizzle) through an mbarrier ring; one thread issues the
+// MMAs; four warps read the accumulator back with tcgen05.ld and run the epilogue:
+//   EPI_PARTIAL  fp32 partial sums per K split (summed later in split order),
+//   EPI_SWIGLU   weight rows interleaved as 64 gate + 64 up features per tile -> silu(g)*u in bf16,
+//   EPI_LMHEAD   per-row max / argmax / sum-exp over the tile's 128 vocabulary entries, so the
+//                logits never leave the SM.
+// Every wait is bounded: on expiry the kernel raises an error word and unwinds.
+//
+// A plain CUDA-core kernel of the same contract is kept for bring-up and as a cross-check.
+#include "kernels.h"
+
+#include <cuda.h>
+#include <math.h>
+#include <stdio.h>
+
+namespace ssd {
+
+int gemm_tiles(int N) { return (N + 127) / 128; }
+
+// =====================================================================================
+// CUDA-core kernel (bring-up / cross-check)
+// =====================================================================================
+namespace {
+
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16* __restrict__ x, const bf16* __restrict__ w,
+                                                        float* __restrict__ out, int R, int N, int K, int x_pitch,
+                                                        int w_pitch, int splits) {
+  __shared__ float Ws[64][33];
+  __shared__ float Xs[32][33];
+  const int n0 = blockIdx.x * 64, r0 = blockIdx.y * 32, split = blockIdx.z;
+  const int kb_total = (K + 63) / 64;
+  const int k_begin = (int)((long long)split * kb_total / splits) * 64;
+  const int k_end = min(K, (int)((long long)(split + 1) * kb_total / splits) * 64);
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  float acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+  for (int k0 = k_begin; k0 < k_end; k0 += 32) {
+    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
+      const int rr = i >> 5, kk = i & 31;
+      const int n = n0 + rr, k = k0 + kk;
+      Ws[rr][kk] = (n < N && k < k_end) ? __bfloat162float(w[(size_t)n * w_pitch + k]) : 0.f;
+    }
+    for (int i = threadIdx.x; i < 32 * 32; i += 256) {
+      const int rr = i >> 5, kk = i & 31;
+      const int r = r0 + rr, k = k0 + kk;
+      Xs[rr][kk] = (r < R && k < k_end) ? __bfloat162float(x[(size_t)r * x_pitch + k]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int kk = 0; kk < 32; ++kk) {
+      const float wv = Ws[tx][kk];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] += wv * Xs[ty * 8 + i][kk];
+    }
+    __syncthreads();
+  }
+  const int n = n0 + tx;
+  if (n < N) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int r = r0 + ty * 8 + i;
+      if (r < R) out[((size_t)split * R + r) * N + n] = acc[i];
+    }
+  }
+}
+
+}  // namespace
+
+void launch_gemm_simt(cudaStream_t st, const GemmArgs& g) {
+  dim3 grid((g.N + 63) / 64, (g.R + 31) / 32, g.splits);
+  gemm_simt_kernel<<<grid, 256, 0, st>>>(g.x, g.w, g.out, g.R, g.N, g.K, g.x_pitch, g.w_pitch, g.splits);
+}
+
+// =====================================================================================
+// Tensor-core kernel
+// =====================================================================================
+namespace {
+
+constexpr int kTileM = 128;          // output features per CTA (MMA M)
+constexpr int kBlockK = 64;          // bf16 elements per stage along K = one 128-byte swizzle row
+constexpr int kTcThreads = 192;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int kMaxStages = 8;
+constexpr int kWTileBytes = kTileM * kBlockK * 2;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
+
+struct TcParams {
+  int R, N, K;
+  int npad;        // MMA N: rows of one row chunk rounded up to 16 (<= 256)
+  int splits;
+  int stages;
+  int epi;
+  uint32_t tmem_cols;
+  float* out;
+  bf16* act;
+  int act_pitch;
+  float* tile_max;
+  float* tile_sum;
+  int* tile_arg;
+  int mask_id;
+  int* err_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the limit expired or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 63) == 0) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// K-major operand tile in shared memory, 128-byte swizzle, rows 128 B apart, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                 // leading-dimension byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride-dimension byte offset: 8 rows * 128 B
+  d |= (uint64_t)1 << 46;                 // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                 // 128-byte swizzle
+  return d;
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kTcThreads, 2)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const TcParams p) {
+  extern __shared__ uint8_t smem_dyn[];
+  // 1024-byte alignment for the swizzled tiles
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  const int x_tile_bytes = p.npad * kBlockK * 2;
+  uint8_t* sW = smem;
+  uint8_t* sX = smem + (size_t)p.stages * kWTileBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sX + (size_t)p.stages * x_tile_bytes);
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = bars + kMaxStages;
+  uint64_t* acc_bar = bars + 2 * kMaxStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x, split = blockIdx.y, row0 = blockIdx.z * 256;
+  const int kb_total = (p.K + kBlockK - 1) / kBlockK;
+  const int kb_begin = (int)((long long)split * kb_total / p.splits);
+  const int kb_end = (int)((long long)(split + 1) * kb_total / p.splits);
+  const int n_kb = kb_end - kb_begin;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_addr(&full_bar[s]), 1);
+      mbar_init(smem_addr(&empty_bar[s]), 1);
+    }
+    mbar_init(smem_addr(acc_bar), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tmW) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tmX) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
+                 "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const uint32_t stage_bytes = (uint32_t)(kWTileBytes + x_tile_bytes);
+      int issued = 0;
+      bool ok = true;
+      for (int it = 0; it < n_kb; ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (uint32_t)((it / p.stages) & 1);
+        if (!mbar_wait(smem_addr(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t fb = smem_addr(&full_bar[s]);
+        mbar_expect_tx(fb, stage_bytes);
+        const int kc = (kb_begin + it) * kBlockK;
+        tma_load_2d(smem_addr(sW + (size_t)s * kWTileBytes), &tmW, fb, kc, tile * kTileM);
+        tma_load_2d(smem_addr(sX + (size_t)s * x_tile_bytes), &tmX, fb, kc, row0);
+        ++issued;
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        atomicExch(p.err_flag, 1);
+        // let the copies already in flight land before the CTA's shared memory goes away
+        const int first = issued > p.stages ? issued - p.stages : 0;
+        for (int j = first; j < issued; ++j) {
+          const unsigned long long t0 = globaltimer_ns();
+          while (!mbar_try_wait(smem_addr(&full_bar[j % p.stages]), (uint32_t)((j / p.stages) & 1)))
+            if (globaltimer_ns() - t0 > kWaitLimitNs) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.npad >> 3) << 17) |
+                             ((uint32_t)(kTileM >> 4) << 24);
+      bool ok = true;
+      for (int it = 0; it < n_kb; ++it) {
+        const int s = it % p.stages;
+        const uint32_t ph = (uint32_t)((it / p.stages) & 1);
+        if (!mbar_wait(smem_addr(&full_bar[s]), ph, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t wa = smem_addr(sW + (size_t)s * kWTileBytes);
+        const uint32_t xa = smem_addr(sX + (size_t)s * x_tile_bytes);
+#pragma unroll
+        for (int k = 0; k < kBlockK / 16; ++k) {
+          tc_mma_bf16(tmem_base, make_smem_desc(wa + k * 32), make_smem_desc(xa + k * 32), idesc,
+                      (uint32_t)((it | k) != 0));
+        }
+        tc_commit(smem_addr(&empty_bar[s]));
+      }
+      if (ok) {
+        tc_commit(smem_addr(acc_bar));
+      } else {
+        *abort_flag = 1;
+        atomicExch(p.err_flag, 2);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps)
+    const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+    const int lrow = quad * 32 + lane;         // accumulator lane = feature inside the tile
+    bool ok = true;
+    if (n_kb > 0) ok = mbar_wait(smem_addr(acc_bar), 0u, abort_flag);
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after();
+    const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const int rows_here = min(p.R - row0, 256);
+    float* scratch = reinterpret_cast<float*>(sW);   // stage 0 of the ring is free once acc_bar fired
+    if (!ok) {
+      if (lane == 0) { *abort_flag = 1; atomicExch(p.err_flag, 3); }
+    } else if (p.epi == EPI_PARTIAL) {
+      const int n = tile * kTileM + lrow;
+      for (int c0 = 0; c0 < p.npad; c0 += 32) {
+        float v[32];
+        if (n_kb > 0) tmem_ld32(taddr + c0, v);
+        else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0.f;
+        }
+        if (n < p.N) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int rr = c0 + j;
+            if (rr < rows_here) p.out[((size_t)split * p.R + row0 + rr) * p.N + n] = v[j];
+          }
+        }
+      }
+    } else if (p.epi == EPI_SWIGLU) {
+      // lanes 0-63 hold gate features, lanes 64-127 the matching up features
+      const int f = tile * 64 + (lrow & 63);
+      for (int c0 = 0; c0 < p.npad; c0 += 32) {
+        float v[32];
+        tmem_ld32(taddr + c0, v);
+        if (lrow >= 64) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) scratch[(lrow - 64) * 33 + j] = v[j];
+        }
+        epi_bar_sync();
+        if (lrow < 64) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int rr = c0 + j;
+            if (rr < rows_here) {
+              const float u = scratch[lrow * 33 + j];
+              const float g = v[j];
+              p.act[(size_t)(row0 + rr) * p.act_pitch + f] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
+            }
+          }
+        }
+        epi_bar_sync();
+      }
+    } else {
+      // EPI_LMHEAD: lane = vocabulary entry; reduce over the 128 lanes per row (= column)
+      const int n = tile * kTileM + lrow;
+      const bool live = (n < p.N) && (n != p.mask_id);
+      float* s_max = scratch;                       // [4][256]
+      float* s_sum = scratch + 4 * 256;
+      int* s_arg = reinterpret_cast<int*>(scratch + 8 * 256);
+      for (int c0 = 0; c0 < p.npad; c0 += 32) {
+        float v[32];
+        tmem_ld32(taddr + c0, v);
+        float my_m = -INFINITY, my_s = 0.f;
+        int my_a = 0x7fffffff;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float x = live ? v[j] : -INFINITY;
+          float m = x;
+          int a = n;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, m, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, a, o);
+            if (om > m || (om == m && oa < a)) { m = om; a = oa; }
+          }
+          float e = (m == -INFINITY) ? 0.f : expf(x - m);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+          if (lane == j) { my_m = m; my_s = e; my_a = a; }
+        }
+        s_max[quad * 256 + c0 + lane] = my_m;
+        s_sum[quad * 256 + c0 + lane] = my_s;
+        s_arg[quad * 256 + c0 + lane] = my_a;
+      }
+      epi_bar_sync();
+      for (int c = (warp - 2) * 32 + lane; c < rows_here; c += 128) {
+        float M = -INFINITY;
+        int A = 0x7fffffff;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float m = s_max[q * 256 + c];
+          if (m > M) { M = m; A = s_arg[q * 256 + c]; }
+        }
+        float S = 0.f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float m = s_max[q * 256 + c];
+          if (m != -INFINITY) S += s_sum[q * 256 + c] * expf(m - M);
+        }
+        const size_t o = (size_t)tile * p.R + row0 + c;
+        p.tile_max[o] = M;
+        p.tile_sum[o] = S;
+        p.tile_arg[o] = A;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+// [rows][pitch] bf16, K contiguous; box = 64 x box_rows; out-of-range elements read as zero
+bool make_tmap(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t pitch_elems, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch_elems * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int gemm_tc_init() {
+  if (g_encode) return 0;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+      q != cudaDriverEntryPointSuccess)
+    return -4;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return 0;
+}
+
+int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
+  if (!g_encode) return -4;
+  if ((g.x_pitch % 8) || (g.w_pitch % 8) || (((uintptr_t)g.x) & 15) || (((uintptr_t)g.w) & 15)) return -2;
+  if (g.R < 1 || g.N < 1 || g.K < 1) return -2;
+  if (g.epi != EPI_PARTIAL && g.splits != 1) return -2;
+  if (g.epi == EPI_SWIGLU && (g.N % 128)) return -2;
+  TcParams p;
+  p.R = g.R; p.N = g.N; p.K = g.K;
+  const int rows_chunk = g.R < 256 ? g.R : 256;
+  p.npad = (rows_chunk + 15) & ~15;
+  p.splits = g.splits;
+  p.epi = g.epi;
+  uint32_t cols = 32;
+  while ((int)cols < p.npad) cols <<= 1;
+  p.tmem_cols = cols;
+  const int stage_bytes = kWTileBytes + p.npad * kBlockK * 2;
+  // two CTAs per SM while the activation tile is small, one deep pipeline otherwise
+  const int budget = (p.npad <= 128) ? 108 * 1024 : 200 * 1024;
+  int stages = budget / stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < 3) stages = 3;
+  p.stages = stages;
+  p.out = g.out; p.act = g.act; p.act_pitch = g.act_pitch;
+  p.tile_max = g.tile_max; p.tile_sum = g.tile_sum; p.tile_arg = g.tile_arg;
+  p.mask_id = g.mask_id; p.err_flag = g.err_flag;
+  const int smem = stages * stage_bytes + 1024 /*alignment slack*/ + (2 * kMaxStages + 1) * 8 + 16;
+  // tensor-memory safety: CTAs that fit by shared memory must also fit by TMEM columns
+  if ((227 * 1024 / smem) * (int)cols > 512) return -2;
+  CUtensorMap tmW, tmX;
+  if (!make_tmap(&tmW, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.w_pitch, kTileM)) return -4;
+  if (!make_tmap(&tmX, g.x, (uint64_t)g.R, (uint64_t)g.K, (uint64_t)g.x_pitch, (uint32_t)p.npad)) return -4;
+  static int smem_set = 0;
+  if (smem > smem_set) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return -4;
+    smem_set = 227 * 1024;
+  }
+  dim3 grid(gemm_tiles(g.N), g.splits, (g.R + 255) / 256);
+  gemm_tc_kernel<<<grid, kTcThreads, smem, st>>>(tmW, tmX, p);
+  return 0;
+}
+
+}  // namespace ssd

@@ -1,0 +1,115 @@
+// Internal launcher declarations shared by the translation units of the library.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+namespace ssd {
+
+// ---------------------------------------------------------------- layout helpers (host+device)
+// Rows of a forward are ordered [sequence slot a][node i][in-block index t].
+struct RowMap {
+  int rows_per_seq;    // n_nodes * T
+  int T;               // rows per node (block tokens, or prompt length for prefill)
+  int pos0;            // absolute position of t = 0 (= cached prefix length S)
+  int seq_base;        // sequence id of slot 0 when seq_map == nullptr
+  const int* seq_map;  // device [slots] slot -> sequence id, or nullptr (identity + seq_base)
+};
+
+// ---------------------------------------------------------------- weight repacking
+// dst[(j / group) * group_stride + group_offset + j % group][c] = bf16(src[j][c]),  j < rows, c < cols
+void launch_convert_rows(cudaStream_t st, const void* src, int src_is_f32, bf16* dst, int rows, int cols,
+                         int dst_pitch, int group, int group_stride, int group_offset);
+void launch_copy_f32(cudaStream_t st, const void* src, int src_is_f32, float* dst, int n);
+
+// ---------------------------------------------------------------- elementwise / reductions
+// h[r] = embed[ids[r]]; xn[r] = bf16(rmsnorm(h[r]) * gain)
+void launch_embed_rmsnorm(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float eps,
+                          float* h, bf16* xn, int R, int d);
+// h[r] += sum_s partial[s][r] (s ascending); if gain: xn[r] = bf16(rmsnorm(h[r]) * gain)
+void launch_residual_rmsnorm(cudaStream_t st, const float* partial, int splits, size_t split_stride,
+                             const float* gain, float eps, float* h, bf16* xn, int R, int d);
+// sums the split-K partials of the fused QKV projection, rotates q and k, writes bf16.
+// kv_to_cache: k/v rows go to cache[(seq*max_seq + pos)*Hkv*hd] else to local [r][Hkv][hd].
+void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H,
+                     int Hkv, int hd, const float2* rope_table, RowMap map, bf16* q, bf16* k_dst, bf16* v_dst,
+                     int kv_to_cache, size_t cache_seq_stride);
+// act[r][f] = bf16(silu(g) * u) from fp32 gate/up laid out in 64-row interleaved groups of 128
+void launch_swiglu(cudaStream_t st, const float* gu, bf16* act, int R, int ffn_pad);
+// per row: argmax / max-softmax-probability over the vocabulary with mask_id excluded
+void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, int V, int mask_id,
+                                 const uint8_t* row_wanted, int* tok, float* conf);
+// merge per-tile (max, sumexp, argmax) in tile order
+void launch_lm_merge(cudaStream_t st, const float* tile_max, const float* tile_sum, const int* tile_arg,
+                     int tiles, int R, const uint8_t* row_wanted, int* tok, float* conf);
+
+// ---------------------------------------------------------------- attention
+struct AttnArgs {
+  const bf16* q;        // [R][H][hd], rotated
+  const bf16* cache_k;  // layer base: [seq][max_seq][Hkv][hd]
+  const bf16* cache_v;
+  const bf16* local_k;  // [R][Hkv][hd] or nullptr (no node-local keys)
+  const bf16* local_v;
+  float* part_o;        // [n_parts][R][H][hd]
+  float2* part_ml;      // [n_parts][R][H]  (running max in log2 domain, sum)
+  bf16* out;            // [R][H*hd]
+  int R, H, Hkv, hd;
+  int S;                // prefix keys read from the cache
+  int kv_split;         // prefix keys per split (a function of S only)
+  size_t cache_seq_stride;
+  RowMap map;
+  int n_seq_slots;
+};
+void launch_attention(cudaStream_t st, const AttnArgs& a, int* launches);
+
+// ---------------------------------------------------------------- projections
+enum { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_LMHEAD = 2 };
+struct GemmArgs {
+  const bf16* x;  // [R][x_pitch] activations (K-major)
+  const bf16* w;  // [N][w_pitch] weights (K-major)
+  int R, N, K, x_pitch, w_pitch;
+  int splits;            // split-K factor (EPI_PARTIAL only)
+  int epi;
+  float* out;            // EPI_PARTIAL: [splits][R][N] fp32
+  bf16* act;             // EPI_SWIGLU: [R][act_pitch], N/2 features
+  int act_pitch;
+  float* tile_max;       // EPI_LMHEAD: [tiles][R]
+  float* tile_sum;
+  int* tile_arg;
+  int mask_id;
+  int* err_flag;         // device int set non-zero when a bounded wait expires
+};
+int gemm_tiles(int N);
+void launch_gemm_simt(cudaStream_t st, const GemmArgs& g);
+// tensor-core path (TMA + tcgen05). Returns 0 or a negative ssd error code.
+int launch_gemm_tc(cudaStream_t st, const GemmArgs& g);
+int gemm_tc_init();   // resolves the driver entry point for tensor-map encoding
+
+// ---------------------------------------------------------------- tree build / acceptance
+struct BlockState {       // device arrays, [max_batch][block_len] unless noted
+  int* ids;
+  uint8_t* masked;
+  int* draft_tok;
+  float* draft_conf;
+  int* has_drafts;        // [max_batch]
+  int* remaining;         // [max_batch] r
+  int* cand_pos;          // [max_batch][block_len]
+  int* cand_tok;
+  int* n_cand;            // [max_batch] N of the current forward
+  int* accept_log;        // [max_batch][block_len] accepted per forward, 0-terminated
+  int* n_forwards;        // [max_batch]
+  int* last_accept;       // [max_batch] accepted by the latest step (0 if not active)
+  int* seq_map;           // [max_batch] slot -> sequence of the current forward
+  int stride;             // block_len (row pitch of the arrays above)
+};
+// slot a (= rank among unfinished sequences): candidates, node rows [a][n_cap][T]
+void launch_tree_build(cudaStream_t st, BlockState s, int batch, int T, int max_drafts, int n_cap, int mask_id,
+                       int* node_ids, uint8_t* node_masked);
+// per slot: per-node best masked position, chain walk, state/draft update
+void launch_accept(cudaStream_t st, BlockState s, int n_slots, int T, int n_cap, const int* tok, const float* conf,
+                   const uint8_t* node_masked, int* nonfinite_flag);
+
+}  // namespace ssd

@@ -1,0 +1,815 @@
+// Host side of the C ABI declared in include/ssd.h: context, weight repacking, the forward pass
+// schedule (one launch sequence per layer), and the per-block decode loop of Algorithm 1.
+#include "../../include/ssd.h"
+#include "kernels.h"
+
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+using namespace ssd;
+
+namespace {
+
+struct LayerW {
+  bf16 *wqkv = nullptr, *wo = nullptr, *wgu = nullptr, *wd = nullptr;
+  float *g_attn = nullptr, *g_ffn = nullptr;
+  uint32_t loaded = 0;   // bit per tensor
+};
+
+struct ProfRec { int fam; cudaEvent_t e0, e1; double bytes; };
+
+char g_create_error[256] = "";
+
+}  // namespace
+
+struct ssd_ctx {
+  ssd_config cfg;
+  cudaStream_t st = nullptr;
+  int H = 0, Hkv = 0, hd = 0, d = 0, ffn = 0, ffn_pad = 0, V = 0, nqkv = 0, qdim = 0, kvdim = 0;
+  std::vector<LayerW> L;
+  bf16 *embed = nullptr, *lm_head = nullptr;
+  float* g_final = nullptr;
+  uint32_t loaded_globals = 0;
+
+  bf16 *cacheK = nullptr, *cacheV = nullptr;
+  size_t cache_seq_stride = 0, cache_layer_stride = 0;
+  float2* rope = nullptr;
+
+  int n_max = 1;         // nodes per sequence the buffers can hold
+  int R_dec = 0;         // max rows of a verification forward
+  int R_cap = 0;         // max rows of any forward
+  size_t partial_elems = 0, part_rows_parts = 0;
+  float* h = nullptr;
+  bf16* xn = nullptr;
+  float* partial = nullptr;
+  bf16 *q = nullptr, *lk = nullptr, *lv = nullptr, *att = nullptr, *act = nullptr;
+  float* part_o = nullptr;
+  float2* part_ml = nullptr;
+  float *tile_max = nullptr, *tile_sum = nullptr;
+  int* tile_arg = nullptr;
+  int* tok = nullptr;
+  float* conf = nullptr;
+  int* node_ids = nullptr;
+  uint8_t* node_masked = nullptr;
+  float* logits = nullptr;
+  size_t logits_elems = 0;
+  int* flags = nullptr;          // [0] bounded-wait expiry, [1] non-finite confidence
+  int* h_pinned = nullptr;       // pinned host staging: [0..1] flags, then 3 * max_batch ints
+  BlockState bs{};
+
+  int batch = 0, prompt_len = 0, cache_len = -1, block_tokens = 0;
+  bool in_block = false;
+  std::vector<int> h_remaining, h_has_drafts;
+
+  int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0, gemm_impl = 1;
+  int64_t launches = 0;
+  bool profiling = false;
+  std::vector<ProfRec> prof;
+  std::vector<void*> allocs;
+  char err[256] = "";
+};
+
+namespace {
+
+int fail(ssd_ctx* c, int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(c ? c->err : g_create_error, 256, fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+#define CUDA_TRY(c, expr)                                                                          \
+  do {                                                                                             \
+    cudaError_t e_ = (expr);                                                                       \
+    if (e_ != cudaSuccess)                                                                         \
+      return fail((c), e_ == cudaErrorMemoryAllocation ? SSD_ERR_OOM : SSD_ERR_CUDA, "%s: %s", #expr, \
+                  cudaGetErrorString(e_));                                                         \
+  } while (0)
+
+template <typename T>
+int dev_alloc(ssd_ctx* c, T** p, size_t n, bool zero = true) {
+  void* v = nullptr;
+  if (n == 0) n = 1;
+  cudaError_t e = cudaMalloc(&v, n * sizeof(T));
+  if (e != cudaSuccess) return fail(c, SSD_ERR_OOM, "cudaMalloc of %zu bytes failed: %s", n * sizeof(T), cudaGetErrorString(e));
+  if (zero) {
+    e = cudaMemsetAsync(v, 0, n * sizeof(T), c->st);
+    if (e != cudaSuccess) return fail(c, SSD_ERR_CUDA, "cudaMemset failed: %s", cudaGetErrorString(e));
+  }
+  c->allocs.push_back(v);
+  *p = reinterpret_cast<T*>(v);
+  return SSD_OK;
+}
+#define ALLOC(c, p, n)                               \
+  do {                                               \
+    int rc_ = dev_alloc((c), &(p), (size_t)(n));     \
+    if (rc_ != SSD_OK) return rc_;                   \
+  } while (0)
+
+int auto_split(int tiles) {
+  int s = 148 / tiles;
+  if (s < 1) s = 1;
+  if (s > 8) s = 8;
+  return s;
+}
+
+int kv_split_for(const ssd_ctx* c, int S) {
+  if (c->kv_split_opt > 0) return c->kv_split_opt;
+  return S <= 4096 ? 256 : 512;      // a function of the prefix length only
+}
+
+// ---- profiling / launch accounting --------------------------------------------------------
+struct Scope {
+  ssd_ctx* c;
+  int fam;
+  double bytes;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  Scope(ssd_ctx* c_, int fam_, double bytes_, int n_launches = 1) : c(c_), fam(fam_), bytes(bytes_) {
+    c->launches += n_launches;
+    if (c->profiling) {
+      cudaEventCreate(&e0);
+      cudaEventCreate(&e1);
+      cudaEventRecord(e0, c->st);
+    }
+  }
+  ~Scope() {
+    if (c->profiling) {
+      cudaEventRecord(e1, c->st);
+      c->prof.push_back({fam, e0, e1, bytes});
+    }
+  }
+};
+
+__global__ void sum_splits_kernel(const float* partial, int splits, size_t stride, float* out, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float v = 0.f;
+  for (int s = 0; s < splits; ++s) v += partial[s * stride + i];
+  out[i] = v;
+}
+
+__global__ void block_init_kernel(BlockState s, int batch, int max_batch, int T, int mask_id) {
+  const int b = blockIdx.x;
+  for (int t = threadIdx.x; t < s.stride; t += blockDim.x) {
+    const size_t o = (size_t)b * s.stride + t;
+    s.ids[o] = mask_id;
+    s.masked[o] = (b < batch && t < T) ? 1 : 0;
+    s.draft_tok[o] = 0;
+    s.draft_conf[o] = 0.f;
+    s.cand_pos[o] = 0;
+    s.cand_tok[o] = 0;
+    s.accept_log[o] = 0;
+  }
+  if (threadIdx.x == 0) {
+    s.has_drafts[b] = 0;
+    s.remaining[b] = (b < batch) ? T : 0;
+    s.n_cand[b] = 0;
+    s.n_forwards[b] = 0;
+    s.last_accept[b] = 0;
+    s.seq_map[b] = b;
+  }
+}
+
+// ---- projections ----------------------------------------------------------------------------
+int run_gemm(ssd_ctx* c, GemmArgs g, int fam) {
+  Scope sc(c, fam, (double)g.N * g.K * 2.0);
+  g.err_flag = c->flags;
+  if (c->gemm_impl == 1) {
+    const int rc = launch_gemm_tc(c->st, g);
+    if (rc != 0) return fail(c, rc, "tensor-core GEMM rejected R=%d N=%d K=%d epi=%d (code %d)", g.R, g.N, g.K, g.epi, rc);
+  } else {
+    if (g.epi != EPI_PARTIAL) return fail(c, SSD_ERR_INVALID_ARG, "bring-up GEMM has no fused epilogue");
+    launch_gemm_simt(c->st, g);
+  }
+  return SSD_OK;
+}
+
+bool all_loaded(const ssd_ctx* c) {
+  if (c->loaded_globals != 7u) return false;
+  for (const LayerW& l : c->L)
+    if (l.loaded != 0x1FFu) return false;
+  return true;
+}
+
+enum { FWD_FILL = 0, FWD_VERIFY = 1 };
+
+// One forward over R rows.  FILL: K/V go to the cache at positions pos0.., attention over the cache
+// only (which then contains the rows themselves), no LM head.  VERIFY: K/V stay node-local, attention
+// over cached prefix + own node, LM head statistics into tok/conf (and logits if wanted).
+int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_slots, bool want_logits,
+            const uint8_t* row_wanted) {
+  const int d = c->d, H = c->H, Hkv = c->Hkv, hd = c->hd;
+  const int S = map.pos0;
+  if (R > c->R_cap) return fail(c, SSD_ERR_OVERFLOW, "forward of %d rows exceeds capacity %d", R, c->R_cap);
+  const int attn_S = (kind == FWD_FILL) ? S + map.T : S;
+  const int kv_split = (kind == FWD_FILL) ? attn_S : kv_split_for(c, S);
+  const int n_parts = (attn_S + kv_split - 1) / kv_split + (kind == FWD_VERIFY ? 1 : 0);
+  if ((size_t)n_parts * R > c->part_rows_parts)
+    return fail(c, SSD_ERR_OVERFLOW, "attention workspace too small for %d parts x %d rows", n_parts, R);
+  const int nl = c->cfg.n_layers;
+  {
+    Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * 8);
+    launch_embed_rmsnorm(c->st, ids_dev, c->embed, c->L[0].g_attn, c->cfg.rms_eps, c->h, c->xn, R, d);
+  }
+  for (int l = 0; l < nl; ++l) {
+    const LayerW& w = c->L[l];
+    // ---- QKV projection, rotary embedding
+    GemmArgs g{};
+    g.x = c->xn; g.w = w.wqkv; g.R = R; g.N = c->nqkv; g.K = d; g.x_pitch = d; g.w_pitch = d;
+    g.splits = c->split_qkv; g.epi = EPI_PARTIAL; g.out = c->partial;
+    if ((size_t)g.splits * R * g.N > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "split-K workspace too small");
+    int rc = run_gemm(c, g, SSD_PROF_GEMM);
+    if (rc) return rc;
+    bf16* kdst = (kind == FWD_FILL) ? c->cacheK + (size_t)l * c->cache_layer_stride : c->lk;
+    bf16* vdst = (kind == FWD_FILL) ? c->cacheV + (size_t)l * c->cache_layer_stride : c->lv;
+    {
+      Scope sc(c, SSD_PROF_ELEMWISE, (double)R * c->nqkv * (4.0 * g.splits + 2.0));
+      launch_qkv_rope(c->st, c->partial, g.splits, (size_t)R * c->nqkv, R, H, Hkv, hd, c->rope, map, c->q, kdst, vdst,
+                      kind == FWD_FILL ? 1 : 0, c->cache_seq_stride);
+    }
+    if (kind == FWD_FILL && l == nl - 1) break;   // only this layer's K/V were still needed
+    // ---- attention
+    {
+      AttnArgs a{};
+      a.q = c->q;
+      a.cache_k = c->cacheK + (size_t)l * c->cache_layer_stride;
+      a.cache_v = c->cacheV + (size_t)l * c->cache_layer_stride;
+      a.local_k = (kind == FWD_VERIFY) ? c->lk : nullptr;
+      a.local_v = (kind == FWD_VERIFY) ? c->lv : nullptr;
+      a.part_o = c->part_o; a.part_ml = c->part_ml; a.out = c->att;
+      a.R = R; a.H = H; a.Hkv = Hkv; a.hd = hd; a.S = attn_S; a.kv_split = kv_split;
+      a.cache_seq_stride = c->cache_seq_stride; a.map = map; a.n_seq_slots = n_slots;
+      const double kvb = (double)n_slots * attn_S * Hkv * hd * 4.0 + (double)R * (H + 2 * Hkv) * hd * 2.0 + (double)R * H * hd * 2.0;
+      Scope sc(c, SSD_PROF_ATTN, kvb, 2);
+      launch_attention(c->st, a, nullptr);
+    }
+    // ---- output projection + residual + norm
+    g = GemmArgs{};
+    g.x = c->att; g.w = w.wo; g.R = R; g.N = d; g.K = c->qdim; g.x_pitch = c->qdim; g.w_pitch = c->qdim;
+    g.splits = c->split_o; g.epi = EPI_PARTIAL; g.out = c->partial;
+    rc = run_gemm(c, g, SSD_PROF_GEMM);
+    if (rc) return rc;
+    {
+      Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * (4.0 * g.splits + 10.0));
+      launch_residual_rmsnorm(c->st, c->partial, g.splits, (size_t)R * d, w.g_ffn, c->cfg.rms_eps, c->h, c->xn, R, d);
+    }
+    // ---- gate/up projection with SwiGLU
+    g = GemmArgs{};
+    g.x = c->xn; g.w = w.wgu; g.R = R; g.N = 2 * c->ffn_pad; g.K = d; g.x_pitch = d; g.w_pitch = d;
+    g.splits = 1;
+    if (c->gemm_impl == 1) {
+      g.epi = EPI_SWIGLU; g.act = c->act; g.act_pitch = c->ffn_pad;
+      rc = run_gemm(c, g, SSD_PROF_GEMM);
+      if (rc) return rc;
+    } else {
+      g.epi = EPI_PARTIAL; g.out = c->partial;
+      if ((size_t)R * g.N > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "workspace too small");
+      rc = run_gemm(c, g, SSD_PROF_GEMM);
+      if (rc) return rc;
+      Scope sc(c, SSD_PROF_ELEMWISE, (double)R * c->ffn_pad * 10.0);
+      launch_swiglu(c->st, c->partial, c->act, R, c->ffn_pad);
+    }
+    // ---- down projection + residual + next norm
+    g = GemmArgs{};
+    g.x = c->act; g.w = w.wd; g.R = R; g.N = d; g.K = c->ffn_pad; g.x_pitch = c->ffn_pad; g.w_pitch = c->ffn_pad;
+    g.splits = c->split_down; g.epi = EPI_PARTIAL; g.out = c->partial;
+    rc = run_gemm(c, g, SSD_PROF_GEMM);
+    if (rc) return rc;
+    {
+      const float* gain = (l + 1 < nl) ? c->L[l + 1].g_attn : c->g_final;
+      Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * (4.0 * g.splits + 10.0));
+      launch_residual_rmsnorm(c->st, c->partial, g.splits, (size_t)R * d, gain, c->cfg.rms_eps, c->h, c->xn, R, d);
+    }
+  }
+  if (kind == FWD_VERIFY) {
+    GemmArgs g{};
+    g.x = c->xn; g.w = c->lm_head; g.R = R; g.N = c->V; g.K = d; g.x_pitch = d; g.w_pitch = d; g.splits = 1;
+    g.mask_id = c->cfg.mask_id;
+    if (want_logits || c->gemm_impl != 1) {
+      const size_t need = (size_t)R * c->V;
+      if (need > c->logits_elems) {
+        float* p = nullptr;
+        if (cudaMalloc(&p, need * sizeof(float)) != cudaSuccess)
+          return fail(c, SSD_ERR_OOM, "cannot allocate %zu bytes for debug logits", need * sizeof(float));
+        c->allocs.push_back(p);
+        c->logits = p;
+        c->logits_elems = need;
+      }
+      g.epi = EPI_PARTIAL; g.out = c->logits;
+      int rc = run_gemm(c, g, SSD_PROF_LMHEAD);
+      if (rc) return rc;
+      Scope sc(c, SSD_PROF_LMHEAD, (double)R * c->V * 4.0);
+      launch_lm_stats_from_logits(c->st, c->logits, R, c->V, c->cfg.mask_id, row_wanted, c->tok, c->conf);
+    } else {
+      g.epi = EPI_LMHEAD; g.tile_max = c->tile_max; g.tile_sum = c->tile_sum; g.tile_arg = c->tile_arg;
+      int rc = run_gemm(c, g, SSD_PROF_LMHEAD);
+      if (rc) return rc;
+      Scope sc(c, SSD_PROF_LMHEAD, (double)gemm_tiles(c->V) * R * 12.0);
+      launch_lm_merge(c->st, c->tile_max, c->tile_sum, c->tile_arg, gemm_tiles(c->V), R, row_wanted, c->tok, c->conf);
+    }
+  }
+  CUDA_TRY(c, cudaGetLastError());
+  return SSD_OK;
+}
+
+int check_flags_after_sync(ssd_ctx* c) {
+  if (c->h_pinned[0] != 0) return fail(c, SSD_ERR_TIMEOUT, "a bounded device-side wait expired (role %d)", c->h_pinned[0]);
+  if (c->h_pinned[1] != 0) return fail(c, SSD_ERR_NONFINITE, "non-finite confidence in the verification forward");
+  return SSD_OK;
+}
+
+int sync_and_check(ssd_ctx* c) {
+  CUDA_TRY(c, cudaMemcpyAsync(c->h_pinned, c->flags, 2 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  return check_flags_after_sync(c);
+}
+
+int parse_layer_name(const char* name, int* layer, const char** rest) {
+  if (strncmp(name, "layers.", 7) != 0) return 0;
+  char* end = nullptr;
+  long l = strtol(name + 7, &end, 10);
+  if (end == name + 7 || *end != '.') return 0;
+  *layer = (int)l;
+  *rest = end + 1;
+  return 1;
+}
+
+}  // namespace
+
+// =============================================================================================
+extern "C" {
+
+const char* ssd_last_error(const ssd_ctx* ctx) { return ctx ? ctx->err : g_create_error; }
+
+int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
+  if (!cfg || !out) return fail(nullptr, SSD_ERR_INVALID_ARG, "null argument");
+  *out = nullptr;
+  const ssd_config& k = *cfg;
+  if (k.n_layers < 1 || k.d_model < 8 || k.n_heads < 1 || k.n_kv_heads < 1 || k.d_ffn < 8 || k.vocab < 2 ||
+      k.max_batch < 1 || k.max_seq < 1 || k.block_len < 1 || k.max_drafts < 0)
+    return fail(nullptr, SSD_ERR_INVALID_ARG, "non-positive size in config");
+  if (k.head_dim != 64 && k.head_dim != 128) return fail(nullptr, SSD_ERR_SHAPE, "head_dim must be 64 or 128");
+  if (k.d_model % 8 || k.d_ffn % 8 || k.n_heads % k.n_kv_heads || k.block_len > 256)
+    return fail(nullptr, SSD_ERR_SHAPE, "d_model, d_ffn must be multiples of 8, heads a multiple of kv heads, block_len <= 256");
+  if (k.mask_id < 0 || k.mask_id >= k.vocab) return fail(nullptr, SSD_ERR_INVALID_ARG, "mask_id outside the vocabulary");
+  if (k.block_len > k.max_seq) return fail(nullptr, SSD_ERR_INVALID_ARG, "block_len exceeds max_seq");
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1)
+    return fail(nullptr, SSD_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  if (gemm_tc_init() != 0) return fail(nullptr, SSD_ERR_CUDA, "cannot resolve the tensor-map encoder of the CUDA driver");
+
+  ssd_ctx* c = new (std::nothrow) ssd_ctx();
+  if (!c) return fail(nullptr, SSD_ERR_OOM, "host allocation failed");
+  c->cfg = k;
+  c->st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  c->H = k.n_heads; c->Hkv = k.n_kv_heads; c->hd = k.head_dim; c->d = k.d_model; c->ffn = k.d_ffn;
+  c->ffn_pad = (k.d_ffn + 63) / 64 * 64; c->V = k.vocab;
+  c->qdim = c->H * c->hd; c->kvdim = c->Hkv * c->hd; c->nqkv = c->qdim + 2 * c->kvdim;
+  c->L.resize(k.n_layers);
+  c->n_max = (k.max_drafts < k.block_len - 1 ? k.max_drafts : k.block_len - 1) + 1;
+  c->R_dec = k.max_batch * c->n_max * k.block_len;
+  c->R_cap = c->R_dec > k.max_seq ? c->R_dec : k.max_seq;
+  c->split_qkv = auto_split(gemm_tiles(c->nqkv));
+  c->split_o = auto_split(gemm_tiles(c->d));
+  c->split_down = auto_split(gemm_tiles(c->d));
+  c->h_remaining.assign(k.max_batch, 0);
+  c->h_has_drafts.assign(k.max_batch, 0);
+
+  int rc = SSD_OK;
+  auto build = [&]() -> int {
+    const int d = c->d;
+    for (LayerW& w : c->L) {
+      ALLOC(c, w.wqkv, (size_t)c->nqkv * d);
+      ALLOC(c, w.wo, (size_t)d * c->qdim);
+      ALLOC(c, w.wgu, (size_t)2 * c->ffn_pad * d);
+      ALLOC(c, w.wd, (size_t)d * c->ffn_pad);
+      ALLOC(c, w.g_attn, d);
+      ALLOC(c, w.g_ffn, d);
+    }
+    ALLOC(c, c->embed, (size_t)c->V * d);
+    ALLOC(c, c->lm_head, (size_t)c->V * d);
+    ALLOC(c, c->g_final, d);
+    c->cache_seq_stride = (size_t)k.max_seq * c->kvdim;
+    c->cache_layer_stride = c->cache_seq_stride * k.max_batch;
+    ALLOC(c, c->cacheK, c->cache_layer_stride * k.n_layers);
+    ALLOC(c, c->cacheV, c->cache_layer_stride * k.n_layers);
+    // rotary table in double precision on the host
+    {
+      const int half = c->hd / 2;
+      std::vector<float2> t((size_t)k.max_seq * half);
+      for (int p = 0; p < k.max_seq; ++p)
+        for (int i = 0; i < half; ++i) {
+          const double inv = pow((double)k.rope_theta, -2.0 * i / (double)c->hd);
+          const double a = (double)p * inv;
+          t[(size_t)p * half + i] = make_float2((float)cos(a), (float)sin(a));
+        }
+      ALLOC(c, c->rope, t.size());
+      CUDA_TRY(c, cudaMemcpyAsync(c->rope, t.data(), t.size() * sizeof(float2), cudaMemcpyHostToDevice, c->st));
+      CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    }
+    const size_t R = (size_t)c->R_cap;
+    ALLOC(c, c->h, R * d);
+    ALLOC(c, c->xn, R * d);
+    size_t widest = (size_t)c->nqkv > (size_t)d ? (size_t)c->nqkv : (size_t)d;
+    c->partial_elems = 8 * R * widest;
+    if (R * 2 * c->ffn_pad > c->partial_elems) c->partial_elems = R * 2 * c->ffn_pad;
+    ALLOC(c, c->partial, c->partial_elems);
+    ALLOC(c, c->q, R * c->qdim);
+    ALLOC(c, c->lk, R * c->kvdim);
+    ALLOC(c, c->lv, R * c->kvdim);
+    ALLOC(c, c->att, R * c->qdim);
+    ALLOC(c, c->act, R * c->ffn_pad);
+    const size_t dec_parts = (size_t)(k.max_seq + 255) / 256 + 1;
+    c->part_rows_parts = (size_t)c->R_dec * dec_parts;
+    if ((size_t)k.max_seq > c->part_rows_parts) c->part_rows_parts = k.max_seq;
+    ALLOC(c, c->part_o, c->part_rows_parts * c->qdim);
+    ALLOC(c, c->part_ml, c->part_rows_parts * c->H);
+    const size_t tiles = gemm_tiles(c->V);
+    ALLOC(c, c->tile_max, tiles * c->R_dec);
+    ALLOC(c, c->tile_sum, tiles * c->R_dec);
+    ALLOC(c, c->tile_arg, tiles * c->R_dec);
+    ALLOC(c, c->tok, R);
+    ALLOC(c, c->conf, R);
+    ALLOC(c, c->node_ids, R);
+    ALLOC(c, c->node_masked, R);
+    ALLOC(c, c->flags, 4);
+    const size_t sb = (size_t)k.max_batch * k.block_len;
+    c->bs.stride = k.block_len;
+    ALLOC(c, c->bs.ids, sb); ALLOC(c, c->bs.masked, sb); ALLOC(c, c->bs.draft_tok, sb); ALLOC(c, c->bs.draft_conf, sb);
+    ALLOC(c, c->bs.cand_pos, sb); ALLOC(c, c->bs.cand_tok, sb); ALLOC(c, c->bs.accept_log, sb);
+    ALLOC(c, c->bs.has_drafts, k.max_batch); ALLOC(c, c->bs.remaining, k.max_batch); ALLOC(c, c->bs.n_cand, k.max_batch);
+    ALLOC(c, c->bs.n_forwards, k.max_batch); ALLOC(c, c->bs.last_accept, k.max_batch); ALLOC(c, c->bs.seq_map, k.max_batch);
+    CUDA_TRY(c, cudaMallocHost(&c->h_pinned, (2 + 3 * (size_t)k.max_batch) * sizeof(int)));
+    CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    return SSD_OK;
+  };
+  rc = build();
+  if (rc != SSD_OK) {
+    snprintf(g_create_error, sizeof(g_create_error), "%s", c->err);
+    ssd_destroy(c);
+    return rc;
+  }
+  *out = c;
+  return SSD_OK;
+}
+
+void ssd_destroy(ssd_ctx* c) {
+  if (!c) return;
+  cudaStreamSynchronize(c->st);
+  for (ProfRec& r : c->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+  for (void* p : c->allocs) cudaFree(p);
+  if (c->h_pinned) cudaFreeHost(c->h_pinned);
+  delete c;
+}
+
+int ssd_load_weights(ssd_ctx* c, const char* name, const void* dev_ptr, int32_t dtype, const int64_t* shape, int32_t ndim) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!name || !dev_ptr || !shape) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  if (dtype != SSD_DTYPE_BF16 && dtype != SSD_DTYPE_F32) return fail(c, SSD_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+  const int f32 = dtype == SSD_DTYPE_F32;
+  const int d = c->d;
+  auto want2 = [&](int64_t r, int64_t k) { return ndim == 2 && shape[0] == r && shape[1] == k; };
+  auto want1 = [&](int64_t n) { return ndim == 1 && shape[0] == n; };
+  int layer = -1;
+  const char* rest = nullptr;
+  bool ok_shape = true;
+  if (!strcmp(name, "embed")) {
+    if ((ok_shape = want2(c->V, d))) { launch_convert_rows(c->st, dev_ptr, f32, c->embed, c->V, d, d, c->V, 0, 0); c->loaded_globals |= 1u; }
+  } else if (!strcmp(name, "lm_head")) {
+    if ((ok_shape = want2(c->V, d))) { launch_convert_rows(c->st, dev_ptr, f32, c->lm_head, c->V, d, d, c->V, 0, 0); c->loaded_globals |= 2u; }
+  } else if (!strcmp(name, "norm_final")) {
+    if ((ok_shape = want1(d))) { launch_copy_f32(c->st, dev_ptr, f32, c->g_final, d); c->loaded_globals |= 4u; }
+  } else if (parse_layer_name(name, &layer, &rest)) {
+    if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, SSD_ERR_INVALID_ARG, "layer %d out of range", layer);
+    LayerW& w = c->L[layer];
+    if (!strcmp(rest, "wq")) {
+      if ((ok_shape = want2(c->qdim, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wqkv, c->qdim, d, d, c->qdim, 0, 0); w.loaded |= 1u; }
+    } else if (!strcmp(rest, "wk")) {
+      if ((ok_shape = want2(c->kvdim, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wqkv, c->kvdim, d, d, c->kvdim, 0, c->qdim); w.loaded |= 2u; }
+    } else if (!strcmp(rest, "wv")) {
+      if ((ok_shape = want2(c->kvdim, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wqkv, c->kvdim, d, d, c->kvdim, 0, c->qdim + c->kvdim); w.loaded |= 4u; }
+    } else if (!strcmp(rest, "wo")) {
+      if ((ok_shape = want2(d, c->qdim))) { launch_convert_rows(c->st, dev_ptr, f32, w.wo, d, c->qdim, c->qdim, d, 0, 0); w.loaded |= 8u; }
+    } else if (!strcmp(rest, "w_gate")) {
+      // 64 gate features then the 64 matching up features per 128-row tile
+      if ((ok_shape = want2(c->ffn, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wgu, c->ffn, d, d, 64, 128, 0); w.loaded |= 16u; }
+    } else if (!strcmp(rest, "w_up")) {
+      if ((ok_shape = want2(c->ffn, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wgu, c->ffn, d, d, 64, 128, 64); w.loaded |= 32u; }
+    } else if (!strcmp(rest, "w_down")) {
+      if ((ok_shape = want2(d, c->ffn))) { launch_convert_rows(c->st, dev_ptr, f32, w.wd, d, c->ffn, c->ffn_pad, d, 0, 0); w.loaded |= 64u; }
+    } else if (!strcmp(rest, "norm_attn")) {
+      if ((ok_shape = want1(d))) { launch_copy_f32(c->st, dev_ptr, f32, w.g_attn, d); w.loaded |= 128u; }
+    } else if (!strcmp(rest, "norm_ffn")) {
+      if ((ok_shape = want1(d))) { launch_copy_f32(c->st, dev_ptr, f32, w.g_ffn, d); w.loaded |= 256u; }
+    } else {
+      return fail(c, SSD_ERR_INVALID_ARG, "unknown tensor '%s'", name);
+    }
+  } else {
+    return fail(c, SSD_ERR_INVALID_ARG, "unknown tensor '%s'", name);
+  }
+  if (!ok_shape) return fail(c, SSD_ERR_SHAPE, "tensor '%s' has the wrong shape", name);
+  c->launches += 1;
+  CUDA_TRY(c, cudaGetLastError());
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  return SSD_OK;
+}
+
+int ssd_prefill_dev(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t* prompt_ids_dev) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!prompt_ids_dev) return fail(c, SSD_ERR_INVALID_ARG, "null prompt");
+  if (batch < 1 || batch > c->cfg.max_batch) return fail(c, SSD_ERR_OVERFLOW, "batch %d outside [1, %d]", batch, c->cfg.max_batch);
+  if (prompt_len < 1 || prompt_len > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "prompt_len %d outside [1, %d]", prompt_len, c->cfg.max_seq);
+  if (!all_loaded(c)) return fail(c, SSD_ERR_STATE, "not every weight tensor has been loaded");
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  for (int b = 0; b < batch; ++b) {
+    RowMap map{prompt_len, prompt_len, 0, b, nullptr};
+    const int rc = forward(c, FWD_FILL, prompt_ids_dev + (size_t)b * prompt_len, prompt_len, map, 1, false, nullptr);
+    if (rc) return rc;
+  }
+  const int rc = sync_and_check(c);
+  if (rc) return rc;
+  c->batch = batch;
+  c->prompt_len = prompt_len;
+  c->cache_len = prompt_len;
+  c->in_block = false;
+  return SSD_OK;
+}
+
+int ssd_prefill(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t* prompt_ids) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!prompt_ids) return fail(c, SSD_ERR_INVALID_ARG, "null prompt");
+  if (batch < 1 || batch > c->cfg.max_batch) return fail(c, SSD_ERR_OVERFLOW, "batch %d outside [1, %d]", batch, c->cfg.max_batch);
+  if (prompt_len < 1 || prompt_len > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "prompt_len %d outside [1, %d]", prompt_len, c->cfg.max_seq);
+  for (size_t i = 0; i < (size_t)batch * prompt_len; ++i)
+    if (prompt_ids[i] < 0 || prompt_ids[i] >= c->V) return fail(c, SSD_ERR_INVALID_ARG, "prompt id %d outside the vocabulary", prompt_ids[i]);
+  int* dev_ids = nullptr;
+  CUDA_TRY(c, cudaMalloc(&dev_ids, (size_t)batch * prompt_len * sizeof(int)));
+  cudaError_t e = cudaMemcpyAsync(dev_ids, prompt_ids, (size_t)batch * prompt_len * sizeof(int), cudaMemcpyHostToDevice, c->st);
+  int rc = (e == cudaSuccess) ? ssd_prefill_dev(c, batch, prompt_len, dev_ids) : fail(c, SSD_ERR_CUDA, "H2D copy failed: %s", cudaGetErrorString(e));
+  cudaStreamSynchronize(c->st);
+  cudaFree(dev_ids);
+  return rc;
+}
+
+int ssd_cache_length(const ssd_ctx* c) { return c ? (c->cache_len < 0 ? SSD_ERR_STATE : c->cache_len) : SSD_ERR_INVALID_ARG; }
+
+int ssd_block_begin(ssd_ctx* c, int32_t T) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
+  if (T < 1 || T > c->cfg.block_len) return fail(c, SSD_ERR_INVALID_ARG, "block_tokens %d outside [1, %d]", T, c->cfg.block_len);
+  if (c->cache_len + T > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "cache %d + block %d exceeds max_seq %d", c->cache_len, T, c->cfg.max_seq);
+  block_init_kernel<<<c->cfg.max_batch, 128, 0, c->st>>>(c->bs, c->batch, c->cfg.max_batch, T, c->cfg.mask_id);
+  c->launches += 1;
+  CUDA_TRY(c, cudaGetLastError());
+  for (int b = 0; b < c->cfg.max_batch; ++b) {
+    c->h_remaining[b] = b < c->batch ? T : 0;
+    c->h_has_drafts[b] = 0;
+  }
+  c->block_tokens = T;
+  c->in_block = true;
+  return SSD_OK;
+}
+
+int ssd_set_block_state(ssd_ctx* c, const int32_t* ids, const uint8_t* masked, const int32_t* draft_tok, const float* draft_conf) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
+  if (!ids || !masked || ((draft_tok == nullptr) != (draft_conf == nullptr))) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  const int T = c->block_tokens, st = c->bs.stride;
+  for (int b = 0; b < c->batch; ++b) {
+    int r = 0;
+    for (int t = 0; t < T; ++t) {
+      r += masked[b * T + t] ? 1 : 0;
+      if (!masked[b * T + t] && (ids[b * T + t] < 0 || ids[b * T + t] >= c->V)) return fail(c, SSD_ERR_INVALID_ARG, "token id outside the vocabulary");
+      if (draft_tok && masked[b * T + t] && (draft_tok[b * T + t] < 0 || draft_tok[b * T + t] >= c->V)) return fail(c, SSD_ERR_INVALID_ARG, "draft id outside the vocabulary");
+    }
+    c->h_remaining[b] = r;
+    c->h_has_drafts[b] = draft_tok ? 1 : 0;
+  }
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->bs.ids, st * sizeof(int), ids, T * sizeof(int), T * sizeof(int), c->batch, cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->bs.masked, st, masked, T, T, c->batch, cudaMemcpyHostToDevice, c->st));
+  if (draft_tok) {
+    CUDA_TRY(c, cudaMemcpy2DAsync(c->bs.draft_tok, st * sizeof(int), draft_tok, T * sizeof(int), T * sizeof(int), c->batch, cudaMemcpyHostToDevice, c->st));
+    CUDA_TRY(c, cudaMemcpy2DAsync(c->bs.draft_conf, st * sizeof(float), draft_conf, T * sizeof(float), T * sizeof(float), c->batch, cudaMemcpyHostToDevice, c->st));
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(c->bs.remaining, c->h_remaining.data(), c->batch * sizeof(int), cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(c->bs.has_drafts, c->h_has_drafts.data(), c->batch * sizeof(int), cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  return SSD_OK;
+}
+
+int ssd_get_block_state(ssd_ctx* c, int32_t* ids, uint8_t* masked, int32_t* draft_tok, float* draft_conf) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
+  const int T = c->block_tokens, st = c->bs.stride;
+  if (ids) CUDA_TRY(c, cudaMemcpy2DAsync(ids, T * sizeof(int), c->bs.ids, st * sizeof(int), T * sizeof(int), c->batch, cudaMemcpyDeviceToHost, c->st));
+  if (masked) CUDA_TRY(c, cudaMemcpy2DAsync(masked, T, c->bs.masked, st, T, c->batch, cudaMemcpyDeviceToHost, c->st));
+  if (draft_tok) CUDA_TRY(c, cudaMemcpy2DAsync(draft_tok, T * sizeof(int), c->bs.draft_tok, st * sizeof(int), T * sizeof(int), c->batch, cudaMemcpyDeviceToHost, c->st));
+  if (draft_conf) CUDA_TRY(c, cudaMemcpy2DAsync(draft_conf, T * sizeof(float), c->bs.draft_conf, st * sizeof(float), T * sizeof(float), c->batch, cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  return SSD_OK;
+}
+
+int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n_nodes) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
+  int md = max_drafts < 0 ? c->cfg.max_drafts : max_drafts;
+  if (md > c->cfg.max_drafts) md = c->cfg.max_drafts;
+  const int T = c->block_tokens, B = c->batch;
+  int active = 0, n_cap = 1;
+  for (int b = 0; b < B; ++b) {
+    if (c->h_remaining[b] <= 0) continue;
+    ++active;
+    const int N = c->h_has_drafts[b] ? (md < c->h_remaining[b] - 1 ? md : c->h_remaining[b] - 1) : 0;
+    if (N + 1 > n_cap) n_cap = N + 1;
+  }
+  if (accepted) memset(accepted, 0, B * sizeof(int));
+  if (n_nodes) memset(n_nodes, 0, B * sizeof(int));
+  if (active == 0) return SSD_OK;
+  const int R = active * n_cap * T;
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  {
+    Scope sc(c, SSD_PROF_TREE, (double)R * 5);
+    launch_tree_build(c->st, c->bs, B, T, md, n_cap, c->cfg.mask_id, c->node_ids, c->node_masked);
+  }
+  RowMap map{n_cap * T, T, c->cache_len, 0, c->bs.seq_map};
+  int rc = forward(c, FWD_VERIFY, c->node_ids, R, map, active, false, c->node_masked);
+  if (rc) return rc;
+  {
+    Scope sc(c, SSD_PROF_TREE, (double)R * 9);
+    launch_accept(c->st, c->bs, active, T, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1);
+  }
+  int* hp = c->h_pinned;
+  const int mb = c->cfg.max_batch;
+  CUDA_TRY(c, cudaMemcpyAsync(hp, c->flags, 2 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(hp + 2, c->bs.remaining, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + mb, c->bs.last_accept, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 2 * mb, c->bs.n_cand, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  rc = check_flags_after_sync(c);
+  if (rc) return rc;
+  for (int b = 0; b < B; ++b) {
+    const bool was_active = c->h_remaining[b] > 0;
+    c->h_remaining[b] = hp[2 + b];
+    if (was_active) c->h_has_drafts[b] = 1;
+    if (accepted) accepted[b] = hp[2 + mb + b];
+    if (n_nodes) n_nodes[b] = was_active ? hp[2 + 2 * mb + b] + 1 : 0;
+  }
+  return SSD_OK;
+}
+
+int ssd_block_commit(ssd_ctx* c) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
+  for (int b = 0; b < c->batch; ++b)
+    if (c->h_remaining[b] > 0) return fail(c, SSD_ERR_STATE, "sequence %d still has %d masked positions", b, c->h_remaining[b]);
+  const int T = c->block_tokens, B = c->batch;
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->node_ids, T * sizeof(int), c->bs.ids, c->bs.stride * sizeof(int), T * sizeof(int), B, cudaMemcpyDeviceToDevice, c->st));
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  RowMap map{T, T, c->cache_len, 0, nullptr};
+  int rc = forward(c, FWD_FILL, c->node_ids, B * T, map, B, false, nullptr);
+  if (rc) return rc;
+  rc = sync_and_check(c);
+  if (rc) return rc;
+  c->cache_len += T;
+  c->in_block = false;
+  return SSD_OK;
+}
+
+int ssd_decode_block(ssd_ctx* c, int32_t mode, int32_t T, int32_t* out_tokens, int32_t* out_accept_counts, int32_t* out_n_forwards) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (mode != SSD_MODE_STEPWISE && mode != SSD_MODE_SSD) return fail(c, SSD_ERR_INVALID_ARG, "unknown mode %d", mode);
+  int rc = ssd_block_begin(c, T);
+  if (rc) return rc;
+  const int md = mode == SSD_MODE_STEPWISE ? 0 : -1;
+  for (int guard = 0; guard <= T; ++guard) {
+    bool any = false;
+    for (int b = 0; b < c->batch; ++b) any = any || c->h_remaining[b] > 0;
+    if (!any) break;
+    rc = ssd_block_step(c, md, nullptr, nullptr);
+    if (rc) return rc;
+  }
+  const int st = c->bs.stride, B = c->batch;
+  if (out_tokens) CUDA_TRY(c, cudaMemcpy2DAsync(out_tokens, T * sizeof(int), c->bs.ids, st * sizeof(int), T * sizeof(int), B, cudaMemcpyDeviceToHost, c->st));
+  if (out_accept_counts) CUDA_TRY(c, cudaMemcpy2DAsync(out_accept_counts, T * sizeof(int), c->bs.accept_log, st * sizeof(int), T * sizeof(int), B, cudaMemcpyDeviceToHost, c->st));
+  if (out_n_forwards) CUDA_TRY(c, cudaMemcpyAsync(out_n_forwards, c->bs.n_forwards, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  return ssd_block_commit(c);
+}
+
+int ssd_verify_forward(ssd_ctx* c, int32_t batch, int32_t n_nodes, int32_t T, const int32_t* node_ids, const uint8_t* node_masked,
+                       int32_t* out_tok, float* out_conf, float* out_logits) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
+  if (!node_ids || !node_masked) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  if (batch < 1 || batch > c->batch) return fail(c, SSD_ERR_INVALID_ARG, "batch %d outside [1, %d]", batch, c->batch);
+  if (T < 1 || T > c->cfg.block_len || n_nodes < 1) return fail(c, SSD_ERR_INVALID_ARG, "bad node shape");
+  const size_t R = (size_t)batch * n_nodes * T;
+  if (R > (size_t)c->R_dec) return fail(c, SSD_ERR_OVERFLOW, "%zu rows exceed the capacity %d set by max_batch/max_drafts/block_len", R, c->R_dec);
+  if (c->cache_len + T > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "cache %d + block %d exceeds max_seq", c->cache_len, T);
+  for (size_t i = 0; i < R; ++i)
+    if (node_ids[i] < 0 || node_ids[i] >= c->V) return fail(c, SSD_ERR_INVALID_ARG, "node id outside the vocabulary");
+  CUDA_TRY(c, cudaMemcpyAsync(c->node_ids, node_ids, R * sizeof(int), cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(c->node_masked, node_masked, R, cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  RowMap map{n_nodes * T, T, c->cache_len, 0, nullptr};
+  int rc = forward(c, FWD_VERIFY, c->node_ids, (int)R, map, batch, out_logits != nullptr, c->node_masked);
+  if (rc) return rc;
+  if (out_tok) CUDA_TRY(c, cudaMemcpyAsync(out_tok, c->tok, R * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  if (out_conf) CUDA_TRY(c, cudaMemcpyAsync(out_conf, c->conf, R * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  if (out_logits) CUDA_TRY(c, cudaMemcpyAsync(out_logits, c->logits, R * (size_t)c->V * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  return sync_and_check(c);
+}
+
+int ssd_read_cache(ssd_ctx* c, int32_t layer, int32_t seq, int32_t length, float* out_k, float* out_v) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= c->cfg.n_layers || seq < 0 || seq >= c->cfg.max_batch || length < 0 || length > c->cfg.max_seq)
+    return fail(c, SSD_ERR_INVALID_ARG, "index out of range");
+  const size_t n = (size_t)length * c->kvdim;
+  std::vector<bf16> tmp(n);
+  for (int which = 0; which < 2; ++which) {
+    float* dst = which ? out_v : out_k;
+    if (!dst) continue;
+    const bf16* src = (which ? c->cacheV : c->cacheK) + (size_t)layer * c->cache_layer_stride + (size_t)seq * c->cache_seq_stride;
+    CUDA_TRY(c, cudaMemcpyAsync(tmp.data(), src, n * sizeof(bf16), cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(c, cudaStreamSynchronize(c->st));
+    for (size_t i = 0; i < n; ++i) dst[i] = __bfloat162float(tmp[i]);
+  }
+  return SSD_OK;
+}
+
+int ssd_gemm_bf16(ssd_ctx* c, const void* x_dev, const void* w_dev, float* out_dev, int32_t rows, int32_t n, int32_t k, int32_t split_k) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!x_dev || !w_dev || !out_dev) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  if (rows < 1 || n < 1 || k < 8 || (k % 8) || split_k < 1 || split_k > 8) return fail(c, SSD_ERR_SHAPE, "bad GEMM shape");
+  if ((size_t)split_k * rows * n > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "GEMM exceeds the workspace");
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  GemmArgs g{};
+  g.x = (const bf16*)x_dev; g.w = (const bf16*)w_dev; g.R = rows; g.N = n; g.K = k; g.x_pitch = k; g.w_pitch = k;
+  g.splits = split_k; g.epi = EPI_PARTIAL; g.out = c->partial;
+  int rc = run_gemm(c, g, SSD_PROF_GEMM);
+  if (rc) return rc;
+  const size_t total = (size_t)rows * n;
+  sum_splits_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->st>>>(c->partial, split_k, total, out_dev, total);
+  c->launches += 1;
+  CUDA_TRY(c, cudaGetLastError());
+  return sync_and_check(c);
+}
+
+int64_t ssd_launch_count(const ssd_ctx* c) { return c ? c->launches : -1; }
+
+int ssd_profile_enable(ssd_ctx* c, int32_t on) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  c->profiling = on != 0;
+  return SSD_OK;
+}
+
+int ssd_profile_read(ssd_ctx* c, int64_t* launches, double* ms, double* bytes) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  for (int f = 0; f < SSD_PROF_FAMILIES; ++f) {
+    if (launches) launches[f] = 0;
+    if (ms) ms[f] = 0;
+    if (bytes) bytes[f] = 0;
+  }
+  for (ProfRec& r : c->prof) {
+    float t = 0.f;
+    cudaEventElapsedTime(&t, r.e0, r.e1);
+    if (launches) launches[r.fam] += 1;
+    if (ms) ms[r.fam] += t;
+    if (bytes) bytes[r.fam] += r.bytes;
+    cudaEventDestroy(r.e0);
+    cudaEventDestroy(r.e1);
+  }
+  c->prof.clear();
+  return SSD_OK;
+}
+
+int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!key) return fail(c, SSD_ERR_INVALID_ARG, "null key");
+  if (!strcmp(key, "split_k_qkv") || !strcmp(key, "split_k_o") || !strcmp(key, "split_k_down")) {
+    if (value < 1 || value > 8) return fail(c, SSD_ERR_INVALID_ARG, "split-K must be in [1, 8]");
+    if (!strcmp(key, "split_k_qkv")) c->split_qkv = value;
+    else if (!strcmp(key, "split_k_o")) c->split_o = value;
+    else c->split_down = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "kv_split")) {
+    if (value != 0 && (value < 64 || value % 64)) return fail(c, SSD_ERR_INVALID_ARG, "kv_split must be 0 (automatic) or a multiple of 64");
+    c->kv_split_opt = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "gemm_impl")) {
+    if (value != 0 && value != 1) return fail(c, SSD_ERR_INVALID_ARG, "gemm_impl is 0 (CUDA cores, bring-up) or 1 (tcgen05)");
+    c->gemm_impl = value;
+    return SSD_OK;
+  }
+  return fail(c, SSD_ERR_INVALID_ARG, "unknown option '%s'", key);
+}
+
+}  // extern "C"

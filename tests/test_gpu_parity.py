@@ -1,0 +1,375 @@
+"""CUDA path vs the CPU oracle, through the C ABI (run with -m gpu on a B200).
+
+Tolerances (bf16 operands, fp32 accumulation; stated by the workload's north star):
+  * logits within 2e-2 absolute of the fp64 oracle, confidences within 2e-2 relative;
+  * against the oracle run with bf16 operand rounding (same arithmetic type as the kernels) the
+    logits agree to 6e-3;
+  * tokens / accept lengths bit-exact wherever the oracle's decision gap exceeds 1e-3;
+  * GPU SSD == GPU stepwise bit-exact, no exemption.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ssd_oracle as so
+from paper_2510_04147_b200 import workloads as wl
+from tests.helpers import make_oracle, oracle_config, oracle_weights
+
+pytestmark = pytest.mark.gpu
+
+GAP = 1e-3
+PEAKED = wl.TINY.replace(name="tiny_peaked", lm_head_scale=8.0)
+
+
+def _binding():
+    from paper_2510_04147_b200 import binding
+    return binding
+
+
+def _make_ssd(w, max_drafts, gemm_impl=1, max_batch=None, max_seq=None):
+    b = _binding()
+    ssd = b.Ssd(b.config_from_workload(w, max_drafts=max_drafts, max_batch=max_batch, max_seq=max_seq))
+    ssd.set_option("gemm_impl", gemm_impl)
+    ssd.load_workload_weights(w)
+    return ssd
+
+
+@pytest.fixture(scope="module")
+def tiny_ssd():
+    ssd = _make_ssd(wl.TINY, max_drafts=wl.TINY.block_len, max_batch=3)
+    yield ssd
+    ssd.destroy()
+
+
+@pytest.fixture(scope="module")
+def peaked_ssd():
+    ssd = _make_ssd(PEAKED, max_drafts=PEAKED.block_len, max_batch=3)
+    yield ssd
+    ssd.destroy()
+
+
+@pytest.fixture(scope="module")
+def tiny_oracles():
+    """(fp64 oracle, bf16-operand oracle) on the bf16-rounded weights of config 1."""
+    return {w.name: (make_oracle(w, as_bf16=True), make_oracle(w, as_bf16=True, operand_rounding="bf16"))
+            for w in (wl.TINY, PEAKED)}
+
+
+# ------------------------------------------------------------------------------------------
+# the projection kernel alone
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", [0, 1], ids=["simt", "tc"])
+@pytest.mark.parametrize("rows,n,k,split", [(16, 128, 64, 1), (32, 256, 256, 1), (100, 688, 688, 1), (37, 1376, 256, 1),
+                                            (128, 4096, 4096, 4), (64, 512, 12288, 8), (300, 384, 512, 2),
+                                            (256, 256, 1024, 3), (1, 130, 72, 1)])
+def test_gemm_against_numpy(tiny_ssd, impl, rows, n, k, split):
+    tiny_ssd.set_option("gemm_impl", impl)
+    try:
+        x = wl.normal_tensor(5, 1, (rows, k), 1.0, device="cuda", dtype=torch.bfloat16)
+        w = wl.normal_tensor(5, 2, (n, k), 0.05, device="cuda", dtype=torch.bfloat16)
+        out = tiny_ssd.gemm_bf16(x, w, split).cpu().numpy()
+        ref = x.cpu().to(torch.float64).numpy() @ w.cpu().to(torch.float64).numpy().T
+        scale = np.sqrt(k) * 0.05
+        assert np.abs(out - ref).max() < 2e-5 * scale * np.sqrt(k) + 1e-6, np.abs(out - ref).max()
+    finally:
+        tiny_ssd.set_option("gemm_impl", 1)
+
+
+# ------------------------------------------------------------------------------------------
+# cache and forward
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("impl", [0, 1], ids=["simt", "tc"])
+def test_prefill_cache_matches_oracle(tiny_ssd, tiny_oracles, impl):
+    w = wl.TINY
+    _, ob = tiny_oracles[w.name]
+    prompts = wl.make_prompts(w, batch=2).numpy()
+    tiny_ssd.set_option("gemm_impl", impl)
+    try:
+        tiny_ssd.prefill(prompts)
+    finally:
+        tiny_ssd.set_option("gemm_impl", 1)
+    assert tiny_ssd.cache_length() == w.prompt_len
+    for b in range(2):
+        cache = ob.prefill(prompts[b])
+        for l in range(w.n_layers):
+            k, v = tiny_ssd.read_cache(l, b, w.prompt_len)
+            assert np.abs(k - cache.k[l]).max() < 2e-2 * max(1.0, np.abs(cache.k[l]).max())
+            assert np.abs(v - cache.v[l]).max() < 2e-2 * max(1.0, np.abs(cache.v[l]).max())
+            # most entries identical after bf16 rounding
+            assert (np.abs(k - cache.k[l]) < 1e-6).mean() > 0.9
+
+
+def _random_nodes(w, rng, n_nodes, T):
+    ids = rng.integers(0, w.vocab - 1, (1, n_nodes, T))
+    masked = rng.random((1, n_nodes, T)) < 0.6
+    masked[:, :, 0] = True
+    return np.where(masked, w.mask_id, ids), masked
+
+
+@pytest.mark.parametrize("impl", [0, 1], ids=["simt", "tc"])
+@pytest.mark.parametrize("which", ["tiny", "tiny_peaked"])
+def test_verify_forward_logits_and_stats(tiny_ssd, peaked_ssd, tiny_oracles, impl, which):
+    w = wl.TINY if which == "tiny" else PEAKED
+    ssd = tiny_ssd if which == "tiny" else peaked_ssd
+    o64, ob = tiny_oracles[w.name]
+    rng = np.random.default_rng(3)
+    prompt = wl.make_prompts(w).numpy()
+    T = w.block_len
+    ssd.set_option("gemm_impl", impl)
+    try:
+        ssd.prefill(prompt)
+        # one committed block so that the prefix is prompt + block
+        blk = rng.integers(0, w.vocab - 1, (1, T))
+        ssd.block_begin(T)
+        ssd.set_block_state(blk, np.zeros((1, T), np.uint8))
+        ssd.block_commit()
+        ids, masked = _random_nodes(w, rng, 5, T)
+        tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
+        tok2, conf2, _ = ssd.verify_forward(ids, masked, want_logits=False)      # fused LM head path
+    finally:
+        ssd.set_option("gemm_impl", 1)
+    for o, tol in ((ob, 6e-3), (o64, 2e-2)):
+        cache = o.prefill(prompt[0])
+        o.commit_block(blk[0], cache)
+        otok, oconf, ogap, ologits = o.verify(ids[0], masked[0], cache)
+        err = np.abs(logits[0] - ologits).max()
+        assert err < tol * w.lm_head_scale, (err, tol)
+        m = masked[0]
+        assert np.allclose(conf[0][m], oconf[m], rtol=2e-2, atol=2e-2 * 1e-3)
+        assert np.allclose(conf2[0][m], oconf[m], rtol=2e-2, atol=2e-2 * 1e-3)
+        sure = m & (ogap > GAP)
+        assert np.array_equal(tok[0][sure], otok[sure])
+        assert np.array_equal(tok2[0][sure], otok[sure])
+        if which == "tiny_peaked":
+            assert sure.sum() > 0.5 * m.sum()          # the peaked variant makes the token check bite
+    # rows that were not asked for
+    assert np.all(tok[0][~masked[0]] == -1) and np.all(conf[0][~masked[0]] == 0)
+    # the two LM-head paths agree (same logits, different reduction order)
+    assert np.array_equal(tok[0][masked[0]], tok2[0][masked[0]]) or impl == 0
+    assert np.allclose(conf[0], conf2[0], rtol=1e-4)
+    assert w.mask_id not in tok
+
+
+def test_row_invariance_of_the_forward(peaked_ssd):
+    """A node's outputs are bit-identical whether it runs alone or among other nodes."""
+    w = PEAKED
+    rng = np.random.default_rng(4)
+    prompt = wl.make_prompts(w).numpy()
+    peaked_ssd.prefill(prompt)
+    T = w.block_len
+    ids, masked = _random_nodes(w, rng, 7, T)
+    tok, conf, _ = peaked_ssd.verify_forward(ids, masked)
+    for i in (0, 3, 6):
+        t1, c1, _ = peaked_ssd.verify_forward(ids[:, i:i + 1], masked[:, i:i + 1])
+        assert np.array_equal(t1[0, 0], tok[0, i])
+        assert np.array_equal(c1[0, 0].view(np.uint32), conf[0, i].view(np.uint32))
+
+
+# ------------------------------------------------------------------------------------------
+# decode loops
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("which", ["tiny", "tiny_peaked"])
+@pytest.mark.parametrize("max_drafts", [0, 1, 3, 5, 16])
+def test_gpu_ssd_equals_gpu_stepwise(tiny_ssd, peaked_ssd, which, max_drafts):
+    w = wl.TINY if which == "tiny" else PEAKED
+    ssd = tiny_ssd if which == "tiny" else peaked_ssd
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    ssd.prefill(prompt)
+    want, acc0, nf0 = ssd.generate(b.MODE_STEPWISE, w.gen_len, w.block_len, 1)
+    ssd.prefill(prompt)
+    toks = []
+    for j in range(w.gen_len // w.block_len):
+        ssd.block_begin(w.block_len)
+        counts = []
+        while True:
+            acc, nn = ssd.block_step(max_drafts, 1)
+            if acc[0] == 0:
+                break
+            assert 1 <= acc[0] <= nn[0] <= max_drafts + 1
+            counts.append(int(acc[0]))
+        assert sum(counts) == w.block_len
+        ids, masked, _, _ = ssd.get_block_state(1, w.block_len)
+        assert masked.sum() == 0
+        toks.append(ids)
+        ssd.block_commit()
+        if max_drafts == 0:
+            assert counts == [1] * w.block_len
+    got = np.concatenate(toks, axis=1)
+    assert np.array_equal(got, want)
+    assert all(int(n[0]) == w.block_len for n in nf0) and all(np.all(a == 1) for a in acc0)
+    assert w.mask_id not in got
+    assert ssd.cache_length() == w.prompt_len + w.gen_len
+
+
+def test_decode_block_postconditions(peaked_ssd):
+    w = PEAKED
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    peaked_ssd.prefill(prompt)
+    tok, accs, nfs = peaked_ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1)
+    for acc, nf in zip(accs, nfs):
+        n = int(nf[0])
+        assert acc[0, :n].sum() == w.block_len and np.all(acc[0, :n] >= 1) and np.all(acc[0, n:] == 0)
+        assert acc[0, 0] == 1                      # first forward of a block has no drafts
+
+
+@pytest.mark.parametrize("which", ["tiny", "tiny_peaked"])
+def test_teacher_forced_ssd_steps_match_oracle(tiny_ssd, peaked_ssd, tiny_oracles, which):
+    """Every verification forward of the oracle's SSD run is replayed on the GPU from the oracle's
+    state and drafts; candidate count, accepted length and the new state must agree wherever the
+    oracle's decisions have a margin above the gap."""
+    w = wl.TINY if which == "tiny" else PEAKED
+    ssd = tiny_ssd if which == "tiny" else peaked_ssd
+    _, ob = tiny_oracles[w.name]
+    prompt = wl.make_prompts(w).numpy()
+    trace = []
+    tokens, _, _ = ob.generate(prompt[0], w.gen_len, w.block_len, mode="ssd", max_drafts=5, trace=trace)
+    ssd.prefill(prompt)
+    T = w.block_len
+    strict = 0
+    cur_block = 0
+    for rec in trace:
+        if rec.block != cur_block:                 # commit the oracle's finished block
+            ssd.block_begin(T)
+            ssd.set_block_state(tokens[cur_block * T:(cur_block + 1) * T][None], np.zeros((1, T), np.uint8))
+            ssd.block_commit()
+            cur_block = rec.block
+        ssd.block_begin(T)
+        if rec.draft_tok is None:
+            ssd.set_block_state(rec.ids_before[None], rec.masked_before[None].astype(np.uint8))
+        else:
+            ssd.set_block_state(rec.ids_before[None], rec.masked_before[None].astype(np.uint8),
+                                rec.draft_tok[None], rec.draft_conf[None])
+        acc, nn = ssd.block_step(5, 1)
+        assert nn[0] == len(rec.cand) + 1
+        ids, masked, dt, dc = ssd.get_block_state(1, T)
+        # margin of every decision that shaped this forward's outcome
+        margin = np.inf
+        if rec.draft_conf is not None:
+            c = np.sort(rec.draft_conf[rec.masked_before])[::-1]
+            if len(c) > 1:
+                margin = min(margin, np.min(c[:-1] - c[1:]) / max(c[0], 1e-30) * 1e3)   # fp32 order of the drafts
+        for i in range(rec.accepted):
+            q, _ = rec.pred[i]
+            cm = np.where(rec.node_masked[i], rec.conf[i], -1.0)
+            srt = np.sort(cm)[::-1]
+            margin = min(margin, rec.gap[i, q], srt[0] - srt[1] if len(srt) > 1 and srt[1] >= 0 else np.inf)
+        if margin > GAP:
+            strict += 1
+            assert acc[0] == rec.accepted
+            want_ids, want_masked = rec.ids_before.copy(), rec.masked_before.copy()
+            for (p, t) in rec.cand[:rec.accepted - 1]:
+                want_ids[p], want_masked[p] = t, False
+            q, t = rec.pred[rec.accepted - 1]
+            want_ids[q], want_masked[q] = t, False
+            assert np.array_equal(masked[0].astype(bool), want_masked)
+            assert np.array_equal(ids[0][~want_masked], want_ids[~want_masked])
+            a = rec.accepted - 1
+            still = want_masked
+            assert np.allclose(dc[0][still], rec.conf[a][still], rtol=2e-2, atol=2e-5)
+            sure = still & (rec.gap[a] > GAP)
+            assert np.array_equal(dt[0][sure], rec.tok[a][sure])
+        else:
+            assert 1 <= acc[0] <= nn[0]
+    if which == "tiny_peaked":
+        assert strict >= len(trace) // 3, (strict, len(trace))
+
+
+def test_batched_sequences_equal_single_runs(peaked_ssd):
+    """Each sequence of a batch has its own tree; batching changes nothing for any of them."""
+    w = PEAKED
+    b = _binding()
+    prompts = wl.make_prompts(w, batch=3).numpy()
+    peaked_ssd.prefill(prompts)
+    tok_b, acc_b, nf_b = peaked_ssd.generate(b.MODE_SSD, 32, w.block_len, 3)
+    for s in range(3):
+        peaked_ssd.prefill(prompts[s:s + 1])
+        tok_s, acc_s, nf_s = peaked_ssd.generate(b.MODE_SSD, 32, w.block_len, 1)
+        assert np.array_equal(tok_s[0], tok_b[s])
+        for j in range(len(acc_s)):
+            assert np.array_equal(acc_s[j][0], acc_b[j][s]) and nf_s[j][0] == nf_b[j][s]
+
+
+def test_ragged_last_block(tiny_ssd):
+    w = wl.TINY
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    tiny_ssd.prefill(prompt)
+    a, _, _ = tiny_ssd.generate(b.MODE_STEPWISE, 40, w.block_len, 1)
+    tiny_ssd.prefill(prompt)
+    c, accs, _ = tiny_ssd.generate(b.MODE_SSD, 40, w.block_len, 1)
+    assert a.shape == (1, 40) and np.array_equal(a, c)
+    assert [int(x.sum()) for x in accs] == [16, 16, 8]
+    assert tiny_ssd.cache_length() == w.prompt_len + 40
+
+
+def test_free_running_tokens_against_oracle(peaked_ssd, tiny_oracles):
+    """Free-running GPU decode vs the oracle's stepwise decode: equal up to the first decision whose
+    oracle margin is below the gap (after which the two runs see different contexts)."""
+    w = PEAKED
+    b = _binding()
+    _, ob = tiny_oracles[w.name]
+    prompt = wl.make_prompts(w).numpy()
+    trace = []
+    want, _, _ = ob.generate(prompt[0], w.gen_len, w.block_len, mode="stepwise", trace=trace)
+    peaked_ssd.prefill(prompt)
+    got, _, _ = peaked_ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1)
+    safe_blocks = 0
+    for j in range(w.gen_len // w.block_len):
+        recs = [r for r in trace if r.block == j]
+        ok = True
+        for r in recs:
+            q, _ = r.pred[0]
+            cm = np.sort(np.where(r.node_masked[0], r.conf[0], -1.0))[::-1]
+            second = cm[1] if len(cm) > 1 and cm[1] >= 0 else -np.inf
+            if min(r.gap[0, q], cm[0] - second) <= GAP:
+                ok = False
+        if not ok:
+            break
+        safe_blocks += 1
+        assert np.array_equal(got[0, j * w.block_len:(j + 1) * w.block_len], want[j * w.block_len:(j + 1) * w.block_len])
+    assert safe_blocks >= 1
+
+
+# ------------------------------------------------------------------------------------------
+# error paths (host-side checks; nothing here faults a GPU)
+# ------------------------------------------------------------------------------------------
+def test_error_codes(tiny_ssd):
+    b = _binding()
+    w = wl.TINY
+    fresh = b.Ssd(b.config_from_workload(w, max_drafts=2))
+    with pytest.raises(b.SsdError) as e:
+        fresh.prefill(wl.make_prompts(w).numpy())          # weights missing
+    assert e.value.code == -7
+    with pytest.raises(b.SsdError) as e:
+        fresh.block_begin(4)                               # no prefill
+    assert e.value.code == -7
+    with pytest.raises(b.SsdError) as e:
+        fresh.load_weights("layers.9.wq", torch.zeros(256, 256, device="cuda"))
+    assert e.value.code == -1
+    with pytest.raises(b.SsdError) as e:
+        fresh.load_weights("embed", torch.zeros(5, 256, device="cuda"))
+    assert e.value.code == -2
+    with pytest.raises(b.SsdError) as e:
+        fresh.set_option("nonsense", 1)
+    assert e.value.code == -1
+    fresh.destroy()
+    prompt = wl.make_prompts(w).numpy()
+    with pytest.raises(b.SsdError) as e:
+        tiny_ssd.prefill(np.full((1, 8), w.vocab, np.int32))    # id outside the vocabulary
+    assert e.value.code == -1
+    with pytest.raises(b.SsdError) as e:
+        tiny_ssd.prefill(np.zeros((9, 8), np.int32))            # batch > max_batch
+    assert e.value.code == -5
+    tiny_ssd.prefill(prompt)
+    for _ in range(w.gen_len // w.block_len):
+        tiny_ssd.decode_block(b.MODE_SSD, w.block_len, 1)
+    with pytest.raises(b.SsdError) as e:
+        tiny_ssd.decode_block(b.MODE_SSD, w.block_len, 1)       # cache full
+    assert e.value.code == -5
+    tiny_ssd.prefill(prompt)
+    tiny_ssd.block_begin(w.block_len)
+    with pytest.raises(b.SsdError) as e:
+        tiny_ssd.block_commit()                                  # block not finished
+    assert e.value.code == -7

@@ -70,7 +70,7 @@ def _context_free_rule(B):
 def test_upper_bound_of_step_reduction(N, pct):
     """With drafts that are always right every forward after the first accepts N+1 tokens, so
     the reduction of forward passes tends to N/(N+1): 75.0 / 80.0 / 83.3 % (Table 2)."""
-    B = 12000
+    B = 4000
     o = ScriptedOracle(64, _context_free_rule(B))
     ids, counts = o.decode_block_ssd(B, NoCache(), max_drafts=N)
     assert np.array_equal(ids, (np.arange(B) * 7 + 3) % 50)
