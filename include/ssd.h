@@ -135,6 +135,11 @@ int ssd_read_cache(ssd_ctx* ctx, int32_t layer, int32_t seq, int32_t length, flo
 /* Cached prefix length S (prompt + committed blocks), or a negative error. */
 int ssd_cache_length(const ssd_ctx* ctx);
 
+/* Forget the blocks committed after position `length` (prompt_len <= length <= current length):
+ * the next block is decoded at `length` again.  The prompt's K/V stay valid, so several
+ * generations from one prefill cost one prefill.  Abandons a block in progress. */
+int ssd_rewind(ssd_ctx* ctx, int32_t length);
+
 /* The skinny projection kernel alone: out[r][n] = sum_k x[r][k] * w[n][k] with bf16 operands and
  * fp32 accumulation, split over `split_k` K ranges that are summed in order.  DEVICE pointers:
  * x [rows, k] bf16, w [n, k] bf16, out [rows, n] fp32.  k a multiple of 8.  Test / tuning hook. */

@@ -26,7 +26,7 @@ PROF_FAMILIES = ("gemm", "lmhead", "attn", "elemwise", "tree")
 
 EXPORTS = ["ssd_create", "ssd_destroy", "ssd_last_error", "ssd_load_weights", "ssd_prefill", "ssd_prefill_dev",
            "ssd_decode_block", "ssd_block_begin", "ssd_set_block_state", "ssd_get_block_state", "ssd_block_step",
-           "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_cache_length", "ssd_gemm_bf16",
+           "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_cache_length", "ssd_rewind", "ssd_gemm_bf16",
            "ssd_launch_count", "ssd_profile_enable", "ssd_profile_read", "ssd_set_option"]
 
 
@@ -74,6 +74,7 @@ def load_library() -> C.CDLL:
     lib.ssd_verify_forward.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.ssd_read_cache.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.ssd_cache_length.argtypes = [vp]
+    lib.ssd_rewind.argtypes = [vp, i32]
     lib.ssd_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
     lib.ssd_launch_count.argtypes = [vp]
     lib.ssd_launch_count.restype = i64
@@ -152,6 +153,17 @@ class Ssd:
         nf = np.zeros(batch, np.int32)
         self._check(self.lib.ssd_decode_block(self._ctx, mode, block_tokens, _np_ptr(tok), _np_ptr(acc), _np_ptr(nf)))
         return tok, acc, nf
+
+    def decode_block_into(self, mode: int, block_tokens: int, tok_ptr: int, acc_ptr: int, nf_ptr: int):
+        """Same call with caller-owned host buffers given as addresses (e.g. pinned memory)."""
+        self._check(self.lib.ssd_decode_block(self._ctx, mode, block_tokens, C.c_void_p(tok_ptr), C.c_void_p(acc_ptr),
+                                              C.c_void_p(nf_ptr)))
+
+    def prefill_ptr(self, batch: int, prompt_len: int, host_ptr: int):
+        self._check(self.lib.ssd_prefill(self._ctx, batch, prompt_len, C.c_void_p(host_ptr)))
+
+    def rewind(self, length: int):
+        self._check(self.lib.ssd_rewind(self._ctx, length))
 
     def block_begin(self, block_tokens: int):
         self._check(self.lib.ssd_block_begin(self._ctx, block_tokens))

@@ -559,6 +559,16 @@ int ssd_prefill(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t* pr
 
 int ssd_cache_length(const ssd_ctx* c) { return c ? (c->cache_len < 0 ? SSD_ERR_STATE : c->cache_len) : SSD_ERR_INVALID_ARG; }
 
+int ssd_rewind(ssd_ctx* c, int32_t length) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
+  if (length < c->prompt_len || length > c->cache_len)
+    return fail(c, SSD_ERR_INVALID_ARG, "rewind target %d outside [%d, %d]", length, c->prompt_len, c->cache_len);
+  c->cache_len = length;
+  c->in_block = false;
+  return SSD_OK;
+}
+
 int ssd_block_begin(ssd_ctx* c, int32_t T) {
   if (!c) return SSD_ERR_INVALID_ARG;
   if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
