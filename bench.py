@@ -1,0 +1,406 @@
+#!/usr/bin/env python
+"""Benchmark of the SSD decode path on synthetic, seeded workloads.
+
+    python bench.py --gpus N --steps K --warmup W [--workload llada8b] [--max-drafts D]
+    python bench.py --impl reference ...        # the CPU oracle, timed on the host cores
+
+One "step" is one pass of the whole hot path over one batch: the generation of all `gen_len`
+tokens of every sequence after its prompt has been prefilled (candidate selection, tree build, one
+batched verification forward per iteration, acceptance, draft update, block commit, for every
+block).  `value` = decode tokens/s with everything resident on the device (prefill excluded);
+`e2e` = tokens/s through the host-buffer C-ABI calls, prefill and host<->device copies included.
+With N > 1 every rank decodes its own replica (independent sequences, no data-path collective):
+weak scaling.  Prints exactly one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode tokens/s at batch 1 (LLaDA-8B-shaped) and % HBM roofline per verify forward"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def forward_bytes(w, n_seq, S):
+    """Algorithmic HBM bytes of one verification forward: every layer weight, the LM head and the
+    cached prefix K/V of each sequence, each read once."""
+    q, kv = w.n_heads * w.head_dim, w.n_kv_heads * w.head_dim
+    per_layer = (q + 2 * kv) * w.d_model + w.d_model * q + 3 * w.d_ffn * w.d_model
+    weights = 2.0 * (per_layer * w.n_layers + w.vocab * w.d_model)
+    kvb = 2.0 * 2.0 * kv * w.n_layers * S * n_seq
+    return weights, kvb
+
+
+class ClockSampler:
+    """nvidia-smi sampled during the timed region (read-only)."""
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.path = f"/tmp/ssd_bench_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                   "samples": len(sm)}
+        return out
+
+
+# --------------------------------------------------------------------------------------------
+# the CPU oracle as baseline / reference arm
+# --------------------------------------------------------------------------------------------
+def oracle_sample(w, layers_sampled, prefix_len, n_rows, repeats=1):
+    """Times the oracle (as it stands) on a bounded sample of the workload: `layers_sampled` layers
+    of one root-only verification forward (`n_rows` rows against `prefix_len` cached positions) plus
+    the LM head, and scales the layer part to the full depth.  Returns (seconds per full forward,
+    description, threads)."""
+    import numpy as np
+    import torch
+    from oracle import ssd_oracle as so
+    from paper_2510_04147_b200 import workloads as wl
+
+    cfg = so.ModelConfig(w.n_layers, w.d_model, w.n_heads, w.n_kv_heads, w.head_dim, w.d_ffn, w.vocab, w.mask_id,
+                         w.rope_theta, w.rms_eps)
+
+    # inputs are drawn before the clock starts: only the oracle's own work is timed
+    names = [f"layers.{l}.{t}" for l in range(layers_sampled)
+             for t in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm_attn", "norm_ffn")]
+    weights = {n: wl.make_tensor(w, n, "cpu").to(torch.float32).numpy() for n in names + ["norm_final", "lm_head"]}
+    o = so.Oracle(cfg, weights)
+    rng = np.random.default_rng(0)
+    pk = rng.standard_normal((prefix_len, w.n_kv_heads, w.head_dim))
+    pv = rng.standard_normal((prefix_len, w.n_kv_heads, w.head_dim))
+    h = [rng.standard_normal((n_rows, w.d_model)) * 0.02]
+    pos = [np.arange(prefix_len, prefix_len + n_rows)]
+    t_layers = 0.0
+    for _ in range(repeats):
+        for l in range(layers_sampled):
+            t0 = time.perf_counter()
+            h2, _, _ = o.layer(l, h, pos, pk, pv)
+            t_layers += time.perf_counter() - t0
+    t_layers /= repeats * layers_sampled
+    t0 = time.perf_counter()
+    logits = so.rmsnorm(h2[0], o._W("norm_final"), cfg.rms_eps) @ o._W("lm_head").T
+    so.token_and_confidence(logits, cfg.mask_id)
+    t_head = time.perf_counter() - t0
+    t_full = t_layers * w.n_layers + t_head
+    desc = (f"oracle (numpy fp64) on {layers_sampled} of {w.n_layers} layers + LM head of one root-only "
+            f"verification forward ({n_rows} rows, prefix {prefix_len}); layer time scaled to full depth; "
+            f"tokens/s = block_len/(block_len+1) / forward time (stepwise: one token per forward, one commit per block)")
+    try:
+        import threadpoolctl
+        threads = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return t_full, desc, threads
+
+
+def run_reference(args):
+    from paper_2510_04147_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.WORKLOADS[args.workload]
+    times = []
+    for i in range(args.warmup + args.steps):
+        t, desc, threads = oracle_sample(w, layers_sampled=1, prefix_len=w.prompt_len, n_rows=w.block_len)
+        if i >= args.warmup:
+            times.append(t)
+    t = sum(times) / len(times)
+    tps = w.block_len / (w.block_len + 1.0) / t
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * t * (w.block_len + 1) * (w.gen_len // w.block_len),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "prompt_len": w.prompt_len, "gen_len": w.gen_len, "block_len": w.block_len,
+                       "batch": 1, "decoding": "stepwise (oracle)"},
+            "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA path
+# --------------------------------------------------------------------------------------------
+def run_ours(args):
+    import numpy as np
+    import torch
+    from paper_2510_04147_b200 import binding, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = load_peaks()
+    w = wl.WORKLOADS[args.workload]
+    B, L, P, bs = w.block_len, w.gen_len, w.prompt_len, w.batch
+    n_blocks = -(-L // B)
+    sweep_drafts = [int(x) for x in args.sweep.split(",")] if args.sweep else []
+    cfg_drafts = max([args.max_drafts if args.max_drafts >= 0 else 0] + sweep_drafts + [3])
+    stream = torch.cuda.current_stream()
+    ssd = binding.Ssd(binding.config_from_workload(w, max_drafts=min(cfg_drafts, B - 1)))
+    for k, v in (("split_k_qkv", args.split_qkv), ("split_k_o", args.split_o), ("split_k_down", args.split_down),
+                 ("kv_split", args.kv_split)):
+        if v is not None:
+            ssd.set_option(k, v)
+    t0 = time.time()
+    ssd.load_workload_weights(w, "cuda")
+    torch.cuda.synchronize()
+    t_load = time.time() - t0
+    # per-rank prompts: rank r decodes sequences r*bs .. r*bs+bs-1 of the seeded prompt set
+    prompts_all = wl.make_prompts(w, "cpu", batch=bs * world)
+    prompts = prompts_all[rank * bs:(rank + 1) * bs].contiguous()
+    prompts_pinned = prompts.clone().pin_memory()
+    prompts_dev = prompts.cuda()
+    out_tok = torch.zeros((bs, B), dtype=torch.int32).pin_memory()
+    out_acc = torch.zeros((bs, B), dtype=torch.int32).pin_memory()
+    out_nf = torch.zeros((bs,), dtype=torch.int32).pin_memory()
+
+    def decode_all(max_drafts, collect=None):
+        """All blocks of one generation through ssd_decode_block (cache must hold exactly the prompt)."""
+        ssd.set_option("max_drafts", max_drafts)
+        mode = binding.MODE_SSD if max_drafts > 0 else binding.MODE_STEPWISE
+        done = 0
+        while done < L:
+            t = min(B, L - done)
+            ssd.decode_block_into(mode, t, out_tok.data_ptr(), out_acc.data_ptr(), out_nf.data_ptr())
+            if collect is not None:
+                collect.append(out_acc.numpy()[:, :t].copy())
+            done += t
+
+    def timed_generation(max_drafts, reps):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(reps):
+            ssd.rewind(P)
+            decode_all(max_drafts)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1) / reps
+
+    def accept_stats(max_drafts):
+        hist = []
+        ssd.rewind(P)
+        decode_all(max_drafts, hist)
+        accs = np.concatenate([a.reshape(-1) for a in hist])
+        return accs[accs > 0]
+
+    t0 = time.time()
+    ssd.prefill_dev(prompts_dev)
+    torch.cuda.synchronize()
+    t_prefill = time.time() - t0
+
+    # ---- choose the draft length: quick sweep (untimed for the headline), or the one given
+    sweep = {}
+    if args.max_drafts >= 0:
+        best = args.max_drafts
+    else:
+        for d in sweep_drafts:
+            ms = timed_generation(d, 1)
+            accs = accept_stats(d)
+            sweep[str(d)] = {"tokens_per_s": bs * L / (ms * 1e-3), "ms_per_generation": ms,
+                             "mean_accepted_per_forward": float(accs.mean()), "forwards": int(len(accs))}
+        best = int(max(sweep, key=lambda k: sweep[k]["tokens_per_s"]))
+    # the configured cap decides buffer sizes only; the draft length used is `best`
+    for _ in range(args.warmup):
+        ssd.rewind(P)
+        decode_all(best)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = ClockSampler(local)
+    clocks.start()
+    launches0 = ssd.launch_count()
+    torch.cuda.synchronize()
+    ms = timed_generation(best, args.steps)
+    launches = ssd.launch_count() - launches0
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clk = clocks.stop()
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * bs * L / (ms * 1e-3)
+
+    # ---- end to end: host prompt -> prefill -> all blocks with host outputs, every step
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(1, min(args.steps, 2))
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for _ in range(e2e_steps):
+        ssd.prefill_ptr(bs, P, prompts_pinned.data_ptr())
+        decode_all(best)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    ms_e2e = ev0.elapsed_time(ev1) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e_value = world * bs * L / (ms_e2e * 1e-3)
+
+    line = None
+    if rank == 0:
+        # ---- accept statistics of the timed configuration
+        accs = accept_stats(best)
+        # ---- per-forward roofline: stepwise (1 node) and the chosen chain, CUDA events per forward
+        fwd = {}
+        for label, d in (("stepwise_1_node", 0), (f"ssd_{best + 1}_nodes", best)):
+            ssd.rewind(P)
+            ssd.block_begin(B)
+            ssd.block_step(d, bs)                       # root-only forward creates the drafts
+            times = []
+            nodes = []
+            for _ in range(6):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                acc, nn = ssd.block_step(d, bs)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if acc.sum() == 0:
+                    break
+                times.append(e0.elapsed_time(e1))
+                nodes.append(int(nn.max()))
+            tmed = statistics.median(times)
+            wb, kvb = forward_bytes(w, bs, P)
+            rows = bs * max(nodes) * B
+            fl = 2.0 * rows * (wb / 2.0)
+            t_hbm = (wb + kvb) / (peaks["hbm_gbs"] * 1e9)
+            t_tc = fl / (peaks["bf16_tflops_sustained"] * 1e12)
+            fwd[label] = {"nodes": max(nodes), "rows": rows, "ms": tmed, "algorithmic_gb": (wb + kvb) / 1e9,
+                          "hbm_frac": t_hbm / (tmed * 1e-3), "frac_of_max_hbm_tensor": max(t_hbm, t_tc) / (tmed * 1e-3)}
+        # ---- dominant kernel: the projection GEMM family, CUDA events around every launch
+        ssd.rewind(P)
+        ssd.block_begin(B)
+        ssd.block_step(best, bs)
+        ssd.profile_enable(True)
+        ssd.profile_read()
+        for _ in range(3):
+            ssd.block_step(best, bs)
+        prof = ssd.profile_read()
+        ssd.profile_enable(False)
+        g = prof["gemm"]
+        achieved = g["bytes"] / (g["ms"] * 1e-3) / 1e9 if g["ms"] > 0 else 0.0
+        total_ms = sum(v["ms"] for v in prof.values())
+        roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel (QKV/O/gate-up/down projections)",
+                    "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                    "peak_source": peaks["_source"], "traffic": None,
+                    "launches": g["launches"], "avg_launch_us": 1e3 * g["ms"] / max(1, g["launches"]),
+                    "bytes_per_launch_avg": g["bytes"] / max(1, g["launches"]),
+                    "family_share_of_device_time": {k: (v["ms"] / total_ms if total_ms else 0) for k, v in prof.items()}}
+        # ---- CPU baseline: the oracle on a bounded sample
+        if args.no_cpu_baseline:
+            cpu = None
+        else:
+            t_fwd, desc, threads = oracle_sample(w, layers_sampled=1, prefix_len=P, n_rows=B)
+            cpu = {"value": B / (B + 1.0) / t_fwd, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                   "sample": desc, "seconds_per_forward": t_fwd}
+        line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": w.name, "prompt_len": P, "gen_len": L, "block_len": B, "batch_per_gpu": bs,
+                           "max_drafts": best, "nodes_per_forward": best + 1,
+                           "l2_policy": "inputs larger than L2 (15 GB of weights streamed per forward)",
+                           "replicas": world, "weights_load_s": t_load, "prefill_s": t_prefill},
+                "clocks": clk, "gpu_launches": int(launches),
+                "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(bs * P * 4),
+                        "d2h_bytes_per_step": int(n_blocks * bs * (2 * B + 1) * 4), "ms_per_step": ms_e2e,
+                        "includes": "host prompt copy + prefill + every block's tokens/accept counts read back"},
+                "roofline": roofline, "forward": fwd, "cpu_baseline": cpu,
+                "accept": {"mean_per_forward": float(accs.mean()), "histogram": np.bincount(accs).tolist(),
+                           "forwards_per_generation": int(len(accs)), "blocks": n_blocks},
+                "sweep": sweep,
+                "paper_context": "paper reports 2.0-3.46x over stepwise decoding on one A100 80GB with trained weights"}
+    ssd.destroy()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if line is not None:
+        print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llada8b")
+    ap.add_argument("--max-drafts", type=int, default=-1, help="draft length N; -1: pick the best of --sweep")
+    ap.add_argument("--sweep", default="0,1,3,5")
+    ap.add_argument("--split-qkv", type=int, default=None)
+    ap.add_argument("--split-o", type=int, default=None)
+    ap.add_argument("--split-down", type=int, default=None)
+    ap.add_argument("--kv-split", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -166,8 +166,9 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
 
 /* Tuning knobs (set before prefill).  key: "split_k_qkv", "split_k_o", "split_k_down" (1..8),
  * "kv_split" (prefix keys per attention split, multiple of 64; 0 = automatic from the prefix
- * length), "gemm_impl" (1 = TMA + tcgen05 kernel, the default; 0 = the plain CUDA-core bring-up
- * kernel, for cross-checks only).  Unknown key: SSD_ERR_INVALID_ARG. */
+ * length), "max_drafts" (lower the draft-length cap below the capacity fixed at creation),
+ * "gemm_impl" (1 = TMA + tcgen05 kernel, the default; 0 = the plain CUDA-core bring-up kernel,
+ * for cross-checks only).  Unknown key: SSD_ERR_INVALID_ARG. */
 int ssd_set_option(ssd_ctx* ctx, const char* key, int32_t value);
 
 #ifdef __cplusplus

@@ -814,6 +814,11 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
     c->kv_split_opt = value;
     return SSD_OK;
   }
+  if (!strcmp(key, "max_drafts")) {
+    if (value < 0 || value + 1 > c->n_max) return fail(c, SSD_ERR_INVALID_ARG, "max_drafts must be in [0, %d] (the capacity fixed at creation)", c->n_max - 1);
+    c->cfg.max_drafts = value;
+    return SSD_OK;
+  }
   if (!strcmp(key, "gemm_impl")) {
     if (value != 0 && value != 1) return fail(c, SSD_ERR_INVALID_ARG, "gemm_impl is 0 (CUDA cores, bring-up) or 1 (tcgen05)");
     c->gemm_impl = value;
