@@ -146,6 +146,25 @@ int ssd_rewind(ssd_ctx* ctx, int32_t length);
 int ssd_gemm_bf16(ssd_ctx* ctx, const void* x_dev, const void* w_dev, float* out_dev,
                   int32_t rows, int32_t n, int32_t k, int32_t split_k);
 
+/* The same projection for callers that cannot allocate device memory while they run (the paper has
+ * no counterpart: this is a deployment aid).  Think of a server that handed the whole GPU to its own
+ * arena at start-up, or of a latency-critical loop that may not make a call which can block on the
+ * device or run out of memory: neither can use a context, whose creation allocates.  This entry point
+ * needs no context and calls no cudaMalloc/cudaFree nor any allocating library routine: its split-K
+ * scratch is a fixed 4 MiB array inside the library image (each GPU that loads the library holds it
+ * until the process exits).
+ *   x_dev [rows,k] bf16, w_dev [n,k] bf16, out_dev [rows,n] fp32: DEVICE memory of the current device,
+ *   owned by the caller; k a multiple of 8; 1 <= split_k <= 8; `cuda_stream` a cudaStream_t.
+ *   Limit: split_k * rows * n <= 1048512 floats (4 MiB minus a 256-byte flag area), else
+ *   SSD_ERR_OVERFLOW; bad shapes SSD_ERR_SHAPE; null pointers SSD_ERR_INVALID_ARG.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call before starting any stream capture.  All calls share the one array, which
+ * keeps the previous call's contents (the error word is cleared at the start of every call): two
+ * calls whose GPU work overlaps - different streams or threads - race on it, so serialise them.
+ * Synchronises the stream before returning; same result as ssd_gemm_bf16. */
+int ssd_gemm_bf16_noalloc(const void* x_dev, const void* w_dev, float* out_dev, int32_t rows, int32_t n,
+                          int32_t k, int32_t split_k, void* cuda_stream);
+
 /* ---- measurement ---------------------------------------------------------------------------- */
 
 /* Kernel launches issued by this context since creation (all streams of the context). */

@@ -27,6 +27,7 @@ PROF_FAMILIES = ("gemm", "lmhead", "attn", "elemwise", "tree")
 EXPORTS = ["ssd_create", "ssd_destroy", "ssd_last_error", "ssd_load_weights", "ssd_prefill", "ssd_prefill_dev",
            "ssd_decode_block", "ssd_block_begin", "ssd_set_block_state", "ssd_get_block_state", "ssd_block_step",
            "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_cache_length", "ssd_rewind", "ssd_gemm_bf16",
+           "ssd_gemm_bf16_noalloc",
            "ssd_launch_count", "ssd_profile_enable", "ssd_profile_read", "ssd_set_option"]
 
 
@@ -76,6 +77,7 @@ def load_library() -> C.CDLL:
     lib.ssd_cache_length.argtypes = [vp]
     lib.ssd_rewind.argtypes = [vp, i32]
     lib.ssd_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
+    lib.ssd_gemm_bf16_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ssd_launch_count.argtypes = [vp]
     lib.ssd_launch_count.restype = i64
     lib.ssd_profile_enable.argtypes = [vp, i32]
@@ -87,6 +89,18 @@ def load_library() -> C.CDLL:
             fn.restype = i32
     _lib = lib
     return lib
+
+
+def gemm_bf16_noalloc(x: torch.Tensor, w: torch.Tensor, out: torch.Tensor, split_k: int = 1) -> int:
+    """ssd_gemm_bf16_noalloc on caller-owned tensors (x [rows,k] bf16, w [n,k] bf16, out [rows,n] fp32, all on the
+    current CUDA device).  Needs no context and allocates nothing; returns the C return code."""
+    lib = load_library()
+    assert x.is_cuda and w.is_cuda and out.is_cuda and x.dtype == w.dtype == torch.bfloat16 and out.dtype == torch.float32
+    assert x.is_contiguous() and w.is_contiguous() and out.is_contiguous()
+    assert x.shape[1] == w.shape[1] and out.shape == (x.shape[0], w.shape[0])
+    return int(lib.ssd_gemm_bf16_noalloc(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(out.data_ptr()),
+                                         x.shape[0], w.shape[0], x.shape[1], split_k,
+                                         C.c_void_p(torch.cuda.current_stream().cuda_stream)))
 
 
 def _np_ptr(a: Optional[np.ndarray]):
