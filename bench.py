@@ -152,12 +152,26 @@ def oracle_sample(w, layers_sampled, prefix_len, n_rows, repeats=1):
     return t_full, desc, threads
 
 
-def run_reference(args):
+def pick_workload(args):
+    """The named workload; --layers / --gen-len / --prompt-len shrink it for profiler captures only
+    (such a run is labelled "reduced" and is not a benchmark of the named configuration)."""
     from paper_2510_04147_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    over = {}
+    if args.layers:
+        over["n_layers"] = args.layers
+    if args.gen_len:
+        over["gen_len"] = args.gen_len
+    if args.prompt_len:
+        over["prompt_len"] = args.prompt_len
+    return (w.replace(**over), True) if over else (w, False)
+
+
+def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = wl.WORKLOADS[args.workload]
+    w, _ = pick_workload(args)
     times = []
     for i in range(args.warmup + args.steps):
         t, desc, threads = oracle_sample(w, layers_sampled=1, prefix_len=w.prompt_len, n_rows=w.block_len)
@@ -181,18 +195,16 @@ def run_reference(args):
 def run_ours(args):
     import numpy as np
     import torch
-    from paper_2510_04147_b200 import binding, workloads as wl
+    from paper_2510_04147_b200 import binding, replicas, workloads as wl
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replicas.rank_world_local()
     torch.cuda.set_device(local)
     dist = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = load_peaks()
-    w = wl.WORKLOADS[args.workload]
+    w, reduced = pick_workload(args)
     B, L, P, bs = w.block_len, w.gen_len, w.prompt_len, w.batch
     n_blocks = -(-L // B)
     sweep_drafts = [int(x) for x in args.sweep.split(",")] if args.sweep else []
@@ -208,8 +220,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     t_load = time.time() - t0
     # per-rank prompts: rank r decodes sequences r*bs .. r*bs+bs-1 of the seeded prompt set
-    prompts_all = wl.make_prompts(w, "cpu", batch=bs * world)
-    prompts = prompts_all[rank * bs:(rank + 1) * bs].contiguous()
+    prompts = replicas.shard_prompts(w, rank, world, bs)
     prompts_pinned = prompts.clone().pin_memory()
     prompts_dev = prompts.cuda()
     out_tok = torch.zeros((bs, B), dtype=torch.int32).pin_memory()
@@ -278,11 +289,8 @@ def run_ours(args):
     if dist is not None:
         dist.barrier()
     clk = clocks.stop()
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * bs * L / (ms * 1e-3)
+    ms = replicas.max_over_ranks(ms, dist, "cuda")
+    value = replicas.job_tokens_per_s(world, bs, L, ms)
 
     # ---- end to end: host prompt -> prefill -> all blocks with host outputs, every step
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -295,11 +303,8 @@ def run_ours(args):
     ev1.record(stream)
     torch.cuda.synchronize()
     ms_e2e = ev0.elapsed_time(ev1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_value = world * bs * L / (ms_e2e * 1e-3)
+    ms_e2e = replicas.max_over_ranks(ms_e2e, dist, "cuda")
+    e2e_value = replicas.job_tokens_per_s(world, bs, L, ms_e2e)
 
     line = None
     if rank == 0:
@@ -363,7 +368,9 @@ def run_ours(args):
                 "config": {"workload": w.name, "prompt_len": P, "gen_len": L, "block_len": B, "batch_per_gpu": bs,
                            "max_drafts": best, "nodes_per_forward": best + 1,
                            "l2_policy": "inputs larger than L2 (15 GB of weights streamed per forward)",
-                           "replicas": world, "weights_load_s": t_load, "prefill_s": t_prefill},
+                           "replicas": world, "weights_load_s": t_load, "prefill_s": t_prefill,
+                           **({"reduced_for_profiling": {"n_layers": w.n_layers, "gen_len": L, "prompt_len": P}}
+                              if reduced else {})},
                 "clocks": clk, "gpu_launches": int(launches),
                 "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(bs * P * 4),
                         "d2h_bytes_per_step": int(n_blocks * bs * (2 * B + 1) * 4), "ms_per_step": ms_e2e,
@@ -395,6 +402,9 @@ def main():
     ap.add_argument("--split-down", type=int, default=None)
     ap.add_argument("--kv-split", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="profiling only: fewer layers of the same shape")
+    ap.add_argument("--gen-len", type=int, default=0, help="profiling only: shorter generation")
+    ap.add_argument("--prompt-len", type=int, default=0, help="profiling only: another prompt length")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
