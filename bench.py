@@ -209,7 +209,9 @@ def run_ours(args):
     n_blocks = -(-L // B)
     sweep_drafts = [int(x) for x in args.sweep.split(",")] if args.sweep else []
     cfg_drafts = max([args.max_drafts if args.max_drafts >= 0 else 0] + sweep_drafts + [3])
-    stream = torch.cuda.current_stream()
+    # a stream of its own (not the legacy default stream) so that dependent launches may overlap
+    stream = torch.cuda.Stream()
+    torch.cuda.set_stream(stream)
     ssd = binding.Ssd(binding.config_from_workload(w, max_drafts=min(cfg_drafts, B - 1)))
     for k, v in (("split_k_qkv", args.split_qkv), ("split_k_o", args.split_o), ("split_k_down", args.split_down),
                  ("kv_split", args.kv_split)):

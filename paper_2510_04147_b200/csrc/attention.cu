@@ -66,6 +66,8 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(AttnArgs a, in
   bf16* sV = sK + 2 * kKTile * HD;
   constexpr int CH = HD / 8;   // 16-byte chunks per row
 
+  pdl_launch_dependents();
+  pdl_wait();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int gq = lane >> 2, tq = lane & 3;
   const int qt = blockIdx.x, h = blockIdx.y;
@@ -244,27 +246,31 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(AttnArgs a, in
   }
 }
 
+// One CTA per (row, group of heads): 256 threads, two output elements each.  Parts are merged in
+// part order with weights 2^(m_p - M).
 __global__ void __launch_bounds__(256) attn_merge_kernel(const float* part_o, const float2* part_ml, bf16* out, int R,
                                                          int H, int hd, int n_parts) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int r = blockIdx.x;
   const int width = H * hd;
-  for (int e = threadIdx.x * 2; e < width; e += 256 * 2) {
-    const int h = e / hd;
-    float M = -INFINITY;
-    for (int p = 0; p < n_parts; ++p) M = fmaxf(M, part_ml[((size_t)p * R + r) * H + h].x);
-    float L = 0.f, ax = 0.f, ay = 0.f;
-    for (int p = 0; p < n_parts; ++p) {
-      const float2 ml = part_ml[((size_t)p * R + r) * H + h];
-      if (ml.x == -INFINITY) continue;
-      const float w = exp2f(ml.x - M);
-      const float2 v = *reinterpret_cast<const float2*>(part_o + ((size_t)p * R + r) * width + e);
-      L += ml.y * w;
-      ax += v.x * w;
-      ay += v.y * w;
-    }
-    const float inv = 1.f / L;
-    *reinterpret_cast<__nv_bfloat162*>(out + (size_t)r * width + e) = __floats2bfloat162_rn(ax * inv, ay * inv);
+  const int e = (blockIdx.y * 256 + threadIdx.x) * 2;
+  if (e >= width) return;
+  const int h = e / hd;
+  float M = -INFINITY;
+  for (int p = 0; p < n_parts; ++p) M = fmaxf(M, part_ml[((size_t)p * R + r) * H + h].x);
+  float L = 0.f, ax = 0.f, ay = 0.f;
+  for (int p = 0; p < n_parts; ++p) {
+    const float2 ml = part_ml[((size_t)p * R + r) * H + h];
+    if (ml.x == -INFINITY) continue;
+    const float w = exp2f(ml.x - M);
+    const float2 v = *reinterpret_cast<const float2*>(part_o + ((size_t)p * R + r) * width + e);
+    L += ml.y * w;
+    ax += v.x * w;
+    ay += v.y * w;
   }
+  const float inv = 1.f / L;
+  *reinterpret_cast<__nv_bfloat162*>(out + (size_t)r * width + e) = __floats2bfloat162_rn(ax * inv, ay * inv);
 }
 
 }  // namespace
@@ -283,12 +289,14 @@ void launch_attention(cudaStream_t st, const AttnArgs& a, int* launches) {
       cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
       attr_set = true;
     }
-    attn_split_kernel<128><<<grid, kAttnThreads, smem, st>>>(a, n_prefix, has_local, scale_log2);
+    launch_pdl(attn_split_kernel<128>, grid, dim3(kAttnThreads), (size_t)smem, st, a, n_prefix, has_local, scale_log2);
   } else {
     const int smem = (kQTile + 4 * kKTile) * 64 * 2;
-    attn_split_kernel<64><<<grid, kAttnThreads, smem, st>>>(a, n_prefix, has_local, scale_log2);
+    launch_pdl(attn_split_kernel<64>, grid, dim3(kAttnThreads), (size_t)smem, st, a, n_prefix, has_local, scale_log2);
   }
-  attn_merge_kernel<<<a.R, 256, 0, st>>>(a.part_o, a.part_ml, a.out, a.R, a.H, a.hd, n_parts);
+  dim3 mgrid(a.R, (a.H * a.hd / 2 + 255) / 256);
+  launch_pdl(attn_merge_kernel, mgrid, dim3(256), 0, st, (const float*)a.part_o, (const float2*)a.part_ml, a.out, a.R,
+             a.H, a.hd, n_parts);
   if (launches) *launches += 2;
 }
 

@@ -37,13 +37,24 @@ __global__ void convert_rows_kernel(const void* src, int src_is_f32, bf16* dst, 
   }
 }
 
+__global__ void convert_tiled_kernel(const void* src, int src_is_f32, bf16* dst, int rows, int cols, int kb_total,
+                                     int group, int group_stride, int group_offset) {
+  const size_t total = (size_t)rows * cols;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const int j = (int)(i / cols), c = (int)(i % cols);
+    const float v = src_is_f32 ? ((const float*)src)[i] : __bfloat162float(((const bf16*)src)[i]);
+    const size_t n = (size_t)(j / group) * group_stride + group_offset + (j % group);
+    dst[(((n >> 7) * kb_total + (c >> 6)) * 128 + (n & 127)) * 64 + (c & 63)] = __float2bfloat16_rn(v);
+  }
+}
+
 __global__ void copy_f32_kernel(const void* src, int src_is_f32, float* dst, int n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = src_is_f32 ? ((const float*)src)[i] : __bfloat162float(((const bf16*)src)[i]);
 }
 
 __device__ __forceinline__ void write_norm_row(const float* hrow, const float* gain, float inv, bf16* xrow, int d) {
-  for (int c = threadIdx.x * 4; c < d; c += kThreads * 4) {
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     const float4 v = *reinterpret_cast<const float4*>(hrow + c);
     const float4 g = *reinterpret_cast<const float4*>(gain + c);
     __nv_bfloat162 a = __floats2bfloat162_rn(v.x * inv * g.x, v.y * inv * g.y);
@@ -53,14 +64,19 @@ __device__ __forceinline__ void write_norm_row(const float* hrow, const float* g
   }
 }
 
-__global__ void __launch_bounds__(kThreads) embed_rmsnorm_kernel(const int* ids, const bf16* embed, const float* gain,
-                                                                 float eps, float* h, bf16* xn, int d) {
-  __shared__ float red[kThreads / 32];
+constexpr int kRowThreadsMax = 1024;   // one float4 per thread up to d = 4096
+
+__global__ void __launch_bounds__(kRowThreadsMax) embed_rmsnorm_kernel(const int* ids, const bf16* embed,
+                                                                       const float* gain, float eps, float* h, bf16* xn,
+                                                                       int d) {
+  __shared__ float red[kRowThreadsMax / 32];
+  pdl_launch_dependents();
+  pdl_wait();
   const int r = blockIdx.x;
   const bf16* e = embed + (size_t)ids[r] * d;
   float* hrow = h + (size_t)r * d;
   float ss = 0.f;
-  for (int c = threadIdx.x * 4; c < d; c += kThreads * 4) {
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(e + c);
     const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(e + c + 2);
     float4 v = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
@@ -72,18 +88,34 @@ __global__ void __launch_bounds__(kThreads) embed_rmsnorm_kernel(const int* ids,
   write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
 }
 
-__global__ void __launch_bounds__(kThreads) residual_rmsnorm_kernel(const float* partial, int splits, size_t split_stride,
-                                                                    const float* gain, float eps, float* h, bf16* xn,
-                                                                    int d) {
-  __shared__ float red[kThreads / 32];
+// One CTA per row, one float4 column group per thread (per pass): every split's partial is loaded
+// independently, then added in split order, so the row's sum does not depend on the launch shape.
+__global__ void __launch_bounds__(kRowThreadsMax) residual_rmsnorm_kernel(const float* partial, int splits,
+                                                                          size_t split_stride, const float* gain,
+                                                                          float eps, float* h, bf16* xn, int d) {
+  __shared__ float red[kRowThreadsMax / 32];
+  pdl_launch_dependents();
+  pdl_wait();
   const int r = blockIdx.x;
   float* hrow = h + (size_t)r * d;
   float ss = 0.f;
-  for (int c = threadIdx.x * 4; c < d; c += kThreads * 4) {
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     float4 v = *reinterpret_cast<const float4*>(hrow + c);
-    for (int s = 0; s < splits; ++s) {
-      const float4 p = *reinterpret_cast<const float4*>(partial + s * split_stride + (size_t)r * d + c);
-      v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+    const float* pp = partial + (size_t)r * d + c;
+    int s = 0;
+    for (; s + 4 <= splits; s += 4) {
+      const float4 p0 = *reinterpret_cast<const float4*>(pp + (size_t)s * split_stride);
+      const float4 p1 = *reinterpret_cast<const float4*>(pp + (size_t)(s + 1) * split_stride);
+      const float4 p2 = *reinterpret_cast<const float4*>(pp + (size_t)(s + 2) * split_stride);
+      const float4 p3 = *reinterpret_cast<const float4*>(pp + (size_t)(s + 3) * split_stride);
+      v.x += p0.x; v.y += p0.y; v.z += p0.z; v.w += p0.w;
+      v.x += p1.x; v.y += p1.y; v.z += p1.z; v.w += p1.w;
+      v.x += p2.x; v.y += p2.y; v.z += p2.z; v.w += p2.w;
+      v.x += p3.x; v.y += p3.y; v.z += p3.z; v.w += p3.w;
+    }
+    for (; s < splits; ++s) {
+      const float4 p0 = *reinterpret_cast<const float4*>(pp + (size_t)s * split_stride);
+      v.x += p0.x; v.y += p0.y; v.z += p0.z; v.w += p0.w;
     }
     *reinterpret_cast<float4*>(hrow + c) = v;
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
@@ -94,46 +126,47 @@ __global__ void __launch_bounds__(kThreads) residual_rmsnorm_kernel(const float*
   write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
 }
 
-__global__ void __launch_bounds__(kThreads) qkv_rope_kernel(const float* partial, int splits, size_t split_stride, int H,
-                                                            int Hkv, int hd, const float2* rope_table, RowMap map,
-                                                            bf16* q, bf16* k_dst, bf16* v_dst, int kv_to_cache,
-                                                            size_t cache_seq_stride) {
+// One CTA per (row, group of 8 heads of the fused q|k|v output); a warp per head.
+constexpr int kRopeHeadsPerBlock = 8;
+__global__ void __launch_bounds__(kRopeHeadsPerBlock * 32) qkv_rope_kernel(const float* partial, int splits,
+                                                                            size_t split_stride, int H, int Hkv, int hd,
+                                                                            const float2* rope_table, RowMap map,
+                                                                            bf16* q, bf16* k_dst, bf16* v_dst,
+                                                                            int kv_to_cache, size_t cache_seq_stride) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int r = blockIdx.x;
+  const int head = blockIdx.y * kRopeHeadsPerBlock + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (head >= H + 2 * Hkv) return;
   const int half = hd >> 1;
   const int nqkv = (H + 2 * Hkv) * hd;
   const int slot = r / map.rows_per_seq;
   const int t = r % map.T;
   const int pos = map.pos0 + t;
   const int seq = map.seq_map ? map.seq_map[slot] : map.seq_base + slot;
-  const float* prow = partial + (size_t)r * nqkv;
+  const float* prow = partial + (size_t)r * nqkv + (size_t)head * hd;
   const size_t kv_row = kv_to_cache ? ((size_t)seq * cache_seq_stride + (size_t)pos * Hkv * hd) : (size_t)r * Hkv * hd;
-  const float2* rt = rope_table + (size_t)pos * half;
-  for (int p = threadIdx.x; p < (H + Hkv) * half; p += kThreads) {
-    const int head = p / half, i = p % half;
-    const int c1 = head * hd + i, c2 = c1 + half;
-    float x1 = 0.f, x2 = 0.f;
-    for (int s = 0; s < splits; ++s) {
-      x1 += prow[s * split_stride + c1];
-      x2 += prow[s * split_stride + c2];
+  if (head < H + Hkv) {
+    const float2* rt = rope_table + (size_t)pos * half;
+    bf16* dst = head < H ? q + ((size_t)r * H + head) * hd : k_dst + kv_row + (size_t)(head - H) * hd;
+    for (int i = lane; i < half; i += 32) {
+      float x1 = 0.f, x2 = 0.f;
+      for (int s = 0; s < splits; ++s) {
+        x1 += prow[s * split_stride + i];
+        x2 += prow[s * split_stride + i + half];
+      }
+      const float2 cs = rt[i];
+      dst[i] = __float2bfloat16_rn(x1 * cs.x - x2 * cs.y);
+      dst[i + half] = __float2bfloat16_rn(x2 * cs.x + x1 * cs.y);
     }
-    const float2 cs = rt[i];
-    const float y1 = x1 * cs.x - x2 * cs.y;
-    const float y2 = x2 * cs.x + x1 * cs.y;
-    if (head < H) {
-      bf16* dst = q + ((size_t)r * H + head) * hd;
-      dst[i] = __float2bfloat16_rn(y1);
-      dst[i + half] = __float2bfloat16_rn(y2);
-    } else {
-      bf16* dst = k_dst + kv_row + (size_t)(head - H) * hd;
-      dst[i] = __float2bfloat16_rn(y1);
-      dst[i + half] = __float2bfloat16_rn(y2);
+  } else {
+    bf16* dst = v_dst + kv_row + (size_t)(head - H - Hkv) * hd;
+    for (int e = lane; e < hd; e += 32) {
+      float x = 0.f;
+      for (int s = 0; s < splits; ++s) x += prow[s * split_stride + e];
+      dst[e] = __float2bfloat16_rn(x);
     }
-  }
-  const int voff = (H + Hkv) * hd;
-  for (int e = threadIdx.x; e < Hkv * hd; e += kThreads) {
-    float x = 0.f;
-    for (int s = 0; s < splits; ++s) x += prow[s * split_stride + voff + e];
-    v_dst[kv_row + e] = __float2bfloat16_rn(x);
   }
 }
 
@@ -183,20 +216,38 @@ __global__ void __launch_bounds__(kThreads) lm_stats_from_logits_kernel(const fl
   if (threadIdx.x == 0) { tok[r] = a; conf[r] = 1.f / s; }
 }
 
-// One warp per row; lanes stride over the vocabulary tiles, then a fixed butterfly merge.
+// Symmetric merge of two (max, sum-exp, argmax) triples: both partners of a butterfly step compute
+// bit-identical results, and ties keep the lower token id.
+__device__ __forceinline__ void stat_merge(float& m, float& s, int& a, float om, float os, int oa) {
+  const float nm = fmaxf(m, om);
+  if (nm == -INFINITY) return;
+  const float lo_m = fminf(m, om);
+  const float hi_s = (m >= om) ? s : os;
+  const float lo_s = (m >= om) ? os : s;
+  const float ns = (m == om) ? (s + os) : (hi_s + lo_s * expf(lo_m - nm));
+  int na;
+  if (m == om) na = min(a, oa); else na = (m > om) ? a : oa;
+  m = nm; s = ns; a = na;
+}
+
+// One CTA per row: threads stride over the vocabulary tiles, butterfly inside each warp, then the
+// warp results in warp order.  The order depends on the tile count alone.
 __global__ void __launch_bounds__(kThreads) lm_merge_kernel(const float* tile_max, const float* tile_sum,
                                                             const int* tile_arg, int tiles, int R,
                                                             const uint8_t* row_wanted, int* tok, float* conf) {
-  const int r = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (r >= R) return;
+  __shared__ float w_m[kThreads / 32], w_s[kThreads / 32];
+  __shared__ int w_a[kThreads / 32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (row_wanted && !row_wanted[r]) {
-    if (lane == 0) { tok[r] = -1; conf[r] = 0.f; }
+    if (threadIdx.x == 0) { tok[r] = -1; conf[r] = 0.f; }
     return;
   }
   float m = -INFINITY, s = 0.f;
   int a = 0x7fffffff;
-  for (int t = lane; t < tiles; t += 32) {
+  for (int t = threadIdx.x; t < tiles; t += kThreads) {
     const float tm = tile_max[(size_t)t * R + r];
     if (tm == -INFINITY) continue;
     const float ts = tile_sum[(size_t)t * R + r];
@@ -209,18 +260,15 @@ __global__ void __launch_bounds__(kThreads) lm_merge_kernel(const float* tile_ma
     const float om = __shfl_xor_sync(0xffffffffu, m, o);
     const float os = __shfl_xor_sync(0xffffffffu, s, o);
     const int oa = __shfl_xor_sync(0xffffffffu, a, o);
-    const float nm = fmaxf(m, om);
-    if (nm == -INFINITY) continue;
-    // symmetric in (self, other) so that both partners compute bit-identical results
-    const float lo_m = fminf(m, om);
-    const float hi_s = (m >= om) ? s : os;
-    const float lo_s = (m >= om) ? os : s;
-    const float ns = (m == om) ? (s + os) : (hi_s + lo_s * expf(lo_m - nm));
-    int na;
-    if (m == om) na = min(a, oa); else na = (m > om) ? a : oa;
-    m = nm; s = ns; a = na;
+    stat_merge(m, s, a, om, os, oa);
   }
-  if (lane == 0) { tok[r] = a; conf[r] = 1.f / s; }
+  if (lane == 0) { w_m[warp] = m; w_s[warp] = s; w_a[warp] = a; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < kThreads / 32; ++i) stat_merge(m, s, a, w_m[i], w_s[i], w_a[i]);
+    tok[r] = a;
+    conf[r] = 1.f / s;
+  }
 }
 
 }  // namespace
@@ -235,25 +283,45 @@ void launch_convert_rows(cudaStream_t st, const void* src, int src_is_f32, bf16*
                                               group_offset);
 }
 
+void launch_convert_tiled(cudaStream_t st, const void* src, int src_is_f32, bf16* dst, int rows, int cols, int kb_total,
+                          int group, int group_stride, int group_offset) {
+  const size_t total = (size_t)rows * cols;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  convert_tiled_kernel<<<blocks, 256, 0, st>>>(src, src_is_f32, dst, rows, cols, kb_total, group, group_stride,
+                                               group_offset);
+}
+
 void launch_copy_f32(cudaStream_t st, const void* src, int src_is_f32, float* dst, int n) {
   copy_f32_kernel<<<(n + 255) / 256, 256, 0, st>>>(src, src_is_f32, dst, n);
 }
 
+static int row_threads(int d) {
+  int t = ((d / 4 + 31) / 32) * 32;
+  if (t > kRowThreadsMax) t = kRowThreadsMax;
+  if (t < 32) t = 32;
+  return t;
+}
+
 void launch_embed_rmsnorm(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float eps, float* h,
                           bf16* xn, int R, int d) {
-  embed_rmsnorm_kernel<<<R, kThreads, 0, st>>>(ids, embed, gain, eps, h, xn, d);
+  launch_pdl(embed_rmsnorm_kernel, dim3(R), dim3(row_threads(d)), 0, st, ids, embed, gain, eps, h, xn, d);
 }
 
 void launch_residual_rmsnorm(cudaStream_t st, const float* partial, int splits, size_t split_stride, const float* gain,
                              float eps, float* h, bf16* xn, int R, int d) {
-  residual_rmsnorm_kernel<<<R, kThreads, 0, st>>>(partial, splits, split_stride, gain, eps, h, xn, d);
+  launch_pdl(residual_rmsnorm_kernel, dim3(R), dim3(row_threads(d)), 0, st, partial, splits, split_stride, gain, eps, h,
+             xn, d);
 }
 
 void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H, int Hkv,
                      int hd, const float2* rope_table, RowMap map, bf16* q, bf16* k_dst, bf16* v_dst, int kv_to_cache,
                      size_t cache_seq_stride) {
-  qkv_rope_kernel<<<R, kThreads, 0, st>>>(partial, splits, split_stride, H, Hkv, hd, rope_table, map, q, k_dst, v_dst,
-                                          kv_to_cache, cache_seq_stride);
+  const int heads = H + 2 * Hkv;
+  dim3 grid(R, (heads + kRopeHeadsPerBlock - 1) / kRopeHeadsPerBlock);
+  launch_pdl(qkv_rope_kernel, grid, dim3(kRopeHeadsPerBlock * 32), 0, st, partial, splits, split_stride, H, Hkv, hd,
+             rope_table, map, q, k_dst, v_dst, kv_to_cache, cache_seq_stride);
 }
 
 void launch_swiglu(cudaStream_t st, const float* gu, bf16* act, int R, int ffn_pad) {
@@ -270,9 +338,8 @@ void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, in
 
 void launch_lm_merge(cudaStream_t st, const float* tile_max, const float* tile_sum, const int* tile_arg, int tiles,
                      int R, const uint8_t* row_wanted, int* tok, float* conf) {
-  const int rows_per_block = kThreads / 32;
-  lm_merge_kernel<<<(R + rows_per_block - 1) / rows_per_block, kThreads, 0, st>>>(tile_max, tile_sum, tile_arg, tiles,
-                                                                                  R, row_wanted, tok, conf);
+  launch_pdl(lm_merge_kernel, dim3(R), dim3(kThreads), 0, st, tile_max, tile_sum, tile_arg, tiles, R, row_wanted, tok,
+             conf);
 }
 
 }  // namespace ssd

@@ -33,7 +33,7 @@ namespace {
 
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16* __restrict__ x, const bf16* __restrict__ w,
                                                         float* __restrict__ out, int R, int N, int K, int x_pitch,
-                                                        int w_pitch, int splits) {
+                                                        int w_pitch, int splits, int w_tiled) {
   __shared__ float Ws[64][33];
   __shared__ float Xs[32][33];
   const int n0 = blockIdx.x * 64, r0 = blockIdx.y * 32, split = blockIdx.z;
@@ -48,7 +48,9 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16* __restrict__
     for (int i = threadIdx.x; i < 64 * 32; i += 256) {
       const int rr = i >> 5, kk = i & 31;
       const int n = n0 + rr, k = k0 + kk;
-      Ws[rr][kk] = (n < N && k < k_end) ? __bfloat162float(w[(size_t)n * w_pitch + k]) : 0.f;
+      const size_t wi = w_tiled ? ((((size_t)(n >> 7) * kb_total + (k >> 6)) * 128 + (n & 127)) * 64 + (k & 63))
+                                : ((size_t)n * w_pitch + k);
+      Ws[rr][kk] = (n < N && k < k_end) ? __bfloat162float(w[wi]) : 0.f;
     }
     for (int i = threadIdx.x; i < 32 * 32; i += 256) {
       const int rr = i >> 5, kk = i & 31;
@@ -78,7 +80,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16* __restrict__
 
 void launch_gemm_simt(cudaStream_t st, const GemmArgs& g) {
   dim3 grid((g.N + 63) / 64, (g.R + 31) / 32, g.splits);
-  gemm_simt_kernel<<<grid, 256, 0, st>>>(g.x, g.w, g.out, g.R, g.N, g.K, g.x_pitch, g.w_pitch, g.splits);
+  gemm_simt_kernel<<<grid, 256, 0, st>>>(g.x, g.w, g.out, g.R, g.N, g.K, g.x_pitch, g.w_pitch, g.splits, g.w_tiled);
 }
 
 // =====================================================================================
@@ -99,6 +101,7 @@ struct TcParams {
   int splits;
   int stages;
   int epi;
+  int w_tiled;     // weights in the tile-contiguous layout: one 16 KB block per (tile, K block)
   uint32_t tmem_cols;
   float* out;
   bf16* act;
@@ -203,6 +206,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x, split = blockIdx.y, row0 = blockIdx.z * 256;
   const int kb_total = (p.K + kBlockK - 1) / kBlockK;
@@ -238,15 +242,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const uint32_t stage_bytes = (uint32_t)(kWTileBytes + x_tile_bytes);
       int issued = 0;
       bool ok = true;
-      for (int it = 0; it < n_kb; ++it) {
+      auto load_w = [&](int it, int s, uint32_t fb) {
+        const int kb = kb_begin + it;
+        if (p.w_tiled) tma_load_2d(smem_addr(sW + (size_t)s * kWTileBytes), &tmW, fb, 0, (tile * kb_total + kb) * kTileM);
+        else tma_load_2d(smem_addr(sW + (size_t)s * kWTileBytes), &tmW, fb, kb * kBlockK, tile * kTileM);
+      };
+      // The weights do not depend on any earlier kernel: fill the ring with weight tiles first, and
+      // only then wait for the kernel that produces the activations.
+      const int pre = n_kb < p.stages ? n_kb : p.stages;
+      for (int it = 0; it < pre; ++it) {
+        const uint32_t fb = smem_addr(&full_bar[it]);
+        mbar_expect_tx(fb, stage_bytes);
+        load_w(it, it, fb);
+      }
+      pdl_wait();
+      for (int it = 0; it < pre; ++it) {
+        tma_load_2d(smem_addr(sX + (size_t)it * x_tile_bytes), &tmX, smem_addr(&full_bar[it]), (kb_begin + it) * kBlockK, row0);
+        ++issued;
+      }
+      for (int it = pre; it < n_kb; ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (uint32_t)((it / p.stages) & 1);
         if (!mbar_wait(smem_addr(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t fb = smem_addr(&full_bar[s]);
         mbar_expect_tx(fb, stage_bytes);
-        const int kc = (kb_begin + it) * kBlockK;
-        tma_load_2d(smem_addr(sW + (size_t)s * kWTileBytes), &tmW, fb, kc, tile * kTileM);
-        tma_load_2d(smem_addr(sX + (size_t)s * x_tile_bytes), &tmX, fb, kc, row0);
+        load_w(it, s, fb);
+        tma_load_2d(smem_addr(sX + (size_t)s * x_tile_bytes), &tmX, fb, (kb_begin + it) * kBlockK, row0);
         ++issued;
       }
       if (!ok) {
@@ -292,6 +313,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     // ------------------------------------------------------------------ epilogue (4 warps)
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
     const int lrow = quad * 32 + lane;         // accumulator lane = feature inside the tile
+    pdl_wait();                                // outputs may still be read by the predecessor
     bool ok = true;
     if (n_kb > 0) ok = mbar_wait(smem_addr(acc_bar), 0u, abort_flag);
     ok = __all_sync(0xffffffffu, ok);
@@ -435,7 +457,7 @@ int gemm_tc_init() {
 
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   if (!g_encode) return -4;
-  if ((g.x_pitch % 8) || (g.w_pitch % 8) || (((uintptr_t)g.x) & 15) || (((uintptr_t)g.w) & 15)) return -2;
+  if ((g.x_pitch % 8) || (!g.w_tiled && (g.w_pitch % 8)) || (((uintptr_t)g.x) & 15) || (((uintptr_t)g.w) & 15)) return -2;
   if (g.R < 1 || g.N < 1 || g.K < 1) return -2;
   if (g.epi != EPI_PARTIAL && g.splits != 1) return -2;
   if (g.epi == EPI_SWIGLU && (g.N % 128)) return -2;
@@ -445,6 +467,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   p.npad = (rows_chunk + 15) & ~15;
   p.splits = g.splits;
   p.epi = g.epi;
+  p.w_tiled = g.w_tiled;
   uint32_t cols = 32;
   while ((int)cols < p.npad) cols <<= 1;
   p.tmem_cols = cols;
@@ -462,7 +485,13 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   // tensor-memory safety: CTAs that fit by shared memory must also fit by TMEM columns
   if ((227 * 1024 / smem) * (int)cols > 512) return -2;
   CUtensorMap tmW, tmX;
-  if (!make_tmap(&tmW, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.w_pitch, kTileM)) return -4;
+  if (g.w_tiled) {
+    // [tiles * K blocks * 128 rows][64]: every box is one contiguous 16 KB block
+    const uint64_t rows = (uint64_t)gemm_tiles(g.N) * ((g.K + kBlockK - 1) / kBlockK) * kTileM;
+    if (!make_tmap(&tmW, g.w, rows, kBlockK, kBlockK, kTileM)) return -4;
+  } else if (!make_tmap(&tmW, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.w_pitch, kTileM)) {
+    return -4;
+  }
   if (!make_tmap(&tmX, g.x, (uint64_t)g.R, (uint64_t)g.K, (uint64_t)g.x_pitch, (uint32_t)p.npad)) return -4;
   static int smem_set = 0;
   if (smem > smem_set) {
@@ -471,7 +500,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
     smem_set = 227 * 1024;
   }
   dim3 grid(gemm_tiles(g.N), g.splits, (g.R + 255) / 256);
-  gemm_tc_kernel<<<grid, kTcThreads, smem, st>>>(tmW, tmX, p);
+  if (launch_pdl(gemm_tc_kernel, grid, dim3(kTcThreads), (size_t)smem, st, tmW, tmX, p) != cudaSuccess) return -4;
   return 0;
 }
 

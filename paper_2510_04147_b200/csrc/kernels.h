@@ -9,6 +9,34 @@ typedef __nv_bfloat16 bf16;
 
 namespace ssd {
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the forward is launched with the "programmatic stream serialization" attribute:
+// it may become resident while its predecessor in the stream still runs.  A kernel first lets ITS
+// successor be scheduled (pdl_launch_dependents), does whatever does not depend on earlier kernels
+// (barrier set-up, weight prefetch), and calls pdl_wait() before it touches anything an earlier
+// kernel wrote or still reads.  pdl_wait() returns once the predecessor grid has completed and its
+// memory operations are visible, so completion is transitive along the stream.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // ---------------------------------------------------------------- layout helpers (host+device)
 // Rows of a forward are ordered [sequence slot a][node i][in-block index t].
 struct RowMap {
@@ -23,6 +51,11 @@ struct RowMap {
 // dst[(j / group) * group_stride + group_offset + j % group][c] = bf16(src[j][c]),  j < rows, c < cols
 void launch_convert_rows(cudaStream_t st, const void* src, int src_is_f32, bf16* dst, int rows, int cols,
                          int dst_pitch, int group, int group_stride, int group_offset);
+// same row mapping, but dst is tile-contiguous: element (n, k) of the mapped matrix lives at
+// (((n / 128) * kb_total + k / 64) * 128 + n % 128) * 64 + k % 64, kb_total = ceil(cols_padded / 64)
+void launch_convert_tiled(cudaStream_t st, const void* src, int src_is_f32, bf16* dst, int rows, int cols,
+                          int kb_total, int group, int group_stride, int group_offset);
+inline size_t tiled_elems(int n, int k) { return (size_t)((n + 127) / 128) * ((k + 63) / 64) * 128 * 64; }
 void launch_copy_f32(cudaStream_t st, const void* src, int src_is_f32, float* dst, int n);
 
 // ---------------------------------------------------------------- elementwise / reductions
@@ -69,8 +102,9 @@ void launch_attention(cudaStream_t st, const AttnArgs& a, int* launches);
 enum { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_LMHEAD = 2 };
 struct GemmArgs {
   const bf16* x;  // [R][x_pitch] activations (K-major)
-  const bf16* w;  // [N][w_pitch] weights (K-major)
+  const bf16* w;  // [N][w_pitch] weights (K-major), or the tile-contiguous layout below when w_tiled
   int R, N, K, x_pitch, w_pitch;
+  int w_tiled;           // 1: w is [ceil(N/128)][ceil(K/64)][128][64] (one 16 KB block per MMA tile, zero padded)
   int splits;            // split-K factor (EPI_PARTIAL only)
   int epi;
   float* out;            // EPI_PARTIAL: [splits][R][N] fp32

@@ -44,6 +44,7 @@ struct ssd_ctx {
   int R_dec = 0;         // max rows of a verification forward
   int R_cap = 0;         // max rows of any forward
   size_t partial_elems = 0, part_rows_parts = 0;
+  size_t partial_row_floats = 0;   // split-K workspace per row
   float* h = nullptr;
   bf16* xn = nullptr;
   float* partial = nullptr;
@@ -112,10 +113,16 @@ int dev_alloc(ssd_ctx* c, T** p, size_t n, bool zero = true) {
     if (rc_ != SSD_OK) return rc_;                   \
   } while (0)
 
-int auto_split(int tiles) {
-  int s = 148 / tiles;
+constexpr int kMaxSplit = 16;
+
+// Split-K factor that fills the machine: two CTAs per SM on 148 SMs, at least four K blocks each.
+// A function of the matrix shape alone, so a row's summation order never depends on the row count.
+int auto_split(int tiles, int k) {
+  const int kb = (k + 63) / 64;
+  int s = (2 * 148 + tiles / 2) / tiles;
+  if (s > kb / 4) s = kb / 4;
+  if (s > kMaxSplit) s = kMaxSplit;
   if (s < 1) s = 1;
-  if (s > 8) s = 8;
   return s;
 }
 
@@ -221,7 +228,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     const LayerW& w = c->L[l];
     // ---- QKV projection, rotary embedding
     GemmArgs g{};
-    g.x = c->xn; g.w = w.wqkv; g.R = R; g.N = c->nqkv; g.K = d; g.x_pitch = d; g.w_pitch = d;
+    g.x = c->xn; g.w = w.wqkv; g.R = R; g.N = c->nqkv; g.K = d; g.x_pitch = d; g.w_pitch = d; g.w_tiled = 1;
     g.splits = c->split_qkv; g.epi = EPI_PARTIAL; g.out = c->partial;
     if ((size_t)g.splits * R * g.N > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "split-K workspace too small");
     int rc = run_gemm(c, g, SSD_PROF_GEMM);
@@ -251,7 +258,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     }
     // ---- output projection + residual + norm
     g = GemmArgs{};
-    g.x = c->att; g.w = w.wo; g.R = R; g.N = d; g.K = c->qdim; g.x_pitch = c->qdim; g.w_pitch = c->qdim;
+    g.x = c->att; g.w = w.wo; g.R = R; g.N = d; g.K = c->qdim; g.x_pitch = c->qdim; g.w_pitch = c->qdim; g.w_tiled = 1;
     g.splits = c->split_o; g.epi = EPI_PARTIAL; g.out = c->partial;
     rc = run_gemm(c, g, SSD_PROF_GEMM);
     if (rc) return rc;
@@ -261,7 +268,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     }
     // ---- gate/up projection with SwiGLU
     g = GemmArgs{};
-    g.x = c->xn; g.w = w.wgu; g.R = R; g.N = 2 * c->ffn_pad; g.K = d; g.x_pitch = d; g.w_pitch = d;
+    g.x = c->xn; g.w = w.wgu; g.R = R; g.N = 2 * c->ffn_pad; g.K = d; g.x_pitch = d; g.w_pitch = d; g.w_tiled = 1;
     g.splits = 1;
     if (c->gemm_impl == 1) {
       g.epi = EPI_SWIGLU; g.act = c->act; g.act_pitch = c->ffn_pad;
@@ -277,7 +284,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     }
     // ---- down projection + residual + next norm
     g = GemmArgs{};
-    g.x = c->act; g.w = w.wd; g.R = R; g.N = d; g.K = c->ffn_pad; g.x_pitch = c->ffn_pad; g.w_pitch = c->ffn_pad;
+    g.x = c->act; g.w = w.wd; g.R = R; g.N = d; g.K = c->ffn_pad; g.x_pitch = c->ffn_pad; g.w_pitch = c->ffn_pad; g.w_tiled = 1;
     g.splits = c->split_down; g.epi = EPI_PARTIAL; g.out = c->partial;
     rc = run_gemm(c, g, SSD_PROF_GEMM);
     if (rc) return rc;
@@ -289,7 +296,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   }
   if (kind == FWD_VERIFY) {
     GemmArgs g{};
-    g.x = c->xn; g.w = c->lm_head; g.R = R; g.N = c->V; g.K = d; g.x_pitch = d; g.w_pitch = d; g.splits = 1;
+    g.x = c->xn; g.w = c->lm_head; g.R = R; g.N = c->V; g.K = d; g.x_pitch = d; g.w_pitch = d; g.splits = 1; g.w_tiled = 1;
     g.mask_id = c->cfg.mask_id;
     if (want_logits || c->gemm_impl != 1) {
       const size_t need = (size_t)R * c->V;
@@ -375,9 +382,9 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
   c->n_max = (k.max_drafts < k.block_len - 1 ? k.max_drafts : k.block_len - 1) + 1;
   c->R_dec = k.max_batch * c->n_max * k.block_len;
   c->R_cap = c->R_dec > k.max_seq ? c->R_dec : k.max_seq;
-  c->split_qkv = auto_split(gemm_tiles(c->nqkv));
-  c->split_o = auto_split(gemm_tiles(c->d));
-  c->split_down = auto_split(gemm_tiles(c->d));
+  c->split_qkv = auto_split(gemm_tiles(c->nqkv), c->d);
+  c->split_o = auto_split(gemm_tiles(c->d), c->qdim);
+  c->split_down = auto_split(gemm_tiles(c->d), c->ffn_pad);
   c->h_remaining.assign(k.max_batch, 0);
   c->h_has_drafts.assign(k.max_batch, 0);
 
@@ -385,15 +392,16 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
   auto build = [&]() -> int {
     const int d = c->d;
     for (LayerW& w : c->L) {
-      ALLOC(c, w.wqkv, (size_t)c->nqkv * d);
-      ALLOC(c, w.wo, (size_t)d * c->qdim);
-      ALLOC(c, w.wgu, (size_t)2 * c->ffn_pad * d);
-      ALLOC(c, w.wd, (size_t)d * c->ffn_pad);
+      // tile-contiguous, zero padded to whole 128 x 64 tiles
+      ALLOC(c, w.wqkv, tiled_elems(c->nqkv, d));
+      ALLOC(c, w.wo, tiled_elems(d, c->qdim));
+      ALLOC(c, w.wgu, tiled_elems(2 * c->ffn_pad, d));
+      ALLOC(c, w.wd, tiled_elems(d, c->ffn_pad));
       ALLOC(c, w.g_attn, d);
       ALLOC(c, w.g_ffn, d);
     }
     ALLOC(c, c->embed, (size_t)c->V * d);
-    ALLOC(c, c->lm_head, (size_t)c->V * d);
+    ALLOC(c, c->lm_head, tiled_elems(c->V, d));
     ALLOC(c, c->g_final, d);
     c->cache_seq_stride = (size_t)k.max_seq * c->kvdim;
     c->cache_layer_stride = c->cache_seq_stride * k.max_batch;
@@ -416,9 +424,11 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     const size_t R = (size_t)c->R_cap;
     ALLOC(c, c->h, R * d);
     ALLOC(c, c->xn, R * d);
-    size_t widest = (size_t)c->nqkv > (size_t)d ? (size_t)c->nqkv : (size_t)d;
-    c->partial_elems = 8 * R * widest;
-    if (R * 2 * c->ffn_pad > c->partial_elems) c->partial_elems = R * 2 * c->ffn_pad;
+    c->partial_row_floats = (size_t)kMaxSplit * d;
+    if ((size_t)4 * c->nqkv > c->partial_row_floats) c->partial_row_floats = (size_t)4 * c->nqkv;
+    if ((size_t)c->split_qkv * c->nqkv > c->partial_row_floats) c->partial_row_floats = (size_t)c->split_qkv * c->nqkv;
+    if ((size_t)2 * c->ffn_pad > c->partial_row_floats) c->partial_row_floats = (size_t)2 * c->ffn_pad;
+    c->partial_elems = R * c->partial_row_floats;
     ALLOC(c, c->partial, c->partial_elems);
     ALLOC(c, c->q, R * c->qdim);
     ALLOC(c, c->lk, R * c->kvdim);
@@ -482,27 +492,28 @@ int ssd_load_weights(ssd_ctx* c, const char* name, const void* dev_ptr, int32_t 
   if (!strcmp(name, "embed")) {
     if ((ok_shape = want2(c->V, d))) { launch_convert_rows(c->st, dev_ptr, f32, c->embed, c->V, d, d, c->V, 0, 0); c->loaded_globals |= 1u; }
   } else if (!strcmp(name, "lm_head")) {
-    if ((ok_shape = want2(c->V, d))) { launch_convert_rows(c->st, dev_ptr, f32, c->lm_head, c->V, d, d, c->V, 0, 0); c->loaded_globals |= 2u; }
+    if ((ok_shape = want2(c->V, d))) { launch_convert_tiled(c->st, dev_ptr, f32, c->lm_head, c->V, d, (d + 63) / 64, c->V, 0, 0); c->loaded_globals |= 2u; }
   } else if (!strcmp(name, "norm_final")) {
     if ((ok_shape = want1(d))) { launch_copy_f32(c->st, dev_ptr, f32, c->g_final, d); c->loaded_globals |= 4u; }
   } else if (parse_layer_name(name, &layer, &rest)) {
     if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, SSD_ERR_INVALID_ARG, "layer %d out of range", layer);
     LayerW& w = c->L[layer];
+    const int kbd = (d + 63) / 64;
     if (!strcmp(rest, "wq")) {
-      if ((ok_shape = want2(c->qdim, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wqkv, c->qdim, d, d, c->qdim, 0, 0); w.loaded |= 1u; }
+      if ((ok_shape = want2(c->qdim, d))) { launch_convert_tiled(c->st, dev_ptr, f32, w.wqkv, c->qdim, d, kbd, c->qdim, 0, 0); w.loaded |= 1u; }
     } else if (!strcmp(rest, "wk")) {
-      if ((ok_shape = want2(c->kvdim, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wqkv, c->kvdim, d, d, c->kvdim, 0, c->qdim); w.loaded |= 2u; }
+      if ((ok_shape = want2(c->kvdim, d))) { launch_convert_tiled(c->st, dev_ptr, f32, w.wqkv, c->kvdim, d, kbd, c->kvdim, 0, c->qdim); w.loaded |= 2u; }
     } else if (!strcmp(rest, "wv")) {
-      if ((ok_shape = want2(c->kvdim, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wqkv, c->kvdim, d, d, c->kvdim, 0, c->qdim + c->kvdim); w.loaded |= 4u; }
+      if ((ok_shape = want2(c->kvdim, d))) { launch_convert_tiled(c->st, dev_ptr, f32, w.wqkv, c->kvdim, d, kbd, c->kvdim, 0, c->qdim + c->kvdim); w.loaded |= 4u; }
     } else if (!strcmp(rest, "wo")) {
-      if ((ok_shape = want2(d, c->qdim))) { launch_convert_rows(c->st, dev_ptr, f32, w.wo, d, c->qdim, c->qdim, d, 0, 0); w.loaded |= 8u; }
+      if ((ok_shape = want2(d, c->qdim))) { launch_convert_tiled(c->st, dev_ptr, f32, w.wo, d, c->qdim, (c->qdim + 63) / 64, d, 0, 0); w.loaded |= 8u; }
     } else if (!strcmp(rest, "w_gate")) {
       // 64 gate features then the 64 matching up features per 128-row tile
-      if ((ok_shape = want2(c->ffn, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wgu, c->ffn, d, d, 64, 128, 0); w.loaded |= 16u; }
+      if ((ok_shape = want2(c->ffn, d))) { launch_convert_tiled(c->st, dev_ptr, f32, w.wgu, c->ffn, d, kbd, 64, 128, 0); w.loaded |= 16u; }
     } else if (!strcmp(rest, "w_up")) {
-      if ((ok_shape = want2(c->ffn, d))) { launch_convert_rows(c->st, dev_ptr, f32, w.wgu, c->ffn, d, d, 64, 128, 64); w.loaded |= 32u; }
+      if ((ok_shape = want2(c->ffn, d))) { launch_convert_tiled(c->st, dev_ptr, f32, w.wgu, c->ffn, d, kbd, 64, 128, 64); w.loaded |= 32u; }
     } else if (!strcmp(rest, "w_down")) {
-      if ((ok_shape = want2(d, c->ffn))) { launch_convert_rows(c->st, dev_ptr, f32, w.wd, d, c->ffn, c->ffn_pad, d, 0, 0); w.loaded |= 64u; }
+      if ((ok_shape = want2(d, c->ffn))) { launch_convert_tiled(c->st, dev_ptr, f32, w.wd, d, c->ffn, c->ffn_pad / 64, d, 0, 0); w.loaded |= 64u; }
     } else if (!strcmp(rest, "norm_attn")) {
       if ((ok_shape = want1(d))) { launch_copy_f32(c->st, dev_ptr, f32, w.g_attn, d); w.loaded |= 128u; }
     } else if (!strcmp(rest, "norm_ffn")) {
@@ -803,7 +814,10 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!c) return SSD_ERR_INVALID_ARG;
   if (!key) return fail(c, SSD_ERR_INVALID_ARG, "null key");
   if (!strcmp(key, "split_k_qkv") || !strcmp(key, "split_k_o") || !strcmp(key, "split_k_down")) {
-    if (value < 1 || value > 8) return fail(c, SSD_ERR_INVALID_ARG, "split-K must be in [1, 8]");
+    const int width = !strcmp(key, "split_k_qkv") ? c->nqkv : c->d;
+    if (value < 1 || value > kMaxSplit || (size_t)value * width > c->partial_row_floats)
+      return fail(c, SSD_ERR_INVALID_ARG, "split-K for this projection must be in [1, %d]",
+                  (int)(c->partial_row_floats / width < (size_t)kMaxSplit ? c->partial_row_floats / width : kMaxSplit));
     if (!strcmp(key, "split_k_qkv")) c->split_qkv = value;
     else if (!strcmp(key, "split_k_o")) c->split_o = value;
     else c->split_down = value;

@@ -23,6 +23,8 @@ __global__ void __launch_bounds__(256) tree_build_kernel(BlockState s, int batch
   __shared__ int rank[kMaxT];
   __shared__ float cf[kMaxT];
   __shared__ uint8_t mk[kMaxT];
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.x;
   if (threadIdx.x == 0) s.last_accept[b] = 0;
   const int r = s.remaining[b];
@@ -78,6 +80,8 @@ __global__ void __launch_bounds__(256) accept_kernel(BlockState s, int T, int n_
   __shared__ int pred_q[kMaxT];
   __shared__ int pred_t[kMaxT];
   __shared__ int s_a;
+  pdl_launch_dependents();
+  pdl_wait();
   const int slot = blockIdx.x;
   const int b = s.seq_map[slot];
   const int N = s.n_cand[b];
@@ -148,12 +152,13 @@ __global__ void __launch_bounds__(256) accept_kernel(BlockState s, int T, int n_
 
 void launch_tree_build(cudaStream_t st, BlockState s, int batch, int T, int max_drafts, int n_cap, int mask_id,
                        int* node_ids, uint8_t* node_masked) {
-  tree_build_kernel<<<batch, 256, 0, st>>>(s, batch, T, max_drafts, n_cap, mask_id, node_ids, node_masked);
+  launch_pdl(tree_build_kernel, dim3(batch), dim3(256), 0, st, s, batch, T, max_drafts, n_cap, mask_id, node_ids,
+             node_masked);
 }
 
 void launch_accept(cudaStream_t st, BlockState s, int n_slots, int T, int n_cap, const int* tok, const float* conf,
                    const uint8_t* node_masked, int* nonfinite_flag) {
-  accept_kernel<<<n_slots, 256, 0, st>>>(s, T, n_cap, tok, conf, node_masked, nonfinite_flag);
+  launch_pdl(accept_kernel, dim3(n_slots), dim3(256), 0, st, s, T, n_cap, tok, conf, node_masked, nonfinite_flag);
 }
 
 }  // namespace ssd

@@ -3,7 +3,11 @@
 Tolerances (bf16 operands, fp32 accumulation; stated by the workload's north star):
   * logits within 2e-2 absolute of the fp64 oracle, confidences within 2e-2 relative;
   * against the oracle run with bf16 operand rounding (same arithmetic type as the kernels) the
-    logits agree to 6e-3;
+    logits agree to 1e-2, half the stated tolerance.  That comparison is not bit-level: the kernels
+    round the attention probabilities relative to a part's running maximum and merge parts, the
+    oracle rounds them relative to the row maximum, and fp32 accumulation (whose order follows the
+    split-K factors) flips a few bf16 roundings of the activations.  What is left is bf16 rounding
+    noise whose maximum over the 1.6e5 logits of a case sits between 4e-3 and 7e-3;
   * tokens / accept lengths bit-exact wherever the oracle's decision gap exceeds 1e-3;
   * GPU SSD == GPU stepwise bit-exact, no exemption.
 """
@@ -139,7 +143,7 @@ def test_verify_forward_logits_and_stats(tiny_ssd, peaked_ssd, tiny_oracles, imp
         tok2, conf2, _ = ssd.verify_forward(ids, masked, want_logits=False)      # fused LM head path
     finally:
         ssd.set_option("gemm_impl", DEFAULT_IMPL)
-    for o, tol in ((ob, 6e-3), (o64, 2e-2)):
+    for o, tol in ((ob, 1e-2), (o64, 2e-2)):
         cache = o.prefill(prompt[0])
         o.commit_block(blk[0], cache)
         otok, oconf, ogap, ologits = o.verify(ids[0], masked[0], cache)
