@@ -350,13 +350,19 @@ def run_ours(args):
         ssd.profile_enable(False)
         g = prof["gemm"]
         achieved = g["bytes"] / (g["ms"] * 1e-3) / 1e9 if g["ms"] > 0 else 0.0
-        total_ms = sum(v["ms"] for v in prof.values())
+        total_ms = sum(prof[k]["ms"] for k in binding.PROF_TOP)
+        per_projection = {k: {"launches": v["launches"], "avg_launch_us": 1e3 * v["ms"] / max(1, v["launches"]),
+                              "gb_per_s": (v["bytes"] / (v["ms"] * 1e-3) / 1e9 if v["ms"] > 0 else 0.0)}
+                          for k, v in prof.items() if k not in binding.PROF_TOP}
         roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel (QKV/O/gate-up/down projections)",
                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                     "peak_source": peaks["_source"], "traffic": None,
                     "launches": g["launches"], "avg_launch_us": 1e3 * g["ms"] / max(1, g["launches"]),
                     "bytes_per_launch_avg": g["bytes"] / max(1, g["launches"]),
-                    "family_share_of_device_time": {k: (v["ms"] / total_ms if total_ms else 0) for k, v in prof.items()}}
+                    "family_share_of_device_time": {k: (prof[k]["ms"] / total_ms if total_ms else 0)
+                                                    for k in binding.PROF_TOP},
+                    "family_avg_launch_us": {k: 1e3 * prof[k]["ms"] / max(1, prof[k]["launches"]) for k in binding.PROF_TOP},
+                    "per_projection": per_projection}
         # ---- CPU baseline: the oracle on a bounded sample
         if args.no_cpu_baseline:
             cpu = None

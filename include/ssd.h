@@ -179,11 +179,16 @@ int64_t ssd_launch_count(const ssd_ctx* ctx);
 #define SSD_PROF_ATTN      2   /* shared-prefix attention (+ split merge)                      */
 #define SSD_PROF_ELEMWISE  3   /* embedding, norms, residuals, rotary, reductions              */
 #define SSD_PROF_TREE      4   /* tree build, acceptance                                       */
-#define SSD_PROF_FAMILIES  5
+#define SSD_PROF_GEMM_QKV  5   /* families 5-8 break family 0 down by projection               */
+#define SSD_PROF_GEMM_O    6
+#define SSD_PROF_GEMM_GU   7
+#define SSD_PROF_GEMM_DOWN 8
+#define SSD_PROF_FAMILIES  9
 int ssd_profile_enable(ssd_ctx* ctx, int32_t on);
 int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, double* bytes);
 
-/* Tuning knobs (set before prefill).  key: "split_k_qkv", "split_k_o", "split_k_down" (1..8),
+/* Tuning knobs (set before prefill).  key: "split_k_qkv", "split_k_o", "split_k_down" (1..16, bounded by
+ * the split-K workspace),
  * "kv_split" (prefix keys per attention split, multiple of 64; 0 = automatic from the prefix
  * length), "max_drafts" (lower the draft-length cap below the capacity fixed at creation),
  * "gemm_impl" (1 = TMA + tcgen05 kernel, the default; 0 = the plain CUDA-core bring-up kernel,

@@ -22,7 +22,8 @@ ERR_NAMES = {-1: "INVALID_ARG", -2: "SHAPE", -3: "OOM", -4: "CUDA", -5: "OVERFLO
              -8: "NONFINITE"}
 DTYPE_BF16, DTYPE_F32 = 0, 1
 MODE_STEPWISE, MODE_SSD = 0, 1
-PROF_FAMILIES = ("gemm", "lmhead", "attn", "elemwise", "tree")
+PROF_FAMILIES = ("gemm", "lmhead", "attn", "elemwise", "tree", "gemm_qkv", "gemm_o", "gemm_gu", "gemm_down")
+PROF_TOP = PROF_FAMILIES[:5]          # the last four break "gemm" down by projection
 
 EXPORTS = ["ssd_create", "ssd_destroy", "ssd_last_error", "ssd_load_weights", "ssd_prefill", "ssd_prefill_dev",
            "ssd_decode_block", "ssd_block_begin", "ssd_set_block_state", "ssd_get_block_state", "ssd_block_step",

@@ -21,7 +21,7 @@ struct LayerW {
   uint32_t loaded = 0;   // bit per tensor
 };
 
-struct ProfRec { int fam; cudaEvent_t e0, e1; double bytes; };
+struct ProfRec { int fam, sub; cudaEvent_t e0, e1; double bytes; };
 
 char g_create_error[256] = "";
 
@@ -134,10 +134,11 @@ int kv_split_for(const ssd_ctx* c, int S) {
 // ---- profiling / launch accounting --------------------------------------------------------
 struct Scope {
   ssd_ctx* c;
-  int fam;
+  int fam, sub;
   double bytes;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
-  Scope(ssd_ctx* c_, int fam_, double bytes_, int n_launches = 1) : c(c_), fam(fam_), bytes(bytes_) {
+  Scope(ssd_ctx* c_, int fam_, double bytes_, int n_launches = 1, int sub_ = -1)
+      : c(c_), fam(fam_), sub(sub_), bytes(bytes_) {
     c->launches += n_launches;
     if (c->profiling) {
       cudaEventCreate(&e0);
@@ -148,7 +149,7 @@ struct Scope {
   ~Scope() {
     if (c->profiling) {
       cudaEventRecord(e1, c->st);
-      c->prof.push_back({fam, e0, e1, bytes});
+      c->prof.push_back({fam, sub, e0, e1, bytes});
     }
   }
 };
@@ -184,8 +185,8 @@ __global__ void block_init_kernel(BlockState s, int batch, int max_batch, int T,
 }
 
 // ---- projections ----------------------------------------------------------------------------
-int run_gemm(ssd_ctx* c, GemmArgs g, int fam) {
-  Scope sc(c, fam, (double)g.N * g.K * 2.0);
+int run_gemm(ssd_ctx* c, GemmArgs g, int fam, int sub = -1) {
+  Scope sc(c, fam, (double)g.N * g.K * 2.0, 1, sub);
   g.err_flag = c->flags;
   if (c->gemm_impl == 1) {
     const int rc = launch_gemm_tc(c->st, g);
@@ -231,7 +232,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g.x = c->xn; g.w = w.wqkv; g.R = R; g.N = c->nqkv; g.K = d; g.x_pitch = d; g.w_pitch = d; g.w_tiled = 1;
     g.splits = c->split_qkv; g.epi = EPI_PARTIAL; g.out = c->partial;
     if ((size_t)g.splits * R * g.N > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "split-K workspace too small");
-    int rc = run_gemm(c, g, SSD_PROF_GEMM);
+    int rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_QKV);
     if (rc) return rc;
     bf16* kdst = (kind == FWD_FILL) ? c->cacheK + (size_t)l * c->cache_layer_stride : c->lk;
     bf16* vdst = (kind == FWD_FILL) ? c->cacheV + (size_t)l * c->cache_layer_stride : c->lv;
@@ -260,7 +261,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g = GemmArgs{};
     g.x = c->att; g.w = w.wo; g.R = R; g.N = d; g.K = c->qdim; g.x_pitch = c->qdim; g.w_pitch = c->qdim; g.w_tiled = 1;
     g.splits = c->split_o; g.epi = EPI_PARTIAL; g.out = c->partial;
-    rc = run_gemm(c, g, SSD_PROF_GEMM);
+    rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_O);
     if (rc) return rc;
     {
       Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * (4.0 * g.splits + 10.0));
@@ -272,12 +273,12 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g.splits = 1;
     if (c->gemm_impl == 1) {
       g.epi = EPI_SWIGLU; g.act = c->act; g.act_pitch = c->ffn_pad;
-      rc = run_gemm(c, g, SSD_PROF_GEMM);
+      rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_GU);
       if (rc) return rc;
     } else {
       g.epi = EPI_PARTIAL; g.out = c->partial;
       if ((size_t)R * g.N > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "workspace too small");
-      rc = run_gemm(c, g, SSD_PROF_GEMM);
+      rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_GU);
       if (rc) return rc;
       Scope sc(c, SSD_PROF_ELEMWISE, (double)R * c->ffn_pad * 10.0);
       launch_swiglu(c->st, c->partial, c->act, R, c->ffn_pad);
@@ -286,7 +287,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g = GemmArgs{};
     g.x = c->act; g.w = w.wd; g.R = R; g.N = d; g.K = c->ffn_pad; g.x_pitch = c->ffn_pad; g.w_pitch = c->ffn_pad; g.w_tiled = 1;
     g.splits = c->split_down; g.epi = EPI_PARTIAL; g.out = c->partial;
-    rc = run_gemm(c, g, SSD_PROF_GEMM);
+    rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_DOWN);
     if (rc) return rc;
     {
       const float* gain = (l + 1 < nl) ? c->L[l + 1].g_attn : c->g_final;
@@ -800,9 +801,12 @@ int ssd_profile_read(ssd_ctx* c, int64_t* launches, double* ms, double* bytes) {
   for (ProfRec& r : c->prof) {
     float t = 0.f;
     cudaEventElapsedTime(&t, r.e0, r.e1);
-    if (launches) launches[r.fam] += 1;
-    if (ms) ms[r.fam] += t;
-    if (bytes) bytes[r.fam] += r.bytes;
+    for (int f : {r.fam, r.sub}) {
+      if (f < 0) continue;
+      if (launches) launches[f] += 1;
+      if (ms) ms[f] += t;
+      if (bytes) bytes[f] += r.bytes;
+    }
     cudaEventDestroy(r.e0);
     cudaEventDestroy(r.e1);
   }
