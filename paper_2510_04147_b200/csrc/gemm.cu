@@ -93,6 +93,7 @@ constexpr int kBlockK = 64;          // bf16 elements per stage along K = one 12
 constexpr int kTcThreads = 192;      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr int kMaxStages = 8;
 constexpr int kWTileBytes = kTileM * kBlockK * 2;
+constexpr int kEpiPitch = 132;       // floats per row of the epilogue's transpose buffer (128 + padding)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
 
 struct TcParams {
@@ -324,7 +325,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (!ok) {
       if (lane == 0) { *abort_flag = 1; atomicExch(p.err_flag, 3); }
     } else if (p.epi == EPI_PARTIAL) {
-      const int n = tile * kTileM + lrow;
+      // Transpose 32 rows x 128 features through shared memory so that a thread stores four
+      // consecutive features of one row: 8 vector stores per thread and chunk instead of 32 scalars.
+      const int n_base = tile * kTileM;
+      const bool vec_ok = ((p.N & 3) == 0) && (n_base + kTileM <= p.N);
+      const int et = threadIdx.x - 64;                 // 0..127 among the epilogue threads
       for (int c0 = 0; c0 < p.npad; c0 += 32) {
         float v[32];
         if (n_kb > 0) tmem_ld32(taddr + c0, v);
@@ -332,35 +337,57 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = 0.f;
         }
-        if (n < p.N) {
+        if (vec_ok) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int rr = c0 + j;
-            if (rr < rows_here) p.out[((size_t)split * p.R + row0 + rr) * p.N + n] = v[j];
+          for (int j = 0; j < 32; ++j) scratch[j * kEpiPitch + lrow] = v[j];
+          epi_bar_sync();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int rr = i * 4 + (et >> 5);          // row inside the chunk
+            const int f4 = (et & 31) * 4;              // first of four features
+            if (c0 + rr < rows_here) {
+              const float4 val = *reinterpret_cast<const float4*>(scratch + rr * kEpiPitch + f4);
+              *reinterpret_cast<float4*>(p.out + ((size_t)split * p.R + row0 + c0 + rr) * p.N + n_base + f4) = val;
+            }
+          }
+          epi_bar_sync();
+        } else {
+          const int n = n_base + lrow;
+          if (n < p.N) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int rr = c0 + j;
+              if (rr < rows_here) p.out[((size_t)split * p.R + row0 + rr) * p.N + n] = v[j];
+            }
           }
         }
       }
     } else if (p.epi == EPI_SWIGLU) {
-      // lanes 0-63 hold gate features, lanes 64-127 the matching up features
-      const int f = tile * 64 + (lrow & 63);
+      // lanes 0-63 hold gate features, lanes 64-127 the matching up features.  After the transpose a
+      // thread owns 16 consecutive features of one row: silu(gate) * up, 32 bytes of bf16 per thread.
+      const int et = threadIdx.x - 64;
+      const int rr = et >> 2, fg = (et & 3) * 16;
       for (int c0 = 0; c0 < p.npad; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + c0, v);
-        if (lrow >= 64) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) scratch[(lrow - 64) * 33 + j] = v[j];
-        }
+        for (int j = 0; j < 32; ++j) scratch[j * kEpiPitch + lrow] = v[j];
         epi_bar_sync();
-        if (lrow < 64) {
+        if (c0 + rr < rows_here) {
+          uint32_t packed[8];
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int rr = c0 + j;
-            if (rr < rows_here) {
-              const float u = scratch[lrow * 33 + j];
-              const float g = v[j];
-              p.act[(size_t)(row0 + rr) * p.act_pitch + f] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
-            }
+          for (int q4 = 0; q4 < 4; ++q4) {
+            const float4 g = *reinterpret_cast<const float4*>(scratch + rr * kEpiPitch + fg + q4 * 4);
+            const float4 u = *reinterpret_cast<const float4*>(scratch + rr * kEpiPitch + 64 + fg + q4 * 4);
+            const float a0 = g.x / (1.f + expf(-g.x)) * u.x, a1 = g.y / (1.f + expf(-g.y)) * u.y;
+            const float a2 = g.z / (1.f + expf(-g.z)) * u.z, a3 = g.w / (1.f + expf(-g.w)) * u.w;
+            __nv_bfloat162 lo = __floats2bfloat162_rn(a0, a1), hi = __floats2bfloat162_rn(a2, a3);
+            packed[q4 * 2] = *reinterpret_cast<uint32_t*>(&lo);
+            packed[q4 * 2 + 1] = *reinterpret_cast<uint32_t*>(&hi);
           }
+          uint4* dst = reinterpret_cast<uint4*>(p.act + (size_t)(row0 + c0 + rr) * p.act_pitch + tile * 64 + fg);
+          dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+          dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
         }
         epi_bar_sync();
       }
