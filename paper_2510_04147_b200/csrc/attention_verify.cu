@@ -1,0 +1,427 @@
+// Shared-prefix bidirectional attention of the verification forward (Eq. 5), one kernel.
+//
+// Rows are ordered [sequence slot][node][in-block index].  A query row attends, without a causal
+// mask, to the cached prefix keys of its sequence and to the keys of ITS OWN node's block.  The
+// keys are cut into parts: prefix parts whose boundaries depend on the prefix length only, plus one
+// node-local part (masked block-diagonally: key and query must belong to the same node).  The
+// parts of one (64-row query tile, head) form a thread-block cluster, one CTA per part, so a
+// prefix K/V tile is read once for all tree nodes of the tile.
+//
+// Prologue: the rotated Q tile - and, in the CTA of the local part, the rotated K and the V of the
+// tile's own nodes - are built straight from the fp32 split-K partials of the QKV projection
+// (sum over splits in split order, rotary embedding at the absolute position), so there is no
+// separate rotary pass and no q/k/v round trip through HBM.  The cached prefix does not depend on
+// any earlier kernel of the forward: its first tiles are requested before the dependency wait.
+//
+// Main loop: eight warps = four groups of 16 query rows x two key sets; key set s takes the
+// 64-key tiles with (tile & 1) == s of the part.  Online softmax in the log2 domain, mma.sync
+// (bf16 in, fp32 accumulate): attention is < 3 % of the forward's flops and latency-bound.
+//
+// Epilogue: every warp publishes (max, sum, unnormalised output) of its (rows, key set) in shared
+// memory; after a cluster barrier CTA p normalises the rows r with r % parts == p, reading all
+// 2 * parts sub-parts through distributed shared memory and merging them in (part, key set) order.
+// Every reduction order depends on the row and the prefix length alone, never on the row count.
+#include "attn_common.cuh"
+
+namespace ssd {
+
+namespace {
+
+using namespace attn;
+
+constexpr int kPairKeys = 2 * kKTile;      // keys per loop step: one tile per key set
+
+__device__ __forceinline__ void cluster_sync_all() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release;\nbarrier.cluster.wait.acquire;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_rank(const void* p, uint32_t rank) {
+  uint32_t out;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_u32(p)), "r"(rank));
+  return out;
+}
+// volatile keeps these after the cluster barrier; no memory clobber, so several can be in flight
+__device__ __forceinline__ float2 ld_cluster_f32x2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+
+template <int HD, int QT>
+__global__ void __launch_bounds__(QT * 4) attn_verify_kernel(AttnArgs a, int n_prefix_parts, int nbuf,
+                                                                     float scale_log2) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  constexpr int kQTile = QT;                                    // query rows per CTA: 32 or 64
+  constexpr int kVerifyThreads = QT * 4;                        // (QT / 16 row groups) x 2 key sets, one warp each
+  bf16* sQ = reinterpret_cast<bf16*>(smem_raw);                 // [QT][HD]
+  bf16* sKV = sQ + kQTile * HD;                                 // nbuf x { K [128][HD], V [128][HD] }
+  constexpr int CH = HD / 8;                                    // 16-byte chunks per row
+  constexpr int HALF = HD / 2;
+  constexpr int kBufElems = 2 * kPairKeys * HD;
+
+  pdl_launch_dependents();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int gq = lane >> 2, tq = lane & 3;
+  const int rg = warp % (QT / 16), kset = warp / (QT / 16);
+  const int n_parts = n_prefix_parts + 1;
+  const int part = blockIdx.x, h = blockIdx.y;                  // the cluster spans x
+  const int q_tiles = (a.map.rows_per_seq + kQTile - 1) / kQTile;
+  const int qt = blockIdx.z % q_tiles, slot = blockIdx.z / q_tiles;
+  const int kvh = h / (a.H / a.Hkv);
+  const int rps = a.map.rows_per_seq, T = a.map.T;
+  const int lr0 = qt * kQTile;                                  // first sequence-local query row
+  const size_t grow0 = (size_t)slot * rps + lr0;                // first global row
+  const bool local = part == n_prefix_parts;
+  const int nqkv = (a.H + 2 * a.Hkv) * HD;
+
+  int k_begin, k_end;
+  if (!local) {
+    k_begin = part * a.kv_split;
+    k_end = min(a.S, k_begin + a.kv_split);
+  } else {
+    const int last = min(lr0 + kQTile - 1, rps - 1);
+    k_begin = (lr0 / T) * T;
+    k_end = (last / T + 1) * T;
+  }
+  const int n_tiles = (k_end - k_begin + kKTile - 1) / kKTile;
+  const int n_pairs = (n_tiles + 1) / 2;
+
+  // ---- prefix K/V: asynchronous copies from the cache, 128 keys per step
+  auto load_prefix = [&](int pair, int buf) {
+    const int seq = seq_of_slot(a.map, slot);
+    const bf16* kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * HD;
+    const bf16* vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * HD;
+    const size_t krow_stride = (size_t)a.Hkv * HD;
+    const int key0 = k_begin + pair * kPairKeys;
+    bf16* dK = sKV + (size_t)buf * kBufElems;
+    bf16* dV = dK + kPairKeys * HD;
+    for (int idx = tid; idx < kPairKeys * CH; idx += kVerifyThreads) {
+      const int row = idx / CH, ch = idx % CH;
+      const int key = key0 + row;
+      const bool valid = key < k_end;
+      const size_t off = (size_t)(valid ? key : k_begin) * krow_stride + ch * 8;
+      cp_async16(dK + swz<HD>(row, ch), kbase + off, valid);
+      cp_async16(dV + swz<HD>(row, ch), vbase + off, valid);
+    }
+  };
+  // ---- rotated (sum over splits of) one head's columns of the fused projection -> swizzled bf16
+  //      rows.  A work item is (row, chunk of 8 rotation pairs): 16-byte loads, splits in flight.
+  auto fill_rotated = [&](bf16* dst, int n_rows, int first_row, int row_limit, int col0) {
+    constexpr int CPR = HALF / 8;
+    for (int idx = tid; idx < n_rows * CPR; idx += kVerifyThreads) {
+      const int row = idx / CPR, c = idx % CPR;
+      const int lr = first_row + row;
+      uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
+      if (lr < row_limit) {
+        float x1[8], x2[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { x1[j] = 0.f; x2[j] = 0.f; }
+        const float* pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + c * 8;
+        const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)(a.map.pos0 + lr % T) * HALF + c * 8);
+        float4 cs[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) cs[j] = cs4[j];            // (cos, sin) of pairs 2j and 2j+1
+        // four splits at a time: every load of the group is issued before the first add
+        for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
+          float4 a0[4], a1[4], b0[4], b1[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+            a0[u] = a1[u] = b0[u] = b1[u] = z;
+            if (s0 + u < a.qkv_splits) {
+              const float* ps = pr + (size_t)(s0 + u) * a.qkv_split_stride;
+              a0[u] = *reinterpret_cast<const float4*>(ps);
+              a1[u] = *reinterpret_cast<const float4*>(ps + 4);
+              b0[u] = *reinterpret_cast<const float4*>(ps + HALF);
+              b1[u] = *reinterpret_cast<const float4*>(ps + HALF + 4);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            if (s0 + u < a.qkv_splits) {
+              x1[0] += a0[u].x; x1[1] += a0[u].y; x1[2] += a0[u].z; x1[3] += a0[u].w;
+              x1[4] += a1[u].x; x1[5] += a1[u].y; x1[6] += a1[u].z; x1[7] += a1[u].w;
+              x2[0] += b0[u].x; x2[1] += b0[u].y; x2[2] += b0[u].z; x2[3] += b0[u].w;
+              x2[4] += b1[u].x; x2[5] += b1[u].y; x2[6] += b1[u].z; x2[7] += b1[u].w;
+            }
+          }
+        }
+        float y1[8], y2[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          y1[2 * j] = x1[2 * j] * cs[j].x - x2[2 * j] * cs[j].y;
+          y2[2 * j] = x2[2 * j] * cs[j].x + x1[2 * j] * cs[j].y;
+          y1[2 * j + 1] = x1[2 * j + 1] * cs[j].z - x2[2 * j + 1] * cs[j].w;
+          y2[2 * j + 1] = x2[2 * j + 1] * cs[j].z + x1[2 * j + 1] * cs[j].w;
+        }
+        lo = make_uint4(pack_bf16(y1[0], y1[1]), pack_bf16(y1[2], y1[3]), pack_bf16(y1[4], y1[5]), pack_bf16(y1[6], y1[7]));
+        hi = make_uint4(pack_bf16(y2[0], y2[1]), pack_bf16(y2[2], y2[3]), pack_bf16(y2[4], y2[5]), pack_bf16(y2[6], y2[7]));
+      }
+      *reinterpret_cast<uint4*>(dst + swz<HD>(row, c)) = lo;
+      *reinterpret_cast<uint4*>(dst + swz<HD>(row, c + CPR)) = hi;
+    }
+  };
+  auto fill_plain = [&](bf16* dst, int n_rows, int first_row, int row_limit, int col0) {
+    for (int idx = tid; idx < n_rows * CH; idx += kVerifyThreads) {
+      const int row = idx / CH, c = idx % CH;
+      const int lr = first_row + row;
+      float x[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) x[j] = 0.f;
+      if (lr < row_limit) {
+        const float* pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + c * 8;
+        for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
+          float4 a0[4], a1[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            a0[u] = a1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (s0 + u < a.qkv_splits) {
+              const float* ps = pr + (size_t)(s0 + u) * a.qkv_split_stride;
+              a0[u] = *reinterpret_cast<const float4*>(ps);
+              a1[u] = *reinterpret_cast<const float4*>(ps + 4);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            if (s0 + u < a.qkv_splits) {
+              x[0] += a0[u].x; x[1] += a0[u].y; x[2] += a0[u].z; x[3] += a0[u].w;
+              x[4] += a1[u].x; x[5] += a1[u].y; x[6] += a1[u].z; x[7] += a1[u].w;
+            }
+          }
+        }
+      }
+      *reinterpret_cast<uint4*>(dst + swz<HD>(row, c)) =
+          make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+    }
+  };
+  // the tile's own nodes: K rotated, V summed, from the projection partials (plain stores)
+  auto fill_local = [&](int pair, int buf) {
+    const int key0 = k_begin + pair * kPairKeys;
+    bf16* dK = sKV + (size_t)buf * kBufElems;
+    bf16* dV = dK + kPairKeys * HD;
+    fill_rotated(dK, kPairKeys, key0, k_end, (a.H + kvh) * HD);
+    fill_plain(dV, kPairKeys, key0, k_end, (a.H + a.Hkv + kvh) * HD);
+  };
+
+  // The cache is not written by any kernel of this forward, so its first tiles may be requested
+  // before the dependency wait - unless the slot -> sequence map is only known on the device.
+  const bool early = a.map.n_inline > 0 || a.map.seq_map == nullptr;
+  if (!local && early) load_prefix(0, 0);
+  pdl_wait();                              // the QKV projection's partials are complete from here on
+  if (!local && !early) load_prefix(0, 0);
+  cp_async_commit();
+  fill_rotated(sQ, kQTile, lr0, rps, h * HD);
+  if (local) fill_local(0, 0);
+
+  float o[HD / 8][4];
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+  uint32_t qf[HD / 16][4];
+  const int qrow_w = rg * 16;                          // the warp's first row inside the query tile
+  const bool rows_live = lr0 + qrow_w < rps;           // otherwise the warp only keeps the barriers
+
+  for (int pair = 0; pair < n_pairs; ++pair) {
+    const int buf = pair % nbuf;
+    if (pair + 1 < n_pairs) {                          // nbuf == 2 whenever a part has several steps
+      if (local) fill_local(pair + 1, (pair + 1) % nbuf);
+      else load_prefix(pair + 1, (pair + 1) % nbuf);
+    }
+    cp_async_commit();
+    cp_async_wait<1>();
+    __syncthreads();
+    if (pair == 0 && rows_live) {
+#pragma unroll
+      for (int kk = 0; kk < HD / 16; ++kk) {
+        const int row = qrow_w + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int ch = kk * 2 + (lane >> 4);
+        ldmatrix_x4(qf[kk], sQ + swz<HD>(row, ch));
+      }
+    }
+    const int tile = 2 * pair + kset;
+    if (rows_live && tile < n_tiles) {
+      const bf16* tK = sKV + (size_t)buf * kBufElems + (size_t)kset * kKTile * HD;
+      const bf16* tV = tK + kPairKeys * HD;
+      float s[kKTile / 8][4];
+#pragma unroll
+      for (int j = 0; j < kKTile / 8; ++j) {
+        s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+#pragma unroll
+        for (int k2 = 0; k2 < HD / 32; ++k2) {
+          uint32_t b[4];
+          ldmatrix_x4(b, tK + swz<HD>(j * 8 + (lane & 7), k2 * 4 + (lane >> 3)));
+          mma_bf16(s[j], qf[2 * k2], b[0], b[1]);
+          mma_bf16(s[j], qf[2 * k2 + 1], b[2], b[3]);
+        }
+      }
+      // ---- scale, mask, online softmax (log2 domain)
+      const int key0 = k_begin + tile * kKTile;
+      float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+      for (int j = 0; j < kKTile / 8; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int key = key0 + j * 8 + 2 * tq + (e & 1);
+          bool ok = key < k_end;
+          if (local) {
+            const int qlr = lr0 + qrow_w + gq + (e >> 1) * 8;
+            ok = ok && (key / T == qlr / T);
+          }
+          const float v = ok ? s[j][e] * scale_log2 : -INFINITY;
+          s[j][e] = v;
+          mx[e >> 1] = fmaxf(mx[e >> 1], v);
+        }
+      }
+      float corr[2], m_use[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 1));
+        mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], 2));
+        const float m_new = fmaxf(m_run[i], mx[i]);
+        m_use[i] = (m_new == -INFINITY) ? 0.f : m_new;
+        corr[i] = exp2f(m_run[i] - m_use[i]);          // exp2(-inf) = 0 while nothing was seen
+        m_run[i] = m_new;
+        l_run[i] *= corr[i];
+      }
+#pragma unroll
+      for (int nb = 0; nb < HD / 8; ++nb) {
+        o[nb][0] *= corr[0]; o[nb][1] *= corr[0];
+        o[nb][2] *= corr[1]; o[nb][3] *= corr[1];
+      }
+#pragma unroll
+      for (int j = 0; j < kKTile / 8; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p = exp2f(s[j][e] - m_use[e >> 1]);
+          s[j][e] = p;
+          l_run[e >> 1] += p;
+        }
+      }
+      // ---- O += P V
+#pragma unroll
+      for (int jj = 0; jj < kKTile / 16; ++jj) {
+        uint32_t pa[4];
+        pa[0] = pack_bf16(s[2 * jj][0], s[2 * jj][1]);
+        pa[1] = pack_bf16(s[2 * jj][2], s[2 * jj][3]);
+        pa[2] = pack_bf16(s[2 * jj + 1][0], s[2 * jj + 1][1]);
+        pa[3] = pack_bf16(s[2 * jj + 1][2], s[2 * jj + 1][3]);
+#pragma unroll
+        for (int n2 = 0; n2 < HD / 16; ++n2) {
+          uint32_t vb[4];
+          const int mtx = lane >> 3;
+          const int krow = jj * 16 + (mtx & 1) * 8 + (lane & 7);
+          ldmatrix_x4_trans(vb, tV + swz<HD>(krow, n2 * 2 + (mtx >> 1)));
+          mma_bf16(o[2 * n2], pa, vb[0], vb[1]);
+          mma_bf16(o[2 * n2 + 1], pa, vb[2], vb[3]);
+        }
+      }
+    }
+    __syncthreads();   // everyone is done with buf before it is refilled
+  }
+  cp_async_wait<0>();
+
+  // ---- publish (max, sum, unnormalised output) of this warp's (rows, key set)
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 1);
+    l_run[i] += __shfl_xor_sync(0xffffffffu, l_run[i], 2);
+  }
+  float* sO = reinterpret_cast<float*>(sKV);            // [2 key sets][64][HD] fp32 (K/V buffers are free now)
+  float2* sML = reinterpret_cast<float2*>(sQ);          // [2 key sets][64] (the Q fragments live in registers)
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int row = qrow_w + gq + i * 8;
+    if (tq == 0) sML[kset * kQTile + row] = make_float2(m_run[i], l_run[i]);
+    float* dst = sO + ((size_t)kset * kQTile + row) * HD + 2 * tq;
+#pragma unroll
+    for (int nb = 0; nb < HD / 8; ++nb) *reinterpret_cast<float2*>(dst + nb * 8) = make_float2(o[nb][2 * i], o[nb][2 * i + 1]);
+  }
+  cluster_sync_all();
+
+  // ---- CTA `part` normalises the rows r with r % n_parts == part: all loads of a row are issued
+  //      before the first use, the sub-parts are merged in (part, key set) order
+  constexpr int TPR = HD / 4;                           // threads per row, four columns each
+  constexpr int kMaxSub = 2 * kAttnMaxClusterParts;
+  const int col = (tid % TPR) * 4;
+  for (int row = part + (tid / TPR) * n_parts; row < kQTile; row += (kVerifyThreads / TPR) * n_parts) {
+    if (lr0 + row >= rps) break;
+    float2 ml[kMaxSub];
+#pragma unroll
+    for (int sp = 0; sp < kMaxSub; ++sp) {
+      ml[sp] = make_float2(-INFINITY, 0.f);
+      if ((sp >> 1) < n_parts) ml[sp] = ld_cluster_f32x2(map_to_rank(sML + (sp & 1) * kQTile + row, (uint32_t)(sp >> 1)));
+    }
+    float4 v[kMaxSub];
+#pragma unroll
+    for (int sp = 0; sp < kMaxSub; ++sp) {
+      v[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if ((sp >> 1) < n_parts)
+        v[sp] = ld_cluster_f32x4(map_to_rank(sO + ((size_t)(sp & 1) * kQTile + row) * HD + col, (uint32_t)(sp >> 1)));
+    }
+    float M = -INFINITY;
+#pragma unroll
+    for (int sp = 0; sp < kMaxSub; ++sp) M = fmaxf(M, ml[sp].x);
+    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int sp = 0; sp < kMaxSub; ++sp) {
+      if (ml[sp].x == -INFINITY) continue;
+      const float w = exp2f(ml[sp].x - M);
+      L += ml[sp].y * w;
+      acc.x += v[sp].x * w; acc.y += v[sp].y * w; acc.z += v[sp].z * w; acc.w += v[sp].w * w;
+    }
+    const float inv = 1.f / L;
+    *reinterpret_cast<uint2*>(a.out + ((grow0 + row) * a.H + h) * HD + col) =
+        make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+  }
+  cluster_sync_all();    // nobody leaves while its shared memory may still be read
+}
+
+}  // namespace
+
+int launch_attention_verify(cudaStream_t st, const AttnArgs& a) {
+  if (a.hd != 64 && a.hd != 128) return -2;
+  if (!a.qkv_partial || !a.rope || a.kv_split < kKTile || (a.kv_split % kKTile)) return -1;
+  const int n_prefix = (a.S + a.kv_split - 1) / a.kv_split;
+  const int n_parts = n_prefix + 1;
+  if (n_parts > kAttnMaxClusterParts) return -2;
+  const float scale_log2 = (1.0f / sqrtf((float)a.hd)) * 1.4426950408889634f;
+  // 32-row query tiles (128 threads) while that still fits the machine in one wave, else 64-row tiles
+  const int tiles32 = (a.map.rows_per_seq + 31) / 32;
+  const int qt_rows = ((long long)a.n_seq_slots * tiles32 * n_parts * a.H <= 3 * 148) ? 32 : 64;
+  const int q_tiles = (a.map.rows_per_seq + qt_rows - 1) / qt_rows;
+  // one 128-key step per part needs one K/V buffer; longer parts double-buffer
+  const int nbuf = (a.kv_split > kPairKeys || a.map.T > 32) ? 2 : 1;
+  const size_t smem = (size_t)(qt_rows + nbuf * 2 * kPairKeys) * a.hd * 2;
+  static bool attr_set = false;
+  if (!attr_set) {
+    const int max_smem = (64 + 2 * 2 * kPairKeys) * 128 * 2;
+    if (cudaFuncSetAttribute(attn_verify_kernel<128, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_verify_kernel<128, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_verify_kernel<64, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_verify_kernel<64, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess)
+      return -4;
+    attr_set = true;
+  }
+  dim3 grid(n_parts, a.H, a.n_seq_slots * q_tiles);
+  dim3 block(qt_rows * 4);
+  cudaError_t e;
+  if (a.hd == 128 && qt_rows == 32)
+    e = launch_pdl_cluster(attn_verify_kernel<128, 32>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, nbuf, scale_log2);
+  else if (a.hd == 128)
+    e = launch_pdl_cluster(attn_verify_kernel<128, 64>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, nbuf, scale_log2);
+  else if (qt_rows == 32)
+    e = launch_pdl_cluster(attn_verify_kernel<64, 32>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, nbuf, scale_log2);
+  else
+    e = launch_pdl_cluster(attn_verify_kernel<64, 64>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, nbuf, scale_log2);
+  return e == cudaSuccess ? 0 : -4;
+}
+
+}  // namespace ssd

@@ -88,8 +88,9 @@ __global__ void __launch_bounds__(kRowThreadsMax) embed_rmsnorm_kernel(const int
   write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
 }
 
-// One CTA per row, one float4 column group per thread (per pass): every split's partial is loaded
-// independently, then added in split order, so the row's sum does not depend on the launch shape.
+// One CTA per row.  A thread owns float4 column groups; for each it issues the loads of h and of
+// up to eight splits before the first add, then adds in split order, so a row's sum does not depend
+// on the launch shape and the latency of the (L2-resident) partials is paid once, not per split.
 __global__ void __launch_bounds__(kRowThreadsMax) residual_rmsnorm_kernel(const float* partial, int splits,
                                                                           size_t split_stride, const float* gain,
                                                                           float eps, float* h, bf16* xn, int d) {
@@ -99,31 +100,40 @@ __global__ void __launch_bounds__(kRowThreadsMax) residual_rmsnorm_kernel(const 
   const int r = blockIdx.x;
   float* hrow = h + (size_t)r * d;
   float ss = 0.f;
+  float4 keep = make_float4(0.f, 0.f, 0.f, 0.f);       // the thread's values when one pass covers the row
   for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     float4 v = *reinterpret_cast<const float4*>(hrow + c);
     const float* pp = partial + (size_t)r * d + c;
-    int s = 0;
-    for (; s + 4 <= splits; s += 4) {
-      const float4 p0 = *reinterpret_cast<const float4*>(pp + (size_t)s * split_stride);
-      const float4 p1 = *reinterpret_cast<const float4*>(pp + (size_t)(s + 1) * split_stride);
-      const float4 p2 = *reinterpret_cast<const float4*>(pp + (size_t)(s + 2) * split_stride);
-      const float4 p3 = *reinterpret_cast<const float4*>(pp + (size_t)(s + 3) * split_stride);
-      v.x += p0.x; v.y += p0.y; v.z += p0.z; v.w += p0.w;
-      v.x += p1.x; v.y += p1.y; v.z += p1.z; v.w += p1.w;
-      v.x += p2.x; v.y += p2.y; v.z += p2.z; v.w += p2.w;
-      v.x += p3.x; v.y += p3.y; v.z += p3.z; v.w += p3.w;
-    }
-    for (; s < splits; ++s) {
-      const float4 p0 = *reinterpret_cast<const float4*>(pp + (size_t)s * split_stride);
-      v.x += p0.x; v.y += p0.y; v.z += p0.z; v.w += p0.w;
+    for (int s0 = 0; s0 < splits; s0 += 8) {
+      float4 p[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        p[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (s0 + u < splits) p[u] = *reinterpret_cast<const float4*>(pp + (size_t)(s0 + u) * split_stride);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (s0 + u < splits) { v.x += p[u].x; v.y += p[u].y; v.z += p[u].z; v.w += p[u].w; }
+      }
     }
     *reinterpret_cast<float4*>(hrow + c) = v;
+    keep = v;
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   if (gain == nullptr) return;
+  const int c = threadIdx.x * 4;
+  float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+  const bool one_pass = d <= (int)blockDim.x * 4;
+  if (one_pass && c < d) g = *reinterpret_cast<const float4*>(gain + c);   // in flight during the reduction
   ss = block_sum(ss, red);
   const float inv = rsqrtf(ss / (float)d + eps);
-  write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
+  if (!one_pass) {
+    write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
+  } else if (c < d) {
+    bf16* xrow = xn + (size_t)r * d;
+    *reinterpret_cast<__nv_bfloat162*>(xrow + c) = __floats2bfloat162_rn(keep.x * inv * g.x, keep.y * inv * g.y);
+    *reinterpret_cast<__nv_bfloat162*>(xrow + c + 2) = __floats2bfloat162_rn(keep.z * inv * g.z, keep.w * inv * g.w);
+  }
 }
 
 // One CTA per (row, group of 8 heads of the fused q|k|v output); a warp per head.

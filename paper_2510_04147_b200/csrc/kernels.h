@@ -20,20 +20,33 @@ namespace ssd {
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// cluster_x > 1 additionally groups that many consecutive CTAs along x into a thread-block cluster.
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                              Args... args) {
+inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                      unsigned cluster_x, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (cluster_x > 1) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster_x;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
+  cfg.attrs = attr;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+  return launch_pdl_cluster(kernel, grid, block, smem, st, 1u, args...);
 }
 #endif
 
@@ -45,7 +58,15 @@ struct RowMap {
   int pos0;            // absolute position of t = 0 (= cached prefix length S)
   int seq_base;        // sequence id of slot 0 when seq_map == nullptr
   const int* seq_map;  // device [slots] slot -> sequence id, or nullptr (identity + seq_base)
+  // The same map by value when the host knows it and it is short: a kernel may then use it before
+  // its dependency wait (the device array is written by an earlier kernel of the same forward).
+  int n_inline;        // 0: not given
+  int inline_seq[8];
 };
+__host__ __device__ inline int seq_of_slot(const RowMap& m, int slot) {
+  if (m.n_inline > 0) return m.inline_seq[slot];
+  return m.seq_map ? m.seq_map[slot] : m.seq_base + slot;
+}
 
 // ---------------------------------------------------------------- weight repacking
 // dst[(j / group) * group_stride + group_offset + j % group][c] = bf16(src[j][c]),  j < rows, c < cols
@@ -81,6 +102,12 @@ void launch_lm_merge(cudaStream_t st, const float* tile_max, const float* tile_s
 
 // ---------------------------------------------------------------- attention
 struct AttnArgs {
+  // verification forward: Q and the node-local K/V come straight from the fp32 split-K partials
+  // of the fused q|k|v projection ([splits][R][(H + 2 Hkv) * hd]) and are rotated in the prologue
+  const float* qkv_partial;
+  int qkv_splits;
+  size_t qkv_split_stride;
+  const float2* rope;         // [max_seq][hd/2] (cos, sin)
   const bf16* q;        // [R][H][hd], rotated
   const bf16* cache_k;  // layer base: [seq][max_seq][Hkv][hd]
   const bf16* cache_v;
@@ -97,6 +124,11 @@ struct AttnArgs {
   int n_seq_slots;
 };
 void launch_attention(cudaStream_t st, const AttnArgs& a, int* launches);
+// Verification-forward form: one kernel; rotary embedding, node-local K/V and the merge of the
+// key parts (through a thread-block cluster) inside.  Needs prefix parts + 1 <= kAttnMaxClusterParts.
+// Returns 0 or a negative ssd error code.
+int launch_attention_verify(cudaStream_t st, const AttnArgs& a);
+constexpr int kAttnMaxClusterParts = 8;
 
 // ---------------------------------------------------------------- projections
 enum { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_LMHEAD = 2 };

@@ -126,9 +126,12 @@ int auto_split(int tiles, int k) {
   return s;
 }
 
+// Prefix keys per attention part: a function of the prefix length (and the option) only.  The
+// verification forward merges the parts inside one cluster, so prefix parts + the local part <= 8.
 int kv_split_for(const ssd_ctx* c, int S) {
-  if (c->kv_split_opt > 0) return c->kv_split_opt;
-  return S <= 4096 ? 256 : 512;      // a function of the prefix length only
+  int ks = c->kv_split_opt > 0 ? c->kv_split_opt : 128;
+  while ((S + ks - 1) / ks > kAttnMaxClusterParts - 1) ks += 64;
+  return ks;
 }
 
 // ---- profiling / launch accounting --------------------------------------------------------
@@ -217,8 +220,8 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   if (R > c->R_cap) return fail(c, SSD_ERR_OVERFLOW, "forward of %d rows exceeds capacity %d", R, c->R_cap);
   const int attn_S = (kind == FWD_FILL) ? S + map.T : S;
   const int kv_split = (kind == FWD_FILL) ? attn_S : kv_split_for(c, S);
-  const int n_parts = (attn_S + kv_split - 1) / kv_split + (kind == FWD_VERIFY ? 1 : 0);
-  if ((size_t)n_parts * R > c->part_rows_parts)
+  const int n_parts = (attn_S + kv_split - 1) / kv_split;
+  if (kind == FWD_FILL && (size_t)n_parts * R > c->part_rows_parts)
     return fail(c, SSD_ERR_OVERFLOW, "attention workspace too small for %d parts x %d rows", n_parts, R);
   const int nl = c->cfg.n_layers;
   {
@@ -234,28 +237,31 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     if ((size_t)g.splits * R * g.N > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "split-K workspace too small");
     int rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_QKV);
     if (rc) return rc;
-    bf16* kdst = (kind == FWD_FILL) ? c->cacheK + (size_t)l * c->cache_layer_stride : c->lk;
-    bf16* vdst = (kind == FWD_FILL) ? c->cacheV + (size_t)l * c->cache_layer_stride : c->lv;
-    {
-      Scope sc(c, SSD_PROF_ELEMWISE, (double)R * c->nqkv * (4.0 * g.splits + 2.0));
-      launch_qkv_rope(c->st, c->partial, g.splits, (size_t)R * c->nqkv, R, H, Hkv, hd, c->rope, map, c->q, kdst, vdst,
-                      kind == FWD_FILL ? 1 : 0, c->cache_seq_stride);
-    }
-    if (kind == FWD_FILL && l == nl - 1) break;   // only this layer's K/V were still needed
-    // ---- attention
-    {
-      AttnArgs a{};
-      a.q = c->q;
-      a.cache_k = c->cacheK + (size_t)l * c->cache_layer_stride;
-      a.cache_v = c->cacheV + (size_t)l * c->cache_layer_stride;
-      a.local_k = (kind == FWD_VERIFY) ? c->lk : nullptr;
-      a.local_v = (kind == FWD_VERIFY) ? c->lv : nullptr;
-      a.part_o = c->part_o; a.part_ml = c->part_ml; a.out = c->att;
-      a.R = R; a.H = H; a.Hkv = Hkv; a.hd = hd; a.S = attn_S; a.kv_split = kv_split;
-      a.cache_seq_stride = c->cache_seq_stride; a.map = map; a.n_seq_slots = n_slots;
-      const double kvb = (double)n_slots * attn_S * Hkv * hd * 4.0 + (double)R * (H + 2 * Hkv) * hd * 2.0 + (double)R * H * hd * 2.0;
+    AttnArgs a{};
+    a.cache_k = c->cacheK + (size_t)l * c->cache_layer_stride;
+    a.cache_v = c->cacheV + (size_t)l * c->cache_layer_stride;
+    a.out = c->att;
+    a.R = R; a.H = H; a.Hkv = Hkv; a.hd = hd; a.S = attn_S; a.kv_split = kv_split;
+    a.cache_seq_stride = c->cache_seq_stride; a.map = map; a.n_seq_slots = n_slots;
+    const double kvb = (double)n_slots * attn_S * Hkv * hd * 4.0 + (double)R * (H + 2 * Hkv) * hd * 2.0 + (double)R * H * hd * 2.0;
+    if (kind == FWD_FILL) {
+      // the rotary pass writes K/V into the cache; attention then reads the cache, which holds the rows themselves
+      {
+        Scope sc(c, SSD_PROF_ELEMWISE, (double)R * c->nqkv * (4.0 * g.splits + 2.0));
+        launch_qkv_rope(c->st, c->partial, g.splits, (size_t)R * c->nqkv, R, H, Hkv, hd, c->rope, map, c->q,
+                        c->cacheK + (size_t)l * c->cache_layer_stride, c->cacheV + (size_t)l * c->cache_layer_stride, 1,
+                        c->cache_seq_stride);
+      }
+      if (l == nl - 1) break;   // only this layer's K/V were still needed
+      a.q = c->q; a.part_o = c->part_o; a.part_ml = c->part_ml;
       Scope sc(c, SSD_PROF_ATTN, kvb, 2);
       launch_attention(c->st, a, nullptr);
+    } else {
+      // rotary embedding, node-local K/V and the merge of the key parts happen inside the attention kernel
+      a.qkv_partial = c->partial; a.qkv_splits = g.splits; a.qkv_split_stride = (size_t)R * c->nqkv; a.rope = c->rope;
+      Scope sc(c, SSD_PROF_ATTN, kvb, 1);
+      const int arc = launch_attention_verify(c->st, a);
+      if (arc != 0) return fail(c, arc, "verification attention rejected S=%d kv_split=%d (code %d)", attn_S, kv_split, arc);
     }
     // ---- output projection + residual + norm
     g = GemmArgs{};
@@ -660,6 +666,10 @@ int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n
     launch_tree_build(c->st, c->bs, B, T, md, n_cap, c->cfg.mask_id, c->node_ids, c->node_masked);
   }
   RowMap map{n_cap * T, T, c->cache_len, 0, c->bs.seq_map};
+  if (active <= 8) {           // the host mirrors `remaining`, so it knows the slot -> sequence map too
+    for (int b = 0; b < B; ++b)
+      if (c->h_remaining[b] > 0) map.inline_seq[map.n_inline++] = b;
+  }
   int rc = forward(c, FWD_VERIFY, c->node_ids, R, map, active, false, c->node_masked);
   if (rc) return rc;
   {
