@@ -31,6 +31,14 @@ using namespace attn;
 
 constexpr int kPairKeys = 2 * kKTile;      // keys per loop step: one tile per key set
 
+__device__ __forceinline__ void cluster_arrive() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+__device__ __forceinline__ void st_cluster_u4(uint32_t addr, uint4 v) {
+  asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 __device__ __forceinline__ void cluster_sync_all() {
   __syncwarp();
   asm volatile("barrier.cluster.arrive.release;\nbarrier.cluster.wait.acquire;" ::: "memory");
@@ -110,114 +118,146 @@ __global__ void __launch_bounds__(QT * 4) attn_verify_kernel(AttnArgs a, int n_p
       cp_async16(dV + swz<HD>(row, ch), vbase + off, valid);
     }
   };
-  // ---- rotated (sum over splits of) one head's columns of the fused projection -> swizzled bf16
-  //      rows.  A work item is (row, chunk of 8 rotation pairs): 16-byte loads, splits in flight.
-  auto fill_rotated = [&](bf16* dst, int n_rows, int first_row, int row_limit, int col0) {
-    constexpr int CPR = HALF / 8;
-    for (int idx = tid; idx < n_rows * CPR; idx += kVerifyThreads) {
-      const int row = idx / CPR, c = idx % CPR;
-      const int lr = first_row + row;
-      uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
-      if (lr < row_limit) {
-        float x1[8], x2[8];
+  // ---- one chunk (8 rotation pairs) of one row of a head of the fused projection: sum over the
+  //      splits in split order (four splits' loads in flight at a time), rotary embedding, bf16
+  auto rot_item = [&](int lr, int c, int col0, uint4& lo, uint4& hi) {
+    float x1[8], x2[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { x1[j] = 0.f; x2[j] = 0.f; }
-        const float* pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + c * 8;
-        const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)(a.map.pos0 + lr % T) * HALF + c * 8);
-        float4 cs[4];
+    for (int j = 0; j < 8; ++j) { x1[j] = 0.f; x2[j] = 0.f; }
+    const float* pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + c * 8;
+    const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)(a.map.pos0 + lr % T) * HALF + c * 8);
+    float4 cs[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) cs[j] = cs4[j];            // (cos, sin) of pairs 2j and 2j+1
-        // four splits at a time: every load of the group is issued before the first add
-        for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
-          float4 a0[4], a1[4], b0[4], b1[4];
+    for (int j = 0; j < 4; ++j) cs[j] = cs4[j];              // (cos, sin) of pairs 2j and 2j+1
+    for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
+      float4 a0[4], a1[4], b0[4], b1[4];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-            a0[u] = a1[u] = b0[u] = b1[u] = z;
-            if (s0 + u < a.qkv_splits) {
-              const float* ps = pr + (size_t)(s0 + u) * a.qkv_split_stride;
-              a0[u] = *reinterpret_cast<const float4*>(ps);
-              a1[u] = *reinterpret_cast<const float4*>(ps + 4);
-              b0[u] = *reinterpret_cast<const float4*>(ps + HALF);
-              b1[u] = *reinterpret_cast<const float4*>(ps + HALF + 4);
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            if (s0 + u < a.qkv_splits) {
-              x1[0] += a0[u].x; x1[1] += a0[u].y; x1[2] += a0[u].z; x1[3] += a0[u].w;
-              x1[4] += a1[u].x; x1[5] += a1[u].y; x1[6] += a1[u].z; x1[7] += a1[u].w;
-              x2[0] += b0[u].x; x2[1] += b0[u].y; x2[2] += b0[u].z; x2[3] += b0[u].w;
-              x2[4] += b1[u].x; x2[5] += b1[u].y; x2[6] += b1[u].z; x2[7] += b1[u].w;
-            }
-          }
-        }
-        float y1[8], y2[8];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          y1[2 * j] = x1[2 * j] * cs[j].x - x2[2 * j] * cs[j].y;
-          y2[2 * j] = x2[2 * j] * cs[j].x + x1[2 * j] * cs[j].y;
-          y1[2 * j + 1] = x1[2 * j + 1] * cs[j].z - x2[2 * j + 1] * cs[j].w;
-          y2[2 * j + 1] = x2[2 * j + 1] * cs[j].z + x1[2 * j + 1] * cs[j].w;
-        }
-        lo = make_uint4(pack_bf16(y1[0], y1[1]), pack_bf16(y1[2], y1[3]), pack_bf16(y1[4], y1[5]), pack_bf16(y1[6], y1[7]));
-        hi = make_uint4(pack_bf16(y2[0], y2[1]), pack_bf16(y2[2], y2[3]), pack_bf16(y2[4], y2[5]), pack_bf16(y2[6], y2[7]));
-      }
-      *reinterpret_cast<uint4*>(dst + swz<HD>(row, c)) = lo;
-      *reinterpret_cast<uint4*>(dst + swz<HD>(row, c + CPR)) = hi;
-    }
-  };
-  auto fill_plain = [&](bf16* dst, int n_rows, int first_row, int row_limit, int col0) {
-    for (int idx = tid; idx < n_rows * CH; idx += kVerifyThreads) {
-      const int row = idx / CH, c = idx % CH;
-      const int lr = first_row + row;
-      float x[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) x[j] = 0.f;
-      if (lr < row_limit) {
-        const float* pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + c * 8;
-        for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
-          float4 a0[4], a1[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            a0[u] = a1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (s0 + u < a.qkv_splits) {
-              const float* ps = pr + (size_t)(s0 + u) * a.qkv_split_stride;
-              a0[u] = *reinterpret_cast<const float4*>(ps);
-              a1[u] = *reinterpret_cast<const float4*>(ps + 4);
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            if (s0 + u < a.qkv_splits) {
-              x[0] += a0[u].x; x[1] += a0[u].y; x[2] += a0[u].z; x[3] += a0[u].w;
-              x[4] += a1[u].x; x[5] += a1[u].y; x[6] += a1[u].z; x[7] += a1[u].w;
-            }
-          }
+      for (int u = 0; u < 4; ++u) {
+        a0[u] = a1[u] = b0[u] = b1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (s0 + u < a.qkv_splits) {
+          const float* ps = pr + (size_t)(s0 + u) * a.qkv_split_stride;
+          a0[u] = *reinterpret_cast<const float4*>(ps);
+          a1[u] = *reinterpret_cast<const float4*>(ps + 4);
+          b0[u] = *reinterpret_cast<const float4*>(ps + HALF);
+          b1[u] = *reinterpret_cast<const float4*>(ps + HALF + 4);
         }
       }
-      *reinterpret_cast<uint4*>(dst + swz<HD>(row, c)) =
-          make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (s0 + u < a.qkv_splits) {
+          x1[0] += a0[u].x; x1[1] += a0[u].y; x1[2] += a0[u].z; x1[3] += a0[u].w;
+          x1[4] += a1[u].x; x1[5] += a1[u].y; x1[6] += a1[u].z; x1[7] += a1[u].w;
+          x2[0] += b0[u].x; x2[1] += b0[u].y; x2[2] += b0[u].z; x2[3] += b0[u].w;
+          x2[4] += b1[u].x; x2[5] += b1[u].y; x2[6] += b1[u].z; x2[7] += b1[u].w;
+        }
+      }
     }
+    float y1[8], y2[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      y1[2 * j] = x1[2 * j] * cs[j].x - x2[2 * j] * cs[j].y;
+      y2[2 * j] = x2[2 * j] * cs[j].x + x1[2 * j] * cs[j].y;
+      y1[2 * j + 1] = x1[2 * j + 1] * cs[j].z - x2[2 * j + 1] * cs[j].w;
+      y2[2 * j + 1] = x2[2 * j + 1] * cs[j].z + x1[2 * j + 1] * cs[j].w;
+    }
+    lo = make_uint4(pack_bf16(y1[0], y1[1]), pack_bf16(y1[2], y1[3]), pack_bf16(y1[4], y1[5]), pack_bf16(y1[6], y1[7]));
+    hi = make_uint4(pack_bf16(y2[0], y2[1]), pack_bf16(y2[2], y2[3]), pack_bf16(y2[4], y2[5]), pack_bf16(y2[6], y2[7]));
   };
-  // the tile's own nodes: K rotated, V summed, from the projection partials (plain stores)
+  // ---- one 16-byte chunk (8 columns) of one row, summed over the splits, bf16 (for V)
+  auto plain_item = [&](int lr, int c, int col0) -> uint4 {
+    float x[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) x[j] = 0.f;
+    const float* pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + c * 8;
+    for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
+      float4 a0[4], a1[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        a0[u] = a1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (s0 + u < a.qkv_splits) {
+          const float* ps = pr + (size_t)(s0 + u) * a.qkv_split_stride;
+          a0[u] = *reinterpret_cast<const float4*>(ps);
+          a1[u] = *reinterpret_cast<const float4*>(ps + 4);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (s0 + u < a.qkv_splits) {
+          x[0] += a0[u].x; x[1] += a0[u].y; x[2] += a0[u].z; x[3] += a0[u].w;
+          x[4] += a1[u].x; x[5] += a1[u].y; x[6] += a1[u].z; x[7] += a1[u].w;
+        }
+      }
+    }
+    return make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+  };
+  // later 128-key steps of a long local part (block length > 32): built by the local CTA alone
   auto fill_local = [&](int pair, int buf) {
+    constexpr int CPR = HALF / 8;
     const int key0 = k_begin + pair * kPairKeys;
     bf16* dK = sKV + (size_t)buf * kBufElems;
     bf16* dV = dK + kPairKeys * HD;
-    fill_rotated(dK, kPairKeys, key0, k_end, (a.H + kvh) * HD);
-    fill_plain(dV, kPairKeys, key0, k_end, (a.H + a.Hkv + kvh) * HD);
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    for (int idx = tid; idx < kPairKeys * CPR; idx += kVerifyThreads) {
+      const int row = idx / CPR, c = idx % CPR;
+      uint4 lo = zero, hi = zero;
+      if (key0 + row < k_end) rot_item(key0 + row, c, (a.H + kvh) * HD, lo, hi);
+      *reinterpret_cast<uint4*>(dK + swz<HD>(row, c)) = lo;
+      *reinterpret_cast<uint4*>(dK + swz<HD>(row, c + CPR)) = hi;
+    }
+    for (int idx = tid; idx < kPairKeys * CH; idx += kVerifyThreads) {
+      const int row = idx / CH, c = idx % CH;
+      *reinterpret_cast<uint4*>(dV + swz<HD>(row, c)) =
+          (key0 + row < k_end) ? plain_item(key0 + row, c, (a.H + a.Hkv + kvh) * HD) : zero;
+    }
   };
 
   // The cache is not written by any kernel of this forward, so its first tiles may be requested
   // before the dependency wait - unless the slot -> sequence map is only known on the device.
   const bool early = a.map.n_inline > 0 || a.map.seq_map == nullptr;
   if (!local && early) load_prefix(0, 0);
+  cluster_arrive();                        // every CTA of the cluster runs before shared memory is written remotely
   pdl_wait();                              // the QKV projection's partials are complete from here on
   if (!local && !early) load_prefix(0, 0);
   cp_async_commit();
-  fill_rotated(sQ, kQTile, lr0, rps, h * HD);
-  if (local) fill_local(0, 0);
+
+  // ---- cooperative prologue: the cluster's threads share the rotary work.  The Q tile is needed by
+  //      every CTA (each chunk is built once and stored into all of them), the first 128 local keys
+  //      only by the CTA of the local part.  Rows past the end are zero (a masked key's V row must
+  //      not hold stale shared memory: 0 * NaN would poison the output).
+  {
+    constexpr int CPR = HALF / 8;
+    const int last = min(lr0 + kQTile - 1, rps - 1);
+    const int lk_begin = (lr0 / T) * T;
+    const int lk_rows = min((last / T + 1) * T - lk_begin, kPairKeys);       // valid local keys of step 0
+    const int lk_fill = min(((lk_rows + kKTile - 1) / kKTile) * kKTile, kPairKeys);   // rows of the tiles in use
+    const int n_q = kQTile * CPR, n_k = lk_fill * CPR, n_v = lk_fill * CH;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    bf16* lK = sKV;                          // buffer 0 of the local CTA
+    bf16* lV = sKV + kPairKeys * HD;
+    cluster_wait();
+    for (int it = part * kVerifyThreads + tid; it < n_q + n_k + n_v; it += n_parts * kVerifyThreads) {
+      if (it < n_q) {
+        const int row = it / CPR, c = it % CPR;
+        uint4 lo = zero, hi = zero;
+        if (lr0 + row < rps) rot_item(lr0 + row, c, h * HD, lo, hi);
+        for (int r = 0; r < n_parts; ++r) {
+          st_cluster_u4(map_to_rank(sQ + swz<HD>(row, c), (uint32_t)r), lo);
+          st_cluster_u4(map_to_rank(sQ + swz<HD>(row, c + CPR), (uint32_t)r), hi);
+        }
+      } else if (it < n_q + n_k) {
+        const int row = (it - n_q) / CPR, c = (it - n_q) % CPR;
+        uint4 lo = zero, hi = zero;
+        if (row < lk_rows) rot_item(lk_begin + row, c, (a.H + kvh) * HD, lo, hi);
+        st_cluster_u4(map_to_rank(lK + swz<HD>(row, c), (uint32_t)n_prefix_parts), lo);
+        st_cluster_u4(map_to_rank(lK + swz<HD>(row, c + CPR), (uint32_t)n_prefix_parts), hi);
+      } else {
+        const int row = (it - n_q - n_k) / CH, c = (it - n_q - n_k) % CH;
+        const uint4 v = (row < lk_rows) ? plain_item(lk_begin + row, c, (a.H + a.Hkv + kvh) * HD) : zero;
+        st_cluster_u4(map_to_rank(lV + swz<HD>(row, c), (uint32_t)n_prefix_parts), v);
+      }
+    }
+    cluster_sync_all();
+  }
 
   float o[HD / 8][4];
 #pragma unroll
