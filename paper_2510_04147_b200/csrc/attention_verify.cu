@@ -291,15 +291,17 @@ __global__ void __launch_bounds__(QT * 4) attn_verify_kernel(AttnArgs a, int n_p
       const bf16* tV = tK + kPairKeys * HD;
       float s[kKTile / 8][4];
 #pragma unroll
-      for (int j = 0; j < kKTile / 8; ++j) {
-        s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+      for (int j = 0; j < kKTile / 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+      // k outer, key group inner: consecutive MMAs update different accumulators
 #pragma unroll
-        for (int k2 = 0; k2 < HD / 32; ++k2) {
-          uint32_t b[4];
-          ldmatrix_x4(b, tK + swz<HD>(j * 8 + (lane & 7), k2 * 4 + (lane >> 3)));
-          mma_bf16(s[j], qf[2 * k2], b[0], b[1]);
-          mma_bf16(s[j], qf[2 * k2 + 1], b[2], b[3]);
-        }
+      for (int k2 = 0; k2 < HD / 32; ++k2) {
+        uint32_t b[kKTile / 8][4];
+#pragma unroll
+        for (int j = 0; j < kKTile / 8; ++j) ldmatrix_x4(b[j], tK + swz<HD>(j * 8 + (lane & 7), k2 * 4 + (lane >> 3)));
+#pragma unroll
+        for (int j = 0; j < kKTile / 8; ++j) mma_bf16(s[j], qf[2 * k2], b[j][0], b[j][1]);
+#pragma unroll
+        for (int j = 0; j < kKTile / 8; ++j) mma_bf16(s[j], qf[2 * k2 + 1], b[j][2], b[j][3]);
       }
       // ---- scale, mask, online softmax (log2 domain)
       const int key0 = k_begin + tile * kKTile;
@@ -383,43 +385,59 @@ __global__ void __launch_bounds__(QT * 4) attn_verify_kernel(AttnArgs a, int n_p
 #pragma unroll
     for (int nb = 0; nb < HD / 8; ++nb) *reinterpret_cast<float2*>(dst + nb * 8) = make_float2(o[nb][2 * i], o[nb][2 * i + 1]);
   }
+  __syncthreads();
+  // ---- the two key sets of this CTA are merged first (set 0, then set 1), in place
+  float2* sML2 = sML + 2 * kQTile;                      // [QT] merged (max, sum)
+  for (int it = tid; it < kQTile * (HD / 4); it += kVerifyThreads) {
+    const int row = it / (HD / 4), c4 = (it % (HD / 4)) * 4;
+    const float2 ml0 = sML[row], ml1 = sML[kQTile + row];
+    const float M = fmaxf(ml0.x, ml1.x);
+    const float w0 = (ml0.x == -INFINITY) ? 0.f : exp2f(ml0.x - M);
+    const float w1 = (ml1.x == -INFINITY) ? 0.f : exp2f(ml1.x - M);
+    float4* p0 = reinterpret_cast<float4*>(sO + (size_t)row * HD + c4);
+    const float4 v0 = *p0;
+    const float4 v1 = *reinterpret_cast<const float4*>(sO + ((size_t)kQTile + row) * HD + c4);
+    *p0 = make_float4(v0.x * w0 + v1.x * w1, v0.y * w0 + v1.y * w1, v0.z * w0 + v1.z * w1, v0.w * w0 + v1.w * w1);
+    if (c4 == 0) sML2[row] = make_float2(M, ml0.y * w0 + ml1.y * w1);
+  }
   cluster_sync_all();
 
-  // ---- CTA `part` normalises the rows r with r % n_parts == part: all loads of a row are issued
-  //      before the first use, the sub-parts are merged in (part, key set) order
-  constexpr int TPR = HD / 4;                           // threads per row, four columns each
-  constexpr int kMaxSub = 2 * kAttnMaxClusterParts;
-  const int col = (tid % TPR) * 4;
+  // ---- CTA `part` normalises the rows r with r % n_parts == part: all remote loads of a row are
+  //      issued before the first use, the parts are merged in part order
+  constexpr int TPR = HD / 8;                           // threads per row, eight columns each
+  const int col = (tid % TPR) * 8;
   for (int row = part + (tid / TPR) * n_parts; row < kQTile; row += (kVerifyThreads / TPR) * n_parts) {
     if (lr0 + row >= rps) break;
-    float2 ml[kMaxSub];
+    float2 ml[kAttnMaxClusterParts];
+    float4 va[kAttnMaxClusterParts], vb[kAttnMaxClusterParts];
 #pragma unroll
-    for (int sp = 0; sp < kMaxSub; ++sp) {
-      ml[sp] = make_float2(-INFINITY, 0.f);
-      if ((sp >> 1) < n_parts) ml[sp] = ld_cluster_f32x2(map_to_rank(sML + (sp & 1) * kQTile + row, (uint32_t)(sp >> 1)));
-    }
-    float4 v[kMaxSub];
-#pragma unroll
-    for (int sp = 0; sp < kMaxSub; ++sp) {
-      v[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if ((sp >> 1) < n_parts)
-        v[sp] = ld_cluster_f32x4(map_to_rank(sO + ((size_t)(sp & 1) * kQTile + row) * HD + col, (uint32_t)(sp >> 1)));
+    for (int pp = 0; pp < kAttnMaxClusterParts; ++pp) {
+      ml[pp] = make_float2(-INFINITY, 0.f);
+      va[pp] = vb[pp] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (pp < n_parts) {
+        ml[pp] = ld_cluster_f32x2(map_to_rank(sML2 + row, (uint32_t)pp));
+        const uint32_t base = map_to_rank(sO + (size_t)row * HD + col, (uint32_t)pp);
+        va[pp] = ld_cluster_f32x4(base);
+        vb[pp] = ld_cluster_f32x4(base + 16);
+      }
     }
     float M = -INFINITY;
 #pragma unroll
-    for (int sp = 0; sp < kMaxSub; ++sp) M = fmaxf(M, ml[sp].x);
+    for (int pp = 0; pp < kAttnMaxClusterParts; ++pp) M = fmaxf(M, ml[pp].x);
     float L = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 acc0 = make_float4(0.f, 0.f, 0.f, 0.f), acc1 = acc0;
 #pragma unroll
-    for (int sp = 0; sp < kMaxSub; ++sp) {
-      if (ml[sp].x == -INFINITY) continue;
-      const float w = exp2f(ml[sp].x - M);
-      L += ml[sp].y * w;
-      acc.x += v[sp].x * w; acc.y += v[sp].y * w; acc.z += v[sp].z * w; acc.w += v[sp].w * w;
+    for (int pp = 0; pp < kAttnMaxClusterParts; ++pp) {
+      if (ml[pp].x == -INFINITY) continue;
+      const float w = exp2f(ml[pp].x - M);
+      L += ml[pp].y * w;
+      acc0.x += va[pp].x * w; acc0.y += va[pp].y * w; acc0.z += va[pp].z * w; acc0.w += va[pp].w * w;
+      acc1.x += vb[pp].x * w; acc1.y += vb[pp].y * w; acc1.z += vb[pp].z * w; acc1.w += vb[pp].w * w;
     }
     const float inv = 1.f / L;
-    *reinterpret_cast<uint2*>(a.out + ((grow0 + row) * a.H + h) * HD + col) =
-        make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+    *reinterpret_cast<uint4*>(a.out + ((grow0 + row) * a.H + h) * HD + col) =
+        make_uint4(pack_bf16(acc0.x * inv, acc0.y * inv), pack_bf16(acc0.z * inv, acc0.w * inv),
+                   pack_bf16(acc1.x * inv, acc1.y * inv), pack_bf16(acc1.z * inv, acc1.w * inv));
   }
   cluster_sync_all();    // nobody leaves while its shared memory may still be read
 }
