@@ -61,8 +61,9 @@ __device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
   return v;
 }
 
-template <int HD, int QT>
-__global__ void __launch_bounds__(QT * 4) attn_verify_kernel(AttnArgs a, int n_prefix_parts, int nbuf,
+// MINB: CTAs per SM the register allocation must allow (3 trades a few spills for one wave at 64 rows)
+template <int HD, int QT, int MINB>
+__global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, int n_prefix_parts, int nbuf,
                                                                      float scale_log2) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   constexpr int kQTile = QT;                                    // query rows per CTA: 32 or 64
@@ -458,27 +459,37 @@ int launch_attention_verify(cudaStream_t st, const AttnArgs& a) {
   // one 128-key step per part needs one K/V buffer; longer parts double-buffer
   const int nbuf = (a.kv_split > kPairKeys || a.map.T > 32) ? 2 : 1;
   const size_t smem = (size_t)(qt_rows + nbuf * 2 * kPairKeys) * a.hd * 2;
+  // two CTAs per SM by default; three (register-capped build) when only that keeps the grid in one wave
+  const long long n_ctas = (long long)a.n_seq_slots * q_tiles * n_parts * a.H;
+  const bool dense = qt_rows == 32 && n_ctas > 2 * 148;
   static bool attr_set = false;
   if (!attr_set) {
     const int max_smem = (64 + 2 * 2 * kPairKeys) * 128 * 2;
-    if (cudaFuncSetAttribute(attn_verify_kernel<128, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
-        cudaFuncSetAttribute(attn_verify_kernel<128, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
-        cudaFuncSetAttribute(attn_verify_kernel<64, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess ||
-        cudaFuncSetAttribute(attn_verify_kernel<64, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess)
+    if (cudaFuncSetAttribute(attn_verify_kernel<128, 32, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_verify_kernel<128, 32, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_verify_kernel<128, 64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_verify_kernel<64, 32, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_verify_kernel<64, 32, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_verify_kernel<64, 64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess)
       return -4;
     attr_set = true;
   }
   dim3 grid(n_parts, a.H, a.n_seq_slots * q_tiles);
   dim3 block(qt_rows * 4);
+  const unsigned cl = (unsigned)n_parts;
   cudaError_t e;
-  if (a.hd == 128 && qt_rows == 32)
-    e = launch_pdl_cluster(attn_verify_kernel<128, 32>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, nbuf, scale_log2);
-  else if (a.hd == 128)
-    e = launch_pdl_cluster(attn_verify_kernel<128, 64>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, nbuf, scale_log2);
-  else if (qt_rows == 32)
-    e = launch_pdl_cluster(attn_verify_kernel<64, 32>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, nbuf, scale_log2);
-  else
-    e = launch_pdl_cluster(attn_verify_kernel<64, 64>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, nbuf, scale_log2);
+#define SSD_LAUNCH_VERIFY(HD_, QT_, MB_) \
+  e = launch_pdl_cluster(attn_verify_kernel<HD_, QT_, MB_>, grid, block, smem, st, cl, a, n_prefix, nbuf, scale_log2)
+  if (a.hd == 128) {
+    if (qt_rows == 64) SSD_LAUNCH_VERIFY(128, 64, 1);
+    else if (dense) SSD_LAUNCH_VERIFY(128, 32, 3);
+    else SSD_LAUNCH_VERIFY(128, 32, 2);
+  } else {
+    if (qt_rows == 64) SSD_LAUNCH_VERIFY(64, 64, 1);
+    else if (dense) SSD_LAUNCH_VERIFY(64, 32, 3);
+    else SSD_LAUNCH_VERIFY(64, 32, 2);
+  }
+#undef SSD_LAUNCH_VERIFY
   return e == cudaSuccess ? 0 : -4;
 }
 
