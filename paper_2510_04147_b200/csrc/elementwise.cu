@@ -88,6 +88,28 @@ __global__ void __launch_bounds__(kRowThreadsMax) embed_rmsnorm_kernel(const int
   write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
 }
 
+__global__ void __launch_bounds__(kRowThreadsMax) embed_prep_kernel(const int* ids, const bf16* embed, const float* gain,
+                                                                    float* h, bf16* hb, float* sq, int sq_stride, int d) {
+  __shared__ float red[kRowThreadsMax / 32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const bf16* e = embed + (size_t)ids[r] * d;
+  float ss = 0.f;
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(e + c);
+    const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(e + c + 2);
+    const float4 g = *reinterpret_cast<const float4*>(gain + c);
+    const float4 v = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
+    *reinterpret_cast<float4*>(h + (size_t)r * d + c) = v;
+    *reinterpret_cast<__nv_bfloat162*>(hb + (size_t)r * d + c) = __floats2bfloat162_rn(v.x * g.x, v.y * g.y);
+    *reinterpret_cast<__nv_bfloat162*>(hb + (size_t)r * d + c + 2) = __floats2bfloat162_rn(v.z * g.z, v.w * g.w);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = block_sum(ss, red);
+  if (threadIdx.x == 0) sq[(size_t)r * sq_stride] = ss;
+}
+
 // One CTA per row.  A thread owns float4 column groups; for each it issues the loads of h and of
 // up to eight splits before the first add, then adds in split order, so a row's sum does not depend
 // on the launch shape and the latency of the (L2-resident) partials is paid once, not per split.
@@ -317,6 +339,11 @@ static int row_threads(int d) {
 void launch_embed_rmsnorm(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float eps, float* h,
                           bf16* xn, int R, int d) {
   launch_pdl(embed_rmsnorm_kernel, dim3(R), dim3(row_threads(d)), 0, st, ids, embed, gain, eps, h, xn, d);
+}
+
+void launch_embed_prep(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float* h, bf16* hb,
+                       float* sq, int sq_stride, int R, int d) {
+  launch_pdl(embed_prep_kernel, dim3(R), dim3(row_threads(d)), 0, st, ids, embed, gain, h, hb, sq, sq_stride, d);
 }
 
 void launch_residual_rmsnorm(cudaStream_t st, const float* partial, int splits, size_t split_stride, const float* gain,

@@ -112,6 +112,14 @@ struct TcParams {
   int* tile_arg;
   int mask_id;
   int* err_flag;
+  const float* sq;
+  int sq_count, sq_stride, norm_dim;
+  float norm_eps;
+  float* h;
+  bf16* hb;
+  const float* gain;
+  float* sq_out;
+  int sq_out_stride;
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -191,6 +199,25 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Cluster-wide barrier in two halves.  All 192 threads of every CTA of the cluster arrive once per
+// phase; only threads that go on to touch remote shared memory need to wait.
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+__device__ __forceinline__ uint32_t map_to_rank(const void* p, uint32_t rank) {
+  uint32_t out;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_addr(p)), "r"(rank));
+  return out;
+}
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
 
 __global__ void __launch_bounds__(kTcThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const TcParams p) {
@@ -206,6 +233,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   uint64_t* acc_bar = bars + 2 * kMaxStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* s_inv = reinterpret_cast<float*>(bars + 32);           // [256] per-row 1/rms of the consumer side
 
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -237,6 +265,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  bool epi_ok = false;       // epilogue threads: the accumulator is complete
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -315,6 +344,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
     const int lrow = quad * 32 + lane;         // accumulator lane = feature inside the tile
     pdl_wait();                                // outputs may still be read by the predecessor
+    const int et = threadIdx.x - 64;           // 0..127 among the epilogue threads
+    if (p.sq != nullptr) {
+      // fused RMSNorm, consumer side: 1/rms of every row from the producers' per-tile sums of squares
+      // (summed in slot order), computed while the main loop still runs
+      for (int rr = et; rr < p.npad; rr += 128) {
+        float inv = 0.f;
+        if (row0 + rr < p.R) {
+          const float* q = p.sq + (size_t)(row0 + rr) * p.sq_stride;
+          float ss = 0.f;
+          for (int t = 0; t < p.sq_count; ++t) ss += q[t];
+          inv = rsqrtf(ss / (float)p.norm_dim + p.norm_eps);
+        }
+        s_inv[rr] = inv;
+      }
+      epi_bar_sync();
+    }
     bool ok = true;
     if (n_kb > 0) ok = mbar_wait(smem_addr(acc_bar), 0u, abort_flag);
     ok = __all_sync(0xffffffffu, ok);
@@ -322,20 +367,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
     const int rows_here = min(p.R - row0, 256);
     float* scratch = reinterpret_cast<float*>(sW);   // stage 0 of the ring is free once acc_bar fired
+    epi_ok = ok;
     if (!ok) {
       if (lane == 0) { *abort_flag = 1; atomicExch(p.err_flag, 3); }
+    } else if (p.epi == EPI_RESIDUAL) {
+      // after the role branches: every thread of the CTA takes part in the cluster barriers
     } else if (p.epi == EPI_PARTIAL) {
       // Transpose 32 rows x 128 features through shared memory so that a thread stores four
       // consecutive features of one row: 8 vector stores per thread and chunk instead of 32 scalars.
       const int n_base = tile * kTileM;
       const bool vec_ok = ((p.N & 3) == 0) && (n_base + kTileM <= p.N);
-      const int et = threadIdx.x - 64;                 // 0..127 among the epilogue threads
       for (int c0 = 0; c0 < p.npad; c0 += 32) {
         float v[32];
         if (n_kb > 0) tmem_ld32(taddr + c0, v);
         else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = 0.f;
+        }
+        if (p.sq != nullptr) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] *= s_inv[c0 + j];
         }
         if (vec_ok) {
 #pragma unroll
@@ -365,11 +416,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     } else if (p.epi == EPI_SWIGLU) {
       // lanes 0-63 hold gate features, lanes 64-127 the matching up features.  After the transpose a
       // thread owns 16 consecutive features of one row: silu(gate) * up, 32 bytes of bf16 per thread.
-      const int et = threadIdx.x - 64;
       const int rr = et >> 2, fg = (et & 3) * 16;
       for (int c0 = 0; c0 < p.npad; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + c0, v);
+        if (p.sq != nullptr) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] *= s_inv[c0 + j];
+        }
 #pragma unroll
         for (int j = 0; j < 32; ++j) scratch[j * kEpiPitch + lrow] = v[j];
         epi_bar_sync();
@@ -401,6 +455,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       for (int c0 = 0; c0 < p.npad; c0 += 32) {
         float v[32];
         tmem_ld32(taddr + c0, v);
+        if (p.sq != nullptr) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] *= s_inv[c0 + j];
+        }
         float my_m = -INFINITY, my_s = 0.f;
         int my_a = 0x7fffffff;
 #pragma unroll
@@ -445,6 +503,71 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
     }
   }
+  if (p.epi == EPI_RESIDUAL) {
+    // ---- split-K reduction inside the cluster + residual + operand of the next projection.
+    // Per chunk of 32 rows: every CTA stages its partial [32 rows][128 features] in shared memory;
+    // after a cluster barrier CTA `rank` owns the rows rank, rank + splits, ... (one warp per row, a
+    // lane per four features): it adds the partials in split order to the residual stream, writes h,
+    // bf16(h * gain) and the tile's sum of squares of the row.  A second barrier frees the staging
+    // buffer.  Every thread of every CTA passes both barriers of every chunk, also after an error.
+    const bool epi_warp = warp >= 2;
+    const int quad = warp & 3;
+    const int lrow = quad * 32 + lane;
+    const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const int rows_here = min(p.R - row0, 256);
+    float* scratch = reinterpret_cast<float*>(sW);
+    const uint32_t n_ranks = (uint32_t)p.splits, rank = cluster_ctarank();
+    const int n_base = tile * kTileM;
+    const int f4 = lane * 4;
+    const bool col_ok = n_base + f4 < p.N;
+    float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (epi_warp && col_ok) g4 = *reinterpret_cast<const float4*>(p.gain + n_base + f4);
+    for (int c0 = 0; c0 < p.npad; c0 += 32) {
+      if (epi_warp && epi_ok) {
+        float v[32];
+        tmem_ld32(taddr + c0, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) scratch[j * kEpiPitch + lrow] = v[j];
+      }
+      __syncwarp();
+      cluster_arrive_release();
+      cluster_wait_acquire();
+      if (epi_warp && epi_ok) {
+        for (int rr = (int)rank + (warp - 2) * (int)n_ranks; rr < 32; rr += 4 * (int)n_ranks) {
+          const int row = c0 + rr;
+          if (row >= rows_here) break;
+          float4 part[kGemmMaxClusterSplits];
+#pragma unroll
+          for (int q = 0; q < kGemmMaxClusterSplits; ++q) {
+            part[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if ((uint32_t)q < n_ranks) part[q] = ld_cluster_f32x4(map_to_rank(scratch + rr * kEpiPitch + f4, (uint32_t)q));
+          }
+          float* hp = p.h + (size_t)(row0 + row) * p.N + n_base + f4;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (col_ok) acc = *reinterpret_cast<const float4*>(hp);
+#pragma unroll
+          for (int q = 0; q < kGemmMaxClusterSplits; ++q) {
+            if ((uint32_t)q < n_ranks) { acc.x += part[q].x; acc.y += part[q].y; acc.z += part[q].z; acc.w += part[q].w; }
+          }
+          float ss = 0.f;
+          if (col_ok) {
+            *reinterpret_cast<float4*>(hp) = acc;
+            __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * g4.x, acc.y * g4.y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * g4.z, acc.w * g4.w);
+            *reinterpret_cast<uint2*>(p.hb + (size_t)(row0 + row) * p.N + n_base + f4) =
+                make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+            ss = acc.x * acc.x + acc.y * acc.y + acc.z * acc.z + acc.w * acc.w;
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+          if (lane == 0) p.sq_out[(size_t)(row0 + row) * p.sq_out_stride + tile] = ss;
+        }
+      }
+      __syncwarp();
+      cluster_arrive_release();
+      cluster_wait_acquire();
+    }
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -486,7 +609,10 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   if (!g_encode) return -4;
   if ((g.x_pitch % 8) || (!g.w_tiled && (g.w_pitch % 8)) || (((uintptr_t)g.x) & 15) || (((uintptr_t)g.w) & 15)) return -2;
   if (g.R < 1 || g.N < 1 || g.K < 1) return -2;
-  if (g.epi != EPI_PARTIAL && g.splits != 1) return -2;
+  if (g.epi != EPI_PARTIAL && g.epi != EPI_RESIDUAL && g.splits != 1) return -2;
+  if (g.epi == EPI_RESIDUAL &&
+      (g.splits < 1 || g.splits > kGemmMaxClusterSplits || (g.N & 3) || !g.h || !g.hb || !g.gain || !g.sq_out)) return -2;
+  if (g.sq != nullptr && (g.sq_count < 1 || g.norm_dim < 1)) return -2;
   if (g.epi == EPI_SWIGLU && (g.N % 128)) return -2;
   TcParams p;
   p.R = g.R; p.N = g.N; p.K = g.K;
@@ -508,7 +634,9 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   p.out = g.out; p.act = g.act; p.act_pitch = g.act_pitch;
   p.tile_max = g.tile_max; p.tile_sum = g.tile_sum; p.tile_arg = g.tile_arg;
   p.mask_id = g.mask_id; p.err_flag = g.err_flag;
-  const int smem = stages * stage_bytes + 1024 /*alignment slack*/ + (2 * kMaxStages + 1) * 8 + 16;
+  p.sq = g.sq; p.sq_count = g.sq_count; p.sq_stride = g.sq_stride; p.norm_dim = g.norm_dim; p.norm_eps = g.norm_eps;
+  p.h = g.h; p.hb = g.hb; p.gain = g.gain; p.sq_out = g.sq_out; p.sq_out_stride = g.sq_out_stride;
+  const int smem = stages * stage_bytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + 1024 /*per-row 1/rms*/;
   // tensor-memory safety: CTAs that fit by shared memory must also fit by TMEM columns
   if ((227 * 1024 / smem) * (int)cols > 512) return -2;
   CUtensorMap tmW, tmX;
@@ -527,7 +655,9 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
     smem_set = 227 * 1024;
   }
   dim3 grid(gemm_tiles(g.N), g.splits, (g.R + 255) / 256);
-  if (launch_pdl(gemm_tc_kernel, grid, dim3(kTcThreads), (size_t)smem, st, tmW, tmX, p) != cudaSuccess) return -4;
+  const unsigned cluster_y = (g.epi == EPI_RESIDUAL) ? (unsigned)g.splits : 1u;
+  if (launch_pdl_cluster_xy(gemm_tc_kernel, grid, dim3(kTcThreads), (size_t)smem, st, 1u, cluster_y, tmW, tmX, p) != cudaSuccess)
+    return -4;
   return 0;
 }
 

@@ -20,10 +20,11 @@ namespace ssd {
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-// cluster_x > 1 additionally groups that many consecutive CTAs along x into a thread-block cluster.
+// A cluster dimension > 1 additionally groups that many consecutive CTAs along x (or y) into a
+// thread-block cluster.
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                                      unsigned cluster_x, Args... args) {
+inline cudaError_t launch_pdl_cluster_xy(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                         unsigned cluster_x, unsigned cluster_y, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -33,10 +34,10 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.numAttrs = 1;
-  if (cluster_x > 1) {
+  if (cluster_x > 1 || cluster_y > 1) {
     attr[1].id = cudaLaunchAttributeClusterDimension;
     attr[1].val.clusterDim.x = cluster_x;
-    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.y = cluster_y;
     attr[1].val.clusterDim.z = 1;
     cfg.numAttrs = 2;
   }
@@ -44,9 +45,14 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                      unsigned cluster_x, Args... args) {
+  return launch_pdl_cluster_xy(kernel, grid, block, smem, st, cluster_x, 1u, args...);
+}
+template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                               Args... args) {
-  return launch_pdl_cluster(kernel, grid, block, smem, st, 1u, args...);
+  return launch_pdl_cluster_xy(kernel, grid, block, smem, st, 1u, 1u, args...);
 }
 #endif
 
@@ -83,6 +89,10 @@ void launch_copy_f32(cudaStream_t st, const void* src, int src_is_f32, float* ds
 // h[r] = embed[ids[r]]; xn[r] = bf16(rmsnorm(h[r]) * gain)
 void launch_embed_rmsnorm(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float eps,
                           float* h, bf16* xn, int R, int d);
+// producer side of the fused RMSNorm: h[r] = embed[ids[r]]; hb[r] = bf16(h[r] * gain);
+// sq[r * sq_stride] = sum of squares of h[r]
+void launch_embed_prep(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float* h, bf16* hb,
+                       float* sq, int sq_stride, int R, int d);
 // h[r] += sum_s partial[s][r] (s ascending); if gain: xn[r] = bf16(rmsnorm(h[r]) * gain)
 void launch_residual_rmsnorm(cudaStream_t st, const float* partial, int splits, size_t split_stride,
                              const float* gain, float eps, float* h, bf16* xn, int R, int d);
@@ -131,7 +141,13 @@ int launch_attention_verify(cudaStream_t st, const AttnArgs& a);
 constexpr int kAttnMaxClusterParts = 8;
 
 // ---------------------------------------------------------------- projections
-enum { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_LMHEAD = 2 };
+// EPI_RESIDUAL: the split-K CTAs of a tile form a cluster; they sum their accumulators through
+// distributed shared memory in split order, add the residual stream, and write the new stream
+// h (fp32), its bf16 copy times the next norm's gain (hb, the next projection's operand) and the
+// tile's share of every row's sum of squares.  The RMSNorm itself is then applied by the consumer:
+// rmsnorm(h) * g . W^T  ==  inv_rms(row) * ((h * g) . W^T), with inv_rms from the sums of squares.
+enum { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_LMHEAD = 2, EPI_RESIDUAL = 3 };
+constexpr int kGemmMaxClusterSplits = 8;
 struct GemmArgs {
   const bf16* x;  // [R][x_pitch] activations (K-major)
   const bf16* w;  // [N][w_pitch] weights (K-major), or the tile-contiguous layout below when w_tiled
@@ -147,6 +163,17 @@ struct GemmArgs {
   int* tile_arg;
   int mask_id;
   int* err_flag;         // device int set non-zero when a bounded wait expires
+  // consumer side of a fused RMSNorm: every output row r is multiplied by
+  // rsqrt(sum_{t < sq_count} sq[r * sq_stride + t] / norm_dim + norm_eps); sq == nullptr: no scaling
+  const float* sq;
+  int sq_count, sq_stride, norm_dim;
+  float norm_eps;
+  // EPI_RESIDUAL: splits = cluster size (<= kGemmMaxClusterSplits)
+  float* h;              // [R][N] fp32 residual stream, updated in place
+  bf16* hb;              // [R][N] bf16(h * gain)
+  const float* gain;     // [N]
+  float* sq_out;         // [R][sq_out_stride]: slot `tile` of a row receives the tile's sum of squares
+  int sq_out_stride;
 };
 int gemm_tiles(int N);
 void launch_gemm_simt(cudaStream_t st, const GemmArgs& g);

@@ -47,6 +47,8 @@ struct ssd_ctx {
   size_t partial_row_floats = 0;   // split-K workspace per row
   float* h = nullptr;
   bf16* xn = nullptr;
+  float* sq = nullptr;           // [R_cap][sq_stride] per-tile sums of squares of h (fused RMSNorm)
+  int sq_stride = 1;
   float* partial = nullptr;
   bf16 *q = nullptr, *lk = nullptr, *lv = nullptr, *att = nullptr, *act = nullptr;
   float* part_o = nullptr;
@@ -224,9 +226,24 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   if (kind == FWD_FILL && (size_t)n_parts * R > c->part_rows_parts)
     return fail(c, SSD_ERR_OVERFLOW, "attention workspace too small for %d parts x %d rows", n_parts, R);
   const int nl = c->cfg.n_layers;
+  // With the tensor-core projections the RMSNorms have no kernel of their own: a producer (the
+  // embedding gather, the O and down projections) writes the residual stream h, bf16(h * gain) in
+  // `xn` and per-tile sums of squares in `sq`; the consuming projection scales its output rows by
+  // 1/rms.  The bring-up projections keep the separate norm kernels.
+  const bool fused = c->gemm_impl == 1;
+  int sq_count = 1;                       // slots of `sq` the next consumer sums per row
+  auto consume_norm = [&](GemmArgs& ga) {
+    if (!fused) return;
+    ga.sq = c->sq; ga.sq_count = sq_count; ga.sq_stride = c->sq_stride; ga.norm_dim = d; ga.norm_eps = c->cfg.rms_eps;
+  };
+  auto produce_norm = [&](GemmArgs& ga, const float* gain, int splits) {
+    ga.epi = EPI_RESIDUAL; ga.splits = splits < kGemmMaxClusterSplits ? splits : kGemmMaxClusterSplits;
+    ga.h = c->h; ga.hb = c->xn; ga.gain = gain; ga.sq_out = c->sq; ga.sq_out_stride = c->sq_stride;
+  };
   {
     Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * 8);
-    launch_embed_rmsnorm(c->st, ids_dev, c->embed, c->L[0].g_attn, c->cfg.rms_eps, c->h, c->xn, R, d);
+    if (fused) launch_embed_prep(c->st, ids_dev, c->embed, c->L[0].g_attn, c->h, c->xn, c->sq, c->sq_stride, R, d);
+    else launch_embed_rmsnorm(c->st, ids_dev, c->embed, c->L[0].g_attn, c->cfg.rms_eps, c->h, c->xn, R, d);
   }
   for (int l = 0; l < nl; ++l) {
     const LayerW& w = c->L[l];
@@ -234,6 +251,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     GemmArgs g{};
     g.x = c->xn; g.w = w.wqkv; g.R = R; g.N = c->nqkv; g.K = d; g.x_pitch = d; g.w_pitch = d; g.w_tiled = 1;
     g.splits = c->split_qkv; g.epi = EPI_PARTIAL; g.out = c->partial;
+    consume_norm(g);
     if ((size_t)g.splits * R * g.N > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "split-K workspace too small");
     int rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_QKV);
     if (rc) return rc;
@@ -267,9 +285,12 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g = GemmArgs{};
     g.x = c->att; g.w = w.wo; g.R = R; g.N = d; g.K = c->qdim; g.x_pitch = c->qdim; g.w_pitch = c->qdim; g.w_tiled = 1;
     g.splits = c->split_o; g.epi = EPI_PARTIAL; g.out = c->partial;
+    if (fused) produce_norm(g, w.g_ffn, c->split_o);
     rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_O);
     if (rc) return rc;
-    {
+    if (fused) {
+      sq_count = gemm_tiles(d);
+    } else {
       Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * (4.0 * g.splits + 10.0));
       launch_residual_rmsnorm(c->st, c->partial, g.splits, (size_t)R * d, w.g_ffn, c->cfg.rms_eps, c->h, c->xn, R, d);
     }
@@ -277,8 +298,9 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g = GemmArgs{};
     g.x = c->xn; g.w = w.wgu; g.R = R; g.N = 2 * c->ffn_pad; g.K = d; g.x_pitch = d; g.w_pitch = d; g.w_tiled = 1;
     g.splits = 1;
-    if (c->gemm_impl == 1) {
+    if (fused) {
       g.epi = EPI_SWIGLU; g.act = c->act; g.act_pitch = c->ffn_pad;
+      consume_norm(g);
       rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_GU);
       if (rc) return rc;
     } else {
@@ -293,10 +315,11 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g = GemmArgs{};
     g.x = c->act; g.w = w.wd; g.R = R; g.N = d; g.K = c->ffn_pad; g.x_pitch = c->ffn_pad; g.w_pitch = c->ffn_pad; g.w_tiled = 1;
     g.splits = c->split_down; g.epi = EPI_PARTIAL; g.out = c->partial;
+    const float* gain = (l + 1 < nl) ? c->L[l + 1].g_attn : c->g_final;
+    if (fused) produce_norm(g, gain, c->split_down);
     rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_DOWN);
     if (rc) return rc;
-    {
-      const float* gain = (l + 1 < nl) ? c->L[l + 1].g_attn : c->g_final;
+    if (!fused) {
       Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * (4.0 * g.splits + 10.0));
       launch_residual_rmsnorm(c->st, c->partial, g.splits, (size_t)R * d, gain, c->cfg.rms_eps, c->h, c->xn, R, d);
     }
@@ -305,6 +328,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     GemmArgs g{};
     g.x = c->xn; g.w = c->lm_head; g.R = R; g.N = c->V; g.K = d; g.x_pitch = d; g.w_pitch = d; g.splits = 1; g.w_tiled = 1;
     g.mask_id = c->cfg.mask_id;
+    consume_norm(g);
     if (want_logits || c->gemm_impl != 1) {
       const size_t need = (size_t)R * c->V;
       if (need > c->logits_elems) {
@@ -431,6 +455,8 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     const size_t R = (size_t)c->R_cap;
     ALLOC(c, c->h, R * d);
     ALLOC(c, c->xn, R * d);
+    c->sq_stride = gemm_tiles(d);
+    ALLOC(c, c->sq, R * c->sq_stride);
     c->partial_row_floats = (size_t)kMaxSplit * d;
     if ((size_t)4 * c->nqkv > c->partial_row_floats) c->partial_row_floats = (size_t)4 * c->nqkv;
     if ((size_t)c->split_qkv * c->nqkv > c->partial_row_floats) c->partial_row_floats = (size_t)c->split_qkv * c->nqkv;

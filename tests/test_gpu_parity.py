@@ -110,8 +110,11 @@ def test_prefill_cache_matches_oracle(tiny_ssd, tiny_oracles, impl):
             k, v = tiny_ssd.read_cache(l, b, w.prompt_len)
             assert np.abs(k - cache.k[l]).max() < 2e-2 * max(1.0, np.abs(cache.k[l]).max())
             assert np.abs(v - cache.v[l]).max() < 2e-2 * max(1.0, np.abs(cache.v[l]).max())
-            # most entries identical after bf16 rounding
-            assert (np.abs(k - cache.k[l]) < 1e-6).mean() > 0.9
+            # Entry by entry the cache stays at bf16 rounding noise of the bf16-operand oracle (entries
+            # are O(0.3), one bf16 step there is 2e-3).  It is not bit-identical: the kernels apply
+            # RMSNorm after the contraction, inv_rms * ((h * g) . W^T), the oracle before it, so the
+            # two round different operands.
+            assert (np.abs(k - cache.k[l]) <= 4e-3).mean() > 0.99
 
 
 def _random_nodes(w, rng, n_nodes, T):
