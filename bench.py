@@ -27,6 +27,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "decode tokens/s at batch 1 (LLaDA-8B-shaped) and % HBM roofline per verify forward"
+# DRAM bytes per projection launch from the ncu capture summarised in
+# profiles/gemm_tc_kernel_llada8b_4layers.md (mean over the four projections of a LLaDA-8B-shaped layer).
+# Valid only for the kernel source it was taken from: reported as null once gemm.cu has changed.
+GEMM_TRAFFIC = {"workload": "llada8b", "bytes_per_launch": 112.97e6, "gemm_cu_sha256_16": "34f85685384169a9"}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -40,6 +44,18 @@ def load_peaks():
     d = dict(FALLBACK_PEAKS)
     d["_source"] = "fallback"
     return d
+
+
+def gemm_traffic(workload_name):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2510_04147_b200", "csrc", "gemm.cu")
+    try:
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    if sha != GEMM_TRAFFIC["gemm_cu_sha256_16"] or workload_name != GEMM_TRAFFIC["workload"]:
+        return None
+    return GEMM_TRAFFIC["bytes_per_launch"]
 
 
 def forward_bytes(w, n_seq, S):
@@ -356,7 +372,7 @@ def run_ours(args):
                           for k, v in prof.items() if k not in binding.PROF_TOP}
         roofline = {"bound": "hbm", "kernel": "gemm_tc_kernel (QKV/O/gate-up/down projections)",
                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                    "peak_source": peaks["_source"], "traffic": None,
+                    "peak_source": peaks["_source"], "traffic": gemm_traffic(args.workload) if not reduced else None,
                     "launches": g["launches"], "avg_launch_us": 1e3 * g["ms"] / max(1, g["launches"]),
                     "bytes_per_launch_avg": g["bytes"] / max(1, g["launches"]),
                     "family_share_of_device_time": {k: (prof[k]["ms"] / total_ms if total_ms else 0)
