@@ -267,6 +267,15 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
   float l_run[2] = {0.f, 0.f};
   uint32_t qf[HD / 16][4];
   const int qrow_w = rg * 16;                          // the warp's first row inside the query tile
+  // keys a query row may see in this part (no division in the inner loop): everything up to k_end for a
+  // prefix part, the row's own node for the local part
+  int node_lo[2], node_hi[2];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int qlr = lr0 + qrow_w + gq + i * 8;
+    node_lo[i] = local ? (qlr / T) * T : 0;
+    node_hi[i] = local ? min(node_lo[i] + T, k_end) : k_end;
+  }
   const bool rows_live = lr0 + qrow_w < rps;           // otherwise the warp only keeps the barriers
 
   for (int pair = 0; pair < n_pairs; ++pair) {
@@ -312,11 +321,8 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const int key = key0 + j * 8 + 2 * tq + (e & 1);
-          bool ok = key < k_end;
-          if (local) {
-            const int qlr = lr0 + qrow_w + gq + (e >> 1) * 8;
-            ok = ok && (key / T == qlr / T);
-          }
+          // local part: the key must lie in the query row's own node [node_lo, node_hi)
+          const bool ok = key >= node_lo[e >> 1] && key < node_hi[e >> 1];
           const float v = ok ? s[j][e] * scale_log2 : -INFINITY;
           s[j][e] = v;
           mx[e >> 1] = fmaxf(mx[e >> 1], v);
