@@ -395,7 +395,8 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
   __syncthreads();
   // ---- the two key sets of this CTA are merged first (set 0, then set 1), in place
   float2* sML2 = sML + 2 * kQTile;                      // [QT] merged (max, sum)
-  for (int it = tid; it < kQTile * (HD / 4); it += kVerifyThreads) {
+#pragma unroll
+  for (int it = tid; it < kQTile * (HD / 4); it += kVerifyThreads) {   // HD / 16 iterations, independent
     const int row = it / (HD / 4), c4 = (it % (HD / 4)) * 4;
     const float2 ml0 = sML[row], ml1 = sML[kQTile + row];
     const float M = fmaxf(ml0.x, ml1.x);
