@@ -505,11 +505,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   }
   if (p.epi == EPI_RESIDUAL) {
     // ---- split-K reduction inside the cluster + residual + operand of the next projection.
-    // Per chunk of 32 rows: every CTA stages its partial [32 rows][128 features] in shared memory;
+    // Per pass (all rows when the tile ring can hold them): every CTA stages its partial [rows][128
+    // features] in shared memory;
     // after a cluster barrier CTA `rank` owns the rows rank, rank + splits, ... (one warp per row, a
     // lane per four features): it adds the partials in split order to the residual stream, writes h,
     // bf16(h * gain) and the tile's sum of squares of the row.  A second barrier frees the staging
-    // buffer.  Every thread of every CTA passes both barriers of every chunk, also after an error.
+    // buffer.  Every thread of every CTA passes both barriers of every pass, also after an error.
     const bool epi_warp = warp >= 2;
     const int quad = warp & 3;
     const int lrow = quad * 32 + lane;
@@ -522,19 +523,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const bool col_ok = n_base + f4 < p.N;
     float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f);
     if (epi_warp && col_ok) g4 = *reinterpret_cast<const float4*>(p.gain + n_base + f4);
-    for (int c0 = 0; c0 < p.npad; c0 += 32) {
+    // as many 32-row chunks per pass as the (now idle) tile ring can stage
+    int pass_rows = (p.stages * (kWTileBytes + x_tile_bytes)) / (kEpiPitch * 4) / 32 * 32;
+    const int npad32 = (p.npad + 31) & ~31;               // whole chunks (TMEM holds a power of two >= 32 columns)
+    if (pass_rows > npad32) pass_rows = npad32;
+    for (int g0 = 0; g0 < npad32; g0 += pass_rows) {
+      const int pass_cnt = min(pass_rows, npad32 - g0);
       if (epi_warp && epi_ok) {
-        float v[32];
-        tmem_ld32(taddr + c0, v);
+        for (int c0 = 0; c0 < pass_cnt; c0 += 32) {
+          float v[32];
+          tmem_ld32(taddr + g0 + c0, v);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) scratch[j * kEpiPitch + lrow] = v[j];
+          for (int j = 0; j < 32; ++j) scratch[(c0 + j) * kEpiPitch + lrow] = v[j];
+        }
       }
       __syncwarp();
       cluster_arrive_release();
       cluster_wait_acquire();
       if (epi_warp && epi_ok) {
-        for (int rr = (int)rank + (warp - 2) * (int)n_ranks; rr < 32; rr += 4 * (int)n_ranks) {
-          const int row = c0 + rr;
+        for (int rr = (int)rank + (warp - 2) * (int)n_ranks; rr < pass_cnt; rr += 4 * (int)n_ranks) {
+          const int row = g0 + rr;
           if (row >= rows_here) break;
           float4 part[kGemmMaxClusterSplits];
 #pragma unroll
