@@ -119,6 +119,12 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
       cp_async16(dV + swz<HD>(row, ch), vbase + off, valid);
     }
   };
+  // block commit: the first query head of a KV group also stores the rows' K/V into the cache.
+  // Sequence-local row lr is in-block index lr (one node per sequence) at position pos0 + lr.
+  const bool commit_kv = a.cache_k_out != nullptr && (h % (a.H / a.Hkv)) == 0;
+  auto cache_row = [&](int lr) -> size_t {
+    return (size_t)seq_of_slot(a.map, slot) * a.cache_seq_stride + ((size_t)(a.map.pos0 + lr) * a.Hkv + kvh) * HD;
+  };
   // ---- one chunk (8 rotation pairs) of one row of a head of the fused projection: sum over the
   //      splits in split order (four splits' loads in flight at a time), rotary embedding, bf16
   auto rot_item = [&](int lr, int c, int col0, uint4& lo, uint4& hi) {
@@ -204,11 +210,17 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
       if (key0 + row < k_end) rot_item(key0 + row, c, (a.H + kvh) * HD, lo, hi);
       *reinterpret_cast<uint4*>(dK + swz<HD>(row, c)) = lo;
       *reinterpret_cast<uint4*>(dK + swz<HD>(row, c + CPR)) = hi;
+      if (commit_kv && key0 + row < k_end) {
+        bf16* dst = a.cache_k_out + cache_row(key0 + row) + c * 8;
+        *reinterpret_cast<uint4*>(dst) = lo;
+        *reinterpret_cast<uint4*>(dst + HALF) = hi;
+      }
     }
     for (int idx = tid; idx < kPairKeys * CH; idx += kVerifyThreads) {
       const int row = idx / CH, c = idx % CH;
-      *reinterpret_cast<uint4*>(dV + swz<HD>(row, c)) =
-          (key0 + row < k_end) ? plain_item(key0 + row, c, (a.H + a.Hkv + kvh) * HD) : zero;
+      const uint4 v = (key0 + row < k_end) ? plain_item(key0 + row, c, (a.H + a.Hkv + kvh) * HD) : zero;
+      *reinterpret_cast<uint4*>(dV + swz<HD>(row, c)) = v;
+      if (commit_kv && key0 + row < k_end) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(key0 + row) + c * 8) = v;
     }
   };
 
@@ -251,10 +263,16 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
         if (row < lk_rows) rot_item(lk_begin + row, c, (a.H + kvh) * HD, lo, hi);
         st_cluster_u4(map_to_rank(lK + swz<HD>(row, c), (uint32_t)n_prefix_parts), lo);
         st_cluster_u4(map_to_rank(lK + swz<HD>(row, c + CPR), (uint32_t)n_prefix_parts), hi);
+        if (commit_kv && row < lk_rows) {
+          bf16* dst = a.cache_k_out + cache_row(lk_begin + row) + c * 8;
+          *reinterpret_cast<uint4*>(dst) = lo;
+          *reinterpret_cast<uint4*>(dst + HALF) = hi;
+        }
       } else {
         const int row = (it - n_q - n_k) / CH, c = (it - n_q - n_k) % CH;
         const uint4 v = (row < lk_rows) ? plain_item(lk_begin + row, c, (a.H + a.Hkv + kvh) * HD) : zero;
         st_cluster_u4(map_to_rank(lV + swz<HD>(row, c), (uint32_t)n_prefix_parts), v);
+        if (commit_kv && row < lk_rows) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(lk_begin + row) + c * 8) = v;
       }
     }
     cluster_sync_all();
@@ -455,6 +473,8 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
 int launch_attention_verify(cudaStream_t st, const AttnArgs& a) {
   if (a.hd != 64 && a.hd != 128) return -2;
   if (!a.qkv_partial || !a.rope || a.kv_split < kKTile || (a.kv_split % kKTile)) return -1;
+  if ((a.cache_k_out != nullptr) != (a.cache_v_out != nullptr)) return -1;
+  if (a.cache_k_out != nullptr && a.map.rows_per_seq != a.map.T) return -1;   // commit: one node per sequence
   const int n_prefix = (a.S + a.kv_split - 1) / a.kv_split;
   const int n_parts = n_prefix + 1;
   if (n_parts > kAttnMaxClusterParts) return -2;

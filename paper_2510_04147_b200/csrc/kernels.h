@@ -118,6 +118,10 @@ struct AttnArgs {
   int qkv_splits;
   size_t qkv_split_stride;
   const float2* rope;         // [max_seq][hd/2] (cos, sin)
+  // block commit through the verification form (one node per sequence, rows_per_seq == T): the
+  // rotated K and the V of the rows are also written to the cache at their absolute positions
+  bf16* cache_k_out;          // layer base like cache_k, or nullptr
+  bf16* cache_v_out;
   const bf16* q;        // [R][H][hd], rotated
   const bf16* cache_k;  // layer base: [seq][max_seq][Hkv][hd]
   const bf16* cache_v;

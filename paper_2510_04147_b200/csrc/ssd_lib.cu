@@ -220,10 +220,16 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   const int d = c->d, H = c->H, Hkv = c->Hkv, hd = c->hd;
   const int S = map.pos0;
   if (R > c->R_cap) return fail(c, SSD_ERR_OVERFLOW, "forward of %d rows exceeds capacity %d", R, c->R_cap);
-  const int attn_S = (kind == FWD_FILL) ? S + map.T : S;
-  const int kv_split = (kind == FWD_FILL) ? attn_S : kv_split_for(c, S);
+  // A block commit is a one-node verification forward whose K/V also go to the cache: it takes the
+  // verification attention kernel.  Only the prefill (many rows, empty cache) fills through the
+  // rotary pass and the cache-reading attention.
+  const bool commit_form = kind == FWD_FILL && c->gemm_impl == 1 && S > 0 && map.rows_per_seq == map.T &&
+                           map.T <= c->cfg.block_len;
+  const bool via_cache = kind == FWD_FILL && !commit_form;
+  const int attn_S = via_cache ? S + map.T : S;
+  const int kv_split = via_cache ? attn_S : kv_split_for(c, S);
   const int n_parts = (attn_S + kv_split - 1) / kv_split;
-  if (kind == FWD_FILL && (size_t)n_parts * R > c->part_rows_parts)
+  if (via_cache && (size_t)n_parts * R > c->part_rows_parts)
     return fail(c, SSD_ERR_OVERFLOW, "attention workspace too small for %d parts x %d rows", n_parts, R);
   const int nl = c->cfg.n_layers;
   // With the tensor-core projections the RMSNorms have no kernel of their own: a producer (the
@@ -262,7 +268,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     a.R = R; a.H = H; a.Hkv = Hkv; a.hd = hd; a.S = attn_S; a.kv_split = kv_split;
     a.cache_seq_stride = c->cache_seq_stride; a.map = map; a.n_seq_slots = n_slots;
     const double kvb = (double)n_slots * attn_S * Hkv * hd * 4.0 + (double)R * (H + 2 * Hkv) * hd * 2.0 + (double)R * H * hd * 2.0;
-    if (kind == FWD_FILL) {
+    if (via_cache) {
       // the rotary pass writes K/V into the cache; attention then reads the cache, which holds the rows themselves
       {
         Scope sc(c, SSD_PROF_ELEMWISE, (double)R * c->nqkv * (4.0 * g.splits + 2.0));
@@ -277,9 +283,14 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     } else {
       // rotary embedding, node-local K/V and the merge of the key parts happen inside the attention kernel
       a.qkv_partial = c->partial; a.qkv_splits = g.splits; a.qkv_split_stride = (size_t)R * c->nqkv; a.rope = c->rope;
+      if (commit_form) {
+        a.cache_k_out = c->cacheK + (size_t)l * c->cache_layer_stride;
+        a.cache_v_out = c->cacheV + (size_t)l * c->cache_layer_stride;
+      }
       Scope sc(c, SSD_PROF_ATTN, kvb, 1);
       const int arc = launch_attention_verify(c->st, a);
       if (arc != 0) return fail(c, arc, "verification attention rejected S=%d kv_split=%d (code %d)", attn_S, kv_split, arc);
+      if (commit_form && l == nl - 1) break;   // the last layer's K/V are in the cache; nothing reads its output
     }
     // ---- output projection + residual + norm
     g = GemmArgs{};
