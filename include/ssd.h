@@ -187,12 +187,16 @@ int64_t ssd_launch_count(const ssd_ctx* ctx);
 int ssd_profile_enable(ssd_ctx* ctx, int32_t on);
 int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, double* bytes);
 
-/* Tuning knobs (set before prefill).  key: "split_k_qkv", "split_k_o", "split_k_down" (1..16, bounded by
- * the split-K workspace),
- * "kv_split" (prefix keys per attention split, multiple of 64; 0 = automatic from the prefix
- * length), "max_drafts" (lower the draft-length cap below the capacity fixed at creation),
- * "gemm_impl" (1 = TMA + tcgen05 kernel, the default; 0 = the plain CUDA-core bring-up kernel,
- * for cross-checks only).  Unknown key: SSD_ERR_INVALID_ARG. */
+/* Tuning knobs (set before prefill).  key:
+ *   "split_k_qkv", "split_k_o", "split_k_down"  split-K factor of a projection, 1..16, bounded by the
+ *        split-K workspace; with the tensor-core kernel the O and down projections reduce their
+ *        splits inside a thread-block cluster and use at most 8;
+ *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically while
+ *        a prefix would need more than 7 parts;
+ *   "max_drafts" lower the draft-length cap below the capacity fixed at creation;
+ *   "gemm_impl"  1 = TMA + tcgen05 kernel with fused RMSNorm / residual epilogues, the default;
+ *        0 = the plain CUDA-core bring-up kernel with separate norm kernels, for cross-checks only.
+ * Unknown key: SSD_ERR_INVALID_ARG. */
 int ssd_set_option(ssd_ctx* ctx, const char* key, int32_t value);
 
 #ifdef __cplusplus

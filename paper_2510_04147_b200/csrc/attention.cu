@@ -1,12 +1,13 @@
-// Shared-prefix bidirectional attention for the verification forward (Eq. 5).
+// Bidirectional attention of the cache-fill forward (prefill of the prompt, and any forward whose
+// rows were first written to the KV cache by the rotary pass): every query row attends, without a
+// causal mask, to the cached keys of its sequence, which include the rows themselves.
 //
-// Rows are ordered [sequence slot][node][in-block index].  Every query row attends, without any
-// causal mask, to the cached prefix keys of its sequence and to the keys of ITS OWN node's block.
-// The prefix is cut into splits whose boundaries depend on the prefix length only; a CTA owns
-// (64 query rows of one sequence, one head, one split) and streams the split's K/V tiles through
-// shared memory once for all of those rows, i.e. once for all tree nodes.  The node-local keys
-// form one more part, masked block-diagonally (key and query must belong to the same node).
-// Parts are merged in part order by a second kernel (log-sum-exp merge, fixed order).
+// Rows are ordered [sequence slot][node][in-block index].  The keys are cut into parts whose
+// boundaries depend on the key count only; a CTA owns (64 query rows of one sequence, one head, one
+// part) and streams the part's K/V tiles through shared memory once for all of those rows.  An
+// optional node-local part (keys given outside the cache, masked block-diagonally) is supported
+// for cross-checks.  Parts are merged in part order by a second kernel (log-sum-exp, fixed order).
+// The verification forward and the block commit use attention_verify.cu instead.
 //
 // Tensor-core work uses warp-level mma.sync (bf16 in, fp32 accumulate): attention is < 3 % of the
 // forward's flops and is bound by the K/V stream and by latency, not by the tensor pipe.

@@ -50,7 +50,7 @@ struct ssd_ctx {
   float* sq = nullptr;           // [R_cap][sq_stride] per-tile sums of squares of h (fused RMSNorm)
   int sq_stride = 1;
   float* partial = nullptr;
-  bf16 *q = nullptr, *lk = nullptr, *lv = nullptr, *att = nullptr, *act = nullptr;
+  bf16 *q = nullptr, *att = nullptr, *act = nullptr;
   float* part_o = nullptr;
   float2* part_ml = nullptr;
   float *tile_max = nullptr, *tile_sum = nullptr;
@@ -475,13 +475,9 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     c->partial_elems = R * c->partial_row_floats;
     ALLOC(c, c->partial, c->partial_elems);
     ALLOC(c, c->q, R * c->qdim);
-    ALLOC(c, c->lk, R * c->kvdim);
-    ALLOC(c, c->lv, R * c->kvdim);
     ALLOC(c, c->att, R * c->qdim);
     ALLOC(c, c->act, R * c->ffn_pad);
-    const size_t dec_parts = (size_t)(k.max_seq + 255) / 256 + 1;
-    c->part_rows_parts = (size_t)c->R_dec * dec_parts;
-    if ((size_t)k.max_seq > c->part_rows_parts) c->part_rows_parts = k.max_seq;
+    c->part_rows_parts = R;      // the cache-fill attention runs one key part per query tile
     ALLOC(c, c->part_o, c->part_rows_parts * c->qdim);
     ALLOC(c, c->part_ml, c->part_rows_parts * c->H);
     const size_t tiles = gemm_tiles(c->V);
