@@ -35,6 +35,8 @@ __device__ __forceinline__ void cluster_arrive() {
   __syncwarp();
   asm volatile("barrier.cluster.arrive.release;" ::: "memory");
 }
+// per-thread form for code where the threads of a warp may have diverged
+__device__ __forceinline__ void cluster_arrive_thread() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
 __device__ __forceinline__ void st_cluster_u4(uint32_t addr, uint4 v) {
   asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -432,8 +434,12 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
   //      issued before the first use, the parts are merged in part order
   constexpr int TPR = HD / 8;                           // threads per row, eight columns each
   const int col = (tid % TPR) * 8;
-  for (int row = part + (tid / TPR) * n_parts; row < kQTile; row += (kVerifyThreads / TPR) * n_parts) {
+  bool arrived = false;     // final barrier: arrive once the last remote read has landed, wait before leaving
+  constexpr int kRowStepUnits = kVerifyThreads / TPR;
+  for (int row = part + (tid / TPR) * n_parts; row < kQTile; row += kRowStepUnits * n_parts) {
     if (lr0 + row >= rps) break;
+    const int next_row = row + kRowStepUnits * n_parts;
+    const bool last_row = next_row >= kQTile || lr0 + next_row >= rps;
     float2 ml[kAttnMaxClusterParts];
     float4 va[kAttnMaxClusterParts], vb[kAttnMaxClusterParts];
 #pragma unroll
@@ -460,12 +466,14 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
       acc0.x += va[pp].x * w; acc0.y += va[pp].y * w; acc0.z += va[pp].z * w; acc0.w += va[pp].w * w;
       acc1.x += vb[pp].x * w; acc1.y += vb[pp].y * w; acc1.z += vb[pp].z * w; acc1.w += vb[pp].w * w;
     }
+    if (last_row) { cluster_arrive_thread(); arrived = true; }
     const float inv = 1.f / L;
     *reinterpret_cast<uint4*>(a.out + ((grow0 + row) * a.H + h) * HD + col) =
         make_uint4(pack_bf16(acc0.x * inv, acc0.y * inv), pack_bf16(acc0.z * inv, acc0.w * inv),
                    pack_bf16(acc1.x * inv, acc1.y * inv), pack_bf16(acc1.z * inv, acc1.w * inv));
   }
-  cluster_sync_all();    // nobody leaves while its shared memory may still be read
+  if (!arrived) cluster_arrive_thread();
+  cluster_wait();        // nobody leaves while its shared memory may still be read
 }
 
 }  // namespace

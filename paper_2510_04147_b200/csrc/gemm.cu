@@ -540,6 +540,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       __syncwarp();
       cluster_arrive_release();
       cluster_wait_acquire();
+      bool arrived = false;
       if (epi_warp && epi_ok) {
         for (int rr = (int)rank + (warp - 2) * (int)n_ranks; rr < pass_cnt; rr += 4 * (int)n_ranks) {
           const int row = g0 + rr;
@@ -557,6 +558,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           for (int q = 0; q < kGemmMaxClusterSplits; ++q) {
             if ((uint32_t)q < n_ranks) { acc.x += part[q].x; acc.y += part[q].y; acc.z += part[q].z; acc.w += part[q].w; }
           }
+          // this warp's last remote read of the pass has landed: arrive now, the stores overlap the barrier
+          if (rr + 4 * (int)n_ranks >= pass_cnt || g0 + rr + 4 * (int)n_ranks >= rows_here) { __syncwarp(); cluster_arrive_release(); arrived = true; }
           float ss = 0.f;
           if (col_ok) {
             *reinterpret_cast<float4*>(hp) = acc;
@@ -571,8 +574,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           if (lane == 0) p.sq_out[(size_t)(row0 + row) * p.sq_out_stride + tile] = ss;
         }
       }
-      __syncwarp();
-      cluster_arrive_release();
+      if (!arrived) { __syncwarp(); cluster_arrive_release(); }
       cluster_wait_acquire();
     }
   }
