@@ -166,3 +166,56 @@ def test_batched_full_width_sequences_equal_single_runs():
         assert np.array_equal(tok_b[i], singles[i][0][0])
         assert np.array_equal(acc_b[i], singles[i][1][0])
         assert nf_b[i] == singles[i][2][0]
+
+
+# ------------------------------------------------------------------------------------------
+# degenerate and extreme shapes of the method
+# ------------------------------------------------------------------------------------------
+EDGE = wl.TINY.replace(name="edge", lm_head_scale=8.0)
+
+
+@pytest.mark.parametrize("block_len,prompt_len,gen_len", [
+    (1, 32, 5),       # B = 1: every block is a single stepwise step, SSD has nothing to draft
+    (16, 1, 32),      # the shortest prompt: one cached key
+    (256, 40, 256),   # the largest block: several 128-key steps in the local attention part, 256-row commit
+    (48, 33, 100),    # odd sizes: block not a multiple of 16 or 32, ragged last block
+])
+def test_extreme_blocks_ssd_equals_stepwise_and_oracle_steps(block_len, prompt_len, gen_len):
+    w = EDGE.replace(block_len=block_len, prompt_len=prompt_len, gen_len=gen_len)
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    ssd = _make(w, max_drafts=min(3, block_len))
+    try:
+        ssd.prefill(prompt)
+        tok_step, acc_step, nf_step = ssd.generate(b.MODE_STEPWISE, gen_len, block_len, 1)
+        ssd.prefill(prompt)
+        tok_ssd, acc_ssd, nf_ssd = ssd.generate(b.MODE_SSD, gen_len, block_len, 1)
+        assert ssd.cache_length() == prompt_len + gen_len
+        # teacher-forced first forward of the second block against the oracle (prefix = prompt + block 0)
+        first = min(block_len, gen_len)
+        ssd.prefill(prompt)
+        ssd.block_begin(first)
+        ssd.set_block_state(tok_step[:, :first], np.zeros((1, first), np.uint8))
+        ssd.block_commit()
+        T = min(block_len, gen_len - first)
+        if T > 0:
+            ids = np.full((1, 1, T), w.mask_id)
+            tok_g, conf_g, _ = ssd.verify_forward(ids, np.ones((1, 1, T), np.uint8))
+    finally:
+        ssd.destroy()
+    assert np.array_equal(tok_step, tok_ssd)                       # losslessness
+    assert tok_step.shape == (1, gen_len)
+    for acc, nf in zip(acc_ssd, nf_ssd):
+        used = acc[0][:nf[0]]
+        assert used.sum() == min(block_len, acc.shape[1]) and np.all(used >= 1) and np.all(used <= 4)
+    for acc, nf in zip(acc_step, nf_step):
+        assert np.all(acc[0][:nf[0]] == 1)
+    if T > 0:
+        o = make_oracle(w, as_bf16=True)
+        cache = o.prefill(prompt[0])
+        o.commit_block(tok_step[0, :first], cache)
+        otok, oconf, ogap, _ = o.verify(ids[0, 0][None], np.ones((1, T), bool), cache)
+        scale = w.lm_head_scale
+        assert np.allclose(conf_g[0, 0], oconf[0], rtol=CONF_RTOL * scale, atol=1e-6)
+        sure = (ogap[0] > GAP) & (ogap[0] > 2 * CONF_RTOL * scale * oconf[0])
+        assert np.array_equal(tok_g[0, 0][sure], otok[0][sure])
