@@ -230,7 +230,7 @@ def run_ours(args):
     torch.cuda.set_stream(stream)
     ssd = binding.Ssd(binding.config_from_workload(w, max_drafts=min(cfg_drafts, B - 1)))
     for k, v in (("split_k_qkv", args.split_qkv), ("split_k_o", args.split_o), ("split_k_down", args.split_down),
-                 ("kv_split", args.kv_split)):
+                 ("kv_split", args.kv_split), ("attn_impl", args.attn_impl)):
         if v is not None:
             ssd.set_option(k, v)
     t0 = time.time()
@@ -425,6 +425,7 @@ def main():
     ap.add_argument("--split-o", type=int, default=None)
     ap.add_argument("--split-down", type=int, default=None)
     ap.add_argument("--kv-split", type=int, default=None)
+    ap.add_argument("--attn-impl", type=int, default=None, help="0: mma.sync attention; 1: tcgen05 attention where eligible")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: fewer layers of the same shape")
     ap.add_argument("--gen-len", type=int, default=0, help="profiling only: shorter generation")

@@ -194,6 +194,9 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically while
  *        a prefix would need more than 7 parts;
  *   "max_drafts" lower the draft-length cap below the capacity fixed at creation;
+ *   "attn_impl"  1 = attention of the verification forward on tcgen05 where the shape allows (head
+ *        dimension 128, prefix <= 896 keys, block length dividing 128), the default; 0 = always the
+ *        mma.sync form;
  *   "gemm_impl"  1 = TMA + tcgen05 kernel with fused RMSNorm / residual epilogues, the default;
  *        0 = the plain CUDA-core bring-up kernel with separate norm kernels, for cross-checks only.
  * Unknown key: SSD_ERR_INVALID_ARG. */

@@ -122,6 +122,7 @@ struct AttnArgs {
   // rotated K and the V of the rows are also written to the cache at their absolute positions
   bf16* cache_k_out;          // layer base like cache_k, or nullptr
   bf16* cache_v_out;
+  int* err_flag;              // device int set non-zero when a bounded wait expires (tcgen05 form)
   const bf16* q;        // [R][H][hd], rotated
   const bf16* cache_k;  // layer base: [seq][max_seq][Hkv][hd]
   const bf16* cache_v;
@@ -142,6 +143,11 @@ void launch_attention(cudaStream_t st, const AttnArgs& a, int* launches);
 // key parts (through a thread-block cluster) inside.  Needs prefix parts + 1 <= kAttnMaxClusterParts.
 // Returns 0 or a negative ssd error code.
 int launch_attention_verify(cudaStream_t st, const AttnArgs& a);
+// The same on the tcgen05 tensor cores, for head dimension 128, kv_split 128 (<= 7 prefix parts) and
+// node-local keys that fit one 128-key tile; needs a.err_flag.  Returns 0 (launched), 1 (shape not
+// covered: use launch_attention_verify) or a negative ssd error code.  v_desc_swap: test hook that
+// swaps the two stride fields of the V operand descriptor.
+int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a, int v_desc_swap);
 constexpr int kAttnMaxClusterParts = 8;
 
 // ---------------------------------------------------------------- projections

@@ -70,6 +70,7 @@ struct ssd_ctx {
   std::vector<int> h_remaining, h_has_drafts;
 
   int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0, gemm_impl = 1;
+  int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
   int64_t launches = 0;
   bool profiling = false;
   std::vector<ProfRec> prof;
@@ -288,7 +289,10 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
         a.cache_v_out = c->cacheV + (size_t)l * c->cache_layer_stride;
       }
       Scope sc(c, SSD_PROF_ATTN, kvb, 1);
-      const int arc = launch_attention_verify(c->st, a);
+      a.err_flag = c->flags;
+      int arc = 1;
+      if (c->attn_impl == 1) arc = launch_attention_verify_tc(c->st, a, 0);   // 1: shape not covered by the tcgen05 form
+      if (arc == 1) arc = launch_attention_verify(c->st, a);
       if (arc != 0) return fail(c, arc, "verification attention rejected S=%d kv_split=%d (code %d)", attn_S, kv_split, arc);
       if (commit_form && l == nl - 1) break;   // the last layer's K/V are in the cache; nothing reads its output
     }
@@ -878,6 +882,11 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "max_drafts")) {
     if (value < 0 || value + 1 > c->n_max) return fail(c, SSD_ERR_INVALID_ARG, "max_drafts must be in [0, %d] (the capacity fixed at creation)", c->n_max - 1);
     c->cfg.max_drafts = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "attn_impl")) {
+    if (value != 0 && value != 1) return fail(c, SSD_ERR_INVALID_ARG, "attn_impl is 0 (mma.sync) or 1 (tcgen05 where the shape allows)");
+    c->attn_impl = value;
     return SSD_OK;
   }
   if (!strcmp(key, "gemm_impl")) {

@@ -219,3 +219,27 @@ def test_extreme_blocks_ssd_equals_stepwise_and_oracle_steps(block_len, prompt_l
         assert np.allclose(conf_g[0, 0], oconf[0], rtol=CONF_RTOL * scale, atol=1e-6)
         sure = (ogap[0] > GAP) & (ogap[0] > 2 * CONF_RTOL * scale * oconf[0])
         assert np.array_equal(tok_g[0, 0][sure], otok[0][sure])
+
+
+def test_both_attention_forms_agree_at_full_width():
+    """The tcgen05 attention (default where the shape allows) and the mma.sync form compute the same
+    forward up to the rounding of a different summation order."""
+    w, n_nodes = WIDTH_CASES["llada_width"]
+    rng = np.random.default_rng(3)
+    T = w.block_len
+    prompt = wl.make_prompts(w).numpy()
+    ids, masked = _nodes(w, rng, n_nodes, T)
+    out = {}
+    ssd = _make(w, max_drafts=n_nodes)
+    try:
+        for impl in (0, 1):
+            ssd.set_option("attn_impl", impl)
+            ssd.prefill(prompt)
+            tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
+            out[impl] = (tok, conf, logits)
+    finally:
+        ssd.destroy()
+    assert np.abs(out[0][2] - out[1][2]).max() < 2e-2          # same bf16 rounding noise level, no bias
+    assert np.sqrt(((out[0][2] - out[1][2]) ** 2).mean()) < 4e-3
+    m = masked[0]
+    assert np.allclose(out[0][1][0][m], out[1][1][0][m], rtol=2e-2)
