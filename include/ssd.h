@@ -191,11 +191,11 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "split_k_qkv", "split_k_o", "split_k_down"  split-K factor of a projection, 1..16, bounded by the
  *        split-K workspace; with the tensor-core kernel the O and down projections reduce their
  *        splits inside a thread-block cluster and use at most 8;
- *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically while
- *        a prefix would need more than 7 parts;
+ *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically (in
+ *        steps of 128) while a prefix would need more than 7 parts;
  *   "max_drafts" lower the draft-length cap below the capacity fixed at creation;
  *   "attn_impl"  1 = attention of the verification forward on tcgen05 where the shape allows (head
- *        dimension 128, prefix <= 896 keys, block length dividing 128), the default; 0 = always the
+ *        dimension 128, parts of whole 128-key tiles, block length dividing 128), the default; 0 = always the
  *        mma.sync form;
  *   "gemm_impl"  1 = TMA + tcgen05 kernel with fused RMSNorm / residual epilogues, the default;
  *        0 = the plain CUDA-core bring-up kernel with separate norm kernels, for cross-checks only.

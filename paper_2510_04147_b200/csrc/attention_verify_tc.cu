@@ -1,5 +1,5 @@
 // Shared-prefix bidirectional attention of the verification forward (Eq. 5) on the tcgen05 tensor
-// cores: the form for head dimension 128 and key parts of at most 128 keys.
+// cores: the form for head dimension 128 and key parts that are whole 128-key tiles.
 //
 // Same decomposition as attention_verify.cu - the key parts of one (query tile, head) form a cluster,
 // one CTA per part, rotary prologue shared by the cluster's threads, parts merged through
@@ -15,7 +15,9 @@
 // Shared-memory tiles are [64-column half][128 rows][64 columns] bf16 with the 128-byte swizzle the
 // tensor core expects (16-byte chunk c of row r at chunk c ^ (r & 7)).  A query tile of 32 or 64
 // rows is replicated to 128, so that 4 or 2 threads share a row's softmax (each takes a slice of
-// the keys) and the read-out of its output row.  P overwrites Q once S is complete.
+// the keys) and the read-out of its output row.  P overwrites the K tile once S is complete.  A part
+// of several tiles runs them in order with a running (max, sum) per row; the output accumulator in
+// tensor memory is rescaled in place before a later tile is added (online softmax).
 #include "attn_common.cuh"
 
 #include <cuda.h>
@@ -27,7 +29,7 @@ namespace {
 using namespace attn;
 
 constexpr int kHD = 128;
-constexpr int kKeys = 128;                  // keys per part (one MMA tile)
+constexpr int kKeys = 128;                  // keys per MMA tile
 constexpr int kTcAttnThreads = 128;
 constexpr int kHalfBytesKV = kKeys * 128;   // one 64-column half of a 128-row tile
 constexpr unsigned long long kAttnWaitLimitNs = 2000000000ull;
@@ -99,6 +101,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// the inverse of tmem_ld32: the thread's lane, 32 consecutive columns
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  uint32_t r[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void cluster_arrive() {
   __syncwarp();
   asm volatile("barrier.cluster.arrive.release;" ::: "memory");
@@ -137,15 +155,17 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
                                                                           int v_desc_swap) {
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;                                   // [2][128][64] bf16; P overwrites it once S is complete
-  uint8_t* sK = sQ + 2 * kHalfBytesKV;                  // [2][128][64]
+  uint8_t* sQ = smem;                                   // [2][128][64] bf16
+  uint8_t* sK = sQ + 2 * kHalfBytesKV;                  // [2][128][64]; P overwrites it once S is complete
   uint8_t* sV = sK + 2 * kHalfBytesKV;                  // [2][128][64]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * kHalfBytesKV);   // [0] S ready, [1] O ready
+  float* sMax = reinterpret_cast<float*>(sV + 2 * kHalfBytesKV);         // [4 copies][128 rows]
+  float* sSum = sMax + 4 * 128;                                          // [4 key groups][128 rows]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sSum + 4 * 128);          // [0] S ready, [1] O ready
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2);
   constexpr int HALF = kHD / 2, CPR = HALF / 8, CH = kHD / 8;
 
   pdl_launch_dependents();
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5;
   const int n_parts = n_prefix_parts + 1;
   const int part = blockIdx.x, h = blockIdx.y;          // the cluster spans x
   const int q_tiles = (a.map.rows_per_seq + QT - 1) / QT;
@@ -159,13 +179,14 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
 
   int k_begin, k_end;
   if (!local) {
-    k_begin = part * kKeys;
-    k_end = min(a.S, k_begin + kKeys);
+    k_begin = part * a.kv_split;                        // a multiple of 128 keys per part
+    k_end = min(a.S, k_begin + a.kv_split);
   } else {
     const int last = min(lr0 + QT - 1, rps - 1);
     k_begin = (lr0 / T) * T;
     k_end = (last / T + 1) * T;                         // the launcher guarantees k_end - k_begin <= 128
   }
+  const int n_tiles = (k_end - k_begin + kKeys - 1) / kKeys;
 
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), 1);
@@ -178,16 +199,17 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   }
 
   // ---- prefix K/V straight from the cache (zero rows past the end of the part)
-  auto load_prefix = [&]() {
+  auto load_prefix = [&](int tile) {
     const int seq = seq_of_slot(a.map, slot);
+    const int kb = k_begin + tile * kKeys;
     const bf16* kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * kHD;
     const bf16* vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * kHD;
     const size_t krow_stride = (size_t)a.Hkv * kHD;
     for (int idx = tid; idx < kKeys * CH; idx += kTcAttnThreads) {
       const int row = idx / CH, ch = idx % CH;
-      const int key = k_begin + row;
+      const int key = kb + row;
       const bool valid = key < k_end;
-      const size_t off = (size_t)(valid ? key : k_begin) * krow_stride + ch * 8;
+      const size_t off = (size_t)(valid ? key : kb) * krow_stride + ch * 8;
       cp_async16(sK + tile_off(row, ch, kKeys), kbase + off, valid);
       cp_async16(sV + tile_off(row, ch, kKeys), vbase + off, valid);
     }
@@ -271,10 +293,10 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   // The cache is not written by any kernel of this forward, so its tiles may be requested before the
   // dependency wait - unless the slot -> sequence map is only known on the device.
   const bool early = a.map.n_inline > 0 || a.map.seq_map == nullptr;
-  if (!local && early) load_prefix();
+  if (!local && early) load_prefix(0);
   cluster_arrive();                        // every CTA of the cluster runs before shared memory is written remotely
   pdl_wait();                              // the QKV projection's partials are complete from here on
-  if (!local && !early) load_prefix();
+  if (!local && !early) load_prefix(0);
   cp_async_commit();
 
   // ---- cooperative prologue: the cluster's threads share the rotary work.  Each chunk of the Q tile
@@ -346,24 +368,9 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   // f32 accumulate, bf16 operands, N = 128, M = 128; bit 16: B is MN-major (V as stored, [key][hd])
   const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
-  bool ok = true;
-  if (tid == 0) {
-    // ---- S = Q . K^T: eight k16 steps over the head dimension (four per 64-column half)
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const uint32_t qa = smem_u32(sQ) + (uint32_t)((k >> 2) * kHalfBytesKV + (k & 3) * 32);
-      const uint32_t ka = smem_u32(sK) + (uint32_t)((k >> 2) * kHalfBytesKV + (k & 3) * 32);
-      tc_mma_bf16(tmem_S, make_desc(qa, 16, 1024), make_desc(ka, 16, 1024), idesc, (uint32_t)(k != 0));
-    }
-    tc_commit(smem_u32(&bars[0]));
-  }
-  ok = mbar_wait(smem_u32(&bars[0]), 0u);
-  tc_fence_after();
-  ok = __syncthreads_and(ok ? 1 : 0) != 0;                // one decision for the CTA (barriers follow)
-
   // ---- softmax, log2 domain.  Thread = TMEM lane: copy `cw` of query row `row`, keys [cw * QT, +QT) of
-  //      the part.  The row maximum is exchanged between the copies through shared memory; the row sum is
-  //      ALWAYS formed as ((g0 + g1) + g2) + g3 over the four 32-key groups, each group summed in key
+  //      a tile.  The row maximum is exchanged between the copies through shared memory; a tile's row sum
+  //      is ALWAYS formed as ((g0 + g1) + g2) + g3 over the four 32-key groups, each group summed in key
   //      order, whatever QT is - a row's bits do not depend on how many rows share the forward.
   const int cw = tid / QT, row = tid % QT;
   const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;       // warp w reads TMEM lanes 32w .. 32w + 31
@@ -374,11 +381,38 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     key_lo = (lr / T) * T;
     key_hi = min(key_lo + T, k_end);
   }
-  float* sMax = reinterpret_cast<float*>(sK);           // [4 groups][128 rows]; K is free once S is complete
-  float* sSum = sMax + 4 * 128;
-  constexpr int NG = QT / 32;                           // 32-key groups this thread owns
-  float m_row = -INFINITY, l_row = 0.f;
-  if (ok) {
+  constexpr int NG = QT / 32;                           // 32-key groups of a tile this thread owns
+  float m_row = -INFINITY, l_row = 0.f;                 // running maximum and sum over the tiles so far
+  bool ok = true;
+#pragma unroll 1
+  for (int t = 0; t < n_tiles; ++t) {
+    const int kb = k_begin + t * kKeys;                 // first key of the tile
+    const uint32_t phase = (uint32_t)(t & 1);
+    if (t > 0) {
+      // the previous tile's MMAs are complete: K (holding P) and V are free
+      load_prefix(t);
+      cp_async_commit();
+      cp_async_wait<0>();
+      asm volatile("fence.proxy.async;" ::: "memory");
+      tc_fence_before();
+      __syncthreads();
+      tc_fence_after();
+    }
+    if (tid == 0) {
+      // ---- S = Q . K^T: eight k16 steps over the head dimension (four per 64-column half)
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint32_t qa = smem_u32(sQ) + (uint32_t)((k >> 2) * kHalfBytesKV + (k & 3) * 32);
+        const uint32_t ka = smem_u32(sK) + (uint32_t)((k >> 2) * kHalfBytesKV + (k & 3) * 32);
+        tc_mma_bf16(tmem_S, make_desc(qa, 16, 1024), make_desc(ka, 16, 1024), idesc, (uint32_t)(k != 0));
+      }
+      tc_commit(smem_u32(&bars[0]));
+    }
+    ok = mbar_wait(smem_u32(&bars[0]), phase);
+    tc_fence_after();
+    ok = __syncthreads_and(ok ? 1 : 0) != 0;              // one decision for the CTA (barriers follow)
+    if (!ok) break;
+
     float m_loc = -INFINITY;
 #pragma unroll 1
     for (int g = 0; g < NG; ++g) {
@@ -387,19 +421,21 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       tmem_ld32(tmem_S + lane_addr + c0, v);
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
-        const int key = k_begin + c0 + j;
+        const int key = kb + c0 + j;
         if (key >= key_lo && key < key_hi) m_loc = fmaxf(m_loc, v[j] * scale_log2);
       }
     }
+    float m_tile = m_loc;
     if (REP > 1) {
       sMax[cw * 128 + row] = m_loc;
       __syncthreads();
+      m_tile = -INFINITY;
 #pragma unroll
-      for (int k = 0; k < REP; ++k) m_row = fmaxf(m_row, sMax[k * 128 + row]);
-    } else {
-      m_row = m_loc;
+      for (int k = 0; k < REP; ++k) m_tile = fmaxf(m_tile, sMax[k * 128 + row]);
     }
-    const float m_use = (m_row == -INFINITY) ? 0.f : m_row;
+    const float m_new = fmaxf(m_row, m_tile);
+    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+    const float corr = exp2f(m_row - m_use);              // 0 for the first tile that holds a visible key
 #pragma unroll 1
     for (int g = 0; g < NG; ++g) {
       const int c0 = cw * QT + g * 32;
@@ -409,7 +445,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       float gsum = 0.f;
 #pragma unroll
       for (int j = 0; j < 32; j += 2) {
-        const int key = k_begin + c0 + j;
+        const int key = kb + c0 + j;
         const float p0 = (key >= key_lo && key < key_hi) ? exp2f(v[j] * scale_log2 - m_use) : 0.f;
         const float p1 = (key + 1 >= key_lo && key + 1 < key_hi) ? exp2f(v[j + 1] * scale_log2 - m_use) : 0.f;
         gsum += p0;
@@ -417,37 +453,54 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
         packed[j >> 1] = pack_bf16(p0, p1);
       }
       sSum[(cw * NG + g) * 128 + row] = gsum;           // group index = c0 / 32
-      // P overwrites Q, in every copy of the row
+      // P overwrites K, in every copy of the row
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const uint4 val = row_live ? make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3])
                                    : make_uint4(0, 0, 0, 0);
 #pragma unroll
         for (int k = 0; k < REP; ++k)
-          *reinterpret_cast<uint4*>(sQ + tile_off(k * QT + row, (c0 >> 3) + q, 128)) = val;
+          *reinterpret_cast<uint4*>(sK + tile_off(k * QT + row, (c0 >> 3) + q, 128)) = val;
       }
     }
-  }
-  asm volatile("fence.proxy.async;" ::: "memory");        // P is read by the tensor core
-  tc_fence_before();
-  __syncthreads();
-  if (tid == 0 && ok) {
-    tc_fence_after();
-    // ---- O = P . V: eight k16 steps over the keys.  P is K-major (keys contiguous); V is used as stored,
-    //      [key][hd] = MN-major: 8-key groups 1024 B apart, the two 64-column halves 16 KB apart.
-    const uint32_t idesc_pv = idesc | (1u << 16);
+    if (t > 0) {
+      // the output so far was accumulated against the old maximum: rescale this thread's columns of its
+      // lane (the columns it reads out at the end; the rest of a copy's lane is never read)
+#pragma unroll 1
+      for (int g = 0; g < NG; ++g) {
+        float v[32];
+        const uint32_t ta = tmem_O + lane_addr + cw * QT + g * 32;
+        tmem_ld32(ta, v);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const uint32_t pa = smem_u32(sQ) + (uint32_t)((k >> 2) * kHalfBytesKV + (k & 3) * 32);
-      const uint32_t va = smem_u32(sV) + (uint32_t)(2 * k * 1024);
-      const uint64_t vdesc = v_desc_swap ? make_desc(va, 1024, kHalfBytesKV) : make_desc(va, kHalfBytesKV, 1024);
-      tc_mma_bf16(tmem_O, make_desc(pa, 16, 1024), vdesc, idesc_pv, (uint32_t)(k != 0));
+        for (int j = 0; j < 32; ++j) v[j] *= corr;
+        tmem_st32(ta, v);
+      }
     }
-    tc_commit(smem_u32(&bars[1]));
+    asm volatile("fence.proxy.async;" ::: "memory");      // P is read by the tensor core
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      // ---- O (+)= P . V: eight k16 steps over the keys.  P is K-major (keys contiguous); V is used as
+      //      stored, [key][hd] = MN-major: 8-key groups 1024 B apart, the two 64-column halves 16 KB apart.
+      const uint32_t idesc_pv = idesc | (1u << 16);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const uint32_t pa = smem_u32(sK) + (uint32_t)((k >> 2) * kHalfBytesKV + (k & 3) * 32);
+        const uint32_t va = smem_u32(sV) + (uint32_t)(2 * k * 1024);
+        const uint64_t vdesc = v_desc_swap ? make_desc(va, 1024, kHalfBytesKV) : make_desc(va, kHalfBytesKV, 1024);
+        tc_mma_bf16(tmem_O, make_desc(pa, 16, 1024), vdesc, idesc_pv, (uint32_t)((t | k) != 0));
+      }
+      tc_commit(smem_u32(&bars[1]));
+    }
+    ok = mbar_wait(smem_u32(&bars[1]), phase);
+    tc_fence_after();
+    ok = __syncthreads_and(ok ? 1 : 0) != 0;              // every MMA is complete: shared memory is free
+    if (!ok) break;
+    const float l_tile = ((sSum[0 * 128 + row] + sSum[1 * 128 + row]) + sSum[2 * 128 + row]) + sSum[3 * 128 + row];
+    l_row = l_row * corr + l_tile;
+    m_row = m_new;
   }
-  if (ok) ok = mbar_wait(smem_u32(&bars[1]), 0u);
-  tc_fence_after();
-  ok = __syncthreads_and(ok ? 1 : 0) != 0;                // every MMA is complete: shared memory is free
 
   // ---- publish (max, sum, unnormalised output) of the rows
   constexpr int kPitch = kHD + 4;                         // floats per staged row
@@ -458,8 +511,6 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     float v[NG][32];
 #pragma unroll
     for (int g = 0; g < NG; ++g) tmem_ld32(tmem_O + lane_addr + cw * QT + g * 32, v[g]);
-    if (cw == 0) l_row = ((sSum[0 * 128 + row] + sSum[1 * 128 + row]) + sSum[2 * 128 + row]) + sSum[3 * 128 + row];
-    __syncthreads();                                      // sSum (in the K buffer) is read before sO overwrites it
 #pragma unroll
     for (int g = 0; g < NG; ++g)
 #pragma unroll
@@ -526,11 +577,11 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
 
 int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a, int v_desc_swap) {
   if (a.hd != kHD || !a.qkv_partial || !a.rope || !a.err_flag) return 1;
-  if (a.kv_split != kKeys) return 1;
+  if (a.kv_split < kKeys || (a.kv_split % kKeys) != 0) return 1;
   if ((a.cache_k_out != nullptr) != (a.cache_v_out != nullptr)) return -1;
   const int rps = a.map.rows_per_seq, T = a.map.T;
   if (a.cache_k_out != nullptr && rps != T) return -1;
-  const int n_prefix = (a.S + kKeys - 1) / kKeys;
+  const int n_prefix = (a.S + a.kv_split - 1) / a.kv_split;
   const int n_parts = n_prefix + 1;
   if (n_parts > kAttnMaxClusterParts) return 1;
   // Eligibility depends on the head dimension, the prefix length and the block length only - never on
@@ -540,11 +591,11 @@ int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a, int v_desc_sw
   const int qt_rows = rps <= 32 ? 32 : (rps <= 64 ? 64 : 128);
   const int q_tiles = (rps + qt_rows - 1) / qt_rows;
   const float scale_log2 = (1.0f / sqrtf((float)a.hd)) * 1.4426950408889634f;
-  // 97 KB: never more than two CTAs per SM, so that two 256-column TMEM allocations always fit
-  const size_t smem = 6 * (size_t)kHalfBytesKV + 64 + 1024;     // Q/P, K, V tiles of 128 rows: two CTAs per SM
+  // 101 KB: never more than two CTAs per SM, so that two 256-column TMEM allocations always fit
+  const size_t smem = 6 * (size_t)kHalfBytesKV + 4096 + 64 + 1024;   // Q, K/P, V tiles of 128 rows + the softmax exchange
   static bool attr_set = false;
   if (!attr_set) {
-    const int max_smem = 6 * kHalfBytesKV + 64 + 1024;
+    const int max_smem = 6 * kHalfBytesKV + 4096 + 64 + 1024;
     if (cudaFuncSetAttribute(attn_verify_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
         cudaFuncSetAttribute(attn_verify_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
         cudaFuncSetAttribute(attn_verify_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)

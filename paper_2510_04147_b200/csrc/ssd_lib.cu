@@ -133,7 +133,8 @@ int auto_split(int tiles, int k) {
 // verification forward merges the parts inside one cluster, so prefix parts + the local part <= 8.
 int kv_split_for(const ssd_ctx* c, int S) {
   int ks = c->kv_split_opt > 0 ? c->kv_split_opt : 128;
-  while ((S + ks - 1) / ks > kAttnMaxClusterParts - 1) ks += 64;
+  // raised in steps of 128 keys: whole tensor-core tiles whenever the starting value is one
+  while ((S + ks - 1) / ks > kAttnMaxClusterParts - 1) ks += 128;
   return ks;
 }
 

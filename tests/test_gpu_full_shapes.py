@@ -239,7 +239,10 @@ def test_both_attention_forms_agree_at_full_width():
             out[impl] = (tok, conf, logits)
     finally:
         ssd.destroy()
-    assert np.abs(out[0][2] - out[1][2]).max() < 2e-2          # same bf16 rounding noise level, no bias
-    assert np.sqrt(((out[0][2] - out[1][2]) ** 2).mean()) < 4e-3
+    # the same fraction of the logit scale as the comparison with the oracle (module docstring)
+    scale = max(1.0, float(out[0][2].std()) / TINY_LOGIT_STD)
+    diff = out[0][2] - out[1][2]
+    assert np.abs(diff).max() < 2e-2 * scale, (np.abs(diff).max(), scale)
+    assert np.sqrt((diff ** 2).mean()) < 4e-3 * scale          # noise, not a bias
     m = masked[0]
-    assert np.allclose(out[0][1][0][m], out[1][1][0][m], rtol=2e-2)
+    assert np.allclose(out[0][1][0][m], out[1][1][0][m], rtol=CONF_RTOL * scale, atol=1e-6)
