@@ -636,10 +636,10 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   p.tmem_cols = cols;
   const int stage_bytes = kWTileBytes + p.npad * kBlockK * 2;
   // two CTAs per SM while the activation tile is small, one deep pipeline otherwise
-  const int budget = (p.npad <= 128) ? 108 * 1024 : 200 * 1024;
+  const int budget = 108 * 1024;
   int stages = budget / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
-  if (stages < 3) stages = 3;
+  if (stages < 2) stages = 2;
   p.stages = stages;
   p.out = g.out; p.act = g.act; p.act_pitch = g.act_pitch;
   p.tile_max = g.tile_max; p.tile_sum = g.tile_sum; p.tile_arg = g.tile_arg;
