@@ -124,6 +124,7 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
   // block commit: the first query head of a KV group also stores the rows' K/V into the cache.
   // Sequence-local row lr is in-block index lr (one node per sequence) at position pos0 + lr.
   const bool commit_kv = a.cache_k_out != nullptr && (h % (a.H / a.Hkv)) == 0;
+  const int commit_rows = a.map.chain_T0 > 0 ? a.map.chain_T0 : rps;   // sequence-local rows whose K/V are cached
   auto cache_row = [&](int lr) -> size_t {
     return (size_t)seq_of_slot(a.map, slot) * a.cache_seq_stride + ((size_t)(a.map.pos0 + lr) * a.Hkv + kvh) * HD;
   };
@@ -212,7 +213,7 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
       if (key0 + row < k_end) rot_item(key0 + row, c, (a.H + kvh) * HD, lo, hi);
       *reinterpret_cast<uint4*>(dK + swz<HD>(row, c)) = lo;
       *reinterpret_cast<uint4*>(dK + swz<HD>(row, c + CPR)) = hi;
-      if (commit_kv && key0 + row < k_end) {
+      if (commit_kv && key0 + row < k_end && key0 + row < commit_rows) {
         bf16* dst = a.cache_k_out + cache_row(key0 + row) + c * 8;
         *reinterpret_cast<uint4*>(dst) = lo;
         *reinterpret_cast<uint4*>(dst + HALF) = hi;
@@ -222,7 +223,7 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
       const int row = idx / CH, c = idx % CH;
       const uint4 v = (key0 + row < k_end) ? plain_item(key0 + row, c, (a.H + a.Hkv + kvh) * HD) : zero;
       *reinterpret_cast<uint4*>(dV + swz<HD>(row, c)) = v;
-      if (commit_kv && key0 + row < k_end) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(key0 + row) + c * 8) = v;
+      if (commit_kv && key0 + row < k_end && key0 + row < commit_rows) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(key0 + row) + c * 8) = v;
     }
   };
 
@@ -265,7 +266,7 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
         if (row < lk_rows) rot_item(lk_begin + row, c, (a.H + kvh) * HD, lo, hi);
         st_cluster_u4(map_to_rank(lK + swz<HD>(row, c), (uint32_t)n_prefix_parts), lo);
         st_cluster_u4(map_to_rank(lK + swz<HD>(row, c + CPR), (uint32_t)n_prefix_parts), hi);
-        if (commit_kv && row < lk_rows) {
+        if (commit_kv && row < lk_rows && lk_begin + row < commit_rows) {
           bf16* dst = a.cache_k_out + cache_row(lk_begin + row) + c * 8;
           *reinterpret_cast<uint4*>(dst) = lo;
           *reinterpret_cast<uint4*>(dst + HALF) = hi;
@@ -274,7 +275,7 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
         const int row = (it - n_q - n_k) / CH, c = (it - n_q - n_k) % CH;
         const uint4 v = (row < lk_rows) ? plain_item(lk_begin + row, c, (a.H + a.Hkv + kvh) * HD) : zero;
         st_cluster_u4(map_to_rank(lV + swz<HD>(row, c), (uint32_t)n_prefix_parts), v);
-        if (commit_kv && row < lk_rows) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(lk_begin + row) + c * 8) = v;
+        if (commit_kv && row < lk_rows && lk_begin + row < commit_rows) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(lk_begin + row) + c * 8) = v;
       }
     }
     cluster_sync_all();
@@ -295,6 +296,8 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
     const int qlr = lr0 + qrow_w + gq + i * 8;
     node_lo[i] = local ? (qlr / T) * T : 0;
     node_hi[i] = local ? min(node_lo[i] + T, k_end) : k_end;
+    // causal chain of two blocks: a row of the finished block does not see the next block
+    if (local && a.map.chain_T0 > 0 && qlr - node_lo[i] < a.map.chain_T0) node_hi[i] = min(node_hi[i], node_lo[i] + a.map.chain_T0);
   }
   const bool rows_live = lr0 + qrow_w < rps;           // otherwise the warp only keeps the barriers
 

@@ -215,6 +215,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     }
   };
   const bool commit_kv = a.cache_k_out != nullptr && (h % (a.H / a.Hkv)) == 0;
+  const int commit_rows = a.map.chain_T0 > 0 ? a.map.chain_T0 : rps;   // sequence-local rows whose K/V are cached
   auto cache_row = [&](int lr) -> size_t {
     return (size_t)seq_of_slot(a.map, slot) * a.cache_seq_stride + ((size_t)(a.map.pos0 + lr) * a.Hkv + kvh) * kHD;
   };
@@ -332,7 +333,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
         if (row < lk_rows) rot_item(lk_begin + row, c, (a.H + kvh) * kHD, lo, hi);
         st_cluster_u4(map_to_rank(sK + tile_off(row, c, kKeys), (uint32_t)n_prefix_parts), lo);
         st_cluster_u4(map_to_rank(sK + tile_off(row, c + 8, kKeys), (uint32_t)n_prefix_parts), hi);
-        if (commit_kv && row < lk_rows) {
+        if (commit_kv && row < lk_rows && lk_begin + row < commit_rows) {
           bf16* dst = a.cache_k_out + cache_row(lk_begin + row) + c * 8;
           *reinterpret_cast<uint4*>(dst) = lo;
           *reinterpret_cast<uint4*>(dst + HALF) = hi;
@@ -341,7 +342,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
         const int row = (it - n_q - n_k) / CH, c = (it - n_q - n_k) % CH;
         const uint4 v = (row < lk_rows) ? plain_item(lk_begin + row, c, (a.H + a.Hkv + kvh) * kHD) : zero;
         st_cluster_u4(map_to_rank(sV + tile_off(row, c, kKeys), (uint32_t)n_prefix_parts), v);
-        if (commit_kv && row < lk_rows) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(lk_begin + row) + c * 8) = v;
+        if (commit_kv && row < lk_rows && lk_begin + row < commit_rows) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(lk_begin + row) + c * 8) = v;
       }
     }
     asm volatile("fence.proxy.async;" ::: "memory");      // these stores are read by the tensor core
@@ -380,6 +381,8 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   if (local) {
     key_lo = (lr / T) * T;
     key_hi = min(key_lo + T, k_end);
+    // causal chain of two blocks: a row of the finished block does not see the next block
+    if (a.map.chain_T0 > 0 && lr - key_lo < a.map.chain_T0) key_hi = min(key_hi, key_lo + a.map.chain_T0);
   }
   constexpr int NG = QT / 32;                           // 32-key groups of a tile this thread owns
   float m_row = -INFINITY, l_row = 0.f;                 // running maximum and sum over the tiles so far

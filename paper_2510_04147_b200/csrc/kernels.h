@@ -68,6 +68,10 @@ struct RowMap {
   // its dependency wait (the device array is written by an earlier kernel of the same forward).
   int n_inline;        // 0: not given
   int inline_seq[8];
+  // > 0: the rows of a sequence are ONE causal chain of two blocks - the first chain_T0 rows are a
+  // finished block (they see the prefix and themselves, and their K/V go to the cache), the rest
+  // is the next block, which also sees the finished one.  rows_per_seq == T then.
+  int chain_T0;
 };
 __host__ __device__ inline int seq_of_slot(const RowMap& m, int slot) {
   if (m.n_inline > 0) return m.inline_seq[slot];
@@ -208,11 +212,15 @@ struct BlockState {       // device arrays, [max_batch][block_len] unless noted
   int* seq_map;           // [max_batch] slot -> sequence of the current forward
   int stride;             // block_len (row pitch of the arrays above)
 };
-// slot a (= rank among unfinished sequences): candidates, node rows [a][n_cap][T]
+// slot a (= rank among unfinished sequences): candidates, node rows [a][n_cap][T].  With prev_ids
+// (device [batch][prev_stride]) the rows of a slot are [prev_T tokens of the finished block, not
+// masked][n_cap][T]: the layout of the forward that also commits the previous block.
 void launch_tree_build(cudaStream_t st, BlockState s, int batch, int T, int max_drafts, int n_cap, int mask_id,
-                       int* node_ids, uint8_t* node_masked);
-// per slot: per-node best masked position, chain walk, state/draft update
+                       int* node_ids, uint8_t* node_masked, const int* prev_ids = nullptr, int prev_T = 0,
+                       int prev_stride = 0);
+// per slot: per-node best masked position, chain walk, state/draft update; a slot's node rows start
+// `row_offset` rows into its `slot_rows` rows (0 and n_cap * T without a finished block in front)
 void launch_accept(cudaStream_t st, BlockState s, int n_slots, int T, int n_cap, const int* tok, const float* conf,
-                   const uint8_t* node_masked, int* nonfinite_flag);
+                   const uint8_t* node_masked, int* nonfinite_flag, int slot_rows = 0, int row_offset = 0);
 
 }  // namespace ssd

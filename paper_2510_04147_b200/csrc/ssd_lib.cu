@@ -67,6 +67,11 @@ struct ssd_ctx {
 
   int batch = 0, prompt_len = 0, cache_len = -1, block_tokens = 0;
   bool in_block = false;
+  // A finished block whose K/V are not in the cache yet: its commit is folded into the next block's
+  // first forward (or run on its own when something else needs the cache first).
+  int pending_T = 0;
+  int* pending_ids = nullptr;    // [max_batch][block_len] tokens of that block
+  int fuse_commit = 1;
   std::vector<int> h_remaining, h_has_drafts;
 
   int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0, gemm_impl = 1;
@@ -285,7 +290,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     } else {
       // rotary embedding, node-local K/V and the merge of the key parts happen inside the attention kernel
       a.qkv_partial = c->partial; a.qkv_splits = g.splits; a.qkv_split_stride = (size_t)R * c->nqkv; a.rope = c->rope;
-      if (commit_form) {
+      if (commit_form || map.chain_T0 > 0) {
         a.cache_k_out = c->cacheK + (size_t)l * c->cache_layer_stride;
         a.cache_v_out = c->cacheV + (size_t)l * c->cache_layer_stride;
       }
@@ -384,6 +389,31 @@ int sync_and_check(ssd_ctx* c) {
   return check_flags_after_sync(c);
 }
 
+// The commit forward of a finished block on its own (Section 3.2.4 leaves open how a block's K/V
+// reach the cache; here: one forward over its final tokens).  ids: device [batch][stride].
+int commit_now(ssd_ctx* c, const int* ids, int stride, int T) {
+  const int B = c->batch;
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->node_ids, T * sizeof(int), ids, stride * sizeof(int), T * sizeof(int), B, cudaMemcpyDeviceToDevice, c->st));
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  RowMap map{T, T, c->cache_len, 0, nullptr};
+  int rc = forward(c, FWD_FILL, c->node_ids, B * T, map, B, false, nullptr);
+  if (rc) return rc;
+  rc = sync_and_check(c);
+  if (rc) return rc;
+  c->cache_len += T;
+  return SSD_OK;
+}
+
+// Whatever needs the whole cache (a test hook, a read-back, a teacher-forced state) first runs the
+// commit that was waiting for the next block's first forward.
+int flush_pending(ssd_ctx* c) {
+  if (c->pending_T <= 0) return SSD_OK;
+  const int rc = commit_now(c, c->pending_ids, c->bs.stride, c->pending_T);
+  if (rc) return rc;
+  c->pending_T = 0;
+  return SSD_OK;
+}
+
 int parse_layer_name(const char* name, int* layer, const char** rest) {
   if (strncmp(name, "layers.", 7) != 0) return 0;
   char* end = nullptr;
@@ -427,7 +457,9 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
   c->qdim = c->H * c->hd; c->kvdim = c->Hkv * c->hd; c->nqkv = c->qdim + 2 * c->kvdim;
   c->L.resize(k.n_layers);
   c->n_max = (k.max_drafts < k.block_len - 1 ? k.max_drafts : k.block_len - 1) + 1;
-  c->R_dec = k.max_batch * c->n_max * k.block_len;
+  // at least two blocks of rows per sequence: the forward that commits a block together with the
+  // first step of the next one
+  c->R_dec = k.max_batch * (c->n_max > 2 ? c->n_max : 2) * k.block_len;
   c->R_cap = c->R_dec > k.max_seq ? c->R_dec : k.max_seq;
   c->split_qkv = auto_split(gemm_tiles(c->nqkv), c->d);
   c->split_o = auto_split(gemm_tiles(c->d), c->qdim);
@@ -498,6 +530,7 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     c->bs.stride = k.block_len;
     ALLOC(c, c->bs.ids, sb); ALLOC(c, c->bs.masked, sb); ALLOC(c, c->bs.draft_tok, sb); ALLOC(c, c->bs.draft_conf, sb);
     ALLOC(c, c->bs.cand_pos, sb); ALLOC(c, c->bs.cand_tok, sb); ALLOC(c, c->bs.accept_log, sb);
+    ALLOC(c, c->pending_ids, sb);
     ALLOC(c, c->bs.has_drafts, k.max_batch); ALLOC(c, c->bs.remaining, k.max_batch); ALLOC(c, c->bs.n_cand, k.max_batch);
     ALLOC(c, c->bs.n_forwards, k.max_batch); ALLOC(c, c->bs.last_accept, k.max_batch); ALLOC(c, c->bs.seq_map, k.max_batch);
     CUDA_TRY(c, cudaMallocHost(&c->h_pinned, (2 + 3 * (size_t)k.max_batch) * sizeof(int)));
@@ -594,6 +627,7 @@ int ssd_prefill_dev(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t
   c->prompt_len = prompt_len;
   c->cache_len = prompt_len;
   c->in_block = false;
+  c->pending_T = 0;
   return SSD_OK;
 }
 
@@ -613,13 +647,21 @@ int ssd_prefill(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t* pr
   return rc;
 }
 
-int ssd_cache_length(const ssd_ctx* c) { return c ? (c->cache_len < 0 ? SSD_ERR_STATE : c->cache_len) : SSD_ERR_INVALID_ARG; }
+int ssd_cache_length(const ssd_ctx* c) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  return c->cache_len < 0 ? SSD_ERR_STATE : c->cache_len + c->pending_T;   // a block waiting for its commit counts
+}
 
 int ssd_rewind(ssd_ctx* c, int32_t length) {
   if (!c) return SSD_ERR_INVALID_ARG;
   if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
-  if (length < c->prompt_len || length > c->cache_len)
-    return fail(c, SSD_ERR_INVALID_ARG, "rewind target %d outside [%d, %d]", length, c->prompt_len, c->cache_len);
+  if (length < c->prompt_len || length > c->cache_len + c->pending_T)
+    return fail(c, SSD_ERR_INVALID_ARG, "rewind target %d outside [%d, %d]", length, c->prompt_len, c->cache_len + c->pending_T);
+  if (length > c->cache_len) {          // part of the waiting block stays: its K/V are needed after all
+    const int rc = flush_pending(c);
+    if (rc) return rc;
+  }
+  c->pending_T = 0;                     // a block cut off entirely is never committed
   c->cache_len = length;
   c->in_block = false;
   return SSD_OK;
@@ -629,7 +671,8 @@ int ssd_block_begin(ssd_ctx* c, int32_t T) {
   if (!c) return SSD_ERR_INVALID_ARG;
   if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
   if (T < 1 || T > c->cfg.block_len) return fail(c, SSD_ERR_INVALID_ARG, "block_tokens %d outside [1, %d]", T, c->cfg.block_len);
-  if (c->cache_len + T > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "cache %d + block %d exceeds max_seq %d", c->cache_len, T, c->cfg.max_seq);
+  if (c->cache_len + c->pending_T + T > c->cfg.max_seq)
+    return fail(c, SSD_ERR_OVERFLOW, "cache %d + block %d exceeds max_seq %d", c->cache_len + c->pending_T, T, c->cfg.max_seq);
   block_init_kernel<<<c->cfg.max_batch, 128, 0, c->st>>>(c->bs, c->batch, c->cfg.max_batch, T, c->cfg.mask_id);
   c->launches += 1;
   CUDA_TRY(c, cudaGetLastError());
@@ -646,6 +689,10 @@ int ssd_set_block_state(ssd_ctx* c, const int32_t* ids, const uint8_t* masked, c
   if (!c) return SSD_ERR_INVALID_ARG;
   if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
   if (!ids || !masked || ((draft_tok == nullptr) != (draft_conf == nullptr))) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  {
+    const int frc = flush_pending(c);   // an injected state continues from a complete cache
+    if (frc) return frc;
+  }
   const int T = c->block_tokens, st = c->bs.stride;
   for (int b = 0; b < c->batch; ++b) {
     int r = 0;
@@ -697,13 +744,34 @@ int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n
   if (accepted) memset(accepted, 0, B * sizeof(int));
   if (n_nodes) memset(n_nodes, 0, B * sizeof(int));
   if (active == 0) return SSD_OK;
-  const int R = active * n_cap * T;
+  // A block waiting for its commit rides in front of the first forward of this block: per sequence
+  // one causal chain [finished block | this block, all MASK].  Only a fresh block qualifies (every
+  // sequence untouched, so one node each); otherwise the commit runs on its own first.
+  int Tp = 0;
+  if (c->pending_T > 0) {
+    bool fresh = active == B && n_cap == 1;
+    for (int b = 0; b < B && fresh; ++b) fresh = c->h_remaining[b] == T && !c->h_has_drafts[b];
+    if (fresh && B * (c->pending_T + T) <= c->R_dec) {
+      Tp = c->pending_T;
+    } else {
+      const int frc = flush_pending(c);
+      if (frc) return frc;
+    }
+  }
+  const int slot_rows = Tp + n_cap * T;
+  const int R = active * slot_rows;
   CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
   {
     Scope sc(c, SSD_PROF_TREE, (double)R * 5);
-    launch_tree_build(c->st, c->bs, B, T, md, n_cap, c->cfg.mask_id, c->node_ids, c->node_masked);
+    launch_tree_build(c->st, c->bs, B, T, md, n_cap, c->cfg.mask_id, c->node_ids, c->node_masked,
+                      Tp > 0 ? c->pending_ids : nullptr, Tp, c->bs.stride);
   }
   RowMap map{n_cap * T, T, c->cache_len, 0, c->bs.seq_map};
+  if (Tp > 0) {                // one chain of Tp + T rows at positions cache_len ...
+    map.rows_per_seq = slot_rows;
+    map.T = slot_rows;
+    map.chain_T0 = Tp;
+  }
   if (active <= 8) {           // the host mirrors `remaining`, so it knows the slot -> sequence map too
     for (int b = 0; b < B; ++b)
       if (c->h_remaining[b] > 0) map.inline_seq[map.n_inline++] = b;
@@ -712,7 +780,7 @@ int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n
   if (rc) return rc;
   {
     Scope sc(c, SSD_PROF_TREE, (double)R * 9);
-    launch_accept(c->st, c->bs, active, T, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1);
+    launch_accept(c->st, c->bs, active, T, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1, slot_rows, Tp);
   }
   int* hp = c->h_pinned;
   const int mb = c->cfg.max_batch;
@@ -723,6 +791,10 @@ int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n
   CUDA_TRY(c, cudaStreamSynchronize(c->st));
   rc = check_flags_after_sync(c);
   if (rc) return rc;
+  if (Tp > 0) {                // the finished block's K/V are in the cache now
+    c->cache_len += Tp;
+    c->pending_T = 0;
+  }
   for (int b = 0; b < B; ++b) {
     const bool was_active = c->h_remaining[b] > 0;
     c->h_remaining[b] = hp[2 + b];
@@ -739,14 +811,19 @@ int ssd_block_commit(ssd_ctx* c) {
   for (int b = 0; b < c->batch; ++b)
     if (c->h_remaining[b] > 0) return fail(c, SSD_ERR_STATE, "sequence %d still has %d masked positions", b, c->h_remaining[b]);
   const int T = c->block_tokens, B = c->batch;
-  CUDA_TRY(c, cudaMemcpy2DAsync(c->node_ids, T * sizeof(int), c->bs.ids, c->bs.stride * sizeof(int), T * sizeof(int), B, cudaMemcpyDeviceToDevice, c->st));
-  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
-  RowMap map{T, T, c->cache_len, 0, nullptr};
-  int rc = forward(c, FWD_FILL, c->node_ids, B * T, map, B, false, nullptr);
+  int rc = flush_pending(c);           // (a block that ended without a single forward of its own)
   if (rc) return rc;
-  rc = sync_and_check(c);
-  if (rc) return rc;
-  c->cache_len += T;
+  if (c->fuse_commit) {
+    // keep the tokens; the next block's first forward (or whoever needs the cache first) commits them
+    CUDA_TRY(c, cudaMemcpy2DAsync(c->pending_ids, c->bs.stride * sizeof(int), c->bs.ids, c->bs.stride * sizeof(int), T * sizeof(int), B,
+                                  cudaMemcpyDeviceToDevice, c->st));
+    rc = sync_and_check(c);
+    if (rc) return rc;
+    c->pending_T = T;
+  } else {
+    rc = commit_now(c, c->bs.ids, c->bs.stride, T);
+    if (rc) return rc;
+  }
   c->in_block = false;
   return SSD_OK;
 }
@@ -778,6 +855,10 @@ int ssd_verify_forward(ssd_ctx* c, int32_t batch, int32_t n_nodes, int32_t T, co
   if (!node_ids || !node_masked) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
   if (batch < 1 || batch > c->batch) return fail(c, SSD_ERR_INVALID_ARG, "batch %d outside [1, %d]", batch, c->batch);
   if (T < 1 || T > c->cfg.block_len || n_nodes < 1) return fail(c, SSD_ERR_INVALID_ARG, "bad node shape");
+  {
+    const int frc = flush_pending(c);
+    if (frc) return frc;
+  }
   const size_t R = (size_t)batch * n_nodes * T;
   if (R > (size_t)c->R_dec) return fail(c, SSD_ERR_OVERFLOW, "%zu rows exceed the capacity %d set by max_batch/max_drafts/block_len", R, c->R_dec);
   if (c->cache_len + T > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "cache %d + block %d exceeds max_seq", c->cache_len, T);
@@ -799,6 +880,10 @@ int ssd_read_cache(ssd_ctx* c, int32_t layer, int32_t seq, int32_t length, float
   if (!c) return SSD_ERR_INVALID_ARG;
   if (layer < 0 || layer >= c->cfg.n_layers || seq < 0 || seq >= c->cfg.max_batch || length < 0 || length > c->cfg.max_seq)
     return fail(c, SSD_ERR_INVALID_ARG, "index out of range");
+  {
+    const int frc = flush_pending(c);
+    if (frc) return frc;
+  }
   const size_t n = (size_t)length * c->kvdim;
   std::vector<bf16> tmp(n);
   for (int which = 0; which < 2; ++which) {
@@ -888,6 +973,15 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "attn_impl")) {
     if (value != 0 && value != 1) return fail(c, SSD_ERR_INVALID_ARG, "attn_impl is 0 (mma.sync) or 1 (tcgen05 where the shape allows)");
     c->attn_impl = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "fuse_commit")) {
+    if (value != 0 && value != 1) return fail(c, SSD_ERR_INVALID_ARG, "fuse_commit is 0 (commit forward of its own) or 1 (folded into the next block's first forward)");
+    if (value == 0) {
+      const int frc = flush_pending(c);
+      if (frc) return frc;
+    }
+    c->fuse_commit = value;
     return SSD_OK;
   }
   if (!strcmp(key, "gemm_impl")) {

@@ -19,7 +19,8 @@ namespace {
 constexpr int kMaxT = 256;
 
 __global__ void __launch_bounds__(256) tree_build_kernel(BlockState s, int batch, int T, int max_drafts, int n_cap,
-                                                         int mask_id, int* node_ids, uint8_t* node_masked) {
+                                                         int mask_id, int* node_ids, uint8_t* node_masked,
+                                                         const int* prev_ids, int prev_T, int prev_stride) {
   __shared__ int rank[kMaxT];
   __shared__ float cf[kMaxT];
   __shared__ uint8_t mk[kMaxT];
@@ -61,7 +62,12 @@ __global__ void __launch_bounds__(256) tree_build_kernel(BlockState s, int batch
     s.seq_map[slot] = b;
   }
   __syncthreads();
-  const size_t base = (size_t)slot * n_cap * T;
+  size_t base = (size_t)slot * (prev_T + n_cap * T);
+  for (int e = threadIdx.x; e < prev_T; e += blockDim.x) {      // the finished block in front: tokens, nothing asked
+    node_ids[base + e] = prev_ids[(size_t)b * prev_stride + e];
+    node_masked[base + e] = 0;
+  }
+  base += prev_T;
   for (int e = threadIdx.x; e < n_cap * T; e += blockDim.x) {
     const int i = e / T, t = e % T;
     const int depth = min(i, N);                 // nodes beyond N repeat node N and ask for nothing
@@ -76,7 +82,8 @@ __global__ void __launch_bounds__(256) tree_build_kernel(BlockState s, int batch
 }
 
 __global__ void __launch_bounds__(256) accept_kernel(BlockState s, int T, int n_cap, const int* tok, const float* conf,
-                                                     const uint8_t* node_masked, int* nonfinite_flag) {
+                                                     const uint8_t* node_masked, int* nonfinite_flag, int slot_rows,
+                                                     int row_offset) {
   __shared__ int pred_q[kMaxT];
   __shared__ int pred_t[kMaxT];
   __shared__ int s_a;
@@ -86,7 +93,7 @@ __global__ void __launch_bounds__(256) accept_kernel(BlockState s, int T, int n_
   const int b = s.seq_map[slot];
   const int N = s.n_cand[b];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
-  const size_t base = (size_t)slot * n_cap * T;
+  const size_t base = (size_t)slot * slot_rows + row_offset;
   for (int i = warp; i <= N; i += nw) {
     float bc = -1.f;
     int bq = 0x7fffffff;
@@ -151,14 +158,17 @@ __global__ void __launch_bounds__(256) accept_kernel(BlockState s, int T, int n_
 }  // namespace
 
 void launch_tree_build(cudaStream_t st, BlockState s, int batch, int T, int max_drafts, int n_cap, int mask_id,
-                       int* node_ids, uint8_t* node_masked) {
+                       int* node_ids, uint8_t* node_masked, const int* prev_ids, int prev_T, int prev_stride) {
+  if (!prev_ids) prev_T = 0;
   launch_pdl(tree_build_kernel, dim3(batch), dim3(256), 0, st, s, batch, T, max_drafts, n_cap, mask_id, node_ids,
-             node_masked);
+             node_masked, prev_ids, prev_T, prev_stride);
 }
 
 void launch_accept(cudaStream_t st, BlockState s, int n_slots, int T, int n_cap, const int* tok, const float* conf,
-                   const uint8_t* node_masked, int* nonfinite_flag) {
-  launch_pdl(accept_kernel, dim3(n_slots), dim3(256), 0, st, s, T, n_cap, tok, conf, node_masked, nonfinite_flag);
+                   const uint8_t* node_masked, int* nonfinite_flag, int slot_rows, int row_offset) {
+  if (slot_rows <= 0) { slot_rows = n_cap * T; row_offset = 0; }
+  launch_pdl(accept_kernel, dim3(n_slots), dim3(256), 0, st, s, T, n_cap, tok, conf, node_masked, nonfinite_flag,
+             slot_rows, row_offset);
 }
 
 }  // namespace ssd

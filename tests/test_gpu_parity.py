@@ -310,6 +310,106 @@ def test_teacher_forced_ssd_steps_match_oracle(tiny_ssd, peaked_ssd, tiny_oracle
     print(f"{which}: {strict} of {len(trace)} forwards had safe margins throughout")
 
 
+@pytest.mark.parametrize("which", ["tiny", "tiny_peaked"])
+def test_commit_folded_into_next_first_forward_matches_oracle(tiny_ssd, peaked_ssd, tiny_oracles, which):
+    """A finished block is committed by the next block's first forward: per sequence one causal chain
+    [finished block | next block, all MASK].  Mathematically that is the commit forward followed by the
+    root forward, so the oracle needs nothing new: its commit_block + verify are the reference for the
+    cache rows the chain writes and for the root predictions it returns."""
+    w = wl.TINY if which == "tiny" else PEAKED
+    ssd = tiny_ssd if which == "tiny" else peaked_ssd
+    _, ob = tiny_oracles[w.name]
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    T, P = w.block_len, w.prompt_len
+    rtol = CONF_RTOL * w.lm_head_scale
+    block0 = np.random.default_rng(11).integers(0, w.vocab - 1, T)
+    # oracle: commit, then the root forward of the next block
+    cache = ob.prefill(prompt[0])
+    ob.commit_block(block0, cache)
+    root_ids = np.full((1, T), w.mask_id)
+    otok, oconf, ogap, _ = ob.verify(root_ids, np.ones((1, T), bool), cache)
+    otok, oconf, ogap = otok[0], oconf[0], ogap[0]
+    # GPU: the commit waits, the next block's first step carries it
+    ssd.prefill(prompt)
+    ssd.block_begin(T)
+    ssd.set_block_state(block0[None], np.zeros((1, T), np.uint8))
+    ssd.block_commit()
+    assert ssd.cache_length() == P + T
+    l0 = ssd.launch_count()
+    ssd.block_begin(T)
+    acc, nn = ssd.block_step(0, 1)
+    fused_launches = ssd.launch_count() - l0
+    assert acc[0] == 1 and nn[0] == 1
+    ids, masked, dt, dc = ssd.get_block_state(1, T)
+    m = masked[0].astype(bool)
+    assert m.sum() == T - 1
+    q = int(np.where(~m)[0][0])
+    assert np.allclose(dc[0][m], oconf[m], rtol=rtol, atol=1e-6)          # next drafts = root predictions
+    sure = m & _token_is_safe(ogap, oconf, w)
+    assert np.array_equal(dt[0][sure], otok[sure])
+    order = np.sort(oconf)[::-1]
+    if order[0] - order[1] > GAP and order[0] - order[1] > 2 * rtol * order[0] and _token_is_safe(ogap, oconf, w)[int(np.argmax(oconf))]:
+        assert q == int(np.argmax(oconf)) and ids[0][q] == otok[q]
+    # the rows the chain wrote into the cache
+    for l in range(w.n_layers):
+        k, v = ssd.read_cache(l, 0, P + T)
+        for got, want in ((k, cache.k[l]), (v, cache.v[l])):
+            assert np.abs(got[P:] - want[P:]).max() < 2e-2 * max(1.0, np.abs(want).max())
+            assert (np.abs(got[P:] - want[P:]) <= 4e-3).mean() > 0.99
+            assert np.abs(got[:P] - want[:P]).max() < 2e-2 * max(1.0, np.abs(want).max())
+    # it really was one forward: a separate commit costs a second pass of the layers
+    ssd.set_option("fuse_commit", 0)
+    try:
+        ssd.prefill(prompt)
+        ssd.block_begin(T)
+        ssd.set_block_state(block0[None], np.zeros((1, T), np.uint8))
+        l1 = ssd.launch_count()
+        ssd.block_commit()
+        ssd.block_begin(T)
+        acc2, _ = ssd.block_step(0, 1)
+        split_launches = ssd.launch_count() - l1
+        ids2, masked2, dt2, dc2 = ssd.get_block_state(1, T)
+    finally:
+        ssd.set_option("fuse_commit", 1)
+    assert fused_launches < split_launches
+    m2 = masked2[0].astype(bool)
+    both = m & m2
+    assert np.allclose(dc[0][both], dc2[0][both], rtol=rtol, atol=1e-6)    # the two forms agree within rounding
+
+
+def test_generation_with_and_without_folded_commit(peaked_ssd):
+    """Both commit forms decode whole generations losslessly (SSD == stepwise bit-exact within a form);
+    the folded form skips the commit of the last block, which nothing reads."""
+    w = PEAKED
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    out = {}
+    try:
+        for fuse in (1, 0):
+            peaked_ssd.set_option("fuse_commit", fuse)
+            peaked_ssd.prefill(prompt)
+            tok_s, _, nf_s = peaked_ssd.generate(b.MODE_STEPWISE, w.gen_len, w.block_len, 1)
+            assert peaked_ssd.cache_length() == w.prompt_len + w.gen_len
+            peaked_ssd.prefill(prompt)
+            l0 = peaked_ssd.launch_count()
+            tok_d, acc_d, nf_d = peaked_ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1)
+            out[fuse] = (tok_d, peaked_ssd.launch_count() - l0)
+            assert np.array_equal(tok_s, tok_d)
+            for a, nf in zip(acc_d, nf_d):
+                assert a[0][:nf[0]].sum() == w.block_len
+    finally:
+        peaked_ssd.set_option("fuse_commit", 1)
+    assert out[1][1] < out[0][1]
+    # rewinding into a block that still waits for its commit keeps its K/V
+    peaked_ssd.prefill(prompt)
+    peaked_ssd.decode_block(b.MODE_SSD, w.block_len, 1)
+    peaked_ssd.rewind(w.prompt_len + w.block_len)
+    assert peaked_ssd.cache_length() == w.prompt_len + w.block_len
+    peaked_ssd.rewind(w.prompt_len)
+    assert peaked_ssd.cache_length() == w.prompt_len
+
+
 def test_batched_sequences_equal_single_runs(peaked_ssd):
     """Each sequence of a batch has its own tree; batching changes nothing for any of them."""
     w = PEAKED
