@@ -85,7 +85,8 @@ int ssd_prefill(ssd_ctx* ctx, int32_t batch, int32_t prompt_len, const int32_t* 
 int ssd_prefill_dev(ssd_ctx* ctx, int32_t batch, int32_t prompt_len, const int32_t* prompt_ids_dev);
 
 /* Decode the next block B_j (Eq. 3) for every sequence of the batch (Algorithm 1 restricted to
- * one block, or stepwise decoding), then append the block's K/V to the cache.
+ * one block, or stepwise decoding), then commit it (see ssd_block_commit: the block's K/V reach
+ * the cache with the first forward of the next call).
  *   mode           SSD_MODE_STEPWISE or SSD_MODE_SSD
  *   block_tokens   number of positions in this block: block_len, or less for a ragged last block
  *   out_tokens         HOST [batch, block_tokens]   decoded ids
@@ -115,7 +116,15 @@ int ssd_get_block_state(ssd_ctx* ctx, int32_t* ids, uint8_t* masked, int32_t* dr
  * 0 gives a stepwise step.  accepted HOST [batch] (0 for finished sequences), n_nodes HOST
  * [batch]; both may be NULL. */
 int ssd_block_step(ssd_ctx* ctx, int32_t max_drafts, int32_t* accepted, int32_t* n_nodes);
-/* Forward over the (fully unmasked) block that appends its K/V to the prefix cache. */
+/* Commit the (fully unmasked) block: its K/V are appended to the prefix cache and
+ * ssd_cache_length grows by the block.  The paper leaves open how a block's K/V reach the cache;
+ * here it is one forward over the block's final tokens, and by default that forward is not run
+ * by itself: the block waits and rides in front of the first ssd_block_step of the next block,
+ * per sequence one causal chain [finished block | next block], which is the commit forward and
+ * the next block's root forward in one weight stream.  A call that needs the complete cache
+ * first (ssd_verify_forward, ssd_read_cache, ssd_set_block_state, a rewind into the waiting
+ * block) runs the waiting commit on its own; a waiting block that is rewound away or followed
+ * by a new prefill is never committed.  Option "fuse_commit" = 0 commits here, at once. */
 int ssd_block_commit(ssd_ctx* ctx);
 
 /* The verification forward alone (Eq. 5) on caller-given node rows, against the current cache;
@@ -132,7 +141,8 @@ int ssd_verify_forward(ssd_ctx* ctx, int32_t batch, int32_t n_nodes, int32_t blo
  * [length, n_kv_heads, head_dim] each, positions [0, length).  Test hook for cache semantics. */
 int ssd_read_cache(ssd_ctx* ctx, int32_t layer, int32_t seq, int32_t length, float* out_k, float* out_v);
 
-/* Cached prefix length S (prompt + committed blocks), or a negative error. */
+/* Cached prefix length S (prompt + committed blocks, a block that waits for its commit
+ * included), or a negative error. */
 int ssd_cache_length(const ssd_ctx* ctx);
 
 /* Forget the blocks committed after position `length` (prompt_len <= length <= current length):
@@ -197,6 +207,8 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "attn_impl"  1 = attention of the verification forward on tcgen05 where the shape allows (head
  *        dimension 128, parts of whole 128-key tiles, block length dividing 128), the default; 0 = always the
  *        mma.sync form;
+ *   "fuse_commit" 1 = a block's commit is folded into the next block's first forward (default); 0 = a
+ *        commit forward of its own inside ssd_block_commit;
  *   "gemm_impl"  1 = TMA + tcgen05 kernel with fused RMSNorm / residual epilogues, the default;
  *        0 = the plain CUDA-core bring-up kernel with separate norm kernels, for cross-checks only.
  * Unknown key: SSD_ERR_INVALID_ARG. */
