@@ -224,7 +224,10 @@ def run_ours(args):
     B, L, P, bs = w.block_len, w.gen_len, w.prompt_len, w.batch
     n_blocks = -(-L // B)
     sweep_drafts = [int(x) for x in args.sweep.split(",")] if args.sweep else []
-    cfg_drafts = max([args.max_drafts if args.max_drafts >= 0 else 0] + sweep_drafts + [3])
+    # the full chain of a block (N = B - 2 drafts, B - 1 nodes) is timed once per run against the tensor
+    # roofline; batches whose full chain would exceed 1024 rows get the longest chain within 1024 rows
+    ft_nodes = max(1, min(w.block_len - 1, 1024 // (w.batch * w.block_len)))
+    cfg_drafts = max([args.max_drafts if args.max_drafts >= 0 else 0] + sweep_drafts + [3, ft_nodes - 1])
     # a stream of its own (not the legacy default stream) so that dependent launches may overlap
     stream = torch.cuda.Stream()
     torch.cuda.set_stream(stream)
@@ -330,13 +333,20 @@ def run_ours(args):
         accs = accept_stats(best)
         # ---- per-forward roofline: stepwise (1 node) and the chosen chain, CUDA events per forward
         fwd = {}
-        for label, d in (("stepwise_1_node", 0), (f"ssd_{best + 1}_nodes", best)):
+        for label, d in (("stepwise_1_node", 0), (f"ssd_{best + 1}_nodes", best), ("full_tree", ft_nodes - 1)):
+            ssd.set_option("max_drafts", d)
             ssd.rewind(P)
             ssd.block_begin(B)
             ssd.block_step(d, bs)                       # root-only forward creates the drafts
             times = []
             nodes = []
-            for _ in range(6):
+            for it in range(6):
+                if label == "full_tree" and it > 0:     # only the first step after the root has the full chain
+                    ssd.rewind(P)
+                    ssd.block_begin(B)
+                    ssd.block_step(d, bs)
+                    if it >= 3:
+                        break
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
                 acc, nn = ssd.block_step(d, bs)
@@ -355,6 +365,7 @@ def run_ours(args):
             fwd[label] = {"nodes": max(nodes), "rows": rows, "ms": tmed, "algorithmic_gb": (wb + kvb) / 1e9,
                           "hbm_frac": t_hbm / (tmed * 1e-3), "frac_of_max_hbm_tensor": max(t_hbm, t_tc) / (tmed * 1e-3)}
         # ---- dominant kernel: the projection GEMM family, CUDA events around every launch
+        ssd.set_option("max_drafts", best)
         ssd.rewind(P)
         ssd.block_begin(B)
         ssd.block_step(best, bs)
