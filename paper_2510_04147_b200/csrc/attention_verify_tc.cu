@@ -219,78 +219,6 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   auto cache_row = [&](int lr) -> size_t {
     return (size_t)seq_of_slot(a.map, slot) * a.cache_seq_stride + ((size_t)(a.map.pos0 + lr) * a.Hkv + kvh) * kHD;
   };
-  // one chunk (8 rotation pairs) of one row of a head of the fused projection: sum over the splits in
-  // split order (four splits' loads in flight at a time), rotary embedding, bf16
-  auto rot_item = [&](int lr, int c, int col0, uint4& lo, uint4& hi) {
-    float x1[8], x2[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) { x1[j] = 0.f; x2[j] = 0.f; }
-    const float* pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + c * 8;
-    const float4* cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)(a.map.pos0 + lr % T) * HALF + c * 8);
-    float4 cs[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) cs[j] = cs4[j];
-    for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
-      float4 a0[4], a1[4], b0[4], b1[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        a0[u] = a1[u] = b0[u] = b1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (s0 + u < a.qkv_splits) {
-          const float* ps = pr + (size_t)(s0 + u) * a.qkv_split_stride;
-          a0[u] = *reinterpret_cast<const float4*>(ps);
-          a1[u] = *reinterpret_cast<const float4*>(ps + 4);
-          b0[u] = *reinterpret_cast<const float4*>(ps + HALF);
-          b1[u] = *reinterpret_cast<const float4*>(ps + HALF + 4);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (s0 + u < a.qkv_splits) {
-          x1[0] += a0[u].x; x1[1] += a0[u].y; x1[2] += a0[u].z; x1[3] += a0[u].w;
-          x1[4] += a1[u].x; x1[5] += a1[u].y; x1[6] += a1[u].z; x1[7] += a1[u].w;
-          x2[0] += b0[u].x; x2[1] += b0[u].y; x2[2] += b0[u].z; x2[3] += b0[u].w;
-          x2[4] += b1[u].x; x2[5] += b1[u].y; x2[6] += b1[u].z; x2[7] += b1[u].w;
-        }
-      }
-    }
-    float y1[8], y2[8];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      y1[2 * j] = x1[2 * j] * cs[j].x - x2[2 * j] * cs[j].y;
-      y2[2 * j] = x2[2 * j] * cs[j].x + x1[2 * j] * cs[j].y;
-      y1[2 * j + 1] = x1[2 * j + 1] * cs[j].z - x2[2 * j + 1] * cs[j].w;
-      y2[2 * j + 1] = x2[2 * j + 1] * cs[j].z + x1[2 * j + 1] * cs[j].w;
-    }
-    lo = make_uint4(pack_bf16(y1[0], y1[1]), pack_bf16(y1[2], y1[3]), pack_bf16(y1[4], y1[5]), pack_bf16(y1[6], y1[7]));
-    hi = make_uint4(pack_bf16(y2[0], y2[1]), pack_bf16(y2[2], y2[3]), pack_bf16(y2[4], y2[5]), pack_bf16(y2[6], y2[7]));
-  };
-  auto plain_item = [&](int lr, int c, int col0) -> uint4 {
-    float x[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) x[j] = 0.f;
-    const float* pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + c * 8;
-    for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
-      float4 a0[4], a1[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        a0[u] = a1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (s0 + u < a.qkv_splits) {
-          const float* ps = pr + (size_t)(s0 + u) * a.qkv_split_stride;
-          a0[u] = *reinterpret_cast<const float4*>(ps);
-          a1[u] = *reinterpret_cast<const float4*>(ps + 4);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (s0 + u < a.qkv_splits) {
-          x[0] += a0[u].x; x[1] += a0[u].y; x[2] += a0[u].z; x[3] += a0[u].w;
-          x[4] += a1[u].x; x[5] += a1[u].y; x[6] += a1[u].z; x[7] += a1[u].w;
-        }
-      }
-    }
-    return make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
-  };
-
   // The cache is not written by any kernel of this forward, so its tiles may be requested before the
   // dependency wait - unless the slot -> sequence map is only known on the device.
   const bool early = a.map.n_inline > 0 || a.map.seq_map == nullptr;
@@ -317,34 +245,113 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
         *reinterpret_cast<uint4*>(sV + tile_off(row, ch, kKeys)) = zero;
       }
     }
-    cluster_wait();
-    for (int it = part * kTcAttnThreads + tid; it < n_q + n_k + n_v; it += n_parts * kTcAttnThreads) {
+    // A thread takes its work items two at a time: the split-K partials of both are requested before
+    // either is used, so the two L2 round trips overlap.
+    struct Item { int kind, row, c; const float* pr; const float4* cs4; };   // kind 0 Q, 1 K, 2 V, -1 none
+    auto decode = [&](int it) -> Item {
+      Item w{-1, 0, 0, nullptr, nullptr};
+      if (it >= n_q + n_k + n_v) return w;
+      int lr, col0;
       if (it < n_q) {
-        const int row = it / CPR, c = it % CPR;
-        uint4 lo = zero, hi = zero;
-        if (lr0 + row < rps) rot_item(lr0 + row, c, h * kHD, lo, hi);
-        for (int r = 0; r < n_parts; ++r) {
-          st_cluster_u4(map_to_rank(sQ + tile_off(row, c, 128), (uint32_t)r), lo);
-          st_cluster_u4(map_to_rank(sQ + tile_off(row, c + 8, 128), (uint32_t)r), hi);
-        }
+        w.kind = 0; w.row = it / CPR; w.c = it % CPR;
+        lr = lr0 + w.row; col0 = h * kHD;
+        if (lr >= rps) return w;                         // rows past the end of the sequence stay zero
       } else if (it < n_q + n_k) {
-        const int row = (it - n_q) / CPR, c = (it - n_q) % CPR;
-        uint4 lo = zero, hi = zero;
-        if (row < lk_rows) rot_item(lk_begin + row, c, (a.H + kvh) * kHD, lo, hi);
-        st_cluster_u4(map_to_rank(sK + tile_off(row, c, kKeys), (uint32_t)n_prefix_parts), lo);
-        st_cluster_u4(map_to_rank(sK + tile_off(row, c + 8, kKeys), (uint32_t)n_prefix_parts), hi);
-        if (commit_kv && row < lk_rows && lk_begin + row < commit_rows) {
-          bf16* dst = a.cache_k_out + cache_row(lk_begin + row) + c * 8;
+        w.kind = 1; w.row = (it - n_q) / CPR; w.c = (it - n_q) % CPR;
+        lr = lk_begin + w.row; col0 = (a.H + kvh) * kHD;
+      } else {
+        w.kind = 2; w.row = (it - n_q - n_k) / CH; w.c = (it - n_q - n_k) % CH;
+        lr = lk_begin + w.row; col0 = (a.H + a.Hkv + kvh) * kHD;
+      }
+      w.pr = a.qkv_partial + ((size_t)slot * rps + lr) * nqkv + col0 + w.c * 8;
+      if (w.kind != 2) w.cs4 = reinterpret_cast<const float4*>(a.rope + (size_t)(a.map.pos0 + lr % T) * HALF + w.c * 8);
+      return w;
+    };
+    // sums over the splits in split order: x1 = the chunk itself, x2 = its rotation partner (rotary items)
+    auto gather2 = [&](const Item& A, const Item& B, float (&xa1)[8], float (&xa2)[8], float (&xb1)[8], float (&xb2)[8]) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { xa1[j] = xa2[j] = xb1[j] = xb2[j] = 0.f; }
+      const bool la = A.pr != nullptr, lb = B.pr != nullptr;
+      const bool ra = la && A.kind != 2, rb = lb && B.kind != 2;
+      for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
+        float4 a0[4], a1[4], a2[4], a3[4], b0[4], b1[4], b2[4], b3[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          a0[u] = a1[u] = a2[u] = a3[u] = b0[u] = b1[u] = b2[u] = b3[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          const bool on = s0 + u < a.qkv_splits;
+          const size_t off = (size_t)(s0 + u) * a.qkv_split_stride;
+          if (on && la) { a0[u] = *reinterpret_cast<const float4*>(A.pr + off); a1[u] = *reinterpret_cast<const float4*>(A.pr + off + 4); }
+          if (on && ra) { a2[u] = *reinterpret_cast<const float4*>(A.pr + off + HALF); a3[u] = *reinterpret_cast<const float4*>(A.pr + off + HALF + 4); }
+          if (on && lb) { b0[u] = *reinterpret_cast<const float4*>(B.pr + off); b1[u] = *reinterpret_cast<const float4*>(B.pr + off + 4); }
+          if (on && rb) { b2[u] = *reinterpret_cast<const float4*>(B.pr + off + HALF); b3[u] = *reinterpret_cast<const float4*>(B.pr + off + HALF + 4); }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (s0 + u < a.qkv_splits) {
+            xa1[0] += a0[u].x; xa1[1] += a0[u].y; xa1[2] += a0[u].z; xa1[3] += a0[u].w;
+            xa1[4] += a1[u].x; xa1[5] += a1[u].y; xa1[6] += a1[u].z; xa1[7] += a1[u].w;
+            xa2[0] += a2[u].x; xa2[1] += a2[u].y; xa2[2] += a2[u].z; xa2[3] += a2[u].w;
+            xa2[4] += a3[u].x; xa2[5] += a3[u].y; xa2[6] += a3[u].z; xa2[7] += a3[u].w;
+            xb1[0] += b0[u].x; xb1[1] += b0[u].y; xb1[2] += b0[u].z; xb1[3] += b0[u].w;
+            xb1[4] += b1[u].x; xb1[5] += b1[u].y; xb1[6] += b1[u].z; xb1[7] += b1[u].w;
+            xb2[0] += b2[u].x; xb2[1] += b2[u].y; xb2[2] += b2[u].z; xb2[3] += b2[u].w;
+            xb2[4] += b3[u].x; xb2[5] += b3[u].y; xb2[6] += b3[u].z; xb2[7] += b3[u].w;
+          }
+        }
+      }
+    };
+    // rotary embedding (Q, K) or plain rounding (V), then the stores of the item
+    auto finish = [&](const Item& w, const float (&x1)[8], const float (&x2)[8]) {
+      if (w.kind < 0) return;
+      uint4 lo = zero, hi = zero;
+      if (w.pr != nullptr) {
+        if (w.kind == 2) {
+          lo = make_uint4(pack_bf16(x1[0], x1[1]), pack_bf16(x1[2], x1[3]), pack_bf16(x1[4], x1[5]), pack_bf16(x1[6], x1[7]));
+        } else {
+          float4 cs[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) cs[j] = w.cs4[j];
+          float y1[8], y2[8];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            y1[2 * j] = x1[2 * j] * cs[j].x - x2[2 * j] * cs[j].y;
+            y2[2 * j] = x2[2 * j] * cs[j].x + x1[2 * j] * cs[j].y;
+            y1[2 * j + 1] = x1[2 * j + 1] * cs[j].z - x2[2 * j + 1] * cs[j].w;
+            y2[2 * j + 1] = x2[2 * j + 1] * cs[j].z + x1[2 * j + 1] * cs[j].w;
+          }
+          lo = make_uint4(pack_bf16(y1[0], y1[1]), pack_bf16(y1[2], y1[3]), pack_bf16(y1[4], y1[5]), pack_bf16(y1[6], y1[7]));
+          hi = make_uint4(pack_bf16(y2[0], y2[1]), pack_bf16(y2[2], y2[3]), pack_bf16(y2[4], y2[5]), pack_bf16(y2[6], y2[7]));
+        }
+      }
+      if (w.kind == 0) {
+        for (int r = 0; r < n_parts; ++r) {
+          st_cluster_u4(map_to_rank(sQ + tile_off(w.row, w.c, 128), (uint32_t)r), lo);
+          st_cluster_u4(map_to_rank(sQ + tile_off(w.row, w.c + 8, 128), (uint32_t)r), hi);
+        }
+      } else if (w.kind == 1) {
+        st_cluster_u4(map_to_rank(sK + tile_off(w.row, w.c, kKeys), (uint32_t)n_prefix_parts), lo);
+        st_cluster_u4(map_to_rank(sK + tile_off(w.row, w.c + 8, kKeys), (uint32_t)n_prefix_parts), hi);
+        if (commit_kv && lk_begin + w.row < commit_rows) {
+          bf16* dst = a.cache_k_out + cache_row(lk_begin + w.row) + w.c * 8;
           *reinterpret_cast<uint4*>(dst) = lo;
           *reinterpret_cast<uint4*>(dst + HALF) = hi;
         }
       } else {
-        const int row = (it - n_q - n_k) / CH, c = (it - n_q - n_k) % CH;
-        const uint4 v = (row < lk_rows) ? plain_item(lk_begin + row, c, (a.H + a.Hkv + kvh) * kHD) : zero;
-        st_cluster_u4(map_to_rank(sV + tile_off(row, c, kKeys), (uint32_t)n_prefix_parts), v);
-        if (commit_kv && row < lk_rows && lk_begin + row < commit_rows) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(lk_begin + row) + c * 8) = v;
+        st_cluster_u4(map_to_rank(sV + tile_off(w.row, w.c, kKeys), (uint32_t)n_prefix_parts), lo);
+        if (commit_kv && lk_begin + w.row < commit_rows) *reinterpret_cast<uint4*>(a.cache_v_out + cache_row(lk_begin + w.row) + w.c * 8) = lo;
       }
+    };
+    const int stride = n_parts * kTcAttnThreads;
+    bool waited = false;
+    for (int it = part * kTcAttnThreads + tid; it < n_q + n_k + n_v; it += 2 * stride) {
+      const Item A = decode(it), B = decode(it + stride);
+      float xa1[8], xa2[8], xb1[8], xb2[8];
+      gather2(A, B, xa1, xa2, xb1, xb2);
+      if (!waited) { cluster_wait(); waited = true; }      // remote stores only once every CTA of the cluster runs
+      finish(A, xa1, xa2);
+      finish(B, xb1, xb2);
     }
+    if (!waited) cluster_wait();
     asm volatile("fence.proxy.async;" ::: "memory");      // these stores are read by the tensor core
     cluster_sync_all();
   }
