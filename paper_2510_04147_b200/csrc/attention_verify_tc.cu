@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   }
 
   // ---- prefix K/V straight from the cache (zero rows past the end of the part)
-  auto load_prefix = [&](int tile) {
+  auto load_prefix = [&](int tile, bool want_k = true, bool want_v = true) {
     const int seq = seq_of_slot(a.map, slot);
     const int kb = k_begin + tile * kKeys;
     const bf16* kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * kHD;
@@ -210,8 +210,8 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       const int key = kb + row;
       const bool valid = key < k_end;
       const size_t off = (size_t)(valid ? key : kb) * krow_stride + ch * 8;
-      cp_async16(sK + tile_off(row, ch, kKeys), kbase + off, valid);
-      cp_async16(sV + tile_off(row, ch, kKeys), vbase + off, valid);
+      if (want_k) cp_async16(sK + tile_off(row, ch, kKeys), kbase + off, valid);
+      if (want_v) cp_async16(sV + tile_off(row, ch, kKeys), vbase + off, valid);
     }
   };
   const bool commit_kv = a.cache_k_out != nullptr && (h % (a.H / a.Hkv)) == 0;
@@ -400,9 +400,12 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     const uint32_t phase = (uint32_t)(t & 1);
     if (t > 0) {
       // the previous tile's MMAs are complete: K (holding P) and V are free
-      load_prefix(t);
+      // (K and V as two groups: S = Q K^T starts when K has landed, V may take until P is ready)
+      load_prefix(t, true, false);
       cp_async_commit();
-      cp_async_wait<0>();
+      load_prefix(t, false, true);
+      cp_async_commit();
+      cp_async_wait<1>();
       asm volatile("fence.proxy.async;" ::: "memory");
       tc_fence_before();
       __syncthreads();
@@ -486,7 +489,8 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
         tmem_st32(ta, v);
       }
     }
-    asm volatile("fence.proxy.async;" ::: "memory");      // P is read by the tensor core
+    cp_async_wait<0>();                                   // V of a later tile
+    asm volatile("fence.proxy.async;" ::: "memory");      // P (and V) are read by the tensor core
     tc_fence_before();
     __syncthreads();
     if (tid == 0) {
