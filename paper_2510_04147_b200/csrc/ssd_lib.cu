@@ -72,7 +72,7 @@ struct ssd_ctx {
   int pending_T = 0;
   int* pending_ids = nullptr;    // [max_batch][block_len] tokens of that block
   int fuse_commit = 1;
-  std::vector<int> h_remaining, h_has_drafts;
+  std::vector<int> h_remaining, h_has_drafts, h_nodes;
 
   int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0, gemm_impl = 1;
   int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
@@ -466,6 +466,7 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
   c->split_down = auto_split(gemm_tiles(c->d), c->ffn_pad);
   c->h_remaining.assign(k.max_batch, 0);
   c->h_has_drafts.assign(k.max_batch, 0);
+  c->h_nodes.assign(k.max_batch, 0);
 
   int rc = SSD_OK;
   auto build = [&]() -> int {
@@ -728,21 +729,29 @@ int ssd_get_block_state(ssd_ctx* c, int32_t* ids, uint8_t* masked, int32_t* draf
   return SSD_OK;
 }
 
-int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n_nodes) {
-  if (!c) return SSD_ERR_INVALID_ARG;
-  if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
+namespace {
+
+int resolve_drafts(const ssd_ctx* c, int max_drafts) {
   int md = max_drafts < 0 ? c->cfg.max_drafts : max_drafts;
-  if (md > c->cfg.max_drafts) md = c->cfg.max_drafts;
+  return md > c->cfg.max_drafts ? c->cfg.max_drafts : md;
+}
+
+// Enqueues one iteration of Algorithm 1's loop for every unfinished sequence - tree build, the batched
+// forward, acceptance - without waiting for it.  The host's mirror of `remaining` / `has_drafts` decides
+// the launch shape; h_nodes[b] receives the nodes sequence b gets (0: finished).  The error flags are
+// sticky and are NOT cleared here.
+int step_enqueue(ssd_ctx* c, int md, bool* launched) {
   const int T = c->block_tokens, B = c->batch;
   int active = 0, n_cap = 1;
   for (int b = 0; b < B; ++b) {
+    c->h_nodes[b] = 0;
     if (c->h_remaining[b] <= 0) continue;
     ++active;
     const int N = c->h_has_drafts[b] ? (md < c->h_remaining[b] - 1 ? md : c->h_remaining[b] - 1) : 0;
+    c->h_nodes[b] = N + 1;
     if (N + 1 > n_cap) n_cap = N + 1;
   }
-  if (accepted) memset(accepted, 0, B * sizeof(int));
-  if (n_nodes) memset(n_nodes, 0, B * sizeof(int));
+  *launched = active > 0;
   if (active == 0) return SSD_OK;
   // A block waiting for its commit rides in front of the first forward of this block: per sequence
   // one causal chain [finished block | this block, all MASK].  Only a fresh block qualifies (every
@@ -756,11 +765,11 @@ int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n
     } else {
       const int frc = flush_pending(c);
       if (frc) return frc;
+      CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
     }
   }
   const int slot_rows = Tp + n_cap * T;
   const int R = active * slot_rows;
-  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
   {
     Scope sc(c, SSD_PROF_TREE, (double)R * 5);
     launch_tree_build(c->st, c->bs, B, T, md, n_cap, c->cfg.mask_id, c->node_ids, c->node_masked,
@@ -782,27 +791,50 @@ int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n
     Scope sc(c, SSD_PROF_TREE, (double)R * 9);
     launch_accept(c->st, c->bs, active, T, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1, slot_rows, Tp);
   }
+  if (Tp > 0) {                // the finished block's K/V are in the cache once this forward has run
+    c->cache_len += Tp;
+    c->pending_T = 0;
+  }
+  for (int b = 0; b < B; ++b)
+    if (c->h_nodes[b] > 0) c->h_has_drafts[b] = 1;
+  return SSD_OK;
+}
+
+// Waits for everything enqueued, checks the error flags and refreshes the host's mirror of `remaining`.
+int step_collect(ssd_ctx* c, int32_t* accepted, int32_t* n_nodes) {
+  const int B = c->batch;
   int* hp = c->h_pinned;
   const int mb = c->cfg.max_batch;
   CUDA_TRY(c, cudaMemcpyAsync(hp, c->flags, 2 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   CUDA_TRY(c, cudaMemcpyAsync(hp + 2, c->bs.remaining, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
-  CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + mb, c->bs.last_accept, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
-  CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 2 * mb, c->bs.n_cand, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  if (accepted) CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + mb, c->bs.last_accept, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  if (n_nodes) CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 2 * mb, c->bs.n_cand, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   CUDA_TRY(c, cudaStreamSynchronize(c->st));
-  rc = check_flags_after_sync(c);
+  const int rc = check_flags_after_sync(c);
   if (rc) return rc;
-  if (Tp > 0) {                // the finished block's K/V are in the cache now
-    c->cache_len += Tp;
-    c->pending_T = 0;
-  }
   for (int b = 0; b < B; ++b) {
-    const bool was_active = c->h_remaining[b] > 0;
     c->h_remaining[b] = hp[2 + b];
-    if (was_active) c->h_has_drafts[b] = 1;
     if (accepted) accepted[b] = hp[2 + mb + b];
-    if (n_nodes) n_nodes[b] = was_active ? hp[2 + 2 * mb + b] + 1 : 0;
+    if (n_nodes) n_nodes[b] = c->h_nodes[b] > 0 ? hp[2 + 2 * mb + b] + 1 : 0;
   }
   return SSD_OK;
+}
+
+}  // namespace
+
+int ssd_block_step(ssd_ctx* c, int32_t max_drafts, int32_t* accepted, int32_t* n_nodes) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
+  const int md = resolve_drafts(c, max_drafts);
+  const int B = c->batch;
+  if (accepted) memset(accepted, 0, B * sizeof(int));
+  if (n_nodes) memset(n_nodes, 0, B * sizeof(int));
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  bool launched = false;
+  int rc = step_enqueue(c, md, &launched);
+  if (rc) return rc;
+  if (!launched) return SSD_OK;
+  return step_collect(c, accepted, n_nodes);
 }
 
 int ssd_block_commit(ssd_ctx* c) {
@@ -833,13 +865,30 @@ int ssd_decode_block(ssd_ctx* c, int32_t mode, int32_t T, int32_t* out_tokens, i
   if (mode != SSD_MODE_STEPWISE && mode != SSD_MODE_SSD) return fail(c, SSD_ERR_INVALID_ARG, "unknown mode %d", mode);
   int rc = ssd_block_begin(c, T);
   if (rc) return rc;
-  const int md = mode == SSD_MODE_STEPWISE ? 0 : -1;
+  const int md = resolve_drafts(c, mode == SSD_MODE_STEPWISE ? 0 : -1);
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  // A forward accepts between 1 and nodes tokens per sequence, so after it at least remaining - nodes
+  // positions are still masked.  While that bound leaves every sequence a full chain (>= md + 1), the
+  // next forward's launch shape is known without its predecessor's result: it is enqueued at once and
+  // the host mirror carries the bound.  The host waits (and learns the true counts) only when the bound
+  // no longer decides the shape - a handful of times per block instead of once per forward.
   for (int guard = 0; guard <= T; ++guard) {
     bool any = false;
     for (int b = 0; b < c->batch; ++b) any = any || c->h_remaining[b] > 0;
     if (!any) break;
-    rc = ssd_block_step(c, md, nullptr, nullptr);
+    bool launched = false;
+    rc = step_enqueue(c, md, &launched);
     if (rc) return rc;
+    bool decided = true;
+    for (int b = 0; b < c->batch; ++b)
+      if (c->h_nodes[b] > 0 && c->h_remaining[b] - c->h_nodes[b] < md + 1) decided = false;
+    if (decided) {
+      for (int b = 0; b < c->batch; ++b) c->h_remaining[b] -= c->h_nodes[b];
+      continue;
+    }
+    rc = step_collect(c, nullptr, nullptr);
+    if (rc) return rc;
+    CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
   }
   const int st = c->bs.stride, B = c->batch;
   if (out_tokens) CUDA_TRY(c, cudaMemcpy2DAsync(out_tokens, T * sizeof(int), c->bs.ids, st * sizeof(int), T * sizeof(int), B, cudaMemcpyDeviceToHost, c->st));
