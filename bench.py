@@ -208,7 +208,20 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------
 # the CUDA path
 # --------------------------------------------------------------------------------------------
+def ensure_library():
+    """Compile the CUDA library when this tree has not been built yet; there is no other implementation to use."""
+    from paper_2510_04147_b200 import binding, build
+    if not os.path.exists(binding.LIB_PATH):
+        if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+            build.build()
+        else:                                   # another rank of this node is compiling
+            t0 = time.time()
+            while not os.path.exists(binding.LIB_PATH) and time.time() - t0 < 900:
+                time.sleep(2.0)
+
+
 def run_ours(args):
+    ensure_library()
     import numpy as np
     import torch
     from paper_2510_04147_b200 import binding, replicas, workloads as wl

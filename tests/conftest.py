@@ -12,6 +12,14 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+def pytest_sessionstart(session):
+    """Build the CUDA library if it has not been built in this tree yet (nvcc cross-compiles without a GPU).
+    The binding itself never builds and never falls back: without the library its calls raise."""
+    from paper_2510_04147_b200 import binding, build
+    if not os.path.exists(binding.LIB_PATH):
+        build.build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
