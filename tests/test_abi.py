@@ -14,7 +14,7 @@ def _declared():
     return sorted(set(re.findall(r"\b(ssd_[a-z0-9_]+)\s*\(", src)))
 
 
-def test_header_declares_the_north_star_calls():
+def test_header_declares_the_three_main_calls():
     names = _declared()
     for n in ("ssd_load_weights", "ssd_prefill", "ssd_decode_block"):
         assert n in names

@@ -1,6 +1,6 @@
 """CUDA path vs the CPU oracle, through the C ABI (run with -m gpu on a B200).
 
-Tolerances (bf16 operands, fp32 accumulation; stated by the workload's north star):
+Tolerances (bf16 operands, fp32 accumulation; the stated parity bar):
   * logits within 2e-2 absolute of the fp64 oracle, confidences within 2e-2 relative;
   * against the oracle run with bf16 operand rounding (same arithmetic type as the kernels) the
     logits agree to 1e-2, half the stated tolerance.  That comparison is not bit-level: the kernels
