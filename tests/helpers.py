@@ -29,6 +29,19 @@ def oracle_weights(w: wl.Workload, as_bf16: bool) -> dict:
     return out
 
 
+class LazyWeights:
+    """The tensors of a LARGE workload one at a time, as the oracle asks for them (fp64, matrices rounded
+    to bfloat16 values): nothing is kept, so a full-size model needs one tensor's worth of host memory.
+    ``device`` is where the seeded generator runs (its output does not depend on it)."""
+
+    def __init__(self, w: wl.Workload, device: str = "cpu"):
+        self.w, self.device = w, device
+
+    def __getitem__(self, name: str) -> np.ndarray:
+        a = wl.make_tensor(self.w, name, self.device).to(torch.float32).cpu().numpy().astype(np.float64)
+        return bf16_round(a) if a.ndim == 2 else a
+
+
 def make_oracle(w: wl.Workload, as_bf16: bool = False, operand_rounding=None) -> Oracle:
     return Oracle(oracle_config(w), oracle_weights(w, as_bf16), operand_rounding)
 
