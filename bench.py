@@ -30,7 +30,7 @@ METRIC = "decode tokens/s at batch 1 (LLaDA-8B-shaped) and % HBM roofline per ve
 # DRAM bytes per projection launch from the ncu capture summarised in
 # profiles/gemm_tc_kernel_llada8b_4layers.md (mean over the four projections of a LLaDA-8B-shaped layer).
 # Valid only for the kernel source it was taken from: reported as null once gemm.cu has changed.
-GEMM_TRAFFIC = {"workload": "llada8b", "bytes_per_launch": 113.0e6, "gemm_cu_sha256_16": "7e5a9fa5033b1eef"}
+GEMM_TRAFFIC = {"workload": "llada8b", "bytes_per_launch": 113.0e6, "gemm_cu_sha256_16": "f728082ded987180"}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -246,7 +246,7 @@ def run_ours(args):
     torch.cuda.set_stream(stream)
     ssd = binding.Ssd(binding.config_from_workload(w, max_drafts=min(cfg_drafts, B - 1)))
     for k, v in (("split_k_qkv", args.split_qkv), ("split_k_o", args.split_o), ("split_k_down", args.split_down),
-                 ("kv_split", args.kv_split), ("attn_impl", args.attn_impl)):
+                 ("kv_split", args.kv_split), ("attn_impl", args.attn_impl), ("two_sm_rows", args.two_sm_rows)):
         if v is not None:
             ssd.set_option(k, v)
     t0 = time.time()
@@ -450,6 +450,8 @@ def main():
     ap.add_argument("--split-down", type=int, default=None)
     ap.add_argument("--kv-split", type=int, default=None)
     ap.add_argument("--attn-impl", type=int, default=None, help="0: mma.sync attention; 1: tcgen05 attention where eligible")
+    ap.add_argument("--two-sm-rows", type=int, default=None,
+                    help="projection tile pairs run as one two-SM MMA from this many rows on (0: never)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: fewer layers of the same shape")
     ap.add_argument("--gen-len", type=int, default=0, help="profiling only: shorter generation")

@@ -103,6 +103,7 @@ struct TcParams {
   int stages;
   int epi;
   int w_tiled;     // weights in the tile-contiguous layout: one 16 KB block per (tile, K block)
+  int two_sm;      // the CTAs of tiles 2i, 2i + 1 issue ONE tcgen05.mma.cta_group::2 (M = 256): each holds half of the activation tile
   uint32_t tmem_cols;
   float* out;
   bf16* act;
@@ -166,6 +167,28 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// ---- forms for a pair of CTAs working as one MMA (cta_group::2).  The even CTA of the pair leads: it
+// owns the "full" barriers (both CTAs' copies count their bytes there - the barrier address with the
+// pair bit cleared), issues the MMAs, and its commits arrive on both CTAs' barriers.
+constexpr uint32_t kPairLeaderMask = 0xFEFFFFFFu;       // shared::cluster address of the same offset in the even CTA
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"((unsigned long long)map), "r"(bar & kPairLeaderMask), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  const uint32_t z = 0;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n}\n"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(z) : "memory");
+}
 // K-major operand tile in shared memory, 128-byte swizzle, rows 128 B apart, 8-row groups 1024 B apart.
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
@@ -219,12 +242,16 @@ __device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
   return v;
 }
 
+// kTwoSm: the instantiation whose CTAs work in pairs (cluster of two along x); the single-CTA
+// instantiation contains none of the pair instructions.
+template <bool kTwoSm>
 __global__ void __launch_bounds__(kTcThreads, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX, const TcParams p) {
   extern __shared__ uint8_t smem_dyn[];
   // 1024-byte alignment for the swizzled tiles
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  const int x_tile_bytes = p.npad * kBlockK * 2;
+  constexpr bool ts = kTwoSm;
+  const int x_tile_bytes = (ts ? p.npad / 2 : p.npad) * kBlockK * 2;    // a pair holds half of the rows each
   uint8_t* sW = smem;
   uint8_t* sX = smem + (size_t)p.stages * kWTileBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sX + (size_t)p.stages * x_tile_bytes);
@@ -242,6 +269,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int kb_begin = (int)((long long)split * kb_total / p.splits);
   const int kb_end = (int)((long long)(split + 1) * kb_total / p.splits);
   const int n_kb = kb_end - kb_begin;
+  uint32_t crank = 0u;
+  if constexpr (ts) crank = cluster_ctarank() & 1u;
+  const bool leader = crank == 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) {
@@ -256,13 +286,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tmX) : "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
-                 "r"(p.tmem_cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (ts) {        // the same warp of both CTAs: the columns are taken in both SMs
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
+                   "r"(p.tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(tmem_slot)),
+                   "r"(p.tmem_cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (ts) {                    // the peer's barriers exist before anything arrives on them
+    cluster_arrive_release();
+    cluster_wait_acquire();
+  }
   const uint32_t tmem_base = *tmem_slot;
 
   bool epi_ok = false;       // epilogue threads: the accumulator is complete
@@ -272,22 +312,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const uint32_t stage_bytes = (uint32_t)(kWTileBytes + x_tile_bytes);
       int issued = 0;
       bool ok = true;
+      // In a pair only the leader's barrier counts: it expects both CTAs' bytes, and both CTAs' copies
+      // complete on it.
+      auto expect = [&](uint32_t fb) {
+        if (!ts) mbar_expect_tx(fb, stage_bytes);
+        else if (leader) mbar_expect_tx(fb, 2u * stage_bytes);
+      };
       auto load_w = [&](int it, int s, uint32_t fb) {
         const int kb = kb_begin + it;
-        if (p.w_tiled) tma_load_2d(smem_addr(sW + (size_t)s * kWTileBytes), &tmW, fb, 0, (tile * kb_total + kb) * kTileM);
-        else tma_load_2d(smem_addr(sW + (size_t)s * kWTileBytes), &tmW, fb, kb * kBlockK, tile * kTileM);
+        const uint32_t dst = smem_addr(sW + (size_t)s * kWTileBytes);
+        const int c0 = p.w_tiled ? 0 : kb * kBlockK, c1 = p.w_tiled ? (tile * kb_total + kb) * kTileM : tile * kTileM;
+        if constexpr (ts) tma_load_2d_pair(dst, &tmW, fb, c0, c1);
+        else tma_load_2d(dst, &tmW, fb, c0, c1);
+      };
+      auto load_x = [&](int it, int s, uint32_t fb) {
+        const uint32_t dst = smem_addr(sX + (size_t)s * x_tile_bytes);
+        if constexpr (ts) tma_load_2d_pair(dst, &tmX, fb, (kb_begin + it) * kBlockK, row0 + (int)crank * (p.npad / 2));
+        else tma_load_2d(dst, &tmX, fb, (kb_begin + it) * kBlockK, row0);
       };
       // The weights do not depend on any earlier kernel: fill the ring with weight tiles first, and
       // only then wait for the kernel that produces the activations.
       const int pre = n_kb < p.stages ? n_kb : p.stages;
       for (int it = 0; it < pre; ++it) {
         const uint32_t fb = smem_addr(&full_bar[it]);
-        mbar_expect_tx(fb, stage_bytes);
+        expect(fb);
         load_w(it, it, fb);
       }
       pdl_wait();
       for (int it = 0; it < pre; ++it) {
-        tma_load_2d(smem_addr(sX + (size_t)it * x_tile_bytes), &tmX, smem_addr(&full_bar[it]), (kb_begin + it) * kBlockK, row0);
+        load_x(it, it, smem_addr(&full_bar[it]));
         ++issued;
       }
       for (int it = pre; it < n_kb; ++it) {
@@ -295,9 +348,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const uint32_t ph = (uint32_t)((it / p.stages) & 1);
         if (!mbar_wait(smem_addr(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t fb = smem_addr(&full_bar[s]);
-        mbar_expect_tx(fb, stage_bytes);
+        expect(fb);
         load_w(it, s, fb);
-        tma_load_2d(smem_addr(sX + (size_t)s * x_tile_bytes), &tmX, fb, (kb_begin + it) * kBlockK, row0);
+        load_x(it, s, fb);
         ++issued;
       }
       if (!ok) {
@@ -305,7 +358,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         atomicExch(p.err_flag, 1);
         // let the copies already in flight land before the CTA's shared memory goes away
         const int first = issued > p.stages ? issued - p.stages : 0;
-        for (int j = first; j < issued; ++j) {
+        for (int j = first; j < issued && (!ts || leader); ++j) {
           const unsigned long long t0 = globaltimer_ns();
           while (!mbar_try_wait(smem_addr(&full_bar[j % p.stages]), (uint32_t)((j / p.stages) & 1)))
             if (globaltimer_ns() - t0 > kWaitLimitNs) break;
@@ -314,9 +367,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && leader) {        // (in a pair the even CTA issues for both)
+      // M = 128 features of this CTA, or 256 = the pair's two weight tiles; N = the padded rows
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.npad >> 3) << 17) |
-                             ((uint32_t)(kTileM >> 4) << 24);
+                             ((uint32_t)((ts ? 2 * kTileM : kTileM) >> 4) << 24);
       bool ok = true;
       for (int it = 0; it < n_kb; ++it) {
         const int s = it % p.stages;
@@ -327,13 +381,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const uint32_t xa = smem_addr(sX + (size_t)s * x_tile_bytes);
 #pragma unroll
         for (int k = 0; k < kBlockK / 16; ++k) {
-          tc_mma_bf16(tmem_base, make_smem_desc(wa + k * 32), make_smem_desc(xa + k * 32), idesc,
-                      (uint32_t)((it | k) != 0));
+          if constexpr (ts) tc_mma_bf16_pair(tmem_base, make_smem_desc(wa + k * 32), make_smem_desc(xa + k * 32), idesc,
+                                   (uint32_t)((it | k) != 0));
+          else tc_mma_bf16(tmem_base, make_smem_desc(wa + k * 32), make_smem_desc(xa + k * 32), idesc,
+                           (uint32_t)((it | k) != 0));
         }
-        tc_commit(smem_addr(&empty_bar[s]));
+        // a pair's commits arrive on both CTAs' barriers; only stages that will be refilled need one
+        if constexpr (!ts) tc_commit(smem_addr(&empty_bar[s]));
+        else if (it + p.stages < n_kb) tc_commit_pair(smem_addr(&empty_bar[s]));
       }
       if (ok) {
-        tc_commit(smem_addr(acc_bar));
+        if constexpr (ts) tc_commit_pair(smem_addr(acc_bar));
+        else tc_commit(smem_addr(acc_bar));
       } else {
         *abort_flag = 1;
         atomicExch(p.err_flag, 2);
@@ -580,8 +639,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   }
   tc_fence_before();
   __syncthreads();
+  if (ts) {                    // both CTAs have read their accumulators; nothing is on its way between them
+    cluster_arrive_release();
+    cluster_wait_acquire();
+  }
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    if constexpr (ts) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
   }
 }
 
@@ -631,10 +695,13 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   p.splits = g.splits;
   p.epi = g.epi;
   p.w_tiled = g.w_tiled;
+  // Pairs of tiles as one two-SM MMA from `two_sm_min_rows` padded rows on (0: never): every SM then takes
+  // in half of the activation tile.  The accumulation order is the same, so the row count may decide.
+  p.two_sm = (g.two_sm_min_rows > 0 && p.npad >= g.two_sm_min_rows && g.epi != EPI_RESIDUAL && (gemm_tiles(g.N) % 2) == 0) ? 1 : 0;
   uint32_t cols = 32;
   while ((int)cols < p.npad) cols <<= 1;
   p.tmem_cols = cols;
-  const int stage_bytes = kWTileBytes + p.npad * kBlockK * 2;
+  const int stage_bytes = kWTileBytes + (p.two_sm ? p.npad / 2 : p.npad) * kBlockK * 2;
   // two CTAs per SM while the activation tile is small, one deep pipeline otherwise
   const int budget = 108 * 1024;
   int stages = budget / stage_bytes;
@@ -657,16 +724,20 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   } else if (!make_tmap(&tmW, g.w, (uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.w_pitch, kTileM)) {
     return -4;
   }
-  if (!make_tmap(&tmX, g.x, (uint64_t)g.R, (uint64_t)g.K, (uint64_t)g.x_pitch, (uint32_t)p.npad)) return -4;
+  if (!make_tmap(&tmX, g.x, (uint64_t)g.R, (uint64_t)g.K, (uint64_t)g.x_pitch, (uint32_t)(p.two_sm ? p.npad / 2 : p.npad))) return -4;
   static int smem_set = 0;
   if (smem > smem_set) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return -4;
     smem_set = 227 * 1024;
   }
   dim3 grid(gemm_tiles(g.N), g.splits, (g.R + 255) / 256);
   const unsigned cluster_y = (g.epi == EPI_RESIDUAL) ? (unsigned)g.splits : 1u;
-  if (launch_pdl_cluster_xy(gemm_tc_kernel, grid, dim3(kTcThreads), (size_t)smem, st, 1u, cluster_y, tmW, tmX, p) != cudaSuccess)
+  const cudaError_t le = p.two_sm
+      ? launch_pdl_cluster_xy(gemm_tc_kernel<true>, grid, dim3(kTcThreads), (size_t)smem, st, 2u, cluster_y, tmW, tmX, p)
+      : launch_pdl_cluster_xy(gemm_tc_kernel<false>, grid, dim3(kTcThreads), (size_t)smem, st, 1u, cluster_y, tmW, tmX, p);
+  if (le != cudaSuccess)
     return -4;
   return 0;
 }

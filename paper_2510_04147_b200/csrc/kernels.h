@@ -168,6 +168,7 @@ struct GemmArgs {
   int R, N, K, x_pitch, w_pitch;
   int w_tiled;           // 1: w is [ceil(N/128)][ceil(K/64)][128][64] (one 16 KB block per MMA tile, zero padded)
   int splits;            // split-K factor (EPI_PARTIAL only)
+  int two_sm_min_rows;   // tensor-core kernel: pairs of tiles run as one cta_group::2 MMA from this many rows on; 0 = never
   int epi;
   float* out;            // EPI_PARTIAL: [splits][R][N] fp32
   bf16* act;             // EPI_SWIGLU: [R][act_pitch], N/2 features

@@ -75,6 +75,7 @@ struct ssd_ctx {
   std::vector<int> h_remaining, h_has_drafts, h_nodes;
 
   int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0, gemm_impl = 1;
+  int two_sm_rows = 256;                   // projections pair their tiles (two-SM MMA) from this many rows on; 0 = never
   int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
   int64_t launches = 0;
   bool profiling = false;
@@ -200,6 +201,7 @@ __global__ void block_init_kernel(BlockState s, int batch, int max_batch, int T,
 int run_gemm(ssd_ctx* c, GemmArgs g, int fam, int sub = -1) {
   Scope sc(c, fam, (double)g.N * g.K * 2.0, 1, sub);
   g.err_flag = c->flags;
+  g.two_sm_min_rows = c->two_sm_rows;
   if (c->gemm_impl == 1) {
     const int rc = launch_gemm_tc(c->st, g);
     if (rc != 0) return fail(c, rc, "tensor-core GEMM rejected R=%d N=%d K=%d epi=%d (code %d)", g.R, g.N, g.K, g.epi, rc);
@@ -1022,6 +1024,11 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "attn_impl")) {
     if (value != 0 && value != 1) return fail(c, SSD_ERR_INVALID_ARG, "attn_impl is 0 (mma.sync) or 1 (tcgen05 where the shape allows)");
     c->attn_impl = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "two_sm_rows")) {
+    if (value < 0 || value > 256) return fail(c, SSD_ERR_INVALID_ARG, "two_sm_rows is 0 (never) or a row count up to 256");
+    c->two_sm_rows = value;
     return SSD_OK;
   }
   if (!strcmp(key, "fuse_commit")) {

@@ -260,6 +260,28 @@ def test_extreme_blocks_ssd_equals_stepwise_and_oracle_steps(block_len, prompt_l
         assert np.array_equal(tok_g[0, 0][sure], otok[0][sure])
 
 
+@pytest.mark.parametrize("case,n_nodes", [("llada_width", 2), ("dream_width", 1), ("llada_width", 8)])
+def test_two_sm_projections_change_no_bit_of_a_forward(case, n_nodes):
+    """All three epilogues that run under the two-SM MMA (split-K partials, SwiGLU, LM-head statistics),
+    at 32 to 256 rows: the forward is bit-identical with the pairs always on and always off."""
+    w, _ = WIDTH_CASES[case]
+    rng = np.random.default_rng(7)
+    T = w.block_len
+    prompt = wl.make_prompts(w).numpy()
+    ids, masked = _nodes(w, rng, n_nodes, T)
+    out = {}
+    ssd = _make(w, max_drafts=n_nodes)
+    try:
+        for rows in (0, 16):
+            ssd.set_option("two_sm_rows", rows)
+            ssd.prefill(prompt)
+            out[rows] = ssd.verify_forward(ids, masked, want_logits=(n_nodes <= 2))
+    finally:
+        ssd.destroy()
+    for a, b in zip(out[0], out[16]):
+        assert (a is None and b is None) or np.array_equal(a, b)
+
+
 def test_both_attention_forms_agree_at_full_width():
     """The tcgen05 attention (default where the shape allows) and the mma.sync form compute the same
     forward up to the rounding of a different summation order."""

@@ -27,6 +27,7 @@ GAP = 1e-3
 CONF_RTOL = 2e-2     # a logit error e moves a softmax probability by a factor within exp(+-2e)
 # which projection kernel the shared contexts use by default (1 = tcgen05, the product path)
 DEFAULT_IMPL = int(os.environ.get("SSD_TEST_GEMM_IMPL", "1"))
+DEFAULT_TWO_SM = 256         # the library's default for "two_sm_rows"
 PEAKED = wl.TINY.replace(name="tiny_peaked", lm_head_scale=8.0)
 
 
@@ -88,6 +89,27 @@ def test_gemm_against_numpy(tiny_ssd, impl, rows, n, k, split):
         assert np.abs(out - ref).max() < 2e-5 * scale * np.sqrt(k) + 1e-6, np.abs(out - ref).max()
     finally:
         tiny_ssd.set_option("gemm_impl", DEFAULT_IMPL)
+
+
+@pytest.mark.parametrize("rows,n,k,split", [(16, 256, 64, 1), (32, 256, 256, 1), (100, 768, 704, 1), (48, 1280, 256, 1),
+                                            (128, 4096, 4096, 4), (64, 512, 12288, 8), (300, 512, 512, 2),
+                                            (256, 256, 1024, 3), (1, 256, 72, 1)])
+def test_gemm_two_sm_pairs_change_no_bit(tiny_ssd, rows, n, k, split):
+    """Pairs of weight tiles as one cta_group::2 MMA (each CTA of the pair holds its own weight tile and
+    half of the activation tile; the even CTA issues, both read their own accumulator): the same products
+    summed in the same order, so the result is bit-identical to the single-CTA launch."""
+    x = wl.normal_tensor(6, 1, (rows, k), 1.0, device="cuda", dtype=torch.bfloat16)
+    w = wl.normal_tensor(6, 2, (n, k), 0.05, device="cuda", dtype=torch.bfloat16)
+    try:
+        tiny_ssd.set_option("two_sm_rows", 0)
+        plain = tiny_ssd.gemm_bf16(x, w, split).cpu().numpy()
+        tiny_ssd.set_option("two_sm_rows", 16)
+        paired = tiny_ssd.gemm_bf16(x, w, split).cpu().numpy()
+    finally:
+        tiny_ssd.set_option("two_sm_rows", DEFAULT_TWO_SM)
+    assert np.array_equal(plain, paired)
+    ref = x.cpu().to(torch.float64).numpy() @ w.cpu().to(torch.float64).numpy().T
+    assert np.abs(paired - ref).max() < 2e-5 * 0.05 * k + 1e-6
 
 
 # ------------------------------------------------------------------------------------------
