@@ -180,8 +180,15 @@ int ssd_gemm_bf16_noalloc(const void* x_dev, const void* w_dev, float* out_dev, 
 /* Kernel launches issued by this context since creation (all streams of the context). */
 int64_t ssd_launch_count(const ssd_ctx* ctx);
 
-/* Per-kernel-family device time.  When enabled, every launch is bracketed by CUDA events on the
- * context's stream (this serialises launches; do not time throughput in this mode).
+/* Per-kernel-family device time.  ssd_profile_enable(ctx, mode):
+ *   0  off;
+ *   1  every launch is bracketed by CUDA events on the context's stream: the kernel alone, without the
+ *      overlap with its neighbours that dependent launches give it (this serialises the stream; do
+ *      not time throughput in this mode);
+ *   2  the live stream: a one-thread marker kernel behind every launch records the time that launch
+ *      completed, and a launch is charged the time from its predecessor's completion to its own (so
+ *      the charges add up to the wall time; each marker adds about a microsecond of dependency
+ *      latency).
  * ssd_profile_read fills, for family f in [0, SSD_PROF_FAMILIES): launches[f], milliseconds[f],
  * algorithmic bytes[f] (operand bytes that must cross HBM once), and resets the counters. */
 #define SSD_PROF_GEMM      0   /* QKV / O / gate-up / down projections                         */

@@ -244,8 +244,9 @@ class Ssd:
     def launch_count(self) -> int:
         return int(self.lib.ssd_launch_count(self._ctx))
 
-    def profile_enable(self, on: bool):
-        self._check(self.lib.ssd_profile_enable(self._ctx, 1 if on else 0))
+    def profile_enable(self, on):
+        """False / 0: off; True / 1: CUDA events around every launch; 2: end-of-launch marks in the live stream."""
+        self._check(self.lib.ssd_profile_enable(self._ctx, int(on)))
 
     def profile_read(self):
         n = len(PROF_FAMILIES)

@@ -22,6 +22,8 @@ struct LayerW {
 };
 
 struct ProfRec { int fam, sub; cudaEvent_t e0, e1; double bytes; };
+struct MarkRec { int fam, sub; double bytes; };
+constexpr int kMaxMarks = 16384;      // launches one in-stream measurement can hold
 
 char g_create_error[256] = "";
 
@@ -78,7 +80,10 @@ struct ssd_ctx {
   int two_sm_rows = 256;                   // projections pair their tiles (two-SM MMA) from this many rows on; 0 = never
   int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
   int64_t launches = 0;
-  bool profiling = false;
+  bool profiling = false;        // mode 1: CUDA events around every launch (serialises the stream)
+  bool marking = false;          // mode 2: a marker kernel after every launch stamps the time it ended, in the live stream
+  unsigned long long* marks = nullptr;   // device [kMaxMarks]
+  std::vector<MarkRec> mark_rec;
   std::vector<ProfRec> prof;
   std::vector<void*> allocs;
   char err[256] = "";
@@ -145,10 +150,21 @@ int kv_split_for(const ssd_ctx* c, int S) {
 }
 
 // ---- profiling / launch accounting --------------------------------------------------------
+// Runs as one more dependent launch behind the kernel it measures: its dependency wait ends when that
+// kernel has completed, and it writes the time.  The kernel after it still starts early and prefetches.
+__global__ void mark_end_kernel(unsigned long long* slot) {
+  pdl_launch_dependents();
+  pdl_wait();
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  *slot = t;
+}
+
 struct Scope {
   ssd_ctx* c;
   int fam, sub;
   double bytes;
+  int mark = -1;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   Scope(ssd_ctx* c_, int fam_, double bytes_, int n_launches = 1, int sub_ = -1)
       : c(c_), fam(fam_), sub(sub_), bytes(bytes_) {
@@ -158,8 +174,13 @@ struct Scope {
       cudaEventCreate(&e1);
       cudaEventRecord(e0, c->st);
     }
+    if (c->marking && (int)c->mark_rec.size() < kMaxMarks) {
+      mark = (int)c->mark_rec.size();
+      c->mark_rec.push_back({fam, sub, bytes});
+    }
   }
   ~Scope() {
+    if (mark >= 0) launch_pdl(mark_end_kernel, dim3(1), dim3(1), 0, c->st, c->marks + mark);
     if (c->profiling) {
       cudaEventRecord(e1, c->st);
       c->prof.push_back({fam, sub, e0, e1, bytes});
@@ -529,6 +550,7 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     ALLOC(c, c->node_ids, R);
     ALLOC(c, c->node_masked, R);
     ALLOC(c, c->flags, 4);
+    ALLOC(c, c->marks, kMaxMarks);
     const size_t sb = (size_t)k.max_batch * k.block_len;
     c->bs.stride = k.block_len;
     ALLOC(c, c->bs.ids, sb); ALLOC(c, c->bs.masked, sb); ALLOC(c, c->bs.draft_tok, sb); ALLOC(c, c->bs.draft_conf, sb);
@@ -970,7 +992,12 @@ int64_t ssd_launch_count(const ssd_ctx* c) { return c ? c->launches : -1; }
 
 int ssd_profile_enable(ssd_ctx* c, int32_t on) {
   if (!c) return SSD_ERR_INVALID_ARG;
-  c->profiling = on != 0;
+  if (on < 0 || on > 2) return fail(c, SSD_ERR_INVALID_ARG, "profile mode is 0 (off), 1 (events around every launch) or 2 (end-of-launch marks in the live stream)");
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  c->profiling = on == 1;
+  c->marking = on == 2;
+  c->mark_rec.clear();
+  if (c->marking) CUDA_TRY(c, cudaMemsetAsync(c->marks, 0, kMaxMarks * sizeof(unsigned long long), c->st));
   return SSD_OK;
 }
 
@@ -995,6 +1022,24 @@ int ssd_profile_read(ssd_ctx* c, int64_t* launches, double* ms, double* bytes) {
     cudaEventDestroy(r.e1);
   }
   c->prof.clear();
+  // mode 2: a launch is charged the time from the end of its predecessor to its own end
+  if (!c->mark_rec.empty()) {
+    std::vector<unsigned long long> t(c->mark_rec.size());
+    CUDA_TRY(c, cudaMemcpy(t.data(), c->marks, t.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+    for (size_t i = 1; i < t.size(); ++i) {
+      if (t[i] == 0 || t[i - 1] == 0 || t[i] < t[i - 1]) continue;
+      const double dt = (double)(t[i] - t[i - 1]) * 1e-6;
+      const MarkRec& r = c->mark_rec[i];
+      for (int f : {r.fam, r.sub}) {
+        if (f < 0) continue;
+        if (launches) launches[f] += 1;
+        if (ms) ms[f] += dt;
+        if (bytes) bytes[f] += r.bytes;
+      }
+    }
+    c->mark_rec.clear();
+    CUDA_TRY(c, cudaMemsetAsync(c->marks, 0, kMaxMarks * sizeof(unsigned long long), c->st));
+  }
   return SSD_OK;
 }
 
