@@ -447,6 +447,32 @@ def test_batched_sequences_equal_single_runs(peaked_ssd):
             assert np.array_equal(acc_s[j][0], acc_b[j][s]) and nf_s[j][0] == nf_b[j][s]
 
 
+def test_profile_modes_account_for_every_launch(tiny_ssd):
+    """Mode 1 brackets every launch with events, mode 2 stamps the end of every launch in the live stream;
+    both count the same launches per family, and decoding is unchanged while they run."""
+    w = wl.TINY
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    tiny_ssd.prefill(prompt)
+    ref, _, _ = tiny_ssd.decode_block(b.MODE_SSD, w.block_len, 1)
+    counts = {}
+    for mode in (1, 2):
+        tiny_ssd.prefill(prompt)
+        tiny_ssd.profile_enable(mode)
+        try:
+            tok, _, nf = tiny_ssd.decode_block(b.MODE_SSD, w.block_len, 1)
+            prof = tiny_ssd.profile_read()
+        finally:
+            tiny_ssd.profile_enable(0)
+        assert np.array_equal(tok, ref)
+        assert prof["gemm"]["launches"] > 0 and prof["gemm"]["ms"] > 0 and prof["attn"]["ms"] > 0
+        assert prof["gemm"]["launches"] == sum(prof[k]["launches"] for k in ("gemm_qkv", "gemm_o", "gemm_gu", "gemm_down"))
+        counts[mode] = {k: v["launches"] for k, v in prof.items()}
+    # mode 2 has no predecessor for its very first launch (a tree kernel)
+    assert counts[1]["gemm"] == counts[2]["gemm"] and counts[1]["attn"] == counts[2]["attn"]
+    assert counts[1]["tree"] == counts[2]["tree"] + 1
+
+
 def test_ragged_last_block(tiny_ssd):
     w = wl.TINY
     b = _binding()
