@@ -236,6 +236,11 @@ __device__ __forceinline__ uint32_t map_to_rank(const void* p, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_addr(p)), "r"(rank));
   return out;
 }
+// x^2 + y^2 + z^2 + w^2 with the roundings spelled out, so that the value does not depend on what the
+// compiler contracts around it
+__device__ __forceinline__ float sumsq4(const float4& a) {
+  return __fmaf_rn(a.w, a.w, __fmaf_rn(a.z, a.z, __fmaf_rn(a.y, a.y, __fmul_rn(a.x, a.x))));
+}
 __device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
@@ -601,36 +606,58 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       cluster_wait_acquire();
       bool arrived = false;
       if (epi_warp && epi_ok) {
-        for (int rr = (int)rank + (warp - 2) * (int)n_ranks; rr < pass_cnt; rr += 4 * (int)n_ranks) {
-          const int row = g0 + rr;
-          if (row >= rows_here) break;
-          float4 part[kGemmMaxClusterSplits];
+        // a warp takes its rows two at a time: the remote reads of both are in flight together
+        const int step = 4 * (int)n_ranks;
+        auto pull = [&](int rr, bool on, float4 (&part)[kGemmMaxClusterSplits]) {
 #pragma unroll
           for (int q = 0; q < kGemmMaxClusterSplits; ++q) {
             part[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if ((uint32_t)q < n_ranks) part[q] = ld_cluster_f32x4(map_to_rank(scratch + rr * kEpiPitch + f4, (uint32_t)q));
+            if (on && (uint32_t)q < n_ranks) part[q] = ld_cluster_f32x4(map_to_rank(scratch + rr * kEpiPitch + f4, (uint32_t)q));
           }
-          float* hp = p.h + (size_t)(row0 + row) * p.N + n_base + f4;
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (col_ok) acc = *reinterpret_cast<const float4*>(hp);
+        };
+        // residual + partials in split order
+        auto reduce = [&](float4 acc, const float4 (&part)[kGemmMaxClusterSplits]) -> float4 {
 #pragma unroll
           for (int q = 0; q < kGemmMaxClusterSplits; ++q) {
             if ((uint32_t)q < n_ranks) { acc.x += part[q].x; acc.y += part[q].y; acc.z += part[q].z; acc.w += part[q].w; }
           }
-          // this warp's last remote read of the pass has landed: arrive now, the stores overlap the barrier
-          if (rr + 4 * (int)n_ranks >= pass_cnt || g0 + rr + 4 * (int)n_ranks >= rows_here) { __syncwarp(); cluster_arrive_release(); arrived = true; }
+          return acc;
+        };
+        // h, bf16(h * gain) and the tile's sum of squares of the row
+        auto store = [&](int row, const float4& acc) {
           float ss = 0.f;
           if (col_ok) {
-            *reinterpret_cast<float4*>(hp) = acc;
+            *reinterpret_cast<float4*>(p.h + (size_t)(row0 + row) * p.N + n_base + f4) = acc;
             __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * g4.x, acc.y * g4.y);
             __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * g4.z, acc.w * g4.w);
             *reinterpret_cast<uint2*>(p.hb + (size_t)(row0 + row) * p.N + n_base + f4) =
                 make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-            ss = acc.x * acc.x + acc.y * acc.y + acc.z * acc.z + acc.w * acc.w;
+            ss = sumsq4(acc);
           }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
           if (lane == 0) p.sq_out[(size_t)(row0 + row) * p.sq_out_stride + tile] = ss;
+        };
+        for (int rrA = (int)rank + (warp - 2) * (int)n_ranks; rrA < pass_cnt; rrA += 2 * step) {
+          if (g0 + rrA >= rows_here) break;
+          const int rrB = rrA + step;
+          const bool onB = rrB < pass_cnt && g0 + rrB < rows_here;
+          float4 partA[kGemmMaxClusterSplits], partB[kGemmMaxClusterSplits];
+          pull(rrA, true, partA);
+          pull(rrB, onB, partB);
+          float4 hA = make_float4(0.f, 0.f, 0.f, 0.f), hB = hA;
+          if (col_ok) hA = *reinterpret_cast<const float4*>(p.h + (size_t)(row0 + g0 + rrA) * p.N + n_base + f4);
+          if (col_ok && onB) hB = *reinterpret_cast<const float4*>(p.h + (size_t)(row0 + g0 + rrB) * p.N + n_base + f4);
+          const float4 accA = reduce(hA, partA), accB = reduce(hB, partB);   // (uses every value read remotely)
+          // this warp's last remote read of the pass has landed: arrive now, the stores overlap the barrier
+          const int nextA = rrA + 2 * step;
+          if (nextA >= pass_cnt || g0 + nextA >= rows_here) {
+            __syncwarp();
+            cluster_arrive_release();
+            arrived = true;
+          }
+          store(g0 + rrA, accA);
+          if (onB) store(g0 + rrB, accB);
         }
       }
       if (!arrived) { __syncwarp(); cluster_arrive_release(); }
