@@ -30,7 +30,9 @@ own predictions from the same forward.
 Precision: everything is fp64.  ``operand_rounding`` optionally rounds the
 operands of every contraction (matmul inputs, attention Q/K/V/P) to bfloat16,
 which is the arithmetic type the accelerated path is specified to use (bf16
-operands, wide accumulation); with ``None`` nothing is rounded.
+operands, wide accumulation); with ``None`` nothing is rounded.  A collection
+of source names (``ROUNDING_SOURCES``) rounds only those operands, which is how
+the share of each rounding point in the total bf16 noise is measured.
 
 Pins: see tests/test_oracle_*.py.  The accept-count VALUES on random-init
 models have no value printed in the paper to compare with: parity unpinned by
@@ -68,6 +70,16 @@ def bf16_round(x: np.ndarray) -> np.ndarray:
     b = f.view(np.uint32).astype(np.uint64)
     b = (b + 0x7FFF + ((b >> 16) & 1)) & 0xFFFF0000
     return b.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
+# The operands a bf16 contraction rounds, by where they enter:
+#   proj_in  normalised hidden state into the q/k/v and gate/up projections
+#   qkv      rotated q and k, and v, into the two attention contractions
+#   p        softmax probabilities into P.V
+#   att      attention output into the output projection
+#   act      SwiGLU activation into the down projection
+#   lm_in    final-norm hidden state into the LM head
+ROUNDING_SOURCES = ("proj_in", "qkv", "p", "att", "act", "lm_in")
 
 
 def block_ranges(gen_len: int, block_len: int) -> List[Tuple[int, int]]:
@@ -249,11 +261,18 @@ class Oracle:
     ``__getitem__`` (so that large models can materialise one tensor at a time).
     """
 
-    def __init__(self, cfg: ModelConfig, weights, operand_rounding: Optional[str] = None):
-        assert operand_rounding in (None, "bf16")
+    def __init__(self, cfg: ModelConfig, weights, operand_rounding=None):
+        if operand_rounding is None:
+            active = ()
+        elif operand_rounding == "bf16":
+            active = ROUNDING_SOURCES
+        else:
+            active = tuple(operand_rounding)
+            assert all(src in ROUNDING_SOURCES for src in active), active
         self.cfg = cfg
         self.w = weights
-        self.rnd = bf16_round if operand_rounding == "bf16" else (lambda a: a)
+        ident = lambda a: a
+        self.r = {src: (bf16_round if src in active else ident) for src in ROUNDING_SOURCES}
 
     def _W(self, name: str) -> np.ndarray:
         return np.asarray(self.w[name], dtype=np.float64)
@@ -264,7 +283,7 @@ class Oracle:
         """Apply layer l to every group (a group = the rows of one node, [T, d]).  Each group
         attends to [prefix ; its own rows].  Returns (new hidden, post-RoPE K, V) per group."""
         c = self.cfg
-        rnd = self.rnd
+        r = self.r
         p = f"layers.{l}."
         wq, wk, wv, wo = self._W(p + "wq"), self._W(p + "wk"), self._W(p + "wv"), self._W(p + "wo")
         wg, wu, wd = self._W(p + "w_gate"), self._W(p + "w_up"), self._W(p + "w_down")
@@ -272,17 +291,17 @@ class Oracle:
         outs, ks, vs = [], [], []
         for h, pos in zip(groups, positions):
             T = h.shape[0]
-            u = rnd(rmsnorm(h, g1, c.rms_eps))
+            u = r["proj_in"](rmsnorm(h, g1, c.rms_eps))
             q = rope((u @ wq.T).reshape(T, c.n_heads, c.head_dim), pos, c.rope_theta)
             k = rope((u @ wk.T).reshape(T, c.n_kv_heads, c.head_dim), pos, c.rope_theta)
             v = (u @ wv.T).reshape(T, c.n_kv_heads, c.head_dim)
-            q, k, v = rnd(q), rnd(k), rnd(v)
+            q, k, v = r["qkv"](q), r["qkv"](k), r["qkv"](v)
             keys = np.concatenate([prefix_k, k], axis=0)
             vals = np.concatenate([prefix_v, v], axis=0)
-            att = rnd(attention(q, keys, vals, rnd))
+            att = r["att"](attention(q, keys, vals, r["p"]))
             h = h + att @ wo.T
-            u = rnd(rmsnorm(h, g2, c.rms_eps))
-            act = rnd(silu(u @ wg.T) * (u @ wu.T))
+            u = r["proj_in"](rmsnorm(h, g2, c.rms_eps))
+            act = r["act"](silu(u @ wg.T) * (u @ wu.T))
             h = h + act @ wd.T
             outs.append(h)
             ks.append(k)
@@ -290,10 +309,12 @@ class Oracle:
         return outs, ks, vs
 
     def forward_rows(self, ids: np.ndarray, pos0: int, cache: Cache, want_logits: bool = True,
-                     logit_rows: Optional[np.ndarray] = None):
+                     logit_rows: Optional[np.ndarray] = None, hidden_trace: Optional[list] = None):
         """f_theta on one or several nodes.  ids [n, T] (or [T]); all nodes sit at absolute
         positions pos0 .. pos0+T-1 and each attends to the cache plus its own T rows.
-        Returns (logits [n, T, V] or None, K list per layer [n,T,Hkv,hd], V list)."""
+        Returns (logits [n, T, V] or None, K list per layer [n,T,Hkv,hd], V list).
+        ``hidden_trace`` (a list) receives the residual stream [n, T, d] entering layer 0,
+        1, ... and, last, the one leaving the final layer (for layer-by-layer comparisons)."""
         c = self.cfg
         ids = np.atleast_2d(np.asarray(ids))
         n, T = ids.shape
@@ -302,13 +323,17 @@ class Oracle:
         pos = [np.arange(pos0, pos0 + T) for _ in range(n)]
         all_k, all_v = [], []
         for l in range(c.n_layers):
+            if hidden_trace is not None:
+                hidden_trace.append(np.stack(groups))
             groups, ks, vs = self.layer(l, groups, pos, cache.k[l], cache.v[l])
             all_k.append(np.stack(ks))
             all_v.append(np.stack(vs))
+        if hidden_trace is not None:
+            hidden_trace.append(np.stack(groups))
         logits = None
         if want_logits:
             gf, wlm = self._W("norm_final"), self._W("lm_head")
-            logits = np.stack([self.rnd(rmsnorm(h, gf, c.rms_eps)) @ wlm.T for h in groups])
+            logits = np.stack([self.r["lm_in"](rmsnorm(h, gf, c.rms_eps)) @ wlm.T for h in groups])
         return logits, all_k, all_v
 
     # ---- cache maintenance ----------------------------------------------------------
@@ -416,11 +441,14 @@ class Oracle:
         return np.concatenate(out), all_counts, cache
 
     # ---- the uncached definition used to pin the cache semantics --------------------
-    def uncached_block_causal(self, tokens: np.ndarray, segment_lengths: Sequence[int]):
+    def uncached_block_causal(self, tokens: np.ndarray, segment_lengths: Sequence[int],
+                              hidden_trace: Optional[list] = None):
         """Forward over the whole sequence with NO cache: position t attends to every
         position of its own segment and of all earlier segments (prompt = first segment).
         Returns (logits [T,V], K list [T,Hkv,hd], V list).  Written as a plain masked
-        attention over the full sequence, independently of ``layer``'s cache handling."""
+        attention over the full sequence, independently of ``layer``'s cache handling.
+        ``hidden_trace`` receives the residual stream [T, d] entering each layer, then the
+        final one."""
         c = self.cfg
         T = len(tokens)
         seg = np.repeat(np.arange(len(segment_lengths)), segment_lengths)
@@ -428,25 +456,29 @@ class Oracle:
         allow = seg[None, :] <= seg[:, None]            # [query, key]
         pos = np.arange(T)
         h = self._W("embed")[np.asarray(tokens)].copy()
-        rnd = self.rnd
+        r = self.r
         Ks, Vs = [], []
         for l in range(c.n_layers):
+            if hidden_trace is not None:
+                hidden_trace.append(h.copy())
             p = f"layers.{l}."
-            u = rnd(rmsnorm(h, self._W(p + "norm_attn"), c.rms_eps))
-            q = rnd(rope((u @ self._W(p + "wq").T).reshape(T, c.n_heads, c.head_dim), pos, c.rope_theta))
-            k = rnd(rope((u @ self._W(p + "wk").T).reshape(T, c.n_kv_heads, c.head_dim), pos, c.rope_theta))
-            v = rnd((u @ self._W(p + "wv").T).reshape(T, c.n_kv_heads, c.head_dim))
+            u = r["proj_in"](rmsnorm(h, self._W(p + "norm_attn"), c.rms_eps))
+            q = r["qkv"](rope((u @ self._W(p + "wq").T).reshape(T, c.n_heads, c.head_dim), pos, c.rope_theta))
+            k = r["qkv"](rope((u @ self._W(p + "wk").T).reshape(T, c.n_kv_heads, c.head_dim), pos, c.rope_theta))
+            v = r["qkv"]((u @ self._W(p + "wv").T).reshape(T, c.n_kv_heads, c.head_dim))
             group = c.n_heads // c.n_kv_heads
             att = np.empty((T, c.n_heads, c.head_dim))
             for hh in range(c.n_heads):
                 s = (q[:, hh, :] @ k[:, hh // group, :].T) / np.sqrt(float(c.head_dim))
                 s = np.where(allow, s, -np.inf)
                 pr = np.exp(s - s.max(axis=-1, keepdims=True))
-                att[:, hh, :] = (rnd(pr) @ v[:, hh // group, :]) / pr.sum(axis=-1, keepdims=True)
-            h = h + rnd(att.reshape(T, -1)) @ self._W(p + "wo").T
-            u = rnd(rmsnorm(h, self._W(p + "norm_ffn"), c.rms_eps))
-            h = h + rnd(silu(u @ self._W(p + "w_gate").T) * (u @ self._W(p + "w_up").T)) @ self._W(p + "w_down").T
+                att[:, hh, :] = (r["p"](pr) @ v[:, hh // group, :]) / pr.sum(axis=-1, keepdims=True)
+            h = h + r["att"](att.reshape(T, -1)) @ self._W(p + "wo").T
+            u = r["proj_in"](rmsnorm(h, self._W(p + "norm_ffn"), c.rms_eps))
+            h = h + r["act"](silu(u @ self._W(p + "w_gate").T) * (u @ self._W(p + "w_up").T)) @ self._W(p + "w_down").T
             Ks.append(k)
             Vs.append(v)
-        logits = rnd(rmsnorm(h, self._W("norm_final"), c.rms_eps)) @ self._W("lm_head").T
+        if hidden_trace is not None:
+            hidden_trace.append(h.copy())
+        logits = r["lm_in"](rmsnorm(h, self._W("norm_final"), c.rms_eps)) @ self._W("lm_head").T
         return logits, Ks, Vs

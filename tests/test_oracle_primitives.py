@@ -204,3 +204,48 @@ def test_operand_rounding_is_small_and_nonzero():
     lb, _, _ = b.forward_rows(np.full(w.block_len, w.mask_id), len(prompt), b.prefill(prompt))
     d = np.abs(la - lb).max()
     assert 0 < d < 2e-2
+
+
+def test_rounding_sources_partition_the_bf16_mode():
+    """Selective operand rounding only switches existing rounding points on and off: every source on is
+    the "bf16" mode bit for bit, none on is the unrounded mode bit for bit, and a single source moves the
+    logits by less than all of them together."""
+    w = SMALL_GQA
+    cfg, wts = oracle_config(w), oracle_weights(w, as_bf16=True)
+    prompt = wl.make_prompts(w).numpy()[0]
+    ids = np.array([[w.mask_id, 3, w.mask_id, 7, 9, w.mask_id]])
+
+    def logits_of(mode):
+        o = so.Oracle(cfg, wts, mode)
+        return o.forward_rows(ids, len(prompt), o.prefill(prompt))[0]
+
+    plain, full = logits_of(None), logits_of("bf16")
+    assert np.array_equal(logits_of(()), plain)
+    assert np.array_equal(logits_of(so.ROUNDING_SOURCES), full)
+    total = np.abs(full - plain).max()
+    assert total > 0
+    for src in so.ROUNDING_SOURCES:
+        one = np.abs(logits_of((src,)) - plain).max()
+        assert 0 < one < 2 * total
+    with pytest.raises(AssertionError):
+        so.Oracle(cfg, wts, ("nonsense",))
+
+
+def test_hidden_trace_is_the_residual_stream():
+    """The recorded residual stream has one entry per layer boundary, starts at the embedding rows, ends
+    at what the LM head normalises, and is the same through the cached and the uncached forward."""
+    w = SMALL
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w).numpy()[0]
+    ids = np.array([5, w.mask_id, 8, w.mask_id, w.mask_id, 2])
+    tr = []
+    logits, _, _ = o.forward_rows(ids[None], len(prompt), o.prefill(prompt), hidden_trace=tr)
+    assert len(tr) == w.n_layers + 1 and tr[0].shape == (1, len(ids), w.d_model)
+    assert np.array_equal(tr[0][0], o._W("embed")[ids])
+    assert np.allclose(so.rmsnorm(tr[-1][0], o._W("norm_final"), w.rms_eps) @ o._W("lm_head").T, logits[0],
+                       rtol=1e-12, atol=1e-14)
+    tr2 = []
+    o.uncached_block_causal(np.concatenate([prompt, ids]), [len(prompt), len(ids)], hidden_trace=tr2)
+    assert len(tr2) == w.n_layers + 1
+    for a, b in zip(tr, tr2):
+        assert np.allclose(a[0], b[len(prompt):], rtol=1e-9, atol=1e-12)
