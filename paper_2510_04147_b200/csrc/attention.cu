@@ -246,10 +246,11 @@ void launch_attention(cudaStream_t st, const AttnArgs& a, int* launches) {
   dim3 grid(q_tiles, a.H, a.n_seq_slots * n_parts);
   if (a.hd == 128) {
     const int smem = (kQTile + 4 * kKTile) * 128 * 2;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices] = {};      // the shared-memory opt-in is per device
+    const int dev = device_slot();
+    if (dev >= 0 && !attr_set[dev]) {
       cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-      attr_set = true;
+      attr_set[dev] = true;
     }
     launch_pdl(attn_split_kernel<128>, grid, dim3(kAttnThreads), (size_t)smem, st, a, n_prefix, has_local, scale_log2);
   } else {

@@ -500,8 +500,10 @@ int launch_attention_verify(cudaStream_t st, const AttnArgs& a) {
   // two CTAs per SM by default; three (register-capped build) when only that keeps the grid in one wave
   const long long n_ctas = (long long)a.n_seq_slots * q_tiles * n_parts * a.H;
   const bool dense = qt_rows == 32 && n_ctas > 2 * 148;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[kMaxDevices] = {};        // the shared-memory opt-in is per device
+  const int dev = device_slot();
+  if (dev < 0) return -4;
+  if (!attr_set[dev]) {
     const int max_smem = (64 + 2 * 2 * kPairKeys) * 128 * 2;
     if (cudaFuncSetAttribute(attn_verify_kernel<128, 32, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
         cudaFuncSetAttribute(attn_verify_kernel<128, 32, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
@@ -510,7 +512,7 @@ int launch_attention_verify(cudaStream_t st, const AttnArgs& a) {
         cudaFuncSetAttribute(attn_verify_kernel<64, 32, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess ||
         cudaFuncSetAttribute(attn_verify_kernel<64, 64, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem / 2) != cudaSuccess)
       return -4;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   dim3 grid(n_parts, a.H, a.n_seq_slots * q_tiles);
   dim3 block(qt_rows * 4);

@@ -151,8 +151,7 @@ __device__ __forceinline__ uint32_t tile_off(int row, int ch, int rows) {
 }
 
 template <int QT>
-__global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnArgs a, int n_prefix_parts, float scale_log2,
-                                                                          int v_desc_swap) {
+__global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnArgs a, int n_prefix_parts, float scale_log2) {
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;                                   // [2][128][64] bf16
@@ -502,8 +501,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       for (int k = 0; k < 8; ++k) {
         const uint32_t pa = smem_u32(sK) + (uint32_t)((k >> 2) * kHalfBytesKV + (k & 3) * 32);
         const uint32_t va = smem_u32(sV) + (uint32_t)(2 * k * 1024);
-        const uint64_t vdesc = v_desc_swap ? make_desc(va, 1024, kHalfBytesKV) : make_desc(va, kHalfBytesKV, 1024);
-        tc_mma_bf16(tmem_O, make_desc(pa, 16, 1024), vdesc, idesc_pv, (uint32_t)((t | k) != 0));
+        tc_mma_bf16(tmem_O, make_desc(pa, 16, 1024), make_desc(va, kHalfBytesKV, 1024), idesc_pv, (uint32_t)((t | k) != 0));
       }
       tc_commit(smem_u32(&bars[1]));
     }
@@ -589,7 +587,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
 
 }  // namespace
 
-int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a, int v_desc_swap) {
+int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a) {
   if (a.hd != kHD || !a.qkv_partial || !a.rope || !a.err_flag) return 1;
   if (a.kv_split < kKeys || (a.kv_split % kKeys) != 0) return 1;
   if ((a.cache_k_out != nullptr) != (a.cache_v_out != nullptr)) return -1;
@@ -607,24 +605,26 @@ int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a, int v_desc_sw
   const float scale_log2 = (1.0f / sqrtf((float)a.hd)) * 1.4426950408889634f;
   // 101 KB: never more than two CTAs per SM, so that two 256-column TMEM allocations always fit
   const size_t smem = 6 * (size_t)kHalfBytesKV + 4096 + 64 + 1024;   // Q, K/P, V tiles of 128 rows + the softmax exchange
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[kMaxDevices] = {};        // the shared-memory opt-in is per device
+  const int dev = device_slot();
+  if (dev < 0) return -4;
+  if (!attr_set[dev]) {
     const int max_smem = 6 * kHalfBytesKV + 4096 + 64 + 1024;
     if (cudaFuncSetAttribute(attn_verify_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
         cudaFuncSetAttribute(attn_verify_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
         cudaFuncSetAttribute(attn_verify_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
       return -4;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   dim3 grid(n_parts, a.H, a.n_seq_slots * q_tiles);
   dim3 block(kTcAttnThreads);
   cudaError_t e;
   if (qt_rows == 32)
-    e = launch_pdl_cluster(attn_verify_tc_kernel<32>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, scale_log2, v_desc_swap);
+    e = launch_pdl_cluster(attn_verify_tc_kernel<32>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, scale_log2);
   else if (qt_rows == 64)
-    e = launch_pdl_cluster(attn_verify_tc_kernel<64>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, scale_log2, v_desc_swap);
+    e = launch_pdl_cluster(attn_verify_tc_kernel<64>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, scale_log2);
   else
-    e = launch_pdl_cluster(attn_verify_tc_kernel<128>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, scale_log2, v_desc_swap);
+    e = launch_pdl_cluster(attn_verify_tc_kernel<128>, grid, block, smem, st, (unsigned)n_parts, a, n_prefix, scale_log2);
   return e == cudaSuccess ? 0 : -4;
 }
 

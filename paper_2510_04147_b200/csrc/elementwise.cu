@@ -1,5 +1,5 @@
-// Small memory-bound kernels around the projections: embedding gather, RMSNorm + residual with
-// split-K reduction, QKV finalisation with rotary embedding, SwiGLU, softmax statistics.
+// Small memory-bound kernels around the projections: weight repacking, embedding gather, QKV
+// finalisation with rotary embedding (cache-fill forward), softmax statistics.
 // Every reduction has a fixed order that depends on the row alone, so a row's result does not
 // depend on how many other rows share the launch.
 #include "kernels.h"
@@ -53,40 +53,7 @@ __global__ void copy_f32_kernel(const void* src, int src_is_f32, float* dst, int
   if (i < n) dst[i] = src_is_f32 ? ((const float*)src)[i] : __bfloat162float(((const bf16*)src)[i]);
 }
 
-__device__ __forceinline__ void write_norm_row(const float* hrow, const float* gain, float inv, bf16* xrow, int d) {
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-    const float4 v = *reinterpret_cast<const float4*>(hrow + c);
-    const float4 g = *reinterpret_cast<const float4*>(gain + c);
-    __nv_bfloat162 a = __floats2bfloat162_rn(v.x * inv * g.x, v.y * inv * g.y);
-    __nv_bfloat162 b = __floats2bfloat162_rn(v.z * inv * g.z, v.w * inv * g.w);
-    *reinterpret_cast<__nv_bfloat162*>(xrow + c) = a;
-    *reinterpret_cast<__nv_bfloat162*>(xrow + c + 2) = b;
-  }
-}
-
 constexpr int kRowThreadsMax = 1024;   // one float4 per thread up to d = 4096
-
-__global__ void __launch_bounds__(kRowThreadsMax) embed_rmsnorm_kernel(const int* ids, const bf16* embed,
-                                                                       const float* gain, float eps, float* h, bf16* xn,
-                                                                       int d) {
-  __shared__ float red[kRowThreadsMax / 32];
-  pdl_launch_dependents();
-  pdl_wait();
-  const int r = blockIdx.x;
-  const bf16* e = embed + (size_t)ids[r] * d;
-  float* hrow = h + (size_t)r * d;
-  float ss = 0.f;
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-    const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(e + c);
-    const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(e + c + 2);
-    float4 v = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
-    *reinterpret_cast<float4*>(hrow + c) = v;
-    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-  }
-  ss = block_sum(ss, red);
-  const float inv = rsqrtf(ss / (float)d + eps);
-  write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
-}
 
 __global__ void __launch_bounds__(kRowThreadsMax) embed_prep_kernel(const int* ids, const bf16* embed, const float* gain,
                                                                     float* h, bf16* hb, float* sq, int sq_stride, int d) {
@@ -108,54 +75,6 @@ __global__ void __launch_bounds__(kRowThreadsMax) embed_prep_kernel(const int* i
   }
   ss = block_sum(ss, red);
   if (threadIdx.x == 0) sq[(size_t)r * sq_stride] = ss;
-}
-
-// One CTA per row.  A thread owns float4 column groups; for each it issues the loads of h and of
-// up to eight splits before the first add, then adds in split order, so a row's sum does not depend
-// on the launch shape and the latency of the (L2-resident) partials is paid once, not per split.
-__global__ void __launch_bounds__(kRowThreadsMax) residual_rmsnorm_kernel(const float* partial, int splits,
-                                                                          size_t split_stride, const float* gain,
-                                                                          float eps, float* h, bf16* xn, int d) {
-  __shared__ float red[kRowThreadsMax / 32];
-  pdl_launch_dependents();
-  pdl_wait();
-  const int r = blockIdx.x;
-  float* hrow = h + (size_t)r * d;
-  float ss = 0.f;
-  float4 keep = make_float4(0.f, 0.f, 0.f, 0.f);       // the thread's values when one pass covers the row
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-    float4 v = *reinterpret_cast<const float4*>(hrow + c);
-    const float* pp = partial + (size_t)r * d + c;
-    for (int s0 = 0; s0 < splits; s0 += 8) {
-      float4 p[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        p[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (s0 + u < splits) p[u] = *reinterpret_cast<const float4*>(pp + (size_t)(s0 + u) * split_stride);
-      }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        if (s0 + u < splits) { v.x += p[u].x; v.y += p[u].y; v.z += p[u].z; v.w += p[u].w; }
-      }
-    }
-    *reinterpret_cast<float4*>(hrow + c) = v;
-    keep = v;
-    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-  }
-  if (gain == nullptr) return;
-  const int c = threadIdx.x * 4;
-  float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-  const bool one_pass = d <= (int)blockDim.x * 4;
-  if (one_pass && c < d) g = *reinterpret_cast<const float4*>(gain + c);   // in flight during the reduction
-  ss = block_sum(ss, red);
-  const float inv = rsqrtf(ss / (float)d + eps);
-  if (!one_pass) {
-    write_norm_row(hrow, gain, inv, xn + (size_t)r * d, d);
-  } else if (c < d) {
-    bf16* xrow = xn + (size_t)r * d;
-    *reinterpret_cast<__nv_bfloat162*>(xrow + c) = __floats2bfloat162_rn(keep.x * inv * g.x, keep.y * inv * g.y);
-    *reinterpret_cast<__nv_bfloat162*>(xrow + c + 2) = __floats2bfloat162_rn(keep.z * inv * g.z, keep.w * inv * g.w);
-  }
 }
 
 // One CTA per (row, group of 8 heads of the fused q|k|v output); a warp per head.
@@ -199,16 +118,6 @@ __global__ void __launch_bounds__(kRopeHeadsPerBlock * 32) qkv_rope_kernel(const
       for (int s = 0; s < splits; ++s) x += prow[s * split_stride + e];
       dst[e] = __float2bfloat16_rn(x);
     }
-  }
-}
-
-__global__ void swiglu_kernel(const float* gu, bf16* act, int R, int ffn_pad) {
-  const size_t total = (size_t)R * ffn_pad;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-    const int r = (int)(i / ffn_pad), f = (int)(i % ffn_pad);
-    const float* row = gu + (size_t)r * 2 * ffn_pad + (size_t)(f >> 6) * 128 + (f & 63);
-    const float g = row[0], u = row[64];
-    act[i] = __float2bfloat16_rn(g / (1.f + expf(-g)) * u);
   }
 }
 
@@ -336,20 +245,9 @@ static int row_threads(int d) {
   return t;
 }
 
-void launch_embed_rmsnorm(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float eps, float* h,
-                          bf16* xn, int R, int d) {
-  launch_pdl(embed_rmsnorm_kernel, dim3(R), dim3(row_threads(d)), 0, st, ids, embed, gain, eps, h, xn, d);
-}
-
 void launch_embed_prep(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float* h, bf16* hb,
                        float* sq, int sq_stride, int R, int d) {
   launch_pdl(embed_prep_kernel, dim3(R), dim3(row_threads(d)), 0, st, ids, embed, gain, h, hb, sq, sq_stride, d);
-}
-
-void launch_residual_rmsnorm(cudaStream_t st, const float* partial, int splits, size_t split_stride, const float* gain,
-                             float eps, float* h, bf16* xn, int R, int d) {
-  launch_pdl(residual_rmsnorm_kernel, dim3(R), dim3(row_threads(d)), 0, st, partial, splits, split_stride, gain, eps, h,
-             xn, d);
 }
 
 void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H, int Hkv,
@@ -359,13 +257,6 @@ void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t s
   dim3 grid(R, (heads + kRopeHeadsPerBlock - 1) / kRopeHeadsPerBlock);
   launch_pdl(qkv_rope_kernel, grid, dim3(kRopeHeadsPerBlock * 32), 0, st, partial, splits, split_stride, H, Hkv, hd,
              rope_table, map, q, k_dst, v_dst, kv_to_cache, cache_seq_stride);
-}
-
-void launch_swiglu(cudaStream_t st, const float* gu, bf16* act, int R, int ffn_pad) {
-  const size_t total = (size_t)R * ffn_pad;
-  int blocks = (int)((total + 255) / 256);
-  if (blocks > 148 * 8) blocks = 148 * 8;
-  swiglu_kernel<<<blocks, 256, 0, st>>>(gu, act, R, ffn_pad);
 }
 
 void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, int V, int mask_id,

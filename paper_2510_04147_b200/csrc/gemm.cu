@@ -14,8 +14,6 @@
 //   EPI_LMHEAD   per-row max / argmax / sum-exp over the tile's 128 vocabulary entries, so the
 //                logits never leave the SM.
 // Every wait is bounded: on expiry the kernel raises an error word and unwinds.
-//
-// A plain CUDA-core kernel of the same contract is kept for bring-up and as a cross-check.
 #include "kernels.h"
 
 #include <cuda.h>
@@ -25,63 +23,6 @@
 namespace ssd {
 
 int gemm_tiles(int N) { return (N + 127) / 128; }
-
-// =====================================================================================
-// CUDA-core kernel (bring-up / cross-check)
-// =====================================================================================
-namespace {
-
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16* __restrict__ x, const bf16* __restrict__ w,
-                                                        float* __restrict__ out, int R, int N, int K, int x_pitch,
-                                                        int w_pitch, int splits, int w_tiled) {
-  __shared__ float Ws[64][33];
-  __shared__ float Xs[32][33];
-  const int n0 = blockIdx.x * 64, r0 = blockIdx.y * 32, split = blockIdx.z;
-  const int kb_total = (K + 63) / 64;
-  const int k_begin = (int)((long long)split * kb_total / splits) * 64;
-  const int k_end = min(K, (int)((long long)(split + 1) * kb_total / splits) * 64);
-  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-  float acc[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-  for (int k0 = k_begin; k0 < k_end; k0 += 32) {
-    for (int i = threadIdx.x; i < 64 * 32; i += 256) {
-      const int rr = i >> 5, kk = i & 31;
-      const int n = n0 + rr, k = k0 + kk;
-      const size_t wi = w_tiled ? ((((size_t)(n >> 7) * kb_total + (k >> 6)) * 128 + (n & 127)) * 64 + (k & 63))
-                                : ((size_t)n * w_pitch + k);
-      Ws[rr][kk] = (n < N && k < k_end) ? __bfloat162float(w[wi]) : 0.f;
-    }
-    for (int i = threadIdx.x; i < 32 * 32; i += 256) {
-      const int rr = i >> 5, kk = i & 31;
-      const int r = r0 + rr, k = k0 + kk;
-      Xs[rr][kk] = (r < R && k < k_end) ? __bfloat162float(x[(size_t)r * x_pitch + k]) : 0.f;
-    }
-    __syncthreads();
-#pragma unroll 8
-    for (int kk = 0; kk < 32; ++kk) {
-      const float wv = Ws[tx][kk];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] += wv * Xs[ty * 8 + i][kk];
-    }
-    __syncthreads();
-  }
-  const int n = n0 + tx;
-  if (n < N) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int r = r0 + ty * 8 + i;
-      if (r < R) out[((size_t)split * R + r) * N + n] = acc[i];
-    }
-  }
-}
-
-}  // namespace
-
-void launch_gemm_simt(cudaStream_t st, const GemmArgs& g) {
-  dim3 grid((g.N + 63) / 64, (g.R + 31) / 32, g.splits);
-  gemm_simt_kernel<<<grid, 256, 0, st>>>(g.x, g.w, g.out, g.R, g.N, g.K, g.x_pitch, g.w_pitch, g.splits, g.w_tiled);
-}
 
 // =====================================================================================
 // Tensor-core kernel
@@ -596,7 +537,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       if (epi_warp && epi_ok) {
         for (int c0 = 0; c0 < pass_cnt; c0 += 32) {
           float v[32];
-          tmem_ld32(taddr + g0 + c0, v);
+          if (n_kb > 0) tmem_ld32(taddr + g0 + c0, v);       // a split without K blocks issued no MMA: it adds zeros
+          else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+          }
 #pragma unroll
           for (int j = 0; j < 32; ++j) scratch[(c0 + j) * kEpiPitch + lrow] = v[j];
         }
@@ -710,6 +655,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   if (!g_encode) return -4;
   if ((g.x_pitch % 8) || (!g.w_tiled && (g.w_pitch % 8)) || (((uintptr_t)g.x) & 15) || (((uintptr_t)g.w) & 15)) return -2;
   if (g.R < 1 || g.N < 1 || g.K < 1) return -2;
+  if (g.splits < 1 || g.splits > (g.K + kBlockK - 1) / kBlockK) return -2;   // every split owns at least one K block
   if (g.epi != EPI_PARTIAL && g.epi != EPI_RESIDUAL && g.splits != 1) return -2;
   if (g.epi == EPI_RESIDUAL &&
       (g.splits < 1 || g.splits > kGemmMaxClusterSplits || (g.N & 3) || !g.h || !g.hb || !g.gain || !g.sq_out)) return -2;
@@ -752,12 +698,15 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
     return -4;
   }
   if (!make_tmap(&tmX, g.x, (uint64_t)g.R, (uint64_t)g.K, (uint64_t)g.x_pitch, (uint32_t)(p.two_sm ? p.npad / 2 : p.npad))) return -4;
-  static int smem_set = 0;
-  if (smem > smem_set) {
+  // the opt-in to more than 48 KB of dynamic shared memory is a per-device attribute of the function
+  static bool smem_set[kMaxDevices] = {};
+  const int dev = device_slot();
+  if (dev < 0) return -4;
+  if (!smem_set[dev]) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return -4;
-    smem_set = 227 * 1024;
+    smem_set[dev] = true;
   }
   dim3 grid(gemm_tiles(g.N), g.splits, (g.R + 255) / 256);
   const unsigned cluster_y = (g.epi == EPI_RESIDUAL) ? (unsigned)g.splits : 1u;

@@ -56,6 +56,16 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 }
 #endif
 
+// ---------------------------------------------------------------- per-device set-up
+// Function attributes (the opt-in to large dynamic shared memory) belong to a device, not to the
+// process: launchers keep one flag per device ordinal and set the attribute on a device's first use.
+constexpr int kMaxDevices = 64;
+inline int device_slot() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
 // ---------------------------------------------------------------- layout helpers (host+device)
 // Rows of a forward are ordered [sequence slot a][node i][in-block index t].
 struct RowMap {
@@ -90,23 +100,15 @@ inline size_t tiled_elems(int n, int k) { return (size_t)((n + 127) / 128) * ((k
 void launch_copy_f32(cudaStream_t st, const void* src, int src_is_f32, float* dst, int n);
 
 // ---------------------------------------------------------------- elementwise / reductions
-// h[r] = embed[ids[r]]; xn[r] = bf16(rmsnorm(h[r]) * gain)
-void launch_embed_rmsnorm(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float eps,
-                          float* h, bf16* xn, int R, int d);
 // producer side of the fused RMSNorm: h[r] = embed[ids[r]]; hb[r] = bf16(h[r] * gain);
 // sq[r * sq_stride] = sum of squares of h[r]
 void launch_embed_prep(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float* h, bf16* hb,
                        float* sq, int sq_stride, int R, int d);
-// h[r] += sum_s partial[s][r] (s ascending); if gain: xn[r] = bf16(rmsnorm(h[r]) * gain)
-void launch_residual_rmsnorm(cudaStream_t st, const float* partial, int splits, size_t split_stride,
-                             const float* gain, float eps, float* h, bf16* xn, int R, int d);
 // sums the split-K partials of the fused QKV projection, rotates q and k, writes bf16.
 // kv_to_cache: k/v rows go to cache[(seq*max_seq + pos)*Hkv*hd] else to local [r][Hkv][hd].
 void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H,
                      int Hkv, int hd, const float2* rope_table, RowMap map, bf16* q, bf16* k_dst, bf16* v_dst,
                      int kv_to_cache, size_t cache_seq_stride);
-// act[r][f] = bf16(silu(g) * u) from fp32 gate/up laid out in 64-row interleaved groups of 128
-void launch_swiglu(cudaStream_t st, const float* gu, bf16* act, int R, int ffn_pad);
 // per row: argmax / max-softmax-probability over the vocabulary with mask_id excluded
 void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, int V, int mask_id,
                                  const uint8_t* row_wanted, int* tok, float* conf);
@@ -149,9 +151,8 @@ void launch_attention(cudaStream_t st, const AttnArgs& a, int* launches);
 int launch_attention_verify(cudaStream_t st, const AttnArgs& a);
 // The same on the tcgen05 tensor cores, for head dimension 128, kv_split 128 (<= 7 prefix parts) and
 // node-local keys that fit one 128-key tile; needs a.err_flag.  Returns 0 (launched), 1 (shape not
-// covered: use launch_attention_verify) or a negative ssd error code.  v_desc_swap: test hook that
-// swaps the two stride fields of the V operand descriptor.
-int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a, int v_desc_swap);
+// covered: use launch_attention_verify) or a negative ssd error code.
+int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a);
 constexpr int kAttnMaxClusterParts = 8;
 
 // ---------------------------------------------------------------- projections
@@ -191,7 +192,6 @@ struct GemmArgs {
   int sq_out_stride;
 };
 int gemm_tiles(int N);
-void launch_gemm_simt(cudaStream_t st, const GemmArgs& g);
 // tensor-core path (TMA + tcgen05). Returns 0 or a negative ssd error code.
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& g);
 int gemm_tc_init();   // resolves the driver entry point for tensor-map encoding

@@ -73,10 +73,11 @@ struct ssd_ctx {
   // first forward (or run on its own when something else needs the cache first).
   int pending_T = 0;
   int* pending_ids = nullptr;    // [max_batch][block_len] tokens of that block
+  int* prompt_stage = nullptr;   // [max_batch][max_seq] device copy of a host prompt (ssd_prefill)
   int fuse_commit = 1;
   std::vector<int> h_remaining, h_has_drafts, h_nodes;
 
-  int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0, gemm_impl = 1;
+  int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0;
   int two_sm_rows = 256;                   // projections pair their tiles (two-SM MMA) from this many rows on; 0 = never
   int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
   int64_t launches = 0;
@@ -223,13 +224,8 @@ int run_gemm(ssd_ctx* c, GemmArgs g, int fam, int sub = -1) {
   Scope sc(c, fam, (double)g.N * g.K * 2.0, 1, sub);
   g.err_flag = c->flags;
   g.two_sm_min_rows = c->two_sm_rows;
-  if (c->gemm_impl == 1) {
-    const int rc = launch_gemm_tc(c->st, g);
-    if (rc != 0) return fail(c, rc, "tensor-core GEMM rejected R=%d N=%d K=%d epi=%d (code %d)", g.R, g.N, g.K, g.epi, rc);
-  } else {
-    if (g.epi != EPI_PARTIAL) return fail(c, SSD_ERR_INVALID_ARG, "bring-up GEMM has no fused epilogue");
-    launch_gemm_simt(c->st, g);
-  }
+  const int rc = launch_gemm_tc(c->st, g);
+  if (rc != 0) return fail(c, rc, "projection kernel rejected R=%d N=%d K=%d epi=%d splits=%d (code %d)", g.R, g.N, g.K, g.epi, g.splits, rc);
   return SSD_OK;
 }
 
@@ -253,7 +249,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   // A block commit is a one-node verification forward whose K/V also go to the cache: it takes the
   // verification attention kernel.  Only the prefill (many rows, empty cache) fills through the
   // rotary pass and the cache-reading attention.
-  const bool commit_form = kind == FWD_FILL && c->gemm_impl == 1 && S > 0 && map.rows_per_seq == map.T &&
+  const bool commit_form = kind == FWD_FILL && S > 0 && map.rows_per_seq == map.T &&
                            map.T <= c->cfg.block_len;
   const bool via_cache = kind == FWD_FILL && !commit_form;
   const int attn_S = via_cache ? S + map.T : S;
@@ -262,14 +258,11 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   if (via_cache && (size_t)n_parts * R > c->part_rows_parts)
     return fail(c, SSD_ERR_OVERFLOW, "attention workspace too small for %d parts x %d rows", n_parts, R);
   const int nl = c->cfg.n_layers;
-  // With the tensor-core projections the RMSNorms have no kernel of their own: a producer (the
-  // embedding gather, the O and down projections) writes the residual stream h, bf16(h * gain) in
-  // `xn` and per-tile sums of squares in `sq`; the consuming projection scales its output rows by
-  // 1/rms.  The bring-up projections keep the separate norm kernels.
-  const bool fused = c->gemm_impl == 1;
+  // The RMSNorms have no kernel of their own: a producer (the embedding gather, the O and down
+  // projections) writes the residual stream h, bf16(h * gain) in `xn` and per-tile sums of squares in
+  // `sq`; the consuming projection scales its output rows by 1/rms.
   int sq_count = 1;                       // slots of `sq` the next consumer sums per row
   auto consume_norm = [&](GemmArgs& ga) {
-    if (!fused) return;
     ga.sq = c->sq; ga.sq_count = sq_count; ga.sq_stride = c->sq_stride; ga.norm_dim = d; ga.norm_eps = c->cfg.rms_eps;
   };
   auto produce_norm = [&](GemmArgs& ga, const float* gain, int splits) {
@@ -278,8 +271,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   };
   {
     Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * 8);
-    if (fused) launch_embed_prep(c->st, ids_dev, c->embed, c->L[0].g_attn, c->h, c->xn, c->sq, c->sq_stride, R, d);
-    else launch_embed_rmsnorm(c->st, ids_dev, c->embed, c->L[0].g_attn, c->cfg.rms_eps, c->h, c->xn, R, d);
+    launch_embed_prep(c->st, ids_dev, c->embed, c->L[0].g_attn, c->h, c->xn, c->sq, c->sq_stride, R, d);
   }
   for (int l = 0; l < nl; ++l) {
     const LayerW& w = c->L[l];
@@ -320,7 +312,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
       Scope sc(c, SSD_PROF_ATTN, kvb, 1);
       a.err_flag = c->flags;
       int arc = 1;
-      if (c->attn_impl == 1) arc = launch_attention_verify_tc(c->st, a, 0);   // 1: shape not covered by the tcgen05 form
+      if (c->attn_impl == 1) arc = launch_attention_verify_tc(c->st, a);   // 1: shape not covered by the tcgen05 form
       if (arc == 1) arc = launch_attention_verify(c->st, a);
       if (arc != 0) return fail(c, arc, "verification attention rejected S=%d kv_split=%d (code %d)", attn_S, kv_split, arc);
       if (commit_form && l == nl - 1) break;   // the last layer's K/V are in the cache; nothing reads its output
@@ -329,51 +321,33 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g = GemmArgs{};
     g.x = c->att; g.w = w.wo; g.R = R; g.N = d; g.K = c->qdim; g.x_pitch = c->qdim; g.w_pitch = c->qdim; g.w_tiled = 1;
     g.splits = c->split_o; g.epi = EPI_PARTIAL; g.out = c->partial;
-    if (fused) produce_norm(g, w.g_ffn, c->split_o);
+    produce_norm(g, w.g_ffn, c->split_o);
     rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_O);
     if (rc) return rc;
-    if (fused) {
-      sq_count = gemm_tiles(d);
-    } else {
-      Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * (4.0 * g.splits + 10.0));
-      launch_residual_rmsnorm(c->st, c->partial, g.splits, (size_t)R * d, w.g_ffn, c->cfg.rms_eps, c->h, c->xn, R, d);
-    }
+    sq_count = gemm_tiles(d);
     // ---- gate/up projection with SwiGLU
     g = GemmArgs{};
     g.x = c->xn; g.w = w.wgu; g.R = R; g.N = 2 * c->ffn_pad; g.K = d; g.x_pitch = d; g.w_pitch = d; g.w_tiled = 1;
     g.splits = 1;
-    if (fused) {
-      g.epi = EPI_SWIGLU; g.act = c->act; g.act_pitch = c->ffn_pad;
-      consume_norm(g);
-      rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_GU);
-      if (rc) return rc;
-    } else {
-      g.epi = EPI_PARTIAL; g.out = c->partial;
-      if ((size_t)R * g.N > c->partial_elems) return fail(c, SSD_ERR_OVERFLOW, "workspace too small");
-      rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_GU);
-      if (rc) return rc;
-      Scope sc(c, SSD_PROF_ELEMWISE, (double)R * c->ffn_pad * 10.0);
-      launch_swiglu(c->st, c->partial, c->act, R, c->ffn_pad);
-    }
+    g.epi = EPI_SWIGLU; g.act = c->act; g.act_pitch = c->ffn_pad;
+    consume_norm(g);
+    rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_GU);
+    if (rc) return rc;
     // ---- down projection + residual + next norm
     g = GemmArgs{};
     g.x = c->act; g.w = w.wd; g.R = R; g.N = d; g.K = c->ffn_pad; g.x_pitch = c->ffn_pad; g.w_pitch = c->ffn_pad; g.w_tiled = 1;
     g.splits = c->split_down; g.epi = EPI_PARTIAL; g.out = c->partial;
     const float* gain = (l + 1 < nl) ? c->L[l + 1].g_attn : c->g_final;
-    if (fused) produce_norm(g, gain, c->split_down);
+    produce_norm(g, gain, c->split_down);
     rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_DOWN);
     if (rc) return rc;
-    if (!fused) {
-      Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * (4.0 * g.splits + 10.0));
-      launch_residual_rmsnorm(c->st, c->partial, g.splits, (size_t)R * d, gain, c->cfg.rms_eps, c->h, c->xn, R, d);
-    }
   }
   if (kind == FWD_VERIFY) {
     GemmArgs g{};
     g.x = c->xn; g.w = c->lm_head; g.R = R; g.N = c->V; g.K = d; g.x_pitch = d; g.w_pitch = d; g.splits = 1; g.w_tiled = 1;
     g.mask_id = c->cfg.mask_id;
     consume_norm(g);
-    if (want_logits || c->gemm_impl != 1) {
+    if (want_logits) {
       const size_t need = (size_t)R * c->V;
       if (need > c->logits_elems) {
         float* p = nullptr;
@@ -556,6 +530,7 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     ALLOC(c, c->bs.ids, sb); ALLOC(c, c->bs.masked, sb); ALLOC(c, c->bs.draft_tok, sb); ALLOC(c, c->bs.draft_conf, sb);
     ALLOC(c, c->bs.cand_pos, sb); ALLOC(c, c->bs.cand_tok, sb); ALLOC(c, c->bs.accept_log, sb);
     ALLOC(c, c->pending_ids, sb);
+    ALLOC(c, c->prompt_stage, (size_t)k.max_batch * k.max_seq);
     ALLOC(c, c->bs.has_drafts, k.max_batch); ALLOC(c, c->bs.remaining, k.max_batch); ALLOC(c, c->bs.n_cand, k.max_batch);
     ALLOC(c, c->bs.n_forwards, k.max_batch); ALLOC(c, c->bs.last_accept, k.max_batch); ALLOC(c, c->bs.seq_map, k.max_batch);
     CUDA_TRY(c, cudaMallocHost(&c->h_pinned, (2 + 3 * (size_t)k.max_batch) * sizeof(int)));
@@ -663,13 +638,9 @@ int ssd_prefill(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t* pr
   if (prompt_len < 1 || prompt_len > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "prompt_len %d outside [1, %d]", prompt_len, c->cfg.max_seq);
   for (size_t i = 0; i < (size_t)batch * prompt_len; ++i)
     if (prompt_ids[i] < 0 || prompt_ids[i] >= c->V) return fail(c, SSD_ERR_INVALID_ARG, "prompt id %d outside the vocabulary", prompt_ids[i]);
-  int* dev_ids = nullptr;
-  CUDA_TRY(c, cudaMalloc(&dev_ids, (size_t)batch * prompt_len * sizeof(int)));
-  cudaError_t e = cudaMemcpyAsync(dev_ids, prompt_ids, (size_t)batch * prompt_len * sizeof(int), cudaMemcpyHostToDevice, c->st);
-  int rc = (e == cudaSuccess) ? ssd_prefill_dev(c, batch, prompt_len, dev_ids) : fail(c, SSD_ERR_CUDA, "H2D copy failed: %s", cudaGetErrorString(e));
-  cudaStreamSynchronize(c->st);
-  cudaFree(dev_ids);
-  return rc;
+  // staged in the context's own buffer (sized max_batch x max_seq at creation): no allocation per call
+  CUDA_TRY(c, cudaMemcpyAsync(c->prompt_stage, prompt_ids, (size_t)batch * prompt_len * sizeof(int), cudaMemcpyHostToDevice, c->st));
+  return ssd_prefill_dev(c, batch, prompt_len, c->prompt_stage);
 }
 
 int ssd_cache_length(const ssd_ctx* c) {
@@ -1047,10 +1018,15 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!c) return SSD_ERR_INVALID_ARG;
   if (!key) return fail(c, SSD_ERR_INVALID_ARG, "null key");
   if (!strcmp(key, "split_k_qkv") || !strcmp(key, "split_k_o") || !strcmp(key, "split_k_down")) {
-    const int width = !strcmp(key, "split_k_qkv") ? c->nqkv : c->d;
-    if (value < 1 || value > kMaxSplit || (size_t)value * width > c->partial_row_floats)
-      return fail(c, SSD_ERR_INVALID_ARG, "split-K for this projection must be in [1, %d]",
-                  (int)(c->partial_row_floats / width < (size_t)kMaxSplit ? c->partial_row_floats / width : kMaxSplit));
+    const bool is_qkv = !strcmp(key, "split_k_qkv");
+    const int width = is_qkv ? c->nqkv : c->d;
+    const int kdim = is_qkv ? c->d : (!strcmp(key, "split_k_o") ? c->qdim : c->ffn_pad);
+    int hi = kMaxSplit;                                   // every split owns at least one 64-wide K block
+    if ((kdim + 63) / 64 < hi) hi = (kdim + 63) / 64;
+    if (!is_qkv && kGemmMaxClusterSplits < hi) hi = kGemmMaxClusterSplits;   // these reduce inside a cluster
+    if (c->partial_row_floats / width < (size_t)hi) hi = (int)(c->partial_row_floats / width);
+    if (value < 1 || value > hi)
+      return fail(c, SSD_ERR_INVALID_ARG, "split-K for this projection must be in [1, %d]", hi);
     if (!strcmp(key, "split_k_qkv")) c->split_qkv = value;
     else if (!strcmp(key, "split_k_o")) c->split_o = value;
     else c->split_down = value;
@@ -1083,11 +1059,6 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
       if (frc) return frc;
     }
     c->fuse_commit = value;
-    return SSD_OK;
-  }
-  if (!strcmp(key, "gemm_impl")) {
-    if (value != 0 && value != 1) return fail(c, SSD_ERR_INVALID_ARG, "gemm_impl is 0 (CUDA cores, bring-up) or 1 (tcgen05)");
-    c->gemm_impl = value;
     return SSD_OK;
   }
   return fail(c, SSD_ERR_INVALID_ARG, "unknown option '%s'", key);

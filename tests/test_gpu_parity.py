@@ -11,7 +11,6 @@ Tolerances (bf16 operands, fp32 accumulation; the stated parity bar):
   * tokens / accept lengths bit-exact wherever the oracle's decision gap exceeds 1e-3;
   * GPU SSD == GPU stepwise bit-exact, no exemption.
 """
-import os
 
 import numpy as np
 import pytest
@@ -25,8 +24,6 @@ pytestmark = pytest.mark.gpu
 
 GAP = 1e-3
 CONF_RTOL = 2e-2     # a logit error e moves a softmax probability by a factor within exp(+-2e)
-# which projection kernel the shared contexts use by default (1 = tcgen05, the product path)
-DEFAULT_IMPL = int(os.environ.get("SSD_TEST_GEMM_IMPL", "1"))
 DEFAULT_TWO_SM = 256         # the library's default for "two_sm_rows"
 PEAKED = wl.TINY.replace(name="tiny_peaked", lm_head_scale=8.0)
 
@@ -42,10 +39,9 @@ def _binding():
     return binding
 
 
-def _make_ssd(w, max_drafts, gemm_impl=DEFAULT_IMPL, max_batch=None, max_seq=None):
+def _make_ssd(w, max_drafts, max_batch=None, max_seq=None):
     b = _binding()
     ssd = b.Ssd(b.config_from_workload(w, max_drafts=max_drafts, max_batch=max_batch, max_seq=max_seq))
-    ssd.set_option("gemm_impl", gemm_impl)
     ssd.load_workload_weights(w)
     return ssd
 
@@ -74,21 +70,16 @@ def tiny_oracles():
 # ------------------------------------------------------------------------------------------
 # the projection kernel alone
 # ------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("impl", [0, 1], ids=["simt", "tc"])
 @pytest.mark.parametrize("rows,n,k,split", [(16, 128, 64, 1), (32, 256, 256, 1), (100, 688, 688, 1), (37, 1376, 256, 1),
                                             (128, 4096, 4096, 4), (64, 512, 12288, 8), (300, 384, 512, 2),
                                             (256, 256, 1024, 3), (1, 130, 72, 1)])
-def test_gemm_against_numpy(tiny_ssd, impl, rows, n, k, split):
-    tiny_ssd.set_option("gemm_impl", impl)
-    try:
-        x = wl.normal_tensor(5, 1, (rows, k), 1.0, device="cuda", dtype=torch.bfloat16)
-        w = wl.normal_tensor(5, 2, (n, k), 0.05, device="cuda", dtype=torch.bfloat16)
-        out = tiny_ssd.gemm_bf16(x, w, split).cpu().numpy()
-        ref = x.cpu().to(torch.float64).numpy() @ w.cpu().to(torch.float64).numpy().T
-        scale = np.sqrt(k) * 0.05
-        assert np.abs(out - ref).max() < 2e-5 * scale * np.sqrt(k) + 1e-6, np.abs(out - ref).max()
-    finally:
-        tiny_ssd.set_option("gemm_impl", DEFAULT_IMPL)
+def test_gemm_against_numpy(tiny_ssd, rows, n, k, split):
+    x = wl.normal_tensor(5, 1, (rows, k), 1.0, device="cuda", dtype=torch.bfloat16)
+    w = wl.normal_tensor(5, 2, (n, k), 0.05, device="cuda", dtype=torch.bfloat16)
+    out = tiny_ssd.gemm_bf16(x, w, split).cpu().numpy()
+    ref = x.cpu().to(torch.float64).numpy() @ w.cpu().to(torch.float64).numpy().T
+    scale = np.sqrt(k) * 0.05
+    assert np.abs(out - ref).max() < 2e-5 * scale * np.sqrt(k) + 1e-6, np.abs(out - ref).max()
 
 
 @pytest.mark.parametrize("rows,n,k,split", [(16, 256, 64, 1), (32, 256, 256, 1), (100, 768, 704, 1), (48, 1280, 256, 1),
@@ -115,16 +106,11 @@ def test_gemm_two_sm_pairs_change_no_bit(tiny_ssd, rows, n, k, split):
 # ------------------------------------------------------------------------------------------
 # cache and forward
 # ------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("impl", [0, 1], ids=["simt", "tc"])
-def test_prefill_cache_matches_oracle(tiny_ssd, tiny_oracles, impl):
+def test_prefill_cache_matches_oracle(tiny_ssd, tiny_oracles):
     w = wl.TINY
     _, ob = tiny_oracles[w.name]
     prompts = wl.make_prompts(w, batch=2).numpy()
-    tiny_ssd.set_option("gemm_impl", impl)
-    try:
-        tiny_ssd.prefill(prompts)
-    finally:
-        tiny_ssd.set_option("gemm_impl", DEFAULT_IMPL)
+    tiny_ssd.prefill(prompts)
     assert tiny_ssd.cache_length() == w.prompt_len
     for b in range(2):
         cache = ob.prefill(prompts[b])
@@ -146,28 +132,23 @@ def _random_nodes(w, rng, n_nodes, T):
     return np.where(masked, w.mask_id, ids), masked
 
 
-@pytest.mark.parametrize("impl", [0, 1], ids=["simt", "tc"])
 @pytest.mark.parametrize("which", ["tiny", "tiny_peaked"])
-def test_verify_forward_logits_and_stats(tiny_ssd, peaked_ssd, tiny_oracles, impl, which):
+def test_verify_forward_logits_and_stats(tiny_ssd, peaked_ssd, tiny_oracles, which):
     w = wl.TINY if which == "tiny" else PEAKED
     ssd = tiny_ssd if which == "tiny" else peaked_ssd
     o64, ob = tiny_oracles[w.name]
     rng = np.random.default_rng(3)
     prompt = wl.make_prompts(w).numpy()
     T = w.block_len
-    ssd.set_option("gemm_impl", impl)
-    try:
-        ssd.prefill(prompt)
-        # one committed block so that the prefix is prompt + block
-        blk = rng.integers(0, w.vocab - 1, (1, T))
-        ssd.block_begin(T)
-        ssd.set_block_state(blk, np.zeros((1, T), np.uint8))
-        ssd.block_commit()
-        ids, masked = _random_nodes(w, rng, 5, T)
-        tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
-        tok2, conf2, _ = ssd.verify_forward(ids, masked, want_logits=False)      # fused LM head path
-    finally:
-        ssd.set_option("gemm_impl", DEFAULT_IMPL)
+    ssd.prefill(prompt)
+    # one committed block so that the prefix is prompt + block
+    blk = rng.integers(0, w.vocab - 1, (1, T))
+    ssd.block_begin(T)
+    ssd.set_block_state(blk, np.zeros((1, T), np.uint8))
+    ssd.block_commit()
+    ids, masked = _random_nodes(w, rng, 5, T)
+    tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
+    tok2, conf2, _ = ssd.verify_forward(ids, masked, want_logits=False)      # fused LM head path
     for o, tol in ((ob, 1e-2), (o64, 2e-2)):
         cache = o.prefill(prompt[0])
         o.commit_block(blk[0], cache)
@@ -185,7 +166,7 @@ def test_verify_forward_logits_and_stats(tiny_ssd, peaked_ssd, tiny_oracles, imp
     # rows that were not asked for
     assert np.all(tok[0][~masked[0]] == -1) and np.all(conf[0][~masked[0]] == 0)
     # the two LM-head paths agree (same logits, different reduction order)
-    assert np.array_equal(tok[0][masked[0]], tok2[0][masked[0]]) or impl == 0
+    assert np.array_equal(tok[0][masked[0]], tok2[0][masked[0]])
     assert np.allclose(conf[0], conf2[0], rtol=1e-4)
     assert w.mask_id not in tok
 
