@@ -17,7 +17,9 @@ What is defined here, and from where:
   greedy verification chain of N+1 nodes (Section 3.2.3), batch verification
   (Eq. 5), parent-prediction-vs-child-draft traversal (Section 3.2.4) and the
   loop of Algorithm 1 -> ``select_candidates``, ``build_chain``,
-  ``node_predictions``, ``accept_length``, ``Oracle.decode_block_ssd``.
+  ``node_predictions``, ``accept_length``, ``Oracle.decode_block_ssd``;
+* the mix-order tree of Section 5.2 (the chain plus one out-of-order branch per chain node
+  that has a grandchild, 2N nodes) -> ``build_mix_order_tree``, ``accept_walk_mix_order``.
 
 Readings where the paper is silent (each also listed in the design notes):
 the forward of a block attends to the cached prefix plus the block itself; a
@@ -213,6 +215,44 @@ def accept_length(pred: Sequence[Tuple[int, int]], cand: Sequence[Tuple[int, int
     return a
 
 
+def build_mix_order_tree(ids: np.ndarray, masked: np.ndarray, cand: Sequence[Tuple[int, int]], mask_id: int
+                         ) -> Tuple[np.ndarray, np.ndarray]:
+    """Greedy chain plus the mix-order branches of Section 5.2: every chain node that has a
+    grandchild (node i, i <= N-2) gets one more child, its own state with candidate i+2
+    written in INSTEAD of candidate i+1 - the state stepwise decoding reaches when it takes
+    the two candidates in the other order.  Branch nodes get no children.  Node order: chain
+    nodes 0..N, then the branch of chain node 0, 1, ..., N-2 (index N+1+i): 2N nodes for
+    N >= 1 (6 / 8 / 10 for N = 3 / 4 / 5, Table 3)."""
+    n_chain = len(cand) + 1
+    chain_ids, chain_masked = build_chain(ids, masked, cand, mask_id)
+    rows_ids, rows_masked = [chain_ids], [chain_masked]
+    for i in range(n_chain - 2):
+        p, t = cand[i + 1]
+        bi, bm = chain_ids[i].copy(), chain_masked[i].copy()
+        bi[p] = t
+        bm[p] = False
+        rows_ids.append(bi[None])
+        rows_masked.append(bm[None])
+    return np.concatenate(rows_ids), np.concatenate(rows_masked)
+
+
+def accept_walk_mix_order(pred: Sequence[Tuple[int, int]], cand: Sequence[Tuple[int, int]]
+                          ) -> Tuple[List[Tuple[int, int]], int]:
+    """Traversal of the mix-order tree.  Along the chain as in ``accept_length``; where chain
+    node a's prediction is not candidate a+1 but equals candidate a+2 (same tokens, other
+    order), that candidate is accepted and the walk moves to node a's branch, whose own
+    prediction is accepted too and ends the walk (branches have no children).  Returns the
+    accepted (position, token) list in stepwise order and the index of the last valid node."""
+    n = len(cand)
+    a = 0
+    while a < n and pred[a] == cand[a]:
+        a += 1
+    if a + 1 < n and pred[a] == cand[a + 1]:
+        branch = n + 1 + a
+        return list(cand[:a]) + [cand[a + 1], pred[branch]], branch
+    return list(cand[:a]) + [pred[a]], a
+
+
 # --------------------------------------------------------------------------------------
 # the model and the decode loops
 # --------------------------------------------------------------------------------------
@@ -250,6 +290,7 @@ class ForwardRecord:
     gap: np.ndarray                 # [n, B] top-1 minus top-2 probability per row
     pred: List[Tuple[int, int]]
     accepted: int                   # a+1
+    last_node: int = -1             # the node whose outputs became the next drafts (-1: not recorded)
 
 
 class Oracle:
@@ -381,13 +422,16 @@ class Oracle:
 
     def decode_block_ssd(self, block_len: int, cache: Cache, max_drafts: int, block_index: int = 0,
                          trace: Optional[List[ForwardRecord]] = None,
-                         draft_override: Optional[Callable] = None):
+                         draft_override: Optional[Callable] = None, tree: str = "greedy"):
         """Algorithm 1 restricted to one block.  Returns (ids [B], accept counts per forward).
 
+        ``tree`` is "greedy" (the chain of N+1 nodes, Section 3.2.3) or "mix_order" (the chain
+        plus one out-of-order branch per chain node with a grandchild, Section 5.2).
         ``draft_override(ids, masked, draft_tok, draft_conf) -> (draft_tok, draft_conf)``
         lets a test replace the drafts (perfect or adversarial) to pin the accept logic
         independently of the model.
         """
+        assert tree in ("greedy", "mix_order")
         mid = self.cfg.mask_id
         ids = np.full(block_len, mid, dtype=np.int64)
         masked = np.ones(block_len, dtype=bool)
@@ -402,30 +446,35 @@ class Oracle:
                 if draft_override is not None:
                     dt, dc = draft_override(ids.copy(), masked.copy(), dt.copy(), dc.copy())
                 cand = select_candidates(dt, dc, masked, max_drafts)
-            node_ids, node_masked = build_chain(ids, masked, cand, mid)
+            if tree == "greedy":
+                node_ids, node_masked = build_chain(ids, masked, cand, mid)
+            else:
+                node_ids, node_masked = build_mix_order_tree(ids, masked, cand, mid)
             tok, conf, gap, _ = self.verify(node_ids, node_masked, cache)
             pred = node_predictions(tok, conf, node_masked)
-            a = accept_length(pred, cand)
+            if tree == "greedy":
+                a = accept_length(pred, cand)
+                accepted, last = list(cand[:a]) + [pred[a]], a
+            else:
+                accepted, last = accept_walk_mix_order(pred, cand)
             if trace is not None:
                 trace.append(ForwardRecord(block_index, cache.length, ids.copy(), masked.copy(),
                                            None if draft_tok is None else draft_tok.copy(),
                                            None if draft_conf is None else draft_conf.copy(),
-                                           list(cand), node_ids, node_masked, tok, conf, gap, pred, a + 1))
-            for (p, t) in cand[:a]:
+                                           list(cand), node_ids, node_masked, tok, conf, gap, pred,
+                                           len(accepted), last))
+            for (p, t) in accepted:
                 ids[p] = t
                 masked[p] = False
-            q, t = pred[a]
-            ids[q] = t
-            masked[q] = False
             # next drafts: the last valid node's own predictions on what is still masked
-            draft_tok = np.where(masked, tok[a], 0).astype(np.int64)
-            draft_conf = np.where(masked, conf[a], 0.0)
-            counts.append(a + 1)
+            draft_tok = np.where(masked, tok[last], 0).astype(np.int64)
+            draft_conf = np.where(masked, conf[last], 0.0)
+            counts.append(len(accepted))
         return ids, counts
 
     def generate(self, prompt: np.ndarray, gen_len: int, block_len: int, mode: str = "ssd",
                  max_drafts: int = 0, trace: Optional[List[ForwardRecord]] = None,
-                 draft_override: Optional[Callable] = None):
+                 draft_override: Optional[Callable] = None, tree: str = "greedy"):
         """Semi-autoregressive generation of gen_len tokens after the prompt.
         Returns (tokens [gen_len], accept counts per block (list of lists), cache)."""
         cache = self.prefill(np.asarray(prompt))
@@ -434,7 +483,7 @@ class Oracle:
             if mode == "stepwise":
                 ids, counts = self.decode_block_stepwise(hi - lo, cache, j, trace)
             else:
-                ids, counts = self.decode_block_ssd(hi - lo, cache, max_drafts, j, trace, draft_override)
+                ids, counts = self.decode_block_ssd(hi - lo, cache, max_drafts, j, trace, draft_override, tree)
             self.commit_block(ids, cache)
             out.append(ids)
             all_counts.append(counts)

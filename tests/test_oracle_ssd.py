@@ -292,3 +292,135 @@ def test_block_order_constraint():
         assert rec.cache_len == w.prompt_len + rec.block * w.block_len
         assert rec.node_ids.shape[1] == w.block_len
         assert all(0 <= p < w.block_len for p, _ in rec.cand)
+
+
+# ---------------------------------------------------------------------------------------
+# mix-order tree (Section 5.2, Table 3)
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N,nodes", _golden("mix_order_verification_batch.txt"))
+def test_mix_order_tree_has_2n_nodes(N, nodes):
+    B = 16
+    o = ScriptedOracle(64, _context_free_rule(B))
+    o.decode_block_ssd(B, NoCache(), max_drafts=N, tree="mix_order")
+    assert o.nodes_per_forward[0] == 1
+    assert o.nodes_per_forward[1] == int(nodes) == 2 * N
+    assert max(o.nodes_per_forward) == 2 * N
+
+
+def test_mix_order_tree_contents():
+    ids = np.array([5, 63, 63, 9, 63, 63])
+    masked = np.array([0, 1, 1, 0, 1, 1], dtype=bool)
+    cand = [(4, 11), (1, 12), (5, 13)]
+    node_ids, node_masked = so.build_mix_order_tree(ids, masked, cand, 63)
+    chain_ids, chain_masked = so.build_chain(ids, masked, cand, 63)
+    assert node_ids.shape == (6, 6)
+    assert np.array_equal(node_ids[:4], chain_ids) and np.array_equal(node_masked[:4], chain_masked)
+    # branch of node 0: candidate 2 alone; branch of node 1: candidates 1 and 3
+    assert node_ids[4].tolist() == [5, 12, 63, 9, 63, 63]
+    assert node_ids[5].tolist() == [5, 63, 63, 9, 11, 13]
+    assert node_masked[4].tolist() == [False, False, True, False, True, True]
+    assert node_masked[5].tolist() == [False, True, True, False, False, False]
+    # fewer than two candidates: nothing to branch to
+    assert so.build_mix_order_tree(ids, masked, cand[:1], 63)[0].shape == (2, 6)
+    assert so.build_mix_order_tree(ids, masked, [], 63)[0].shape == (1, 6)
+
+
+def test_mix_order_walk():
+    cand = [(4, 11), (1, 12), (5, 13)]
+    # node order: chain 0..3, branch of 0, branch of 1
+    chain_ok = [(4, 11), (1, 12), (5, 13), (2, 7), (0, 0), (0, 0)]
+    assert so.accept_walk_mix_order(chain_ok, cand) == ([(4, 11), (1, 12), (5, 13), (2, 7)], 3)
+    swapped_at_root = [(1, 12), (0, 0), (0, 0), (0, 0), (4, 99), (0, 0)]
+    assert so.accept_walk_mix_order(swapped_at_root, cand) == ([(1, 12), (4, 99)], 4)
+    swapped_at_one = [(4, 11), (5, 13), (0, 0), (0, 0), (0, 0), (2, 8)]
+    assert so.accept_walk_mix_order(swapped_at_one, cand) == ([(4, 11), (5, 13), (2, 8)], 5)
+    # a skip of two, a wrong token at the other position, and the last chain node have no branch
+    assert so.accept_walk_mix_order([(5, 13), (0, 0), (0, 0), (0, 0), (0, 0), (0, 0)], cand) == ([(5, 13)], 0)
+    assert so.accept_walk_mix_order([(1, 99), (0, 0), (0, 0), (0, 0), (0, 0), (0, 0)], cand) == ([(1, 99)], 0)
+    assert so.accept_walk_mix_order([(4, 11), (1, 12), (2, 7), (0, 0), (0, 0), (0, 0)], cand) == \
+        ([(4, 11), (1, 12), (2, 7)], 2)
+    assert so.accept_walk_mix_order([(3, 3)], []) == ([(3, 3)], 0)
+
+
+def test_mix_order_recovers_the_swapped_order_case():
+    """Section 5.2 / Fig. 4(b): drafts that hold the right tokens in another order cost the greedy chain
+    everything but one token per forward; the mix-order branch accepts the swapped candidate and its
+    own prediction."""
+    B = 24
+    base = ScriptedOracle(64, _context_free_rule(B))
+    want, _ = base.decode_block_stepwise(B, NoCache())
+    conf = np.linspace(0.9, 0.1, B)
+
+    def swap_first_two(ids, masked, dt, dc):
+        pos = [p for p in range(B) if masked[p]]
+        order = sorted(pos, key=lambda p: -conf[p])
+        dc = conf.copy()
+        if len(order) >= 2:
+            dc[order[0]], dc[order[1]] = conf[order[1]], conf[order[0]]
+        return dt, dc
+
+    g = ScriptedOracle(64, _context_free_rule(B))
+    ids_g, counts_g = g.decode_block_ssd(B, NoCache(), max_drafts=4, draft_override=swap_first_two)
+    m = ScriptedOracle(64, _context_free_rule(B))
+    ids_m, counts_m = m.decode_block_ssd(B, NoCache(), max_drafts=4, draft_override=swap_first_two, tree="mix_order")
+    assert np.array_equal(ids_g, want) and np.array_equal(ids_m, want)
+    assert all(c == 1 for c in counts_g[:-1])
+    assert all(c == 2 for c in counts_m[1:-3]) and len(counts_m) < len(counts_g)
+
+
+def test_mix_order_matches_bruteforce_and_never_loses_to_greedy():
+    """Context-dependent scripted model: the tokens a mix-order forward accepts are exactly the next
+    stepwise steps from the same state, their number is the greedy count or one more, and the output
+    is the stepwise output."""
+    B, V = 14, 40
+    table_rng = np.random.default_rng(7)
+    # tokens mostly stable, confidences jitter with the context: the drafts usually hold the right
+    # tokens, but their order goes stale - the out-of-order case of Fig. 4(a)
+    tok_tab = np.tile(table_rng.integers(0, V - 1, B), (B + 1, 1))
+    tok_tab[::4] = table_rng.integers(0, V - 1, (len(tok_tab[::4]), B))
+    conf_tab = np.linspace(0.9, 0.2, B)[None, :] + 0.12 * table_rng.random((B + 1, B))
+
+    def rule(ids, masked):
+        r = int(masked.sum())
+        return tok_tab[r].copy(), conf_tab[r].copy()
+
+    ref = ScriptedOracle(V, rule)
+    want, _ = ref.decode_block_stepwise(B, NoCache())
+    order = []
+    ids = np.full(B, V - 1)
+    masked = np.ones(B, dtype=bool)
+    while masked.any():
+        t, c = rule(ids, masked)
+        q = so.best_masked_position(c, masked)
+        order.append((q, int(t[q])))
+        ids[q] = t[q]
+        masked[q] = False
+    gained = 0
+    for N in (2, 3, 5, B):
+        trace = []
+        o = ScriptedOracle(V, rule)
+        got, counts = o.decode_block_ssd(B, NoCache(), max_drafts=N, trace=trace, tree="mix_order")
+        assert np.array_equal(got, want)
+        done = 0
+        for rec in trace:
+            n = len(rec.cand)
+            accepted, last = so.accept_walk_mix_order(rec.pred, rec.cand)
+            assert accepted == order[done:done + rec.accepted]            # exactly the stepwise continuation
+            greedy = so.accept_length(rec.pred[:n + 1], rec.cand) + 1
+            assert rec.accepted in (greedy, greedy + 1)
+            assert rec.node_ids.shape[0] == n + 1 + max(0, n - 1)
+            gained += rec.accepted - greedy
+            done += rec.accepted
+        assert done == B
+    assert gained > 0                                                     # the branch is exercised
+
+
+@pytest.mark.parametrize("w", [SMALL, SMALL_GQA], ids=lambda w: w.name)
+@pytest.mark.parametrize("max_drafts", [1, 2, 3, 5, 64])
+def test_mix_order_equals_stepwise_small(w, max_drafts):
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    a, _, _ = o.generate(prompt, w.gen_len, w.block_len, mode="stepwise")
+    b, counts, _ = o.generate(prompt, w.gen_len, w.block_len, mode="ssd", max_drafts=max_drafts, tree="mix_order")
+    assert np.array_equal(a, b)
+    assert all(sum(c) == w.block_len for c in counts)
