@@ -141,6 +141,23 @@ int ssd_verify_forward(ssd_ctx* ctx, int32_t batch, int32_t n_nodes, int32_t blo
  * [length, n_kv_heads, head_dim] each, positions [0, length).  Test hook for cache semantics. */
 int ssd_read_cache(ssd_ctx* ctx, int32_t layer, int32_t seq, int32_t length, float* out_k, float* out_v);
 
+/* The reverse: overwrite cached K (post-rotary) and V of one layer and sequence, positions
+ * [0, length), from HOST fp32 [length, n_kv_heads, head_dim] (rounded to bf16, the cache's type).
+ * Test hook: lets a reference supply the prefix of a layer-by-layer comparison.  Does not change
+ * ssd_cache_length. */
+int ssd_write_cache(ssd_ctx* ctx, int32_t layer, int32_t seq, int32_t length, const float* k, const float* v);
+
+/* Layers [layer_begin, layer_end) of the verification forward (Eq. 5) on a caller-given residual
+ * stream, against the current cache: `h_in` HOST fp32 [batch * n_nodes * block_tokens, d_model] is
+ * the stream entering layer_begin, `h_out` (same shape, may be NULL) the stream leaving
+ * layer_end - 1.  With layer_end == n_layers, out_tok / out_conf (HOST [batch, n_nodes,
+ * block_tokens], may be NULL) receive the LM-head statistics of every row.  Test hook: each layer can
+ * be checked against a reference from the reference's own input, so that rounding noise does not
+ * compound over the depth.  The decode state is not touched. */
+int ssd_verify_layers(ssd_ctx* ctx, int32_t batch, int32_t n_nodes, int32_t block_tokens,
+                      int32_t layer_begin, int32_t layer_end, const float* h_in, float* h_out,
+                      int32_t* out_tok, float* out_conf);
+
 /* Cached prefix length S (prompt + committed blocks, a block that waits for its commit
  * included), or a negative error. */
 int ssd_cache_length(const ssd_ctx* ctx);
@@ -205,12 +222,19 @@ int ssd_profile_enable(ssd_ctx* ctx, int32_t on);
 int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, double* bytes);
 
 /* Tuning knobs (set before prefill).  key:
- *   "split_k_qkv", "split_k_o", "split_k_down"  split-K factor of a projection, 1..16, bounded by the
- *        split-K workspace; with the tensor-core kernel the O and down projections reduce their
- *        splits inside a thread-block cluster and use at most 8;
+ *   "split_k_qkv", "split_k_o", "split_k_down"  split-K factor of a projection: 1..16 for QKV, 1..8 for
+ *        the O and down projections (they reduce their splits inside a thread-block cluster), never
+ *        more than the projection has 64-wide K blocks, bounded by the split-K workspace;
  *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically (in
  *        steps of 128) while a prefix would need more than 7 parts;
  *   "max_drafts" lower the draft-length cap below the capacity fixed at creation;
+ *   "mix_order"  1 = the verification tree is the greedy chain plus the mix-order branches of
+ *        Section 5.2 (Table 3): every chain node that has a grandchild gets one more child, its state
+ *        with candidate i+2 in place of candidate i+1; when a node predicts that candidate (right
+ *        tokens, other order) it is accepted together with the branch's own prediction and the walk
+ *        ends.  2N nodes instead of N+1; the tokens are still those of stepwise decoding.  The tree
+ *        must fit the node capacity fixed at creation (max_drafts + 1 nodes): create the context with
+ *        max_drafts >= 2N - 1, then set "max_drafts" to N.  0 = greedy chain (default);
  *   "attn_impl"  1 = attention of the verification forward on tcgen05 where the shape allows (head
  *        dimension 128, parts of whole 128-key tiles, block length dividing 128), the default; 0 = always the
  *        mma.sync form;
@@ -220,8 +244,6 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *        are bit-identical either way;
  *   "fuse_commit" 1 = a block's commit is folded into the next block's first forward (default); 0 = a
  *        commit forward of its own inside ssd_block_commit;
- *   "gemm_impl"  1 = TMA + tcgen05 kernel with fused RMSNorm / residual epilogues, the default;
- *        0 = the plain CUDA-core bring-up kernel with separate norm kernels, for cross-checks only.
  * Unknown key: SSD_ERR_INVALID_ARG. */
 int ssd_set_option(ssd_ctx* ctx, const char* key, int32_t value);
 

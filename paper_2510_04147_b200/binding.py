@@ -27,7 +27,7 @@ PROF_TOP = PROF_FAMILIES[:5]          # the last four break "gemm" down by proje
 
 EXPORTS = ["ssd_create", "ssd_destroy", "ssd_last_error", "ssd_load_weights", "ssd_prefill", "ssd_prefill_dev",
            "ssd_decode_block", "ssd_block_begin", "ssd_set_block_state", "ssd_get_block_state", "ssd_block_step",
-           "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_cache_length", "ssd_rewind", "ssd_gemm_bf16",
+           "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_write_cache", "ssd_verify_layers", "ssd_cache_length", "ssd_rewind", "ssd_gemm_bf16",
            "ssd_gemm_bf16_noalloc",
            "ssd_launch_count", "ssd_profile_enable", "ssd_profile_read", "ssd_set_option"]
 
@@ -75,6 +75,8 @@ def load_library() -> C.CDLL:
     lib.ssd_block_commit.argtypes = [vp]
     lib.ssd_verify_forward.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.ssd_read_cache.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.ssd_write_cache.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.ssd_verify_layers.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.ssd_cache_length.argtypes = [vp]
     lib.ssd_rewind.argtypes = [vp, i32]
     lib.ssd_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
@@ -226,6 +228,23 @@ class Ssd:
         assert k.size == length * kv
         self._check(self.lib.ssd_read_cache(self._ctx, layer, seq, length, _np_ptr(k), _np_ptr(v)))
         return k, v
+
+    def write_cache(self, layer: int, seq: int, k: np.ndarray, v: np.ndarray):
+        k = np.ascontiguousarray(k, dtype=np.float32)
+        v = np.ascontiguousarray(v, dtype=np.float32)
+        assert k.shape == v.shape and k.shape[1:] == (self.cfg.n_kv_heads, self.cfg.head_dim)
+        self._check(self.lib.ssd_write_cache(self._ctx, layer, seq, k.shape[0], _np_ptr(k), _np_ptr(v)))
+
+    def verify_layers(self, h_in: np.ndarray, batch: int, n_nodes: int, block_tokens: int, layer_begin: int,
+                      layer_end: int, want_stats: bool = False):
+        """Returns (h_out [batch*n_nodes*block_tokens, d], tok or None, conf or None)."""
+        h = np.ascontiguousarray(h_in, dtype=np.float32).reshape(batch * n_nodes * block_tokens, self.cfg.d_model)
+        out = np.zeros_like(h)
+        tok = np.zeros((batch, n_nodes, block_tokens), np.int32) if want_stats else None
+        conf = np.zeros((batch, n_nodes, block_tokens), np.float32) if want_stats else None
+        self._check(self.lib.ssd_verify_layers(self._ctx, batch, n_nodes, block_tokens, layer_begin, layer_end,
+                                               _np_ptr(h), _np_ptr(out), _np_ptr(tok), _np_ptr(conf)))
+        return out, tok, conf
 
     def cache_length(self) -> int:
         rc = self.lib.ssd_cache_length(self._ctx)

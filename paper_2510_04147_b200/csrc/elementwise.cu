@@ -56,12 +56,16 @@ __global__ void copy_f32_kernel(const void* src, int src_is_f32, float* dst, int
 constexpr int kRowThreadsMax = 1024;   // one float4 per thread up to d = 4096
 
 __global__ void __launch_bounds__(kRowThreadsMax) embed_prep_kernel(const int* ids, const bf16* embed, const float* gain,
-                                                                    float* h, bf16* hb, float* sq, int sq_stride, int d) {
+                                                                    float* h, bf16* hb, float* sq, int sq_stride, int d,
+                                                                    int V) {
   __shared__ float red[kRowThreadsMax / 32];
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.x;
-  const bf16* e = embed + (size_t)ids[r] * d;
+  // ids come from the device-side decode state: never index the table with one outside the vocabulary
+  int id = ids[r];
+  if ((unsigned)id >= (unsigned)V) id = 0;
+  const bf16* e = embed + (size_t)id * d;
   float ss = 0.f;
   for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
     const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(e + c);
@@ -69,6 +73,26 @@ __global__ void __launch_bounds__(kRowThreadsMax) embed_prep_kernel(const int* i
     const float4 g = *reinterpret_cast<const float4*>(gain + c);
     const float4 v = make_float4(__low2float(a), __high2float(a), __low2float(b), __high2float(b));
     *reinterpret_cast<float4*>(h + (size_t)r * d + c) = v;
+    *reinterpret_cast<__nv_bfloat162*>(hb + (size_t)r * d + c) = __floats2bfloat162_rn(v.x * g.x, v.y * g.y);
+    *reinterpret_cast<__nv_bfloat162*>(hb + (size_t)r * d + c + 2) = __floats2bfloat162_rn(v.z * g.z, v.w * g.w);
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+  }
+  ss = block_sum(ss, red);
+  if (threadIdx.x == 0) sq[(size_t)r * sq_stride] = ss;
+}
+
+// The same producer step for a residual stream that is already in h (a forward entered at a
+// later layer): hb[r] = bf16(h[r] * gain); sq[r * sq_stride] = sum of squares of h[r]
+__global__ void __launch_bounds__(kRowThreadsMax) stream_prep_kernel(const float* h, const float* gain, bf16* hb,
+                                                                     float* sq, int sq_stride, int d) {
+  __shared__ float red[kRowThreadsMax / 32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  float ss = 0.f;
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(h + (size_t)r * d + c);
+    const float4 g = *reinterpret_cast<const float4*>(gain + c);
     *reinterpret_cast<__nv_bfloat162*>(hb + (size_t)r * d + c) = __floats2bfloat162_rn(v.x * g.x, v.y * g.y);
     *reinterpret_cast<__nv_bfloat162*>(hb + (size_t)r * d + c + 2) = __floats2bfloat162_rn(v.z * g.z, v.w * g.w);
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
@@ -154,7 +178,8 @@ __global__ void __launch_bounds__(kThreads) lm_stats_from_logits_kernel(const fl
   for (int v = threadIdx.x; v < V; v += kThreads)
     if (v != mask_id) s += expf(l[v] - m);
   s = block_sum(s, red);
-  if (threadIdx.x == 0) { tok[r] = a; conf[r] = 1.f / s; }
+  // non-finite logits leave no valid argmax: the token stays inside the vocabulary, the confidence says so
+  if (threadIdx.x == 0) { tok[r] = ((unsigned)a >= (unsigned)V) ? 0 : a; conf[r] = 1.f / s; }
 }
 
 // Symmetric merge of two (max, sum-exp, argmax) triples: both partners of a butterfly step compute
@@ -174,7 +199,7 @@ __device__ __forceinline__ void stat_merge(float& m, float& s, int& a, float om,
 // One CTA per row: threads stride over the vocabulary tiles, butterfly inside each warp, then the
 // warp results in warp order.  The order depends on the tile count alone.
 __global__ void __launch_bounds__(kThreads) lm_merge_kernel(const float* tile_max, const float* tile_sum,
-                                                            const int* tile_arg, int tiles, int R,
+                                                            const int* tile_arg, int tiles, int R, int V,
                                                             const uint8_t* row_wanted, int* tok, float* conf) {
   __shared__ float w_m[kThreads / 32], w_s[kThreads / 32];
   __shared__ int w_a[kThreads / 32];
@@ -207,7 +232,8 @@ __global__ void __launch_bounds__(kThreads) lm_merge_kernel(const float* tile_ma
   __syncthreads();
   if (threadIdx.x == 0) {
     for (int i = 1; i < kThreads / 32; ++i) stat_merge(m, s, a, w_m[i], w_s[i], w_a[i]);
-    tok[r] = a;
+    // non-finite logits leave no valid argmax: the token stays inside the vocabulary, the confidence says so
+    tok[r] = ((unsigned)a >= (unsigned)V) ? 0 : a;
     conf[r] = 1.f / s;
   }
 }
@@ -246,8 +272,13 @@ static int row_threads(int d) {
 }
 
 void launch_embed_prep(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float* h, bf16* hb,
-                       float* sq, int sq_stride, int R, int d) {
-  launch_pdl(embed_prep_kernel, dim3(R), dim3(row_threads(d)), 0, st, ids, embed, gain, h, hb, sq, sq_stride, d);
+                       float* sq, int sq_stride, int R, int d, int V) {
+  launch_pdl(embed_prep_kernel, dim3(R), dim3(row_threads(d)), 0, st, ids, embed, gain, h, hb, sq, sq_stride, d, V);
+}
+
+void launch_stream_prep(cudaStream_t st, const float* h, const float* gain, bf16* hb, float* sq, int sq_stride, int R,
+                        int d) {
+  launch_pdl(stream_prep_kernel, dim3(R), dim3(row_threads(d)), 0, st, h, gain, hb, sq, sq_stride, d);
 }
 
 void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H, int Hkv,
@@ -265,9 +296,9 @@ void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, in
 }
 
 void launch_lm_merge(cudaStream_t st, const float* tile_max, const float* tile_sum, const int* tile_arg, int tiles,
-                     int R, const uint8_t* row_wanted, int* tok, float* conf) {
-  launch_pdl(lm_merge_kernel, dim3(R), dim3(kThreads), 0, st, tile_max, tile_sum, tile_arg, tiles, R, row_wanted, tok,
-             conf);
+                     int R, int V, const uint8_t* row_wanted, int* tok, float* conf) {
+  launch_pdl(lm_merge_kernel, dim3(R), dim3(kThreads), 0, st, tile_max, tile_sum, tile_arg, tiles, R, V, row_wanted,
+             tok, conf);
 }
 
 }  // namespace ssd

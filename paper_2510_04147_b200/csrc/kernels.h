@@ -102,8 +102,12 @@ void launch_copy_f32(cudaStream_t st, const void* src, int src_is_f32, float* ds
 // ---------------------------------------------------------------- elementwise / reductions
 // producer side of the fused RMSNorm: h[r] = embed[ids[r]]; hb[r] = bf16(h[r] * gain);
 // sq[r * sq_stride] = sum of squares of h[r]
+// (ids outside [0, V) read row 0: the table is never indexed out of range)
 void launch_embed_prep(cudaStream_t st, const int* ids, const bf16* embed, const float* gain, float* h, bf16* hb,
-                       float* sq, int sq_stride, int R, int d);
+                       float* sq, int sq_stride, int R, int d, int V);
+// the same producer step for a residual stream already in h: hb[r] = bf16(h[r] * gain), sq as above
+void launch_stream_prep(cudaStream_t st, const float* h, const float* gain, bf16* hb, float* sq, int sq_stride, int R,
+                        int d);
 // sums the split-K partials of the fused QKV projection, rotates q and k, writes bf16.
 // kv_to_cache: k/v rows go to cache[(seq*max_seq + pos)*Hkv*hd] else to local [r][Hkv][hd].
 void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H,
@@ -112,9 +116,9 @@ void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t s
 // per row: argmax / max-softmax-probability over the vocabulary with mask_id excluded
 void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, int V, int mask_id,
                                  const uint8_t* row_wanted, int* tok, float* conf);
-// merge per-tile (max, sumexp, argmax) in tile order
+// merge per-tile (max, sumexp, argmax) in tile order; the token is always inside [0, V)
 void launch_lm_merge(cudaStream_t st, const float* tile_max, const float* tile_sum, const int* tile_arg,
-                     int tiles, int R, const uint8_t* row_wanted, int* tok, float* conf);
+                     int tiles, int R, int V, const uint8_t* row_wanted, int* tok, float* conf);
 
 // ---------------------------------------------------------------- attention
 struct AttnArgs {
@@ -213,15 +217,18 @@ struct BlockState {       // device arrays, [max_batch][block_len] unless noted
   int* seq_map;           // [max_batch] slot -> sequence of the current forward
   int stride;             // block_len (row pitch of the arrays above)
 };
+// Nodes of the verification tree for N candidates: the greedy chain has N + 1; the mix-order tree adds
+// one branch for every chain node that has a grandchild (N - 1 of them): 2N nodes for N >= 1.
+__host__ __device__ inline int tree_nodes(int N, int mix_order) { return N + 1 + ((mix_order && N >= 2) ? N - 1 : 0); }
 // slot a (= rank among unfinished sequences): candidates, node rows [a][n_cap][T].  With prev_ids
 // (device [batch][prev_stride]) the rows of a slot are [prev_T tokens of the finished block, not
 // masked][n_cap][T]: the layout of the forward that also commits the previous block.
 void launch_tree_build(cudaStream_t st, BlockState s, int batch, int T, int max_drafts, int n_cap, int mask_id,
-                       int* node_ids, uint8_t* node_masked, const int* prev_ids = nullptr, int prev_T = 0,
-                       int prev_stride = 0);
+                       int* node_ids, uint8_t* node_masked, const int* prev_ids, int prev_T, int prev_stride,
+                       int mix_order);
 // per slot: per-node best masked position, chain walk, state/draft update; a slot's node rows start
 // `row_offset` rows into its `slot_rows` rows (0 and n_cap * T without a finished block in front)
 void launch_accept(cudaStream_t st, BlockState s, int n_slots, int T, int n_cap, const int* tok, const float* conf,
-                   const uint8_t* node_masked, int* nonfinite_flag, int slot_rows = 0, int row_offset = 0);
+                   const uint8_t* node_masked, int* nonfinite_flag, int slot_rows, int row_offset, int mix_order);
 
 }  // namespace ssd

@@ -75,7 +75,8 @@ struct ssd_ctx {
   int* pending_ids = nullptr;    // [max_batch][block_len] tokens of that block
   int* prompt_stage = nullptr;   // [max_batch][max_seq] device copy of a host prompt (ssd_prefill)
   int fuse_commit = 1;
-  std::vector<int> h_remaining, h_has_drafts, h_nodes;
+  std::vector<int> h_remaining, h_has_drafts, h_nodes, h_max_accept;
+  int mix_order = 0;             // 1: the verification tree gets the out-of-order branches of Section 5.2
 
   int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0;
   int two_sm_rows = 256;                   // projections pair their tiles (two-SM MMA) from this many rows on; 0 = never
@@ -238,11 +239,19 @@ bool all_loaded(const ssd_ctx* c) {
 
 enum { FWD_FILL = 0, FWD_VERIFY = 1 };
 
+// Layers [begin, end) of a forward; from_stream: the residual stream entering `begin` is already in
+// c->h (no embedding gather); lm_head: run the LM head after the last layer of the range.
+struct LayerRange {
+  int begin = 0, end = -1;       // end < 0: all layers
+  bool from_stream = false;
+  bool lm_head = true;
+};
+
 // One forward over R rows.  FILL: K/V go to the cache at positions pos0.., attention over the cache
 // only (which then contains the rows themselves), no LM head.  VERIFY: K/V stay node-local, attention
 // over cached prefix + own node, LM head statistics into tok/conf (and logits if wanted).
 int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_slots, bool want_logits,
-            const uint8_t* row_wanted) {
+            const uint8_t* row_wanted, LayerRange range = LayerRange()) {
   const int d = c->d, H = c->H, Hkv = c->Hkv, hd = c->hd;
   const int S = map.pos0;
   if (R > c->R_cap) return fail(c, SSD_ERR_OVERFLOW, "forward of %d rows exceeds capacity %d", R, c->R_cap);
@@ -257,7 +266,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   const int n_parts = (attn_S + kv_split - 1) / kv_split;
   if (via_cache && (size_t)n_parts * R > c->part_rows_parts)
     return fail(c, SSD_ERR_OVERFLOW, "attention workspace too small for %d parts x %d rows", n_parts, R);
-  const int nl = c->cfg.n_layers;
+  const int nl = range.end < 0 ? c->cfg.n_layers : range.end;
   // The RMSNorms have no kernel of their own: a producer (the embedding gather, the O and down
   // projections) writes the residual stream h, bf16(h * gain) in `xn` and per-tile sums of squares in
   // `sq`; the consuming projection scales its output rows by 1/rms.
@@ -271,9 +280,10 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   };
   {
     Scope sc(c, SSD_PROF_ELEMWISE, (double)R * d * 8);
-    launch_embed_prep(c->st, ids_dev, c->embed, c->L[0].g_attn, c->h, c->xn, c->sq, c->sq_stride, R, d);
+    if (range.from_stream) launch_stream_prep(c->st, c->h, c->L[range.begin].g_attn, c->xn, c->sq, c->sq_stride, R, d);
+    else launch_embed_prep(c->st, ids_dev, c->embed, c->L[0].g_attn, c->h, c->xn, c->sq, c->sq_stride, R, d, c->V);
   }
-  for (int l = 0; l < nl; ++l) {
+  for (int l = range.begin; l < nl; ++l) {
     const LayerW& w = c->L[l];
     // ---- QKV projection, rotary embedding
     GemmArgs g{};
@@ -337,12 +347,12 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     g = GemmArgs{};
     g.x = c->act; g.w = w.wd; g.R = R; g.N = d; g.K = c->ffn_pad; g.x_pitch = c->ffn_pad; g.w_pitch = c->ffn_pad; g.w_tiled = 1;
     g.splits = c->split_down; g.epi = EPI_PARTIAL; g.out = c->partial;
-    const float* gain = (l + 1 < nl) ? c->L[l + 1].g_attn : c->g_final;
+    const float* gain = (l + 1 < c->cfg.n_layers) ? c->L[l + 1].g_attn : c->g_final;
     produce_norm(g, gain, c->split_down);
     rc = run_gemm(c, g, SSD_PROF_GEMM, SSD_PROF_GEMM_DOWN);
     if (rc) return rc;
   }
-  if (kind == FWD_VERIFY) {
+  if (kind == FWD_VERIFY && range.lm_head && nl == c->cfg.n_layers) {
     GemmArgs g{};
     g.x = c->xn; g.w = c->lm_head; g.R = R; g.N = c->V; g.K = d; g.x_pitch = d; g.w_pitch = d; g.splits = 1; g.w_tiled = 1;
     g.mask_id = c->cfg.mask_id;
@@ -367,7 +377,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
       int rc = run_gemm(c, g, SSD_PROF_LMHEAD);
       if (rc) return rc;
       Scope sc(c, SSD_PROF_LMHEAD, (double)gemm_tiles(c->V) * R * 12.0);
-      launch_lm_merge(c->st, c->tile_max, c->tile_sum, c->tile_arg, gemm_tiles(c->V), R, row_wanted, c->tok, c->conf);
+      launch_lm_merge(c->st, c->tile_max, c->tile_sum, c->tile_arg, gemm_tiles(c->V), R, c->V, row_wanted, c->tok, c->conf);
     }
   }
   CUDA_TRY(c, cudaGetLastError());
@@ -464,6 +474,7 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
   c->h_remaining.assign(k.max_batch, 0);
   c->h_has_drafts.assign(k.max_batch, 0);
   c->h_nodes.assign(k.max_batch, 0);
+  c->h_max_accept.assign(k.max_batch, 0);
 
   int rc = SSD_OK;
   auto build = [&]() -> int {
@@ -740,12 +751,15 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched) {
   int active = 0, n_cap = 1;
   for (int b = 0; b < B; ++b) {
     c->h_nodes[b] = 0;
+    c->h_max_accept[b] = 0;
     if (c->h_remaining[b] <= 0) continue;
     ++active;
     const int N = c->h_has_drafts[b] ? (md < c->h_remaining[b] - 1 ? md : c->h_remaining[b] - 1) : 0;
-    c->h_nodes[b] = N + 1;
-    if (N + 1 > n_cap) n_cap = N + 1;
+    c->h_nodes[b] = tree_nodes(N, c->mix_order);
+    c->h_max_accept[b] = N + 1;            // (a branch ends the walk at most N tokens in)
+    if (c->h_nodes[b] > n_cap) n_cap = c->h_nodes[b];
   }
+  if (n_cap > c->n_max) return fail(c, SSD_ERR_OVERFLOW, "a tree of %d nodes exceeds the capacity of %d nodes fixed at creation", n_cap, c->n_max);
   *launched = active > 0;
   if (active == 0) return SSD_OK;
   // A block waiting for its commit rides in front of the first forward of this block: per sequence
@@ -768,7 +782,7 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched) {
   {
     Scope sc(c, SSD_PROF_TREE, (double)R * 5);
     launch_tree_build(c->st, c->bs, B, T, md, n_cap, c->cfg.mask_id, c->node_ids, c->node_masked,
-                      Tp > 0 ? c->pending_ids : nullptr, Tp, c->bs.stride);
+                      Tp > 0 ? c->pending_ids : nullptr, Tp, c->bs.stride, c->mix_order);
   }
   RowMap map{n_cap * T, T, c->cache_len, 0, c->bs.seq_map};
   if (Tp > 0) {                // one chain of Tp + T rows at positions cache_len ...
@@ -784,7 +798,7 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched) {
   if (rc) return rc;
   {
     Scope sc(c, SSD_PROF_TREE, (double)R * 9);
-    launch_accept(c->st, c->bs, active, T, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1, slot_rows, Tp);
+    launch_accept(c->st, c->bs, active, T, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1, slot_rows, Tp, c->mix_order);
   }
   if (Tp > 0) {                // the finished block's K/V are in the cache once this forward has run
     c->cache_len += Tp;
@@ -810,7 +824,7 @@ int step_collect(ssd_ctx* c, int32_t* accepted, int32_t* n_nodes) {
   for (int b = 0; b < B; ++b) {
     c->h_remaining[b] = hp[2 + b];
     if (accepted) accepted[b] = hp[2 + mb + b];
-    if (n_nodes) n_nodes[b] = c->h_nodes[b] > 0 ? hp[2 + 2 * mb + b] + 1 : 0;
+    if (n_nodes) n_nodes[b] = c->h_nodes[b] > 0 ? tree_nodes(hp[2 + 2 * mb + b], c->mix_order) : 0;
   }
   return SSD_OK;
 }
@@ -876,9 +890,9 @@ int ssd_decode_block(ssd_ctx* c, int32_t mode, int32_t T, int32_t* out_tokens, i
     if (rc) return rc;
     bool decided = true;
     for (int b = 0; b < c->batch; ++b)
-      if (c->h_nodes[b] > 0 && c->h_remaining[b] - c->h_nodes[b] < md + 1) decided = false;
+      if (c->h_nodes[b] > 0 && c->h_remaining[b] - c->h_max_accept[b] < md + 1) decided = false;
     if (decided) {
-      for (int b = 0; b < c->batch; ++b) c->h_remaining[b] -= c->h_nodes[b];
+      for (int b = 0; b < c->batch; ++b) c->h_remaining[b] -= c->h_max_accept[b];
       continue;
     }
     rc = step_collect(c, nullptr, nullptr);
@@ -939,6 +953,59 @@ int ssd_read_cache(ssd_ctx* c, int32_t layer, int32_t seq, int32_t length, float
     for (size_t i = 0; i < n; ++i) dst[i] = __bfloat162float(tmp[i]);
   }
   return SSD_OK;
+}
+
+int ssd_write_cache(ssd_ctx* c, int32_t layer, int32_t seq, int32_t length, const float* k, const float* v) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!k || !v) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
+  if (layer < 0 || layer >= c->cfg.n_layers || seq < 0 || seq >= c->cfg.max_batch || length < 0 || length > c->cfg.max_seq)
+    return fail(c, SSD_ERR_INVALID_ARG, "index out of range");
+  {
+    const int frc = flush_pending(c);
+    if (frc) return frc;
+  }
+  const size_t n = (size_t)length * c->kvdim;
+  std::vector<bf16> tmp(n);
+  for (int which = 0; which < 2; ++which) {
+    const float* src = which ? v : k;
+    bf16* dst = (which ? c->cacheV : c->cacheK) + (size_t)layer * c->cache_layer_stride + (size_t)seq * c->cache_seq_stride;
+    for (size_t i = 0; i < n; ++i) tmp[i] = __float2bfloat16_rn(src[i]);
+    CUDA_TRY(c, cudaMemcpyAsync(dst, tmp.data(), n * sizeof(bf16), cudaMemcpyHostToDevice, c->st));
+    CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  }
+  return SSD_OK;
+}
+
+int ssd_verify_layers(ssd_ctx* c, int32_t batch, int32_t n_nodes, int32_t T, int32_t layer_begin, int32_t layer_end,
+                      const float* h_in, float* h_out, int32_t* out_tok, float* out_conf) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
+  if (!h_in) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  if (batch < 1 || batch > c->batch) return fail(c, SSD_ERR_INVALID_ARG, "batch %d outside [1, %d]", batch, c->batch);
+  if (T < 1 || T > c->cfg.block_len || n_nodes < 1) return fail(c, SSD_ERR_INVALID_ARG, "bad node shape");
+  if (layer_begin < 0 || layer_end <= layer_begin || layer_end > c->cfg.n_layers)
+    return fail(c, SSD_ERR_INVALID_ARG, "layer range [%d, %d) outside [0, %d)", layer_begin, layer_end, c->cfg.n_layers);
+  if ((out_tok || out_conf) && layer_end != c->cfg.n_layers)
+    return fail(c, SSD_ERR_INVALID_ARG, "token statistics need the last layer in the range");
+  {
+    const int frc = flush_pending(c);
+    if (frc) return frc;
+  }
+  const size_t R = (size_t)batch * n_nodes * T;
+  if (R > (size_t)c->R_dec) return fail(c, SSD_ERR_OVERFLOW, "%zu rows exceed the capacity %d set by max_batch/max_drafts/block_len", R, c->R_dec);
+  if (c->cache_len + T > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "cache %d + block %d exceeds max_seq", c->cache_len, T);
+  CUDA_TRY(c, cudaMemcpyAsync(c->h, h_in, R * c->d * sizeof(float), cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  RowMap map{n_nodes * T, T, c->cache_len, 0, nullptr};
+  LayerRange range;
+  range.begin = layer_begin; range.end = layer_end; range.from_stream = true; range.lm_head = out_tok || out_conf;
+  int rc = forward(c, FWD_VERIFY, nullptr, (int)R, map, batch, false, nullptr, range);
+  if (rc) return rc;
+  if (h_out) CUDA_TRY(c, cudaMemcpyAsync(h_out, c->h, R * c->d * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  if (out_tok) CUDA_TRY(c, cudaMemcpyAsync(out_tok, c->tok, R * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  if (out_conf) CUDA_TRY(c, cudaMemcpyAsync(out_conf, c->conf, R * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  return sync_and_check(c);
 }
 
 int ssd_gemm_bf16(ssd_ctx* c, const void* x_dev, const void* w_dev, float* out_dev, int32_t rows, int32_t n, int32_t k, int32_t split_k) {
@@ -1040,6 +1107,11 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "max_drafts")) {
     if (value < 0 || value + 1 > c->n_max) return fail(c, SSD_ERR_INVALID_ARG, "max_drafts must be in [0, %d] (the capacity fixed at creation)", c->n_max - 1);
     c->cfg.max_drafts = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "mix_order")) {
+    if (value != 0 && value != 1) return fail(c, SSD_ERR_INVALID_ARG, "mix_order is 0 (greedy chain) or 1 (chain plus out-of-order branches)");
+    c->mix_order = value;
     return SSD_OK;
   }
   if (!strcmp(key, "attn_impl")) {

@@ -1,23 +1,28 @@
 """CUDA path at the widths and sizes the benchmark runs (run with -m gpu on a B200).
 
-Two kinds of checks, because a full-depth fp64 oracle forward of an 8B-parameter model does not
-finish in seconds:
+Three kinds of checks:
   * full WIDTH, two layers, reduced vocabulary: element-by-element parity with the CPU oracle for the
-    LLaDA-8B-shaped, the Dream-7B-shaped (grouped KV heads) and the long-context launch shapes.
-    The stated tolerance (logits 2e-2 absolute, confidences 2e-2 relative) is quoted at config 1,
-    whose logits have standard deviation 0.02 * sqrt(256) = 0.32.  At d = 3584 / 4096 the logits are
-    four times larger (0.02 * sqrt(d) = 1.2 / 1.28) and so is the rounding noise of bf16 operands
-    (every contraction rounds its activations to 8 bits of mantissa: 2^-9 / sqrt(3) relative per
-    stage; both projection kernels of this library, and the bf16-operand oracle against either of
-    them, sit at 0.7-0.9 % of the logit scale rms, 3.5-5 % at the maximum over 4e5 logits).  The
-    tolerance is therefore kept at the same fraction of the logit scale: 2e-2 * std / 0.32, as the
-    tests of the scaled-LM-head variant already do; tokens are compared where the oracle's gap is safe;
-  * full SIZE (all layers, full vocabulary, the launch configuration bench.py times): properties
-    that hold at any size - SSD tokens == stepwise tokens bit for bit, a node's outputs do not depend
-    on the nodes it shares a forward with, accept counts are a valid decomposition of the block.
-"""
-import os
+    LLaDA-8B-shaped, the Dream-7B-shaped (grouped KV heads) and the long-context launch shapes, plain and
+    "peaked" (LM head scaled so that top-1/top-2 gaps are common and the exact-token rule bites);
+  * full DEPTH: all 32 layers and the full vocabulary of the benchmarked model against the oracle, once
+    free-running and once layer by layer from the oracle's own residual stream and prefix K/V;
+  * full SIZE in the launch configuration bench.py times: properties that hold at any size - SSD tokens
+    == stepwise tokens bit for bit, a node's outputs do not depend on the nodes it shares a forward
+    with, accept counts are a valid decomposition of the block.
 
+Tolerance.  The stated bar is 2e-2 absolute on logits / 2e-2 relative on confidences for bf16 operands
+with fp32 accumulation; it is asserted as stated wherever the logits are of the scale it is quoted at
+(config 1, standard deviation 0.02 * sqrt(256) = 0.32).  At d = 3584 / 4096 the logits are four times
+larger (std 1.2 - 1.28), and bf16 operands (8 bits of mantissa) cannot hold an absolute 2e-2 there: the
+ORACLE ITSELF, run with its operands rounded to bf16, is further than that from its own unrounded
+result (two layers: 0.010 rms / 0.05 maximum over 4e5 logits at std 1.28; 32 layers: see
+test_full_depth_*).  The bound used here is therefore the arithmetic's own: the CUDA path may be no
+further from the unrounded fp64 oracle than NOISE_RMS (rms) / NOISE_MAX (maximum) times the distance of
+the bf16-operand oracle from it, both measured in the same test on the same inputs.  The factors leave
+room for the roundings the kernels add to the oracle's (fp32 accumulation, probabilities rounded
+relative to a key part's maximum, the RMSNorm applied after the contraction) and for the statistics of a
+maximum.  Tokens are compared wherever the oracle's gap exceeds 1e-3 and the logit bound cannot flip it.
+"""
 import numpy as np
 import pytest
 import torch
@@ -28,8 +33,22 @@ from tests.helpers import make_oracle
 pytestmark = pytest.mark.gpu
 
 GAP = 1e-3
-CONF_RTOL = 2e-2
-TINY_LOGIT_STD = 0.32        # 0.02 * sqrt(256): the logit scale the stated tolerances are quoted at
+STATED_TOL = 2e-2            # logits absolute / confidences relative, quoted at logit std 0.32
+TINY_LOGIT_STD = 0.32
+NOISE_RMS = 1.25             # CUDA-vs-oracle error as a multiple of the bf16-operand oracle's own distance
+NOISE_MAX = 1.5
+
+
+def _noise_bounds(ologits_plain, ologits_bf16):
+    """(rms bound, max bound) for logits of the CUDA path against the unrounded oracle."""
+    d = ologits_bf16 - ologits_plain
+    return NOISE_RMS * float(np.sqrt((d ** 2).mean())), NOISE_MAX * float(np.abs(d).max())
+
+
+def _sure_tokens(ogap, oconf, e_max):
+    """Rows whose argmax cannot be flipped by logit errors up to e_max: the oracle's top-1/top-2
+    probability gap exceeds 1e-3 and the log-ratio of the two exceeds 2 * e_max."""
+    return (ogap > GAP) & (ogap > (1.0 - np.exp(-2.0 * e_max)) * oconf)
 
 
 def _binding():
@@ -58,6 +77,11 @@ WIDTH_CASES = {
     # long prefix, 64-token blocks: several 128-key steps per attention part, double-buffered K/V
     "long_width": (wl.LLADA_8B_LONG.replace(name="long_width", n_layers=1, vocab=2048, prompt_len=1100, gen_len=128,
                                             batch=1), 2),
+    # "peaked": LM head x 4, so that most rows have a top-1/top-2 gap the rounding noise cannot flip
+    "llada_width_peaked": (wl.LLADA_8B.replace(name="llada_width_peaked", n_layers=2, vocab=4096, prompt_len=160,
+                                               gen_len=64, lm_head_scale=4.0), 3),
+    "dream_width_peaked": (wl.DREAM_7B.replace(name="dream_width_peaked", n_layers=2, vocab=4096, prompt_len=200,
+                                               gen_len=64, lm_head_scale=4.0), 2),
 }
 
 
@@ -79,20 +103,33 @@ def test_full_width_forward_matches_oracle(case):
         tok2, conf2, _ = ssd.verify_forward(ids, masked)     # fused LM-head statistics
     finally:
         ssd.destroy()
-    o = make_oracle(w, as_bf16=True)                         # fp64 arithmetic on the bf16 weight values
-    cache = o.prefill(prompt[0])
-    o.commit_block(blk[0], cache)
-    otok, oconf, ogap, ologits = o.verify(ids[0], masked[0], cache)
-    scale = max(1.0, float(ologits.std()) / TINY_LOGIT_STD)       # logit scale relative to config 1
-    err = np.abs(logits[0] - ologits)
-    assert err.max() < 2e-2 * scale, (err.max(), scale)
-    assert np.sqrt((err ** 2).mean()) < 4e-3 * scale             # and it is noise, not a bias: rms 5x below
+    res = {}
+    for mode in (None, "bf16"):                              # fp64 arithmetic on the bf16 weight values
+        o = make_oracle(w, as_bf16=True, operand_rounding=mode)
+        cache = o.prefill(prompt[0])
+        o.commit_block(blk[0], cache)
+        res[mode] = o.verify(ids[0], masked[0], cache)
+    otok, oconf, ogap, ologits = res[None]
+    rms_bound, max_bound = _noise_bounds(ologits, res["bf16"][3])
+    err = logits[0] - ologits
+    rms, mx = float(np.sqrt((err ** 2).mean())), float(np.abs(err).max())
     m = masked[0]
-    assert np.allclose(conf[0][m], oconf[m], rtol=CONF_RTOL * scale, atol=1e-6)
-    assert np.allclose(conf2[0][m], oconf[m], rtol=CONF_RTOL * scale, atol=1e-6)
-    sure = m & (ogap > GAP) & (ogap > 2 * CONF_RTOL * scale * oconf)
+    sure = m & _sure_tokens(ogap, oconf, max_bound)
+    print(f"{case}: logit std {ologits.std():.3f}; CUDA vs fp64 oracle rms {rms:.4f} max {mx:.4f}; bf16-operand oracle "
+          f"vs fp64 oracle rms {rms_bound / NOISE_RMS:.4f} max {max_bound / NOISE_MAX:.4f}; stated {STATED_TOL} "
+          f"{'met' if mx < STATED_TOL else 'not attainable with bf16 operands at this logit scale'}; "
+          f"sure rows {int(sure.sum())} of {int(m.sum())}")
+    assert rms < rms_bound and mx < max_bound, (rms, rms_bound, mx, max_bound)
+    if ologits.std() <= 1.25 * TINY_LOGIT_STD:
+        assert mx < STATED_TOL
+    # a logit error e moves a softmax probability by a factor within exp(+-2e)
+    rtol = np.exp(2.0 * max_bound) - 1.0
+    assert np.allclose(conf[0][m], oconf[m], rtol=rtol, atol=1e-6)
+    assert np.allclose(conf2[0][m], oconf[m], rtol=rtol, atol=1e-6)
     assert np.array_equal(tok[0][sure], otok[sure])
     assert np.array_equal(tok2[0][sure], otok[sure])
+    if w.lm_head_scale > 1:
+        assert sure.sum() > 0.25 * m.sum()                   # the peaked variants make the token rule bite
     assert np.all(tok2[0][~m] == -1)
 
 
@@ -126,41 +163,67 @@ def test_full_size_ssd_equals_stepwise_and_accounts_for_the_block(llada_full):
     assert ssd.cache_length() == w.prompt_len + B
 
 
-@pytest.mark.skipif(os.environ.get("SSD_FULL_DEPTH_ORACLE") != "1",
-                    reason="minutes of CPU work (two fp64 passes over 8 B parameters): set SSD_FULL_DEPTH_ORACLE=1")
-def test_full_depth_forward_matches_oracle(llada_full):
-    """All 32 layers and the full vocabulary against the oracle, on a short prompt so that the oracle's
-    prefill stays affordable: one root forward (all 32 positions masked) after an 8-token prefill.
-    Tolerance: the full-width tests hold two layers to 2e-2 of the logit scale.  The rounding of bf16
-    operands is independent noise added to the residual stream layer after layer (kernel and oracle
-    round different intermediates), so its rms grows like sqrt(layers): sqrt(32 / 2) = 4 times the
-    two-layer bound.  Measured on B200: confidence relative error 0.089 max, 0.033 mean (logit std
-    1.28), 31 of 32 argmax tokens equal on a random-init model whose top-1 margins are ~1e-4."""
-    from tests.helpers import LazyWeights, oracle_config
-    from oracle.ssd_oracle import Oracle
+def test_full_depth_forward_and_every_layer_match_oracle(llada_full):
+    """All 32 layers and the full vocabulary of the benchmarked model against the oracle, on a short
+    prompt so that the oracle stays affordable (one pass over the 8 B parameters for the unrounded and the
+    bf16-operand arithmetic together): one root forward, all 32 positions masked, after an 8-token prefill.
+      free-running  - logits / confidences of the CUDA forward against the unrounded oracle, bounded by the
+                      bf16-operand oracle's own distance from it (module docstring);
+      layer by layer - every layer of the CUDA path is run from the ORACLE's residual stream and the
+                      ORACLE's prefix K/V for that layer, so rounding noise cannot compound and a wrong
+                      layer cannot hide behind it: the update a layer adds to the stream must agree
+                      with the oracle's to a small fraction of its size, the same for all 32 layers."""
+    from tests.helpers import LayerCachedWeights, lockstep_root_forward
     w, ssd = llada_full
     P8 = 8
     prompt = wl.make_prompts(w).numpy()[:, :P8]
     T = w.block_len
     ids = np.full((1, 1, T), w.mask_id)
     masked = np.ones((1, 1, T), bool)
+    ref = lockstep_root_forward(w, LayerCachedWeights(w, "cuda"), prompt[0], ids[0, 0], (None, "bf16"))
+    plain, rounded = ref[None], ref["bf16"]
     try:
         ssd.prefill(prompt)
-        tok, conf, _ = ssd.verify_forward(ids, masked)
+        tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
+        tok2, conf2, _ = ssd.verify_forward(ids, masked)
+        # ---- layer by layer, teacher-forced from the bf16-operand oracle (its K/V are bf16 values)
+        for l in range(w.n_layers):
+            ssd.write_cache(l, 0, rounded["prefix_k"][l], rounded["prefix_v"][l])
+        worst = (0.0, -1)
+        for l in range(w.n_layers):
+            h_in, h_ref = rounded["hidden"][l], rounded["hidden"][l + 1]
+            h_out, _, _ = ssd.verify_layers(h_in, 1, 1, T, l, l + 1)
+            upd, upd_ref = h_out - h_in.astype(np.float32), h_ref - h_in
+            rel = float(np.sqrt(((upd - upd_ref) ** 2).mean()) / np.sqrt((upd_ref ** 2).mean()))
+            worst = max(worst, (rel, l))
+            # bf16 operands: 2^-9 relative per rounded operand, a handful of independent roundings per layer
+            assert rel < 1e-2, (l, rel)
+            assert np.abs(upd - upd_ref).max() < 0.1 * np.abs(upd_ref).max(), l
+        _, tok_l, conf_l = ssd.verify_layers(rounded["hidden"][w.n_layers - 1], 1, 1, T, w.n_layers - 1, w.n_layers,
+                                             want_stats=True)
     finally:
         ssd.prefill_dev(wl.make_prompts(w, "cuda"))          # what the other tests of this module expect
-    o = Oracle(oracle_config(w), LazyWeights(w, "cuda"), "bf16")
-    cache = o.prefill(prompt[0])
-    otok, oconf, ogap, ologits = o.verify(ids[0], masked[0], cache)
-    scale = max(1.0, float(ologits.std()) / TINY_LOGIT_STD)
-    rel = np.abs(conf[0, 0] / oconf[0] - 1.0)
-    print(f"full depth: logit std {ologits.std():.3f}, confidence relative error max {rel.max():.4f} "
-          f"mean {rel.mean():.4f}, tokens equal {int((tok[0, 0] == otok[0]).sum())} of {T}")
-    rtol = CONF_RTOL * scale * np.sqrt(w.n_layers / 2.0)
-    assert np.allclose(conf[0, 0], oconf[0], rtol=rtol, atol=1e-6)
-    assert rel.mean() < rtol / 4                                  # noise around the oracle, not a bias
-    sure = (ogap[0] > GAP) & (ogap[0] > 2 * rtol * oconf[0])
-    assert np.array_equal(tok[0, 0][sure], otok[0][sure])
+    from oracle.ssd_oracle import token_and_confidence, top2_gap
+    otok, oconf = token_and_confidence(plain["logits"], w.mask_id)
+    ogap = top2_gap(plain["logits"], w.mask_id)
+    rtok, rconf = token_and_confidence(rounded["logits"], w.mask_id)
+    rms_bound, max_bound = _noise_bounds(plain["logits"], rounded["logits"])
+    err = logits[0, 0] - plain["logits"]
+    rms, mx = float(np.sqrt((err ** 2).mean())), float(np.abs(err).max())
+    rel_conf = np.abs(conf[0, 0] / oconf - 1.0)
+    sure = _sure_tokens(ogap, oconf, max_bound)
+    print(f"full depth: logit std {plain['logits'].std():.3f}; CUDA vs fp64 oracle rms {rms:.4f} max {mx:.4f}; "
+          f"bf16-operand oracle vs fp64 oracle rms {rms_bound / NOISE_RMS:.4f} max {max_bound / NOISE_MAX:.4f}; "
+          f"confidence relative error max {rel_conf.max():.4f} mean {rel_conf.mean():.4f}; tokens equal "
+          f"{int((tok[0, 0] == otok).sum())} of {T} (bf16-operand oracle: {int((rtok == otok).sum())}); sure rows "
+          f"{int(sure.sum())}; worst layer update error {worst[0]:.4f} at layer {worst[1]}")
+    assert rms < rms_bound and mx < max_bound, (rms, rms_bound, mx, max_bound)
+    rtol = np.exp(2.0 * max_bound) - 1.0
+    assert np.allclose(conf[0, 0], oconf, rtol=rtol, atol=1e-6)
+    assert np.allclose(conf2[0, 0], oconf, rtol=rtol, atol=1e-6)
+    assert np.array_equal(tok[0, 0][sure], otok[sure]) and np.array_equal(tok2[0, 0][sure], otok[sure])
+    # the last layer + LM head from the oracle's stream: one layer of noise only
+    assert np.allclose(conf_l[0, 0], rconf, rtol=5 * STATED_TOL, atol=1e-6)
 
 
 def test_full_size_row_invariance(llada_full):
@@ -254,9 +317,9 @@ def test_extreme_blocks_ssd_equals_stepwise_and_oracle_steps(block_len, prompt_l
         cache = o.prefill(prompt[0])
         o.commit_block(tok_step[0, :first], cache)
         otok, oconf, ogap, _ = o.verify(ids[0, 0][None], np.ones((1, T), bool), cache)
-        scale = w.lm_head_scale
-        assert np.allclose(conf_g[0, 0], oconf[0], rtol=CONF_RTOL * scale, atol=1e-6)
-        sure = (ogap[0] > GAP) & (ogap[0] > 2 * CONF_RTOL * scale * oconf[0])
+        tol = STATED_TOL * w.lm_head_scale        # config-1 width; the scaled LM head scales logits and their errors alike
+        assert np.allclose(conf_g[0, 0], oconf[0], rtol=tol, atol=1e-6)
+        sure = _sure_tokens(ogap[0], oconf[0], tol)
         assert np.array_equal(tok_g[0, 0][sure], otok[0][sure])
 
 
@@ -300,10 +363,16 @@ def test_both_attention_forms_agree_at_full_width():
             out[impl] = (tok, conf, logits)
     finally:
         ssd.destroy()
-    # the same fraction of the logit scale as the comparison with the oracle (module docstring)
-    scale = max(1.0, float(out[0][2].std()) / TINY_LOGIT_STD)
-    diff = out[0][2] - out[1][2]
-    assert np.abs(diff).max() < 2e-2 * scale, (np.abs(diff).max(), scale)
-    assert np.sqrt((diff ** 2).mean()) < 4e-3 * scale          # noise, not a bias
+    # both forms stay within the bf16-operand noise of the oracle (module docstring), so they differ from each
+    # other by at most twice that
+    prm = prompt[0]
+    ol = {}
+    for mode in (None, "bf16"):
+        o = make_oracle(w, as_bf16=True, operand_rounding=mode)
+        ol[mode] = o.verify(ids[0], masked[0], o.prefill(prm))[3]
+    rms_bound, max_bound = _noise_bounds(ol[None], ol["bf16"])
+    diff = out[0][2][0] - out[1][2][0]
+    assert np.abs(diff).max() < 2 * max_bound, (np.abs(diff).max(), max_bound)
+    assert np.sqrt((diff ** 2).mean()) < 2 * rms_bound
     m = masked[0]
-    assert np.allclose(out[0][1][0][m], out[1][1][0][m], rtol=CONF_RTOL * scale, atol=1e-6)
+    assert np.allclose(out[0][1][0][m], out[1][1][0][m], rtol=np.exp(4.0 * max_bound) - 1.0, atol=1e-6)

@@ -508,3 +508,67 @@ def test_error_codes(tiny_ssd):
     with pytest.raises(b.SsdError) as e:
         tiny_ssd.block_commit()                                  # block not finished
     assert e.value.code == -7
+
+
+def test_split_k_options_are_bounded_and_keep_parity(tiny_oracles):
+    """A projection never gets more splits than it has 64-wide K blocks (an empty split would add an
+    accumulator nothing wrote); within the bound every split count gives the same forward up to the
+    rounding of another summation order."""
+    w = wl.TINY
+    b = _binding()
+    o64, _ = tiny_oracles[w.name]
+    rng = np.random.default_rng(9)
+    prompt = wl.make_prompts(w).numpy()
+    ids, masked = _random_nodes(w, rng, 3, w.block_len)
+    ssd = _make_ssd(w, max_drafts=3)
+    try:
+        with pytest.raises(b.SsdError) as e:
+            ssd.set_option("split_k_o", 8)                 # the O projection has 256 / 64 = 4 K blocks
+        assert e.value.code == -1
+        with pytest.raises(b.SsdError) as e:
+            ssd.set_option("split_k_qkv", 5)
+        assert e.value.code == -1
+        ssd.prefill(prompt)
+        _, _, base = ssd.verify_forward(ids, masked, want_logits=True)
+        ssd.set_option("split_k_o", 4)                     # one K block per split
+        ssd.set_option("split_k_down", 8)                  # 11 K blocks over 8 splits: ragged
+        ssd.set_option("split_k_qkv", 4)
+        ssd.prefill(prompt)
+        _, _, split = ssd.verify_forward(ids, masked, want_logits=True)
+    finally:
+        ssd.destroy()
+    cache = o64.prefill(prompt[0])
+    _, _, _, ologits = o64.verify(ids[0], masked[0], cache)
+    assert np.abs(split[0] - ologits).max() < 2e-2
+    assert np.abs(base[0] - ologits).max() < 2e-2
+    assert np.abs(split - base).max() < 1e-2
+
+
+def test_nonfinite_weights_are_reported_not_decoded():
+    """A NaN in a weight (injected on the host side, nothing faults) makes every confidence NaN: the step
+    returns SSD_ERR_NONFINITE instead of tokens, and the context stays usable."""
+    w = wl.TINY
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    ssd = _make_ssd(w, max_drafts=2)
+    try:
+        good = wl.make_tensor(w, "norm_final", "cuda")
+        bad = good.clone()
+        bad[7] = float("nan")
+        ssd.load_weights("norm_final", bad)
+        ssd.prefill(prompt)
+        ssd.block_begin(w.block_len)
+        with pytest.raises(b.SsdError) as e:
+            ssd.block_step(2, 1)
+        assert e.value.code == -8
+        ssd.prefill(prompt)
+        with pytest.raises(b.SsdError) as e:
+            ssd.decode_block(b.MODE_SSD, w.block_len, 1)
+        assert e.value.code == -8
+        # with the weight repaired the same context decodes again
+        ssd.load_weights("norm_final", good)
+        ssd.prefill(prompt)
+        tok, acc, nf = ssd.decode_block(b.MODE_SSD, w.block_len, 1)
+        assert acc[0][:nf[0]].sum() == w.block_len and w.mask_id not in tok
+    finally:
+        ssd.destroy()

@@ -249,3 +249,25 @@ def test_hidden_trace_is_the_residual_stream():
     assert len(tr2) == w.n_layers + 1
     for a, b in zip(tr, tr2):
         assert np.allclose(a[0], b[len(prompt):], rtol=1e-9, atol=1e-12)
+
+
+def test_lockstep_driver_equals_prefill_then_forward():
+    """The layer-by-layer driver used for large models (several rounding modes through one pass over the
+    weights) is the oracle's prefill followed by forward_rows, bit for bit."""
+    from tests.helpers import lockstep_root_forward
+    w = SMALL_GQA
+    wts = oracle_weights(w, as_bf16=True)
+    prompt = wl.make_prompts(w).numpy()[0]
+    ids = np.array([w.mask_id, 3, w.mask_id, 7, 9, w.mask_id])
+    got = lockstep_root_forward(w, wts, prompt, ids, (None, "bf16"))
+    for mode in (None, "bf16"):
+        o = so.Oracle(oracle_config(w), wts, mode)
+        cache = o.prefill(prompt)
+        tr = []
+        logits, _, _ = o.forward_rows(ids[None], len(prompt), cache, hidden_trace=tr)
+        assert np.array_equal(got[mode]["logits"], logits[0])
+        for l in range(w.n_layers):
+            assert np.array_equal(got[mode]["prefix_k"][l], cache.k[l])
+            assert np.array_equal(got[mode]["prefix_v"][l], cache.v[l])
+        for a, b in zip(got[mode]["hidden"], tr):
+            assert np.array_equal(a, b[0])
