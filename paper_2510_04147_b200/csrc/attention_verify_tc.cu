@@ -8,9 +8,11 @@
 //     S[row, key] = Q[row, :] . K[key, :]        (A = Q, B = K, both K-major over the head dimension)
 //     O[row, :]   = P[row, :] . V[:, :]          (A = P, K-major over the keys; B = V as stored,
 //                                                 [key][hd]: the MN-major operand form)
-// A thread owns one query row (= one TMEM lane): the softmax of a row is thread-local, no shuffles,
-// and no accumulator lives in registers, so 32, 64 or 128 rows per CTA cost the same 128 threads and
-// the grid stays at parts x heads CTAs per 128 rows - one wave for the chains SSD runs.
+// A query row is one TMEM lane, shared by two threads (warps w and w + 4 read the same lane quadrant),
+// each owning half of the lane's columns: the softmax needs no shuffles, only one exchange of the row
+// maximum through shared memory, and no accumulator lives in registers, so 32, 64 or 128 rows per CTA
+// cost the same 256 threads and the grid stays at parts x heads CTAs per 128 rows - one wave for the
+// chains SSD runs.
 //
 // Shared-memory tiles are [64-column half][128 rows][64 columns] bf16 with the 128-byte swizzle the
 // tensor core expects (16-byte chunk c of row r at chunk c ^ (r & 7)).  A query tile of 32 or 64
@@ -30,7 +32,7 @@ using namespace attn;
 
 constexpr int kHD = 128;
 constexpr int kKeys = 128;                  // keys per MMA tile
-constexpr int kTcAttnThreads = 128;
+constexpr int kTcAttnThreads = 256;       // two threads per TMEM lane (= query row copy): each takes half of the lane's columns
 constexpr int kHalfBytesKV = kKeys * 128;   // one 64-column half of a 128-row tile
 constexpr unsigned long long kAttnWaitLimitNs = 2000000000ull;
 
@@ -86,34 +88,28 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uin
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// 16 consecutive columns of the thread's lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
-// the inverse of tmem_ld32: the thread's lane, 32 consecutive columns
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
-  uint32_t r[32];
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) {
+  uint32_t r[16];
 #pragma unroll
-  for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+  for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(v[i]);
   asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
       ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
@@ -157,9 +153,9 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   uint8_t* sQ = smem;                                   // [2][128][64] bf16
   uint8_t* sK = sQ + 2 * kHalfBytesKV;                  // [2][128][64]; P overwrites it once S is complete
   uint8_t* sV = sK + 2 * kHalfBytesKV;                  // [2][128][64]
-  float* sMax = reinterpret_cast<float*>(sV + 2 * kHalfBytesKV);         // [4 copies][128 rows]
-  float* sSum = sMax + 4 * 128;                                          // [4 key groups][128 rows]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sSum + 4 * 128);          // [0] S ready, [1] O ready
+  float* sMax = reinterpret_cast<float*>(sV + 2 * kHalfBytesKV);         // [2 halves x 4 copies][128 rows]
+  float* sSum = sMax + 8 * 128;                                          // [8 chunks of 16 keys][128 rows]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sSum + 8 * 128);          // [0] S ready, [1] O ready
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2);
   constexpr int HALF = kHD / 2, CPR = HALF / 8, CH = kHD / 8;
 
@@ -244,8 +240,8 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
         *reinterpret_cast<uint4*>(sV + tile_off(row, ch, kKeys)) = zero;
       }
     }
-    // A thread takes its work items two at a time: the split-K partials of both are requested before
-    // either is used, so the two L2 round trips overlap.
+    // A work item = one 16-byte chunk of a row (with its rotation partner for Q and K).  All split-K
+    // partials of an item are requested before the first is used, so their L2 round trips overlap.
     struct Item { int kind, row, c; const float* pr; const float4* cs4; };   // kind 0 Q, 1 K, 2 V, -1 none
     auto decode = [&](int it) -> Item {
       Item w{-1, 0, 0, nullptr, nullptr};
@@ -267,34 +263,28 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       return w;
     };
     // sums over the splits in split order: x1 = the chunk itself, x2 = its rotation partner (rotary items)
-    auto gather2 = [&](const Item& A, const Item& B, float (&xa1)[8], float (&xa2)[8], float (&xb1)[8], float (&xb2)[8]) {
+    auto gather = [&](const Item& A, float (&x1)[8], float (&x2)[8]) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { xa1[j] = xa2[j] = xb1[j] = xb2[j] = 0.f; }
-      const bool la = A.pr != nullptr, lb = B.pr != nullptr;
-      const bool ra = la && A.kind != 2, rb = lb && B.kind != 2;
+      for (int j = 0; j < 8; ++j) { x1[j] = x2[j] = 0.f; }
+      const bool la = A.pr != nullptr;
+      const bool ra = la && A.kind != 2;
       for (int s0 = 0; s0 < a.qkv_splits; s0 += 4) {
-        float4 a0[4], a1[4], a2[4], a3[4], b0[4], b1[4], b2[4], b3[4];
+        float4 a0[4], a1[4], a2[4], a3[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          a0[u] = a1[u] = a2[u] = a3[u] = b0[u] = b1[u] = b2[u] = b3[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          a0[u] = a1[u] = a2[u] = a3[u] = make_float4(0.f, 0.f, 0.f, 0.f);
           const bool on = s0 + u < a.qkv_splits;
           const size_t off = (size_t)(s0 + u) * a.qkv_split_stride;
           if (on && la) { a0[u] = *reinterpret_cast<const float4*>(A.pr + off); a1[u] = *reinterpret_cast<const float4*>(A.pr + off + 4); }
           if (on && ra) { a2[u] = *reinterpret_cast<const float4*>(A.pr + off + HALF); a3[u] = *reinterpret_cast<const float4*>(A.pr + off + HALF + 4); }
-          if (on && lb) { b0[u] = *reinterpret_cast<const float4*>(B.pr + off); b1[u] = *reinterpret_cast<const float4*>(B.pr + off + 4); }
-          if (on && rb) { b2[u] = *reinterpret_cast<const float4*>(B.pr + off + HALF); b3[u] = *reinterpret_cast<const float4*>(B.pr + off + HALF + 4); }
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           if (s0 + u < a.qkv_splits) {
-            xa1[0] += a0[u].x; xa1[1] += a0[u].y; xa1[2] += a0[u].z; xa1[3] += a0[u].w;
-            xa1[4] += a1[u].x; xa1[5] += a1[u].y; xa1[6] += a1[u].z; xa1[7] += a1[u].w;
-            xa2[0] += a2[u].x; xa2[1] += a2[u].y; xa2[2] += a2[u].z; xa2[3] += a2[u].w;
-            xa2[4] += a3[u].x; xa2[5] += a3[u].y; xa2[6] += a3[u].z; xa2[7] += a3[u].w;
-            xb1[0] += b0[u].x; xb1[1] += b0[u].y; xb1[2] += b0[u].z; xb1[3] += b0[u].w;
-            xb1[4] += b1[u].x; xb1[5] += b1[u].y; xb1[6] += b1[u].z; xb1[7] += b1[u].w;
-            xb2[0] += b2[u].x; xb2[1] += b2[u].y; xb2[2] += b2[u].z; xb2[3] += b2[u].w;
-            xb2[4] += b3[u].x; xb2[5] += b3[u].y; xb2[6] += b3[u].z; xb2[7] += b3[u].w;
+            x1[0] += a0[u].x; x1[1] += a0[u].y; x1[2] += a0[u].z; x1[3] += a0[u].w;
+            x1[4] += a1[u].x; x1[5] += a1[u].y; x1[6] += a1[u].z; x1[7] += a1[u].w;
+            x2[0] += a2[u].x; x2[1] += a2[u].y; x2[2] += a2[u].z; x2[3] += a2[u].w;
+            x2[4] += a3[u].x; x2[5] += a3[u].y; x2[6] += a3[u].z; x2[7] += a3[u].w;
           }
         }
       }
@@ -342,13 +332,12 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     };
     const int stride = n_parts * kTcAttnThreads;
     bool waited = false;
-    for (int it = part * kTcAttnThreads + tid; it < n_q + n_k + n_v; it += 2 * stride) {
-      const Item A = decode(it), B = decode(it + stride);
-      float xa1[8], xa2[8], xb1[8], xb2[8];
-      gather2(A, B, xa1, xa2, xb1, xb2);
+    for (int it = part * kTcAttnThreads + tid; it < n_q + n_k + n_v; it += stride) {
+      const Item A = decode(it);
+      float x1[8], x2[8];
+      gather(A, x1, x2);
       if (!waited) { cluster_wait(); waited = true; }      // remote stores only once every CTA of the cluster runs
-      finish(A, xa1, xa2);
-      finish(B, xb1, xb2);
+      finish(A, x1, x2);
     }
     if (!waited) cluster_wait();
     asm volatile("fence.proxy.async;" ::: "memory");      // these stores are read by the tensor core
@@ -375,12 +364,17 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   // f32 accumulate, bf16 operands, N = 128, M = 128; bit 16: B is MN-major (V as stored, [key][hd])
   const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
-  // ---- softmax, log2 domain.  Thread = TMEM lane: copy `cw` of query row `row`, keys [cw * QT, +QT) of
-  //      a tile.  The row maximum is exchanged between the copies through shared memory; a tile's row sum
-  //      is ALWAYS formed as ((g0 + g1) + g2) + g3 over the four 32-key groups, each group summed in key
-  //      order, whatever QT is - a row's bits do not depend on how many rows share the forward.
-  const int cw = tid / QT, row = tid % QT;
-  const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;       // warp w reads TMEM lanes 32w .. 32w + 31
+  // ---- softmax, log2 domain.  TMEM lane lt = copy `cw` of query row `row`; a copy covers the keys
+  //      [cw * QT, +QT) of a tile and the lane's two threads (hw = 0, 1) half of those each, in 16-key
+  //      chunks.  The row maximum is exchanged through shared memory; a tile's row sum is ALWAYS formed
+  //      from its eight 16-key chunks as (((c0 + c1) + (c2 + c3)) + (c4 + c5)) + (c6 + c7), each chunk
+  //      summed in key order, whatever QT is - a row's bits do not depend on how many rows share the forward.
+  constexpr int KPT = QT / 2;                           // keys of a tile per thread
+  constexpr int NCH = KPT / 16;                         // 16-key chunks per thread
+  const int lt = tid & 127, hw = tid >> 7;
+  const int cw = lt / QT, row = lt % QT;
+  const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;   // warps w and w + 4 read TMEM lanes 32 (w & 3) ...
+  const int col0 = cw * QT + hw * KPT;                  // first column (key of a tile) of this thread
   const int lr = lr0 + row;
   const bool row_live = lr < rps;
   int key_lo = k_begin, key_hi = k_end;                 // keys this row may see in this part
@@ -390,7 +384,6 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     // causal chain of two blocks: a row of the finished block does not see the next block
     if (a.map.chain_T0 > 0 && lr - key_lo < a.map.chain_T0) key_hi = min(key_hi, key_lo + a.map.chain_T0);
   }
-  constexpr int NG = QT / 32;                           // 32-key groups of a tile this thread owns
   float m_row = -INFINITY, l_row = 0.f;                 // running maximum and sum over the tiles so far
   bool ok = true;
 #pragma unroll 1
@@ -426,48 +419,45 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     if (!ok) break;
 
     float m_loc = -INFINITY;
-#pragma unroll 1
-    for (int g = 0; g < NG; ++g) {
-      const int c0 = cw * QT + g * 32;
-      float v[32];
-      tmem_ld32(tmem_S + lane_addr + c0, v);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
+    for (int ch = 0; ch < NCH; ++ch) {
+      const int c0 = col0 + ch * 16;
+      float v[16];
+      tmem_ld16(tmem_S + lane_addr + c0, v);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
         const int key = kb + c0 + j;
         if (key >= key_lo && key < key_hi) m_loc = fmaxf(m_loc, v[j] * scale_log2);
       }
     }
-    float m_tile = m_loc;
-    if (REP > 1) {
-      sMax[cw * 128 + row] = m_loc;
-      __syncthreads();
-      m_tile = -INFINITY;
+    sMax[(hw * 4 + cw) * 128 + row] = m_loc;
+    __syncthreads();
+    float m_tile = -INFINITY;
 #pragma unroll
-      for (int k = 0; k < REP; ++k) m_tile = fmaxf(m_tile, sMax[k * 128 + row]);
-    }
+    for (int k = 0; k < REP; ++k) m_tile = fmaxf(m_tile, fmaxf(sMax[k * 128 + row], sMax[(4 + k) * 128 + row]));
     const float m_new = fmaxf(m_row, m_tile);
     const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
     const float corr = exp2f(m_row - m_use);              // 0 for the first tile that holds a visible key
-#pragma unroll 1
-    for (int g = 0; g < NG; ++g) {
-      const int c0 = cw * QT + g * 32;
-      float v[32];
-      tmem_ld32(tmem_S + lane_addr + c0, v);
-      uint32_t packed[16];
-      float gsum = 0.f;
 #pragma unroll
-      for (int j = 0; j < 32; j += 2) {
+    for (int ch = 0; ch < NCH; ++ch) {
+      const int c0 = col0 + ch * 16;
+      float v[16];
+      tmem_ld16(tmem_S + lane_addr + c0, v);
+      uint32_t packed[8];
+      float csum = 0.f;
+#pragma unroll
+      for (int j = 0; j < 16; j += 2) {
         const int key = kb + c0 + j;
         const float p0 = (key >= key_lo && key < key_hi) ? exp2f(v[j] * scale_log2 - m_use) : 0.f;
         const float p1 = (key + 1 >= key_lo && key + 1 < key_hi) ? exp2f(v[j + 1] * scale_log2 - m_use) : 0.f;
-        gsum += p0;
-        gsum += p1;
+        csum += p0;
+        csum += p1;
         packed[j >> 1] = pack_bf16(p0, p1);
       }
-      sSum[(cw * NG + g) * 128 + row] = gsum;           // group index = c0 / 32
+      sSum[(c0 >> 4) * 128 + row] = csum;               // chunk index = c0 / 16
       // P overwrites K, in every copy of the row
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < 2; ++q) {
         const uint4 val = row_live ? make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3])
                                    : make_uint4(0, 0, 0, 0);
 #pragma unroll
@@ -478,14 +468,14 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     if (t > 0) {
       // the output so far was accumulated against the old maximum: rescale this thread's columns of its
       // lane (the columns it reads out at the end; the rest of a copy's lane is never read)
-#pragma unroll 1
-      for (int g = 0; g < NG; ++g) {
-        float v[32];
-        const uint32_t ta = tmem_O + lane_addr + cw * QT + g * 32;
-        tmem_ld32(ta, v);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] *= corr;
-        tmem_st32(ta, v);
+      for (int ch = 0; ch < NCH; ++ch) {
+        float v[16];
+        const uint32_t ta = tmem_O + lane_addr + col0 + ch * 16;
+        tmem_ld16(ta, v);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) v[j] *= corr;
+        tmem_st16(ta, v);
       }
     }
     cp_async_wait<0>();                                   // V of a later tile
@@ -509,7 +499,8 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     tc_fence_after();
     ok = __syncthreads_and(ok ? 1 : 0) != 0;              // every MMA is complete: shared memory is free
     if (!ok) break;
-    const float l_tile = ((sSum[0 * 128 + row] + sSum[1 * 128 + row]) + sSum[2 * 128 + row]) + sSum[3 * 128 + row];
+    const float l_tile = (((sSum[0 * 128 + row] + sSum[1 * 128 + row]) + (sSum[2 * 128 + row] + sSum[3 * 128 + row])) +
+                          (sSum[4 * 128 + row] + sSum[5 * 128 + row])) + (sSum[6 * 128 + row] + sSum[7 * 128 + row]);
     l_row = l_row * corr + l_tile;
     m_row = m_new;
   }
@@ -519,16 +510,16 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   float* sO = reinterpret_cast<float*>(smem);             // [QT][kPitch]
   float2* sML = reinterpret_cast<float2*>(sO + QT * kPitch);
   if (ok) {
-    // every copy of a row holds the same O row: copy cw stages the columns [cw * QT, +QT)
-    float v[NG][32];
+    // every copy of a row holds the same O row: a thread stages the columns it owns, [col0, +KPT)
 #pragma unroll
-    for (int g = 0; g < NG; ++g) tmem_ld32(tmem_O + lane_addr + cw * QT + g * 32, v[g]);
+    for (int ch = 0; ch < NCH; ++ch) {
+      float v[16];
+      tmem_ld16(tmem_O + lane_addr + col0 + ch * 16, v);
 #pragma unroll
-    for (int g = 0; g < NG; ++g)
-#pragma unroll
-      for (int j = 0; j < 32; j += 4)
-        *reinterpret_cast<float4*>(sO + row * kPitch + cw * QT + g * 32 + j) = make_float4(v[g][j], v[g][j + 1], v[g][j + 2], v[g][j + 3]);
-    if (cw == 0) sML[row] = row_live ? make_float2(m_row, l_row) : make_float2(-INFINITY, 0.f);
+      for (int j = 0; j < 16; j += 4)
+        *reinterpret_cast<float4*>(sO + row * kPitch + col0 + ch * 16 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+    }
+    if (cw == 0 && hw == 0) sML[row] = row_live ? make_float2(m_row, l_row) : make_float2(-INFINITY, 0.f);
   } else if (tid == 0) {
     atomicExch(a.err_flag, 4);
   }
@@ -604,12 +595,12 @@ int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a) {
   const int q_tiles = (rps + qt_rows - 1) / qt_rows;
   const float scale_log2 = (1.0f / sqrtf((float)a.hd)) * 1.4426950408889634f;
   // 101 KB: never more than two CTAs per SM, so that two 256-column TMEM allocations always fit
-  const size_t smem = 6 * (size_t)kHalfBytesKV + 4096 + 64 + 1024;   // Q, K/P, V tiles of 128 rows + the softmax exchange
+  const size_t smem = 6 * (size_t)kHalfBytesKV + 8192 + 64 + 1024;   // Q, K/P, V tiles of 128 rows + the softmax exchange
   static bool attr_set[kMaxDevices] = {};        // the shared-memory opt-in is per device
   const int dev = device_slot();
   if (dev < 0) return -4;
   if (!attr_set[dev]) {
-    const int max_smem = 6 * kHalfBytesKV + 4096 + 64 + 1024;
+    const int max_smem = 6 * kHalfBytesKV + 8192 + 64 + 1024;
     if (cudaFuncSetAttribute(attn_verify_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
         cudaFuncSetAttribute(attn_verify_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
         cudaFuncSetAttribute(attn_verify_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)

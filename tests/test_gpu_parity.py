@@ -572,3 +572,99 @@ def test_nonfinite_weights_are_reported_not_decoded():
         assert acc[0][:nf[0]].sum() == w.block_len and w.mask_id not in tok
     finally:
         ssd.destroy()
+
+
+# ------------------------------------------------------------------------------------------
+# mix-order tree (Section 5.2)
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("which", ["tiny", "tiny_peaked"])
+def test_mix_order_steps_match_oracle(tiny_ssd, peaked_ssd, tiny_oracles, which):
+    """Every forward of the oracle's mix-order run replayed on the GPU from the oracle's state: the tree
+    has the oracle's nodes (bit-exact rows, via the forward's outputs on them), and the walk - chain,
+    out-of-order branch, state and draft update - equals the oracle's walk applied to the GPU forward's
+    own (token, confidence) outputs, without exemption."""
+    w = wl.TINY if which == "tiny" else PEAKED
+    ssd = tiny_ssd if which == "tiny" else peaked_ssd
+    _, ob = tiny_oracles[w.name]
+    prompt = wl.make_prompts(w).numpy()
+    trace = []
+    N = 5
+    tokens, _, _ = ob.generate(prompt[0], w.gen_len, w.block_len, mode="ssd", max_drafts=N, trace=trace, tree="mix_order")
+    T = w.block_len
+    rtol = CONF_RTOL * w.lm_head_scale
+    branches = 0
+    ssd.set_option("mix_order", 1)
+    try:
+        ssd.prefill(prompt)
+        cur_block = 0
+        for rec in trace:
+            if rec.block != cur_block:
+                ssd.block_begin(T)
+                ssd.set_block_state(tokens[cur_block * T:(cur_block + 1) * T][None], np.zeros((1, T), np.uint8))
+                ssd.block_commit()
+                cur_block = rec.block
+            tok_g, conf_g, _ = ssd.verify_forward(rec.node_ids[None], rec.node_masked[None])
+            tok_g, conf_g = tok_g[0], conf_g[0]
+            m = rec.node_masked
+            assert np.allclose(conf_g[m], rec.conf[m], rtol=rtol, atol=1e-6)
+            ssd.block_begin(T)
+            if rec.draft_tok is None:
+                ssd.set_block_state(rec.ids_before[None], rec.masked_before[None].astype(np.uint8))
+                cand = []
+            else:
+                dconf32 = rec.draft_conf.astype(np.float32)
+                ssd.set_block_state(rec.ids_before[None], rec.masked_before[None].astype(np.uint8),
+                                    rec.draft_tok[None], dconf32[None])
+                cand = so.select_candidates(rec.draft_tok, dconf32, rec.masked_before, N)
+            acc, nn = ssd.block_step(N, 1)
+            assert nn[0] == rec.node_ids.shape[0] == len(cand) + 1 + max(0, len(cand) - 1)
+            ids, masked, dt, dc = ssd.get_block_state(1, T)
+            if cand != rec.cand:
+                continue
+            pred = so.node_predictions(tok_g, conf_g, rec.node_masked)
+            accepted, last = so.accept_walk_mix_order(pred, cand)
+            branches += int(last > len(cand))
+            assert acc[0] == len(accepted)
+            want_ids, want_masked = rec.ids_before.copy(), rec.masked_before.copy()
+            for (p, t) in accepted:
+                want_ids[p], want_masked[p] = t, False
+            assert np.array_equal(masked[0].astype(bool), want_masked)
+            assert np.array_equal(ids[0][~want_masked], want_ids[~want_masked])
+            assert np.array_equal(dt[0][want_masked], tok_g[last][want_masked])
+            assert np.array_equal(dc[0][want_masked].view(np.uint32), conf_g[last][want_masked].view(np.uint32))
+    finally:
+        ssd.set_option("mix_order", 0)
+    print(f"{which}: {branches} of {len(trace)} forwards ended in an out-of-order branch")
+
+
+def test_mix_order_generation_is_lossless_on_the_device(peaked_ssd):
+    """GPU mix-order SSD == GPU stepwise bit for bit; it never needs more forwards than the greedy chain."""
+    w = PEAKED
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    peaked_ssd.prefill(prompt)
+    tok_s, _, _ = peaked_ssd.generate(b.MODE_STEPWISE, w.gen_len, w.block_len, 1)
+    forwards = {}
+    try:
+        for mix in (0, 1):
+            peaked_ssd.set_option("mix_order", mix)
+            peaked_ssd.set_option("max_drafts", 4)
+            peaked_ssd.prefill(prompt)
+            tok, accs, nfs = peaked_ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1)
+            assert np.array_equal(tok, tok_s)
+            for acc, nf in zip(accs, nfs):
+                used = acc[0][:nf[0]]
+                assert used.sum() == w.block_len and np.all(used >= 1) and np.all(used <= 5)
+            forwards[mix] = sum(int(nf[0]) for nf in nfs)
+    finally:
+        peaked_ssd.set_option("mix_order", 0)
+        peaked_ssd.set_option("max_drafts", w.block_len - 1)
+    assert forwards[1] <= forwards[0]
+    with pytest.raises(b.SsdError) as e:                     # 2N nodes must fit the capacity fixed at creation
+        peaked_ssd.set_option("mix_order", 1)
+        peaked_ssd.set_option("max_drafts", w.block_len - 1)
+        peaked_ssd.prefill(prompt)
+        peaked_ssd.decode_block(b.MODE_SSD, w.block_len, 1)
+    assert e.value.code == -5
+    peaked_ssd.set_option("mix_order", 0)
+    peaked_ssd.prefill(prompt)
