@@ -122,11 +122,21 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 # the CPU oracle as baseline / reference arm
 # --------------------------------------------------------------------------------------------
-def oracle_sample(w, layers_sampled, prefix_len, n_rows, repeats=1):
-    """Times the oracle (as it stands) on a bounded sample of the workload: `layers_sampled` layers
-    of one root-only verification forward (`n_rows` rows against `prefix_len` cached positions) plus
-    the LM head, and scales the layer part to the full depth.  Returns (seconds per full forward,
-    description, threads)."""
+def _oracle_threads():
+    try:
+        import threadpoolctl
+        return max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_forward_times(w, layers, prefix_len, node_counts, device="cpu", with_head=True):
+    """Times the oracle (as it stands) on verification forwards of `w`: for every layer index in `layers`
+    the layer's tensors are drawn (outside the clock, one layer in memory at a time) and ``Oracle.layer`` is
+    timed once per entry of `node_counts` (that many nodes of block_len rows against `prefix_len` cached
+    positions); then the LM head on the same rows.  The inputs of a layer are seeded stand-ins (the cost of
+    the oracle's arithmetic does not depend on the values).  Returns ({nodes: seconds over `layers`},
+    {nodes: seconds of the LM head}, threads)."""
     import numpy as np
     import torch
     from oracle import ssd_oracle as so
@@ -135,37 +145,35 @@ def oracle_sample(w, layers_sampled, prefix_len, n_rows, repeats=1):
     cfg = so.ModelConfig(w.n_layers, w.d_model, w.n_heads, w.n_kv_heads, w.head_dim, w.d_ffn, w.vocab, w.mask_id,
                          w.rope_theta, w.rms_eps)
 
-    # inputs are drawn before the clock starts: only the oracle's own work is timed
-    names = [f"layers.{l}.{t}" for l in range(layers_sampled)
-             for t in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "norm_attn", "norm_ffn")]
-    weights = {n: wl.make_tensor(w, n, "cpu").to(torch.float32).numpy() for n in names + ["norm_final", "lm_head"]}
-    o = so.Oracle(cfg, weights)
+    def draw(names):
+        return {n: wl.make_tensor(w, n, device).to(torch.float32).cpu().numpy().astype(np.float64) for n in names}
+
     rng = np.random.default_rng(0)
+    B = w.block_len
     pk = rng.standard_normal((prefix_len, w.n_kv_heads, w.head_dim))
     pv = rng.standard_normal((prefix_len, w.n_kv_heads, w.head_dim))
-    h = [rng.standard_normal((n_rows, w.d_model)) * 0.02]
-    pos = [np.arange(prefix_len, prefix_len + n_rows)]
-    t_layers = 0.0
-    for _ in range(repeats):
-        for l in range(layers_sampled):
+    t_layers = {n: 0.0 for n in node_counts}
+    t_head = {n: 0.0 for n in node_counts}
+    for l in layers:
+        o = so.Oracle(cfg, draw([f"layers.{l}.{t}" for t in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down",
+                                                             "norm_attn", "norm_ffn")]))
+        for n in node_counts:
+            groups = [rng.standard_normal((B, w.d_model)) for _ in range(n)]
+            pos = [np.arange(prefix_len, prefix_len + B) for _ in range(n)]
             t0 = time.perf_counter()
-            h2, _, _ = o.layer(l, h, pos, pk, pv)
-            t_layers += time.perf_counter() - t0
-    t_layers /= repeats * layers_sampled
-    t0 = time.perf_counter()
-    logits = so.rmsnorm(h2[0], o._W("norm_final"), cfg.rms_eps) @ o._W("lm_head").T
-    so.token_and_confidence(logits, cfg.mask_id)
-    t_head = time.perf_counter() - t0
-    t_full = t_layers * w.n_layers + t_head
-    desc = (f"oracle (numpy fp64) on {layers_sampled} of {w.n_layers} layers + LM head of one root-only "
-            f"verification forward ({n_rows} rows, prefix {prefix_len}); layer time scaled to full depth; "
-            f"tokens/s = block_len/(block_len+1) / forward time (stepwise: one token per forward, one commit per block)")
-    try:
-        import threadpoolctl
-        threads = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] + [1])
-    except Exception:
-        threads = os.cpu_count() or 1
-    return t_full, desc, threads
+            o.layer(l, groups, pos, pk, pv)
+            t_layers[n] += time.perf_counter() - t0
+        del o
+    if with_head:
+        o = so.Oracle(cfg, draw(["norm_final", "lm_head"]))
+        for n in node_counts:
+            h = rng.standard_normal((n * B, w.d_model))
+            t0 = time.perf_counter()
+            logits = so.rmsnorm(h, o._W("norm_final"), cfg.rms_eps) @ o._W("lm_head").T
+            so.token_and_confidence(logits, cfg.mask_id)
+            t_head[n] = time.perf_counter() - t0
+            del logits
+    return t_layers, t_head, _oracle_threads()
 
 
 def pick_workload(args):
@@ -184,22 +192,43 @@ def pick_workload(args):
 
 
 def run_reference(args):
+    """The oracle as reference arm.  A step is a bounded sample of the workload: `--ref-layers` layers of one
+    stepwise forward (one node of block_len rows against the prompt's prefix) plus the LM head, actually
+    timed; step i takes the next layers in turn, so that 32 / ref-layers steps visit every layer.  `value`
+    scales the mean per-layer time to the full depth (stepwise decoding: one token per forward, one commit
+    forward per block); `ms_per_step` is the time the step's sample really took."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     w, _ = pick_workload(args)
-    times = []
+    ls = max(1, min(args.ref_layers, w.n_layers))
+    per_layer, head, step_ms = [], [], []
+    device = "cpu"
+    try:
+        import torch
+        if torch.cuda.is_available():
+            device = "cuda"                     # where the seeded generator draws (its output does not depend on it)
+    except Exception:
+        pass
+    threads = 1
     for i in range(args.warmup + args.steps):
-        t, desc, threads = oracle_sample(w, layers_sampled=1, prefix_len=w.prompt_len, n_rows=w.block_len)
+        layers = [(i * ls + j) % w.n_layers for j in range(ls)]
+        tl, th, threads = oracle_forward_times(w, layers, w.prompt_len, [1], device)
         if i >= args.warmup:
-            times.append(t)
-    t = sum(times) / len(times)
-    tps = w.block_len / (w.block_len + 1.0) / t
+            per_layer.append(tl[1] / ls)
+            head.append(th[1])
+            step_ms.append(1e3 * (tl[1] + th[1]))
+    t_fwd = (sum(per_layer) / len(per_layer)) * w.n_layers + sum(head) / len(head)
+    tps = w.block_len / (w.block_len + 1.0) / t_fwd
+    desc = (f"oracle (numpy fp64), per step {ls} of {w.n_layers} layers (next layers each step) + LM head of one stepwise "
+            f"forward ({w.block_len} rows, prefix {w.prompt_len}), timed; {args.steps} steps timed; tokens/s = "
+            f"block_len/(block_len+1) / (mean layer time x {w.n_layers} + LM head)")
     line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": 1e3 * t * (w.block_len + 1) * (w.gen_len // w.block_len),
+            "warmup": args.warmup, "ms_per_step": sum(step_ms) / len(step_ms),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "prompt_len": w.prompt_len, "gen_len": w.gen_len, "block_len": w.block_len,
-                       "batch": 1, "decoding": "stepwise (oracle)"},
+                       "batch_per_gpu": w.batch, "decoding": "stepwise (oracle)", "step": f"{ls} layers + LM head of one forward",
+                       "seconds_per_full_forward": t_fwd},
             "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -220,6 +249,74 @@ def ensure_library():
                 time.sleep(2.0)
 
 
+def quick_workload(w, peaks, stream, drafts=(0, 1)):
+    """The other configurations in short: one generation per draft length (decode tokens/s, accept
+    histogram) and CUDA-event times of single forwards, on a context of its own."""
+    import numpy as np
+    import torch
+    from paper_2510_04147_b200 import binding, workloads as wl
+
+    B, L, P, bs = w.block_len, w.gen_len, w.prompt_len, w.batch
+    ssd = binding.Ssd(binding.config_from_workload(w, max_drafts=max(drafts)))
+    try:
+        ssd.load_workload_weights(w, "cuda")
+        ssd.prefill_dev(wl.make_prompts(w, "cuda"))
+        out_tok = torch.zeros((bs, B), dtype=torch.int32).pin_memory()
+        out_acc = torch.zeros((bs, B), dtype=torch.int32).pin_memory()
+        out_nf = torch.zeros((bs,), dtype=torch.int32).pin_memory()
+        res = {"batch": bs, "prompt_len": P, "gen_len": L, "block_len": B, "per_draft_length": {}}
+        for d in drafts:
+            ssd.set_option("max_drafts", d)
+            mode = binding.MODE_SSD if d > 0 else binding.MODE_STEPWISE
+            ssd.rewind(P)
+            ssd.decode_block_into(mode, B, out_tok.data_ptr(), out_acc.data_ptr(), out_nf.data_ptr())   # warm-up block
+            ssd.rewind(P)
+            accs = []
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(stream)
+            done = 0
+            while done < L:
+                t = min(B, L - done)
+                ssd.decode_block_into(mode, t, out_tok.data_ptr(), out_acc.data_ptr(), out_nf.data_ptr())
+                accs.append(out_acc.numpy()[:, :t].copy())
+                done += t
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            ms = ev0.elapsed_time(ev1)
+            a = np.concatenate([x.reshape(-1) for x in accs])
+            a = a[a > 0]
+            # one forward of this chain length in the middle of a block, CUDA events around the step
+            ssd.rewind(P)
+            ssd.block_begin(B)
+            ssd.block_step(d, bs)
+            times = []
+            for _ in range(4):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                acc, nn = ssd.block_step(d, bs)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if acc.sum() == 0:
+                    break
+                times.append(e0.elapsed_time(e1))
+            tmed = statistics.median(times)
+            wb, kvb = forward_bytes(w, bs, P)
+            rows = bs * (d + 1) * B
+            t_hbm = (wb + kvb) / (peaks["hbm_gbs"] * 1e9)
+            t_tc = 2.0 * rows * (wb / 2.0) / (peaks["bf16_tflops_sustained"] * 1e12)
+            res["per_draft_length"][str(d)] = {
+                "tokens_per_s": bs * L / (ms * 1e-3), "ms_per_generation": ms, "forwards_per_sequence": int(len(a) / bs),
+                "mean_accepted_per_forward": float(a.mean()), "accept_histogram": np.bincount(a).tolist(),
+                "forward": {"rows": rows, "ms": tmed, "algorithmic_gb": (wb + kvb) / 1e9, "hbm_frac": t_hbm / (tmed * 1e-3),
+                            "frac_of_max_hbm_tensor": max(t_hbm, t_tc) / (tmed * 1e-3)}}
+        best = max(res["per_draft_length"], key=lambda k: res["per_draft_length"][k]["tokens_per_s"])
+        res["best_draft_length"] = int(best)
+        res["tokens_per_s"] = res["per_draft_length"][best]["tokens_per_s"]
+        return res
+    finally:
+        ssd.destroy()
+
+
 def run_ours(args):
     ensure_library()
     import numpy as np
@@ -236,7 +333,8 @@ def run_ours(args):
     w, reduced = pick_workload(args)
     B, L, P, bs = w.block_len, w.gen_len, w.prompt_len, w.batch
     n_blocks = -(-L // B)
-    sweep_drafts = [int(x) for x in args.sweep.split(",")] if args.sweep else []
+    sweep_drafts = sorted({(w.block_len - 2 if x == "full" else int(x)) for x in args.sweep.split(",")}) if args.sweep else []
+    sweep_drafts = [d for d in sweep_drafts if 0 <= d <= w.block_len - 1 and w.batch * (d + 1) * w.block_len <= 1024]
     # the full chain of a block (N = B - 2 drafts, B - 1 nodes) is timed once per run against the tensor
     # roofline; batches whose full chain would exceed 1024 rows get the longest chain within 1024 rows
     ft_nodes = max(1, min(w.block_len - 1, 1024 // (w.batch * w.block_len)))
@@ -328,7 +426,7 @@ def run_ours(args):
 
     # ---- end to end: host prompt -> prefill -> all blocks with host outputs, every step
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e2e_steps = max(1, min(args.steps, 2))
+    e2e_steps = max(1, args.steps)
     torch.cuda.synchronize()
     ev0.record(stream)
     for _ in range(e2e_steps):
@@ -346,7 +444,12 @@ def run_ours(args):
         accs = accept_stats(best)
         # ---- per-forward roofline: stepwise (1 node) and the chosen chain, CUDA events per forward
         fwd = {}
-        for label, d in (("stepwise_1_node", 0), (f"ssd_{best + 1}_nodes", best), ("full_tree", ft_nodes - 1)):
+        labels = [("stepwise_1_node", 0), (f"ssd_{best + 1}_nodes", best)]
+        for extra in (1, 3):                            # 2 and 4 nodes always: forward time against the row count
+            if extra != best and extra + 1 <= ft_nodes:
+                labels.append((f"ssd_{extra + 1}_nodes", extra))
+        labels.append(("full_tree", ft_nodes - 1))
+        for label, d in labels:
             ssd.set_option("max_drafts", d)
             ssd.rewind(P)
             ssd.block_begin(B)
@@ -425,9 +528,17 @@ def run_ours(args):
         if args.no_cpu_baseline:
             cpu = None
         else:
-            t_fwd, desc, threads = oracle_sample(w, layers_sampled=1, prefix_len=P, n_rows=B)
+            nodes_timed = sorted({1, best + 1})
+            tl, th, threads = oracle_forward_times(w, range(w.n_layers), P, nodes_timed, "cuda")
+            t_fwd = tl[1] + th[1]                               # one stepwise forward, every layer timed
+            t_ver = tl[best + 1] + th[best + 1]                 # one verification forward of the benchmarked chain
+            desc = (f"oracle (numpy fp64), {w.n_layers} of {w.n_layers} layers + LM head actually timed, once as a stepwise "
+                    f"forward (1 node, {B} rows) and once as the verification forward of the benchmarked chain "
+                    f"({best + 1} nodes), prefix {P}; weights drawn one layer at a time outside the clock; value = "
+                    f"stepwise tokens/s = block_len/(block_len+1) / forward time (one token per forward, one commit per block)")
             cpu = {"value": B / (B + 1.0) / t_fwd, "unit": "tokens/s", "cores": threads, "kind": "oracle",
-                   "sample": desc, "seconds_per_forward": t_fwd}
+                   "sample": desc, "seconds_per_forward": t_fwd, "seconds_per_verify_forward": t_ver,
+                   "ssd_tokens_per_s_at_measured_acceptance": float(accs.mean()) / t_ver}
         line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -447,6 +558,20 @@ def run_ours(args):
                 "sweep": sweep,
                 "paper_context": "paper reports 2.0-3.46x over stepwise decoding on one A100 80GB with trained weights"}
     ssd.destroy()
+    if line is not None and world == 1 and not reduced and args.workload == "llada8b" and not args.no_other_workloads:
+        # the other configurations, each on a context of its own (one generation per draft length)
+        others = {}
+        torch.cuda.empty_cache()
+        for name, batches in (("dream7b", (1,)), ("llada8b_batch", (1, 2, 4, 8)), ("llada8b_long", (4,))):
+            for b in batches:
+                wo = wl.WORKLOADS[name].replace(batch=b)
+                key = name if len(batches) == 1 else f"{name}_{b}"
+                try:
+                    others[key] = quick_workload(wo, peaks, stream)
+                except Exception as e:                    # report, do not lose the headline line
+                    others[key] = {"error": str(e)}
+                torch.cuda.empty_cache()
+        line["workloads"] = others
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
@@ -462,7 +587,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llada8b")
     ap.add_argument("--max-drafts", type=int, default=-1, help="draft length N; -1: pick the best of --sweep")
-    ap.add_argument("--sweep", default="0,1,3,5")
+    ap.add_argument("--sweep", default="0,1,3,5,7,full", help="draft lengths tried; full = block_len - 2 (the whole block as one chain)")
+    ap.add_argument("--ref-layers", type=int, default=4, help="--impl reference: layers timed per step")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the short runs of the other configurations")
     ap.add_argument("--split-qkv", type=int, default=None)
     ap.add_argument("--split-o", type=int, default=None)
     ap.add_argument("--split-down", type=int, default=None)

@@ -18,6 +18,9 @@ What is defined here, and from where:
   (Eq. 5), parent-prediction-vs-child-draft traversal (Section 3.2.4) and the
   loop of Algorithm 1 -> ``select_candidates``, ``build_chain``,
   ``node_predictions``, ``accept_length``, ``Oracle.decode_block_ssd``;
+* the acceptance-rate limit of self-drafting, Section 5.1 / Table 2 (how many stepwise
+  tokens lie within the draft forward's top-k candidates) -> ``token_topk``,
+  ``Oracle.acceptance_limit``;
 * the mix-order tree of Section 5.2 (the chain plus one out-of-order branch per chain node
   that has a grandchild, 2N nodes) -> ``build_mix_order_tree``, ``accept_walk_mix_order``.
 
@@ -146,6 +149,17 @@ def token_and_confidence(logits: np.ndarray, mask_id: int) -> Tuple[np.ndarray, 
     m = l.max(axis=-1, keepdims=True)
     conf = 1.0 / np.exp(l - m).sum(axis=-1)
     return tok.astype(np.int64), conf
+
+
+def token_topk(logits: np.ndarray, mask_id: int, k: int) -> Tuple[np.ndarray, np.ndarray]:
+    """The k most probable tokens per row of logits [T, V] (mask token excluded), most probable
+    first, lower id first among equals, and their softmax probabilities."""
+    l = np.array(logits, dtype=np.float64, copy=True)
+    l[:, mask_id] = -np.inf
+    order = np.argsort(-l, axis=-1, kind="stable")[:, :k]
+    m = l.max(axis=-1, keepdims=True)
+    z = np.exp(l - m).sum(axis=-1, keepdims=True)
+    return order.astype(np.int64), np.exp(np.take_along_axis(l, order, axis=-1) - m) / z
 
 
 def top2_gap(logits: np.ndarray, mask_id: int) -> np.ndarray:
@@ -488,6 +502,49 @@ class Oracle:
             out.append(ids)
             all_counts.append(counts)
         return np.concatenate(out), all_counts, cache
+
+    # ---- acceptance-rate limit of self-drafting (Section 5.1, Table 2) ---------------
+    def acceptance_limit_block(self, block_len: int, cache: Cache, draft_len: int, k_max: int):
+        """Stepwise decoding of one block in rounds of draft_len + 1 steps.  The forward that opens a
+        round is the draft: its k most probable tokens per masked position are recorded; every token
+        the round then decodes (the first one comes from the draft forward itself and is not counted)
+        is "matched at k" if it is among the draft's top k at its position - such a token could have
+        been accepted without a forward of its own.  Returns (ids [B], matched [k_max] with
+        matched[k-1] = tokens matched at k, steps = forwards stepwise decoding took)."""
+        mid = self.cfg.mask_id
+        ids = np.full(block_len, mid, dtype=np.int64)
+        masked = np.ones(block_len, dtype=bool)
+        matched = np.zeros(k_max, dtype=np.int64)
+        steps, in_round, draft_top = 0, 0, None
+        while masked.any():
+            node_ids, node_masked = build_chain(ids, masked, [], mid)
+            tok, conf, _, logits = self.verify(node_ids, node_masked, cache)
+            q, t = node_predictions(tok, conf, node_masked)[0]
+            if in_round == 0:
+                draft_top, _ = token_topk(logits[0], mid, k_max)
+            else:
+                hit = np.nonzero(draft_top[q] == t)[0]
+                if len(hit):
+                    matched[int(hit[0]):] += 1          # matched at every k above the rank it was found at
+            ids[q] = t
+            masked[q] = False
+            steps += 1
+            in_round = (in_round + 1) % (draft_len + 1)
+        return ids, matched, steps
+
+    def acceptance_limit(self, prompt: np.ndarray, gen_len: int, block_len: int, draft_len: int, k_max: int):
+        """Table 2's quantity for one generation: the fraction of stepwise forwards that drafts
+        matched within their top k would save, for k = 1 .. k_max (bounded by N/(N+1)).  Returns
+        (tokens [gen_len], reduction [k_max])."""
+        cache = self.prefill(np.asarray(prompt))
+        out, matched, steps = [], np.zeros(k_max, dtype=np.int64), 0
+        for (lo, hi) in block_ranges(gen_len, block_len):
+            ids, m, s = self.acceptance_limit_block(hi - lo, cache, draft_len, k_max)
+            self.commit_block(ids, cache)
+            out.append(ids)
+            matched += m
+            steps += s
+        return np.concatenate(out), matched / float(steps)
 
     # ---- the uncached definition used to pin the cache semantics --------------------
     def uncached_block_causal(self, tokens: np.ndarray, segment_lengths: Sequence[int],

@@ -424,3 +424,98 @@ def test_mix_order_equals_stepwise_small(w, max_drafts):
     b, counts, _ = o.generate(prompt, w.gen_len, w.block_len, mode="ssd", max_drafts=max_drafts, tree="mix_order")
     assert np.array_equal(a, b)
     assert all(sum(c) == w.block_len for c in counts)
+
+
+# ---------------------------------------------------------------------------------------
+# acceptance-rate limit of self-drafting (Section 5.1, Table 2)
+# ---------------------------------------------------------------------------------------
+def test_token_topk_matches_torch_and_top1():
+    import torch
+    rng = np.random.default_rng(3)
+    logits = rng.standard_normal((9, 50))
+    logits[2, 7] = logits[2, 11] = logits[2].max() + 1.0          # a tie: the lower id comes first
+    mask_id = 49
+    tok, prob = so.token_topk(logits, mask_id, 5)
+    l = torch.tensor(logits)
+    l[:, mask_id] = -float("inf")
+    ref_p, ref_i = torch.topk(torch.softmax(l, -1), 5, dim=-1)
+    assert np.allclose(prob, ref_p.numpy(), rtol=1e-12)
+    assert tok[2, 0] == 7 and tok[2, 1] == 11
+    rows = [r for r in range(9) if r != 2]
+    assert np.array_equal(tok[rows], ref_i.numpy()[rows])
+    t1, c1 = so.token_and_confidence(logits, mask_id)
+    assert np.array_equal(tok[:, 0], t1) and np.allclose(prob[:, 0], c1, rtol=1e-12)
+    assert mask_id not in tok
+
+
+class ScriptedLogitsOracle(so.Oracle):
+    """verify() answers logits from a script: rule(ids_row, masked_row) -> logits [B, V]."""
+
+    def __init__(self, vocab, rule):
+        super().__init__(so.ModelConfig(0, 0, 0, 0, 0, 0, vocab, vocab - 1, 1.0, 0.0), {})
+        self.rule = rule
+
+    def verify(self, node_ids, node_masked, cache):
+        logits = np.stack([self.rule(node_ids[i], node_masked[i]) for i in range(node_ids.shape[0])])
+        n, T, V = logits.shape
+        tok, conf = so.token_and_confidence(logits.reshape(n * T, V), self.cfg.mask_id)
+        return tok.reshape(n, T), conf.reshape(n, T), np.ones((n, T)), logits
+
+
+@pytest.mark.parametrize("N,pct", _golden("step_reduction_upper_bound.txt"))
+def test_acceptance_limit_reaches_the_printed_bound_when_drafts_never_go_stale(N, pct):
+    """A model whose predictions do not depend on the context: every stepwise token is the draft's
+    top-1, so the limit is the bound N/(N+1) of Table 2 already at k = 1."""
+    B, V = 60 * (N + 1), 40
+    rng = np.random.default_rng(N)
+    fixed = rng.standard_normal((B, V)) * 3.0
+    o = ScriptedLogitsOracle(V, lambda ids, masked: fixed)
+    ids, matched, steps = o.acceptance_limit_block(B, NoCache(), N, 3)
+    assert steps == B and np.all(matched == B - B // (N + 1))
+    assert round(100.0 * matched[0] / steps, 1) == pct
+
+
+def test_acceptance_limit_counts_match_bruteforce_and_grow_with_k():
+    """Context-dependent scripted logits: the counts equal a direct recount from the stepwise trajectory,
+    are non-decreasing in k, and k = vocabulary size matches everything (the bound)."""
+    B, V, N = 18, 12, 2
+    rng = np.random.default_rng(9)
+    tabs = rng.standard_normal((B + 1, B, V)) * 2.0
+
+    def rule(ids, masked):
+        return tabs[int(masked.sum())]
+
+    o = ScriptedLogitsOracle(V, rule)
+    ids, matched, steps = o.acceptance_limit_block(B, NoCache(), N, V - 1)
+    want, _ = o.decode_block_stepwise(B, NoCache())
+    assert np.array_equal(ids, want) and steps == B
+    # recount: replay stepwise, remember the ranking of every position at each round start
+    cur = np.full(B, V - 1)
+    msk = np.ones(B, dtype=bool)
+    expect = np.zeros(V - 1, dtype=int)
+    for step in range(B):
+        logits = rule(cur, msk).copy()
+        logits[:, V - 1] = -np.inf
+        if step % (N + 1) == 0:
+            rank_of = np.argsort(np.argsort(-logits, axis=-1, kind="stable"), axis=-1, kind="stable")
+        conf = np.exp(logits - logits.max(-1, keepdims=True))
+        conf = (conf / conf.sum(-1, keepdims=True)).max(-1)
+        q = so.best_masked_position(conf, msk)
+        t = int(np.argmax(logits[q]))
+        if step % (N + 1) != 0:
+            expect[rank_of[q, t]:] += 1
+        cur[q], msk[q] = t, False
+    assert np.array_equal(matched, expect)
+    assert np.all(np.diff(matched) >= 0)
+    assert matched[-1] == B - B // (N + 1)               # every token is within the top V-1
+    assert 0 < matched[0] < matched[-1]                  # stale drafts: k = 1 misses some
+
+
+def test_acceptance_limit_on_the_model_keeps_stepwise_tokens():
+    w = SMALL
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    want, _, _ = o.generate(prompt, w.gen_len, w.block_len, mode="stepwise")
+    got, red = o.acceptance_limit(prompt, w.gen_len, w.block_len, 2, 4)
+    assert np.array_equal(got, want)
+    assert np.all(np.diff(red) >= 0) and np.all(red >= 0) and np.all(red <= 2.0 / 3.0 + 1e-12)
