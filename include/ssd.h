@@ -137,6 +137,28 @@ int ssd_verify_forward(ssd_ctx* ctx, int32_t batch, int32_t n_nodes, int32_t blo
                        const int32_t* node_ids, const uint8_t* node_masked,
                        int32_t* out_tok, float* out_conf, float* out_logits);
 
+/* The verification forward with the `k` most probable tokens per wanted row instead of the single best
+ * (Section 5.1: the candidates a k-ary verification tree would draw from).  1 <= k <= 8.  HOST outputs
+ * out_tok / out_prob [batch, n_nodes, block_tokens, k]: tokens by descending softmax probability (mask id
+ * excluded, lower id first among equals) and those probabilities; -1 / 0 on rows not masked.  out_tok[..., 0]
+ * and out_prob[..., 0] are what ssd_verify_forward returns.  The logits still never reach HBM: the LM-head
+ * epilogue ranks every 128-entry vocabulary tile on chip and a merge kernel ranks the tiles' lists. */
+int ssd_verify_forward_topk(ssd_ctx* ctx, int32_t batch, int32_t n_nodes, int32_t block_tokens,
+                            const int32_t* node_ids, const uint8_t* node_masked, int32_t k,
+                            int32_t* out_tok, float* out_prob);
+
+/* Acceptance-rate limit of self-drafting (Section 5.1, Table 2), measured on the next block: the block is
+ * decoded stepwise (the tokens are those of SSD_MODE_STEPWISE) in rounds of draft_len + 1 forwards; the
+ * forward that opens a round is the draft and its top-k_max tokens per position are kept on the device;
+ * every later token of the round is looked up in them.  out_matched HOST [k_max]: tokens, summed over the
+ * batch, that lay within the draft's top k for k = 1 .. k_max - tokens a verification tree over the top-k
+ * candidates could have accepted without a forward of their own; out_steps HOST [1]: forwards x sequences
+ * stepwise decoding took.  matched[k-1] / steps is Table 2's reduction ratio, bounded by
+ * draft_len / (draft_len + 1).  out_tokens HOST [batch, block_tokens] or NULL.  Commits the block like
+ * ssd_decode_block. */
+int ssd_probe_acceptance_limit(ssd_ctx* ctx, int32_t block_tokens, int32_t draft_len, int32_t k_max,
+                               int32_t* out_tokens, int64_t* out_matched, int64_t* out_steps);
+
 /* Read cached K (post-rotary) and V of one layer and sequence: HOST fp32
  * [length, n_kv_heads, head_dim] each, positions [0, length).  Test hook for cache semantics. */
 int ssd_read_cache(ssd_ctx* ctx, int32_t layer, int32_t seq, int32_t length, float* out_k, float* out_v);

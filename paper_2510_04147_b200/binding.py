@@ -27,7 +27,8 @@ PROF_TOP = PROF_FAMILIES[:5]          # the last four break "gemm" down by proje
 
 EXPORTS = ["ssd_create", "ssd_destroy", "ssd_last_error", "ssd_load_weights", "ssd_prefill", "ssd_prefill_dev",
            "ssd_decode_block", "ssd_block_begin", "ssd_set_block_state", "ssd_get_block_state", "ssd_block_step",
-           "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_write_cache", "ssd_verify_layers", "ssd_cache_length", "ssd_rewind", "ssd_gemm_bf16",
+           "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_write_cache", "ssd_verify_layers",
+           "ssd_verify_forward_topk", "ssd_probe_acceptance_limit", "ssd_cache_length", "ssd_rewind", "ssd_gemm_bf16",
            "ssd_gemm_bf16_noalloc",
            "ssd_launch_count", "ssd_profile_enable", "ssd_profile_read", "ssd_set_option"]
 
@@ -77,6 +78,8 @@ def load_library() -> C.CDLL:
     lib.ssd_read_cache.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.ssd_write_cache.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.ssd_verify_layers.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.ssd_verify_forward_topk.argtypes = [vp, i32, i32, i32, vp, vp, i32, vp, vp]
+    lib.ssd_probe_acceptance_limit.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     lib.ssd_cache_length.argtypes = [vp]
     lib.ssd_rewind.argtypes = [vp, i32]
     lib.ssd_gemm_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32]
@@ -220,6 +223,26 @@ class Ssd:
         self._check(self.lib.ssd_verify_forward(self._ctx, b, n, t, _np_ptr(ids), _np_ptr(mk), _np_ptr(tok),
                                                 _np_ptr(conf), _np_ptr(logits)))
         return tok, conf, logits
+
+    def verify_forward_topk(self, node_ids: np.ndarray, node_masked: np.ndarray, k: int):
+        ids = np.ascontiguousarray(node_ids, dtype=np.int32)
+        mk = np.ascontiguousarray(node_masked, dtype=np.uint8)
+        assert ids.ndim == 3 and ids.shape == mk.shape
+        b, n, t = ids.shape
+        tok = np.zeros((b, n, t, k), np.int32)
+        prob = np.zeros((b, n, t, k), np.float32)
+        self._check(self.lib.ssd_verify_forward_topk(self._ctx, b, n, t, _np_ptr(ids), _np_ptr(mk), k, _np_ptr(tok),
+                                                     _np_ptr(prob)))
+        return tok, prob
+
+    def probe_acceptance_limit(self, block_tokens: int, draft_len: int, k_max: int, batch: int):
+        """Returns (tokens [batch, block_tokens], matched [k_max], steps)."""
+        tok = np.zeros((batch, block_tokens), np.int32)
+        matched = np.zeros(k_max, np.int64)
+        steps = np.zeros(1, np.int64)
+        self._check(self.lib.ssd_probe_acceptance_limit(self._ctx, block_tokens, draft_len, k_max, _np_ptr(tok),
+                                                        _np_ptr(matched), _np_ptr(steps)))
+        return tok, matched, int(steps[0])
 
     def read_cache(self, layer: int, seq: int, length: int):
         kv = self.cfg.n_kv_heads * self.cfg.head_dim

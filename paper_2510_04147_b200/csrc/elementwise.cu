@@ -238,6 +238,87 @@ __global__ void __launch_bounds__(kThreads) lm_merge_kernel(const float* tile_ma
   }
 }
 
+// The k most probable tokens of a row from the per-tile candidate lists.  One CTA per row: a thread
+// keeps the best k of the tiles it strides over (tile order, so equal values keep the lower index), the
+// threads' sorted lists are merged per warp by k rounds of a warp-wide argmax over the list heads, and
+// thread 0 merges the warps' lists the same way.  prob = exp(logit - max) * conf, conf = 1 / sum-exp.
+__global__ void __launch_bounds__(kThreads) lm_merge_topk_kernel(const float* tile_topv, const int* tile_topi, int tiles,
+                                                                 int R, int V, int k, const uint8_t* row_wanted,
+                                                                 const float* conf, int* topk_tok, float* topk_prob) {
+  __shared__ float w_v[kThreads / 32][kLmTopKMax];
+  __shared__ int w_i[kThreads / 32][kLmTopKMax];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (row_wanted && !row_wanted[r]) {
+    for (int j = threadIdx.x; j < kLmTopKMax; j += kThreads) { topk_tok[(size_t)r * kLmTopKMax + j] = -1; topk_prob[(size_t)r * kLmTopKMax + j] = 0.f; }
+    return;
+  }
+  float bv[kLmTopKMax];
+  int bi[kLmTopKMax];
+#pragma unroll
+  for (int j = 0; j < kLmTopKMax; ++j) { bv[j] = -INFINITY; bi[j] = 0x7fffffff; }
+  for (int t = threadIdx.x; t < tiles; t += kThreads) {
+    const size_t o = ((size_t)t * R + r) * kLmTopKMax;
+    for (int c = 0; c < k; ++c) {
+      float v = tile_topv[o + c];
+      int i = tile_topi[o + c];
+      if (!(v > bv[k - 1] || (v == bv[k - 1] && i < bi[k - 1]))) break;      // a tile's list is sorted: the rest is worse
+#pragma unroll
+      for (int j = 0; j < kLmTopKMax; ++j) {                                   // insert, keeping (value desc, index asc)
+        if (j < k && (v > bv[j] || (v == bv[j] && i < bi[j]))) {
+          const float tv = bv[j]; const int ti = bi[j];
+          bv[j] = v; bi[j] = i; v = tv; i = ti;
+        }
+      }
+    }
+  }
+  // warp merge: k rounds over the heads of the 32 sorted lists
+  int head = 0;
+  for (int c = 0; c < k; ++c) {
+    float m = -INFINITY;
+    int a = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < kLmTopKMax; ++j)
+      if (j == head) { m = bv[j]; a = bi[j]; }
+    float wm = m;
+    int wa = a;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, wm, o);
+      const int oa = __shfl_xor_sync(0xffffffffu, wa, o);
+      if (om > wm || (om == wm && oa < wa)) { wm = om; wa = oa; }
+    }
+    if (wm == m && wa == a && a != 0x7fffffff) ++head;      // (indices are unique: exactly one lane advances)
+    if (lane == 0) { w_v[warp][c] = wm; w_i[warp][c] = wa; }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int hd[kThreads / 32];
+    for (int q = 0; q < kThreads / 32; ++q) hd[q] = 0;
+    float top = -INFINITY;
+    for (int c = 0; c < k; ++c) {
+      float bm = -INFINITY;
+      int ba = 0x7fffffff, bq = 0;
+      for (int q = 0; q < kThreads / 32; ++q) {
+        if (hd[q] < k) {
+          const float m = w_v[q][hd[q]];
+          const int a = w_i[q][hd[q]];
+          if (m > bm || (m == bm && a < ba)) { bm = m; ba = a; bq = q; }
+        }
+      }
+      ++hd[bq];
+      if (c == 0) top = bm;
+      const bool valid = (unsigned)ba < (unsigned)V && bm != -INFINITY;
+      topk_tok[(size_t)r * kLmTopKMax + c] = valid ? ba : -1;
+      topk_prob[(size_t)r * kLmTopKMax + c] = valid ? expf(bm - top) * conf[r] : 0.f;
+    }
+    for (int c = k; c < kLmTopKMax; ++c) { topk_tok[(size_t)r * kLmTopKMax + c] = -1; topk_prob[(size_t)r * kLmTopKMax + c] = 0.f; }
+  }
+}
+
+
 }  // namespace
 
 void launch_convert_rows(cudaStream_t st, const void* src, int src_is_f32, bf16* dst, int rows, int cols, int dst_pitch,
@@ -299,6 +380,12 @@ void launch_lm_merge(cudaStream_t st, const float* tile_max, const float* tile_s
                      int R, int V, const uint8_t* row_wanted, int* tok, float* conf) {
   launch_pdl(lm_merge_kernel, dim3(R), dim3(kThreads), 0, st, tile_max, tile_sum, tile_arg, tiles, R, V, row_wanted,
              tok, conf);
+}
+
+void launch_lm_merge_topk(cudaStream_t st, const float* tile_topv, const int* tile_topi, int tiles, int R, int V, int k,
+                          const uint8_t* row_wanted, const float* conf, int* topk_tok, float* topk_prob) {
+  launch_pdl(lm_merge_topk_kernel, dim3(R), dim3(kThreads), 0, st, tile_topv, tile_topi, tiles, R, V, k, row_wanted,
+             conf, topk_tok, topk_prob);
 }
 
 }  // namespace ssd

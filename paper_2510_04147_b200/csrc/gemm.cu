@@ -52,6 +52,9 @@ struct TcParams {
   float* tile_max;
   float* tile_sum;
   int* tile_arg;
+  int topk;        // EPI_LMHEAD: > 0 also writes the tile's `topk` largest logits per row (value, vocabulary index)
+  float* tile_topv;
+  int* tile_topi;
   int mask_id;
   int* err_flag;
   const float* sq;
@@ -485,6 +488,64 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         s_max[quad * 256 + c0 + lane] = my_m;
         s_sum[quad * 256 + c0 + lane] = my_s;
         s_arg[quad * 256 + c0 + lane] = my_a;
+        if (p.topk > 0) {
+          // The tile's `topk` largest logits of every row of the chunk (value descending, lower index first):
+          // per warp by repeated warp-wide argmax with the winner struck out, then the four warps' sorted
+          // lists are merged by one thread per row.
+          float* s_tv = scratch + 12 * 256;              // [4 warps][kLmTopKMax][32 rows]
+          int* s_ti = reinterpret_cast<int*>(s_tv + 4 * kLmTopKMax * 32);
+          float tv[kLmTopKMax];
+          int ti[kLmTopKMax];
+#pragma unroll
+          for (int r = 0; r < kLmTopKMax; ++r) { tv[r] = -INFINITY; ti[r] = 0x7fffffff; }
+          float w[32];                                   // a copy of its own: indexed by a loop variable below
+          tmem_ld32(taddr + c0, w);
+#pragma unroll 1
+          for (int j = 0; j < 32; ++j) {
+            float x = live ? (p.sq != nullptr ? w[j] * s_inv[c0 + j] : w[j]) : -INFINITY;
+#pragma unroll
+            for (int r = 0; r < kLmTopKMax; ++r) {
+              if (r < p.topk) {
+                float m = x;
+                int a = n;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                  const float om = __shfl_xor_sync(0xffffffffu, m, o);
+                  const int oa = __shfl_xor_sync(0xffffffffu, a, o);
+                  if (om > m || (om == m && oa < a)) { m = om; a = oa; }
+                }
+                if (a == n) x = -INFINITY;               // struck out for the next round
+                if (lane == j) { tv[r] = m; ti[r] = (m == -INFINITY) ? 0x7fffffff : a; }
+              }
+            }
+          }
+#pragma unroll
+          for (int r = 0; r < kLmTopKMax; ++r) {
+            s_tv[(quad * kLmTopKMax + r) * 32 + lane] = tv[r];
+            s_ti[(quad * kLmTopKMax + r) * 32 + lane] = ti[r];
+          }
+          epi_bar_sync();
+          if (warp == 2 && c0 + lane < rows_here) {
+            int head[4] = {0, 0, 0, 0};
+            const size_t o = ((size_t)tile * p.R + row0 + c0 + lane) * kLmTopKMax;
+            for (int r = 0; r < p.topk; ++r) {
+              float bm = -INFINITY;
+              int ba = 0x7fffffff, bq = 0;
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                if (head[q] < p.topk) {
+                  const float m = s_tv[(q * kLmTopKMax + head[q]) * 32 + lane];
+                  const int a = s_ti[(q * kLmTopKMax + head[q]) * 32 + lane];
+                  if (m > bm || (m == bm && a < ba)) { bm = m; ba = a; bq = q; }
+                }
+              }
+              ++head[bq];
+              p.tile_topv[o + r] = bm;
+              p.tile_topi[o + r] = ba;
+            }
+          }
+          epi_bar_sync();
+        }
       }
       epi_bar_sync();
       for (int c = (warp - 2) * 32 + lane; c < rows_here; c += 128) {
@@ -683,6 +744,8 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   p.stages = stages;
   p.out = g.out; p.act = g.act; p.act_pitch = g.act_pitch;
   p.tile_max = g.tile_max; p.tile_sum = g.tile_sum; p.tile_arg = g.tile_arg;
+  p.topk = g.topk; p.tile_topv = g.tile_topv; p.tile_topi = g.tile_topi;
+  if (g.topk < 0 || g.topk > kLmTopKMax || (g.topk > 0 && (g.epi != EPI_LMHEAD || !g.tile_topv || !g.tile_topi))) return -2;
   p.mask_id = g.mask_id; p.err_flag = g.err_flag;
   p.sq = g.sq; p.sq_count = g.sq_count; p.sq_stride = g.sq_stride; p.norm_dim = g.norm_dim; p.norm_eps = g.norm_eps;
   p.h = g.h; p.hb = g.hb; p.gain = g.gain; p.sq_out = g.sq_out; p.sq_out_stride = g.sq_out_stride;

@@ -120,6 +120,11 @@ void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, in
 void launch_lm_merge(cudaStream_t st, const float* tile_max, const float* tile_sum, const int* tile_arg,
                      int tiles, int R, int V, const uint8_t* row_wanted, int* tok, float* conf);
 
+// the k most probable tokens per row from the per-tile candidate lists (merged in tile order, lower index
+// first among equals): topk_tok [R][kLmTopKMax], topk_prob likewise = exp(logit - max) * conf[row]
+void launch_lm_merge_topk(cudaStream_t st, const float* tile_topv, const int* tile_topi, int tiles, int R, int V, int k,
+                          const uint8_t* row_wanted, const float* conf, int* topk_tok, float* topk_prob);
+
 // ---------------------------------------------------------------- attention
 struct AttnArgs {
   // verification forward: Q and the node-local K/V come straight from the fp32 split-K partials
@@ -167,6 +172,7 @@ constexpr int kAttnMaxClusterParts = 8;
 // rmsnorm(h) * g . W^T  ==  inv_rms(row) * ((h * g) . W^T), with inv_rms from the sums of squares.
 enum { EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_LMHEAD = 2, EPI_RESIDUAL = 3 };
 constexpr int kGemmMaxClusterSplits = 8;
+constexpr int kLmTopKMax = 8;   // most candidates per row the LM-head epilogue can rank
 struct GemmArgs {
   const bf16* x;  // [R][x_pitch] activations (K-major)
   const bf16* w;  // [N][w_pitch] weights (K-major), or the tile-contiguous layout below when w_tiled
@@ -181,6 +187,9 @@ struct GemmArgs {
   float* tile_max;       // EPI_LMHEAD: [tiles][R]
   float* tile_sum;
   int* tile_arg;
+  int topk;              // EPI_LMHEAD: 0, or how many of the tile's largest logits per row to write as well (<= kLmTopKMax)
+  float* tile_topv;      // [tiles][R][kLmTopKMax] values, descending
+  int* tile_topi;        // [tiles][R][kLmTopKMax] vocabulary indices (lower index first among equals)
   int mask_id;
   int* err_flag;         // device int set non-zero when a bounded wait expires
   // consumer side of a fused RMSNorm: every output row r is multiplied by
@@ -214,6 +223,8 @@ struct BlockState {       // device arrays, [max_batch][block_len] unless noted
   int* accept_log;        // [max_batch][block_len] accepted per forward, 0-terminated
   int* n_forwards;        // [max_batch]
   int* last_accept;       // [max_batch] accepted by the latest step (0 if not active)
+  int* last_pos;          // [max_batch] position and token of the last token the latest step accepted
+  int* last_tok;          //             (the last valid node's own prediction)
   int* seq_map;           // [max_batch] slot -> sequence of the current forward
   int stride;             // block_len (row pitch of the arrays above)
 };

@@ -63,6 +63,14 @@ struct ssd_ctx {
   uint8_t* node_masked = nullptr;
   float* logits = nullptr;
   size_t logits_elems = 0;
+  // acceptance-limit probe (allocated on first use): per-tile candidate lists of the LM head, the merged
+  // top-k per row, the draft forward's top-k per block position, match counters
+  float* tile_topv = nullptr;
+  int* tile_topi = nullptr;
+  int* topk_tok = nullptr;       // [R_dec][kLmTopKMax]
+  float* topk_prob = nullptr;
+  int* draft_top = nullptr;      // [max_batch][block_len][kLmTopKMax]
+  unsigned long long* probe_counts = nullptr;   // [kLmTopKMax] tokens matched at k = 1.., then [kLmTopKMax] = steps counted
   int* flags = nullptr;          // [0] bounded-wait expiry, [1] non-finite confidence
   int* h_pinned = nullptr;       // pinned host staging: [0..1] flags, then 3 * max_batch ints
   BlockState bs{};
@@ -245,6 +253,7 @@ struct LayerRange {
   int begin = 0, end = -1;       // end < 0: all layers
   bool from_stream = false;
   bool lm_head = true;
+  int topk = 0;                  // > 0: the LM head also ranks the `topk` most probable tokens of every wanted row
 };
 
 // One forward over R rows.  FILL: K/V go to the cache at positions pos0.., attention over the cache
@@ -374,14 +383,57 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
       launch_lm_stats_from_logits(c->st, c->logits, R, c->V, c->cfg.mask_id, row_wanted, c->tok, c->conf);
     } else {
       g.epi = EPI_LMHEAD; g.tile_max = c->tile_max; g.tile_sum = c->tile_sum; g.tile_arg = c->tile_arg;
+      if (range.topk > 0) { g.topk = range.topk; g.tile_topv = c->tile_topv; g.tile_topi = c->tile_topi; }
       int rc = run_gemm(c, g, SSD_PROF_LMHEAD);
       if (rc) return rc;
-      Scope sc(c, SSD_PROF_LMHEAD, (double)gemm_tiles(c->V) * R * 12.0);
+      Scope sc(c, SSD_PROF_LMHEAD, (double)gemm_tiles(c->V) * R * 12.0, range.topk > 0 ? 2 : 1);
       launch_lm_merge(c->st, c->tile_max, c->tile_sum, c->tile_arg, gemm_tiles(c->V), R, c->V, row_wanted, c->tok, c->conf);
+      if (range.topk > 0)
+        launch_lm_merge_topk(c->st, c->tile_topv, c->tile_topi, gemm_tiles(c->V), R, c->V, range.topk, row_wanted, c->conf,
+                             c->topk_tok, c->topk_prob);
     }
   }
   CUDA_TRY(c, cudaGetLastError());
   return SSD_OK;
+}
+
+// Buffers of the acceptance-limit probe; allocated the first time a top-k forward is asked for.
+int ensure_topk_buffers(ssd_ctx* c) {
+  if (c->tile_topv) return SSD_OK;
+  const size_t tiles = gemm_tiles(c->V);
+  ALLOC(c, c->tile_topv, tiles * c->R_dec * kLmTopKMax);
+  ALLOC(c, c->tile_topi, tiles * c->R_dec * kLmTopKMax);
+  ALLOC(c, c->topk_tok, (size_t)c->R_dec * kLmTopKMax);
+  ALLOC(c, c->topk_prob, (size_t)c->R_dec * kLmTopKMax);
+  ALLOC(c, c->draft_top, (size_t)c->cfg.max_batch * c->cfg.block_len * kLmTopKMax);
+  ALLOC(c, c->probe_counts, kLmTopKMax + 1);
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  return SSD_OK;
+}
+
+// round opening: the draft forward's top-k of every block position of every sequence
+__global__ void probe_store_kernel(const int* topk_tok, int* draft_top, const int* seq_map, int T, int stride,
+                                   int slot_rows, int row_offset) {
+  const int slot = blockIdx.x, b = seq_map[slot];
+  for (int e = threadIdx.x; e < T * kLmTopKMax; e += blockDim.x)
+    draft_top[(size_t)b * stride * kLmTopKMax + e] = topk_tok[((size_t)slot * slot_rows + row_offset) * kLmTopKMax + e];
+}
+
+// after a stepwise step: is the token just decoded among the draft's top k at its position?
+__global__ void probe_count_kernel(BlockState s, const int* draft_top, int n_slots, int k_max, int count_matches,
+                                   unsigned long long* counts) {
+  const int slot = threadIdx.x;
+  if (slot >= n_slots) return;
+  const int b = s.seq_map[slot];
+  atomicAdd(&counts[kLmTopKMax], 1ull);
+  if (!count_matches) return;
+  const int q = s.last_pos[b], t = s.last_tok[b];
+  for (int r = 0; r < k_max; ++r) {
+    if (draft_top[((size_t)b * s.stride + q) * kLmTopKMax + r] == t) {
+      for (int k = r; k < k_max; ++k) atomicAdd(&counts[k], 1ull);      // matched at every k above its rank
+      break;
+    }
+  }
 }
 
 int check_flags_after_sync(ssd_ctx* c) {
@@ -544,6 +596,7 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     ALLOC(c, c->prompt_stage, (size_t)k.max_batch * k.max_seq);
     ALLOC(c, c->bs.has_drafts, k.max_batch); ALLOC(c, c->bs.remaining, k.max_batch); ALLOC(c, c->bs.n_cand, k.max_batch);
     ALLOC(c, c->bs.n_forwards, k.max_batch); ALLOC(c, c->bs.last_accept, k.max_batch); ALLOC(c, c->bs.seq_map, k.max_batch);
+    ALLOC(c, c->bs.last_pos, k.max_batch); ALLOC(c, c->bs.last_tok, k.max_batch);
     CUDA_TRY(c, cudaMallocHost(&c->h_pinned, (2 + 3 * (size_t)k.max_batch) * sizeof(int)));
     CUDA_TRY(c, cudaStreamSynchronize(c->st));
     return SSD_OK;
@@ -746,7 +799,9 @@ int resolve_drafts(const ssd_ctx* c, int max_drafts) {
 // forward, acceptance - without waiting for it.  The host's mirror of `remaining` / `has_drafts` decides
 // the launch shape; h_nodes[b] receives the nodes sequence b gets (0: finished).  The error flags are
 // sticky and are NOT cleared here.
-int step_enqueue(ssd_ctx* c, int md, bool* launched) {
+struct ProbeStep { int k_max; bool open_round; };
+
+int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nullptr) {
   const int T = c->block_tokens, B = c->batch;
   int active = 0, n_cap = 1;
   for (int b = 0; b < B; ++b) {
@@ -794,11 +849,22 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched) {
     for (int b = 0; b < B; ++b)
       if (c->h_remaining[b] > 0) map.inline_seq[map.n_inline++] = b;
   }
-  int rc = forward(c, FWD_VERIFY, c->node_ids, R, map, active, false, c->node_masked);
+  LayerRange range;
+  if (probe && probe->open_round) range.topk = probe->k_max;
+  int rc = forward(c, FWD_VERIFY, c->node_ids, R, map, active, false, c->node_masked, range);
   if (rc) return rc;
   {
     Scope sc(c, SSD_PROF_TREE, (double)R * 9);
     launch_accept(c->st, c->bs, active, T, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1, slot_rows, Tp, c->mix_order);
+  }
+  if (probe) {
+    // the forward that opens a round is the draft: keep its top-k per block position; every later token of
+    // the round is looked up in it
+    Scope sc(c, SSD_PROF_TREE, (double)active * T * kLmTopKMax * 4, probe->open_round ? 2 : 1);
+    if (probe->open_round)
+      probe_store_kernel<<<active, 128, 0, c->st>>>(c->topk_tok, c->draft_top, c->bs.seq_map, T, c->bs.stride, slot_rows, Tp);
+    probe_count_kernel<<<1, (active + 31) / 32 * 32, 0, c->st>>>(c->bs, c->draft_top, active, probe->k_max,
+                                                               probe->open_round ? 0 : 1, c->probe_counts);
   }
   if (Tp > 0) {                // the finished block's K/V are in the cache once this forward has run
     c->cache_len += Tp;
@@ -1006,6 +1072,76 @@ int ssd_verify_layers(ssd_ctx* c, int32_t batch, int32_t n_nodes, int32_t T, int
   if (out_tok) CUDA_TRY(c, cudaMemcpyAsync(out_tok, c->tok, R * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   if (out_conf) CUDA_TRY(c, cudaMemcpyAsync(out_conf, c->conf, R * sizeof(float), cudaMemcpyDeviceToHost, c->st));
   return sync_and_check(c);
+}
+
+int ssd_verify_forward_topk(ssd_ctx* c, int32_t batch, int32_t n_nodes, int32_t T, const int32_t* node_ids,
+                            const uint8_t* node_masked, int32_t k, int32_t* out_tok, float* out_prob) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
+  if (!node_ids || !node_masked || !out_tok || !out_prob) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  if (batch < 1 || batch > c->batch) return fail(c, SSD_ERR_INVALID_ARG, "batch %d outside [1, %d]", batch, c->batch);
+  if (T < 1 || T > c->cfg.block_len || n_nodes < 1) return fail(c, SSD_ERR_INVALID_ARG, "bad node shape");
+  if (k < 1 || k > kLmTopKMax) return fail(c, SSD_ERR_INVALID_ARG, "k %d outside [1, %d]", k, kLmTopKMax);
+  int rc = flush_pending(c);
+  if (rc) return rc;
+  rc = ensure_topk_buffers(c);
+  if (rc) return rc;
+  const size_t R = (size_t)batch * n_nodes * T;
+  if (R > (size_t)c->R_dec) return fail(c, SSD_ERR_OVERFLOW, "%zu rows exceed the capacity %d set by max_batch/max_drafts/block_len", R, c->R_dec);
+  if (c->cache_len + T > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "cache %d + block %d exceeds max_seq", c->cache_len, T);
+  for (size_t i = 0; i < R; ++i)
+    if (node_ids[i] < 0 || node_ids[i] >= c->V) return fail(c, SSD_ERR_INVALID_ARG, "node id outside the vocabulary");
+  CUDA_TRY(c, cudaMemcpyAsync(c->node_ids, node_ids, R * sizeof(int), cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(c->node_masked, node_masked, R, cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  RowMap map{n_nodes * T, T, c->cache_len, 0, nullptr};
+  LayerRange range;
+  range.topk = k;
+  rc = forward(c, FWD_VERIFY, c->node_ids, (int)R, map, batch, false, c->node_masked, range);
+  if (rc) return rc;
+  std::vector<int> tk(R * kLmTopKMax);
+  std::vector<float> tp(R * kLmTopKMax);
+  CUDA_TRY(c, cudaMemcpyAsync(tk.data(), c->topk_tok, tk.size() * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(tp.data(), c->topk_prob, tp.size() * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  rc = sync_and_check(c);
+  if (rc) return rc;
+  for (size_t i = 0; i < R; ++i)
+    for (int j = 0; j < k; ++j) {
+      out_tok[i * k + j] = tk[i * kLmTopKMax + j];
+      out_prob[i * k + j] = tp[i * kLmTopKMax + j];
+    }
+  return SSD_OK;
+}
+
+int ssd_probe_acceptance_limit(ssd_ctx* c, int32_t T, int32_t draft_len, int32_t k_max, int32_t* out_tokens,
+                               int64_t* out_matched, int64_t* out_steps) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!out_matched || !out_steps) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  if (draft_len < 0 || k_max < 1 || k_max > kLmTopKMax) return fail(c, SSD_ERR_INVALID_ARG, "draft_len >= 0 and k_max in [1, %d]", kLmTopKMax);
+  int rc = ensure_topk_buffers(c);
+  if (rc) return rc;
+  rc = ssd_block_begin(c, T);
+  if (rc) return rc;
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  CUDA_TRY(c, cudaMemsetAsync(c->probe_counts, 0, (kLmTopKMax + 1) * sizeof(unsigned long long), c->st));
+  // stepwise decoding (every sequence accepts exactly one token per forward, so all stay in lockstep) in rounds
+  // of draft_len + 1 forwards; nothing depends on a forward's result, so the whole block is enqueued at once
+  for (int step = 0; step < T; ++step) {
+    ProbeStep ps{k_max, step % (draft_len + 1) == 0};
+    bool launched = false;
+    rc = step_enqueue(c, 0, &launched, &ps);
+    if (rc) return rc;
+    for (int b = 0; b < c->batch; ++b) c->h_remaining[b] -= 1;
+  }
+  rc = step_collect(c, nullptr, nullptr);
+  if (rc) return rc;
+  unsigned long long counts[kLmTopKMax + 1];
+  CUDA_TRY(c, cudaMemcpyAsync(counts, c->probe_counts, sizeof(counts), cudaMemcpyDeviceToHost, c->st));
+  if (out_tokens) CUDA_TRY(c, cudaMemcpy2DAsync(out_tokens, T * sizeof(int), c->bs.ids, c->bs.stride * sizeof(int), T * sizeof(int), c->batch, cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  for (int k = 0; k < k_max; ++k) out_matched[k] = (int64_t)counts[k];
+  *out_steps = (int64_t)counts[kLmTopKMax];
+  return ssd_block_commit(c);
 }
 
 int ssd_gemm_bf16(ssd_ctx* c, const void* x_dev, const void* w_dev, float* out_dev, int32_t rows, int32_t n, int32_t k, int32_t split_k) {

@@ -166,6 +166,8 @@ __global__ void __launch_bounds__(256) accept_kernel(BlockState s, int T, int n_
     s.accept_log[(size_t)b * s.stride + f] = n_acc;
     s.n_forwards[b] = f + 1;
     s.last_accept[b] = n_acc;
+    s.last_pos[b] = pred_q[last];
+    s.last_tok[b] = pred_t[last];
   }
 }
 

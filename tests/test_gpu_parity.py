@@ -668,3 +668,86 @@ def test_mix_order_generation_is_lossless_on_the_device(peaked_ssd):
     assert e.value.code == -5
     peaked_ssd.set_option("mix_order", 0)
     peaked_ssd.prefill(prompt)
+
+
+# ------------------------------------------------------------------------------------------
+# top-k LM head and the acceptance-limit probe (Section 5.1, Table 2)
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("which", ["tiny", "tiny_peaked"])
+def test_topk_forward_matches_oracle(tiny_ssd, peaked_ssd, tiny_oracles, which):
+    w = wl.TINY if which == "tiny" else PEAKED
+    ssd = tiny_ssd if which == "tiny" else peaked_ssd
+    _, ob = tiny_oracles[w.name]
+    rng = np.random.default_rng(21)
+    prompt = wl.make_prompts(w).numpy()
+    T, K = w.block_len, 5
+    ids, masked = _random_nodes(w, rng, 3, T)
+    ssd.prefill(prompt)
+    tok1, conf1, _ = ssd.verify_forward(ids, masked)
+    tok, prob = ssd.verify_forward_topk(ids, masked, K)
+    m = masked[0]
+    # rank 0 is the fused top-1 path, bit for bit
+    assert np.array_equal(tok[0][..., 0], tok1[0])
+    assert np.array_equal(prob[0][..., 0].view(np.uint32)[m], conf1[0].view(np.uint32)[m])
+    assert np.all(tok[0][~m] == -1) and np.all(prob[0][~m] == 0)
+    # sorted, distinct, never the mask token
+    assert np.all(np.diff(prob[0][m], axis=-1) <= 0)
+    assert all(len(set(row)) == K for row in tok[0][m]) and w.mask_id not in tok[0][m]
+    cache = ob.prefill(prompt[0])
+    _, _, _, ologits = ob.verify(ids[0], masked[0], cache)
+    otok, oprob = so.token_topk(ologits.reshape(-1, w.vocab), w.mask_id, K + 1)
+    otok, oprob = otok.reshape(3, T, K + 1), oprob.reshape(3, T, K + 1)
+    rtol = CONF_RTOL * w.lm_head_scale
+    assert np.allclose(prob[0][m], oprob[m][:, :K], rtol=rtol, atol=1e-7)
+    # a rank is comparable where the oracle separates it from both neighbours by more than the tolerance
+    sep = (oprob[..., :-1] - oprob[..., 1:]) > 2 * rtol * oprob[..., :-1]          # rank r vs r + 1
+    safe = sep[..., :K].copy()
+    safe[..., 1:] &= sep[..., :K - 1]
+    safe &= m[..., None]
+    assert np.array_equal(tok[0][safe], otok[..., :K][safe])
+    if which == "tiny_peaked":
+        assert safe.sum() > 0.25 * m.sum() * K
+
+
+def test_acceptance_limit_probe_matches_a_recount_and_the_oracle(peaked_ssd, tiny_oracles):
+    """The probe decodes the block stepwise and counts on the device; a host recount through
+    ssd_verify_forward_topk (same forwards, same bits) gives the same numbers, and so does the oracle's
+    procedure when it takes the same stepwise trajectory."""
+    w = PEAKED
+    b = _binding()
+    _, ob = tiny_oracles[w.name]
+    prompt = wl.make_prompts(w).numpy()
+    T, N, K = w.block_len, 3, 4
+    peaked_ssd.prefill(prompt)
+    tok_step, _, _ = peaked_ssd.decode_block(b.MODE_STEPWISE, T, 1)
+    peaked_ssd.prefill(prompt)
+    tok, matched, steps = peaked_ssd.probe_acceptance_limit(T, N, K, 1)
+    assert steps == T and np.array_equal(tok, tok_step)
+    assert peaked_ssd.cache_length() == w.prompt_len + T
+    assert np.all(np.diff(matched) >= 0) and 0 <= matched[0] and matched[-1] <= T - -(-T // (N + 1))
+    # host recount with the library's own forwards
+    peaked_ssd.prefill(prompt)
+    ids = np.full((1, 1, T), w.mask_id)
+    msk = np.ones((1, 1, T), bool)
+    expect = np.zeros(K, np.int64)
+    for step in range(T):
+        tk, pr = peaked_ssd.verify_forward_topk(ids, msk, K)
+        conf = np.where(msk[0, 0], pr[0, 0, :, 0], -1.0)
+        q = int(np.argmax(conf))
+        t = int(tk[0, 0, q, 0])
+        if step % (N + 1) == 0:
+            draft = tk[0, 0].copy()
+        else:
+            hit = np.nonzero(draft[q] == t)[0]
+            if len(hit):
+                expect[hit[0]:] += 1
+        ids[0, 0, q], msk[0, 0, q] = t, False
+    assert np.array_equal(ids[0], tok_step)
+    assert np.array_equal(matched, expect)
+    # the oracle's own procedure
+    cache = ob.prefill(prompt[0])
+    oids, omatched, osteps = ob.acceptance_limit_block(T, cache, N, K)
+    print(f"acceptance limit, N = {N}: device {matched.tolist()} of {steps}, oracle {omatched.tolist()} of {osteps}")
+    assert osteps == steps
+    if np.array_equal(oids, tok_step[0]):
+        assert np.all(np.abs(matched - omatched) <= 1)
