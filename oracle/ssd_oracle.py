@@ -18,6 +18,9 @@ What is defined here, and from where:
   (Eq. 5), parent-prediction-vs-child-draft traversal (Section 3.2.4) and the
   loop of Algorithm 1 -> ``select_candidates``, ``build_chain``,
   ``node_predictions``, ``accept_length``, ``Oracle.decode_block_ssd``;
+* candidates that run on into the next block when the current one cannot fill the chain
+  (Section 3.2.2), under the block order of Section 3.1 -> ``Oracle.verify_window``,
+  ``Oracle.generate_spill``;
 * the acceptance-rate limit of self-drafting, Section 5.1 / Table 2 (how many stepwise
   tokens lie within the draft forward's top-k candidates) -> ``token_topk``,
   ``Oracle.acceptance_limit``;
@@ -186,12 +189,14 @@ def best_masked_position(conf: np.ndarray, masked: np.ndarray) -> int:
 
 
 def select_candidates(draft_tok: np.ndarray, draft_conf: np.ndarray, masked: np.ndarray,
-                      max_drafts: int) -> List[Tuple[int, int]]:
+                      max_drafts: int, keep_one: bool = True) -> List[Tuple[int, int]]:
     """Greedy selection: the N = min(max_drafts, r-1) masked positions of the current block
     with the highest draft confidence, in descending confidence (lower position first on
-    ties).  r-1 because every node of the chain must keep one masked position to predict."""
+    ties).  r-1 because every node of the chain must keep one masked position to predict;
+    ``keep_one=False`` (the chain goes on into the next block, whose positions the last nodes
+    predict) lets all r positions be candidates."""
     pos = [p for p in range(len(masked)) if masked[p]]
-    n = max(0, min(max_drafts, len(pos) - 1))
+    n = max(0, min(max_drafts, len(pos) - (1 if keep_one else 0)))
     order = sorted(pos, key=lambda p: (-draft_conf[p], p))
     return [(p, int(draft_tok[p])) for p in order[:n]]
 
@@ -502,6 +507,102 @@ class Oracle:
             out.append(ids)
             all_counts.append(counts)
         return np.concatenate(out), all_counts, cache
+
+    # ---- candidates from the next block (Section 3.2.2) -------------------------------
+    def verify_window(self, node_ids: np.ndarray, node_masked: np.ndarray, T: int, cache: Cache):
+        """Eq. 5 on nodes that span two consecutive blocks: rows [0, T) are the current block,
+        rows [T, T+T2) the next one, at positions cache.length ...  The window is block-causal
+        like the whole sequence: a row of the current block sees the prefix and its own block, a
+        row of the next block sees the prefix, the node's current block and its own block - which
+        is the current block's forward followed by the next block's forward with the current
+        block's K/V appended to the prefix.  Returns (tok, conf, gap), each [n, T+T2]."""
+        n, W = node_ids.shape
+        S = cache.length
+        toks, confs, gaps = [], [], []
+        for i in range(n):
+            la, ks, vs = self.forward_rows(node_ids[i, :T], S, cache)
+            ext = Cache(self.cfg)
+            ext.k = [np.concatenate([cache.k[l], ks[l][0]], axis=0) for l in range(self.cfg.n_layers)]
+            ext.v = [np.concatenate([cache.v[l], vs[l][0]], axis=0) for l in range(self.cfg.n_layers)]
+            lb, _, _ = self.forward_rows(node_ids[i, T:], S + T, ext)
+            logits = np.concatenate([la[0], lb[0]], axis=0)
+            t, c = token_and_confidence(logits, self.cfg.mask_id)
+            toks.append(t)
+            confs.append(c)
+            gaps.append(top2_gap(logits, self.cfg.mask_id))
+        return np.stack(toks), np.stack(confs), np.stack(gaps)
+
+    def generate_spill(self, prompt: np.ndarray, gen_len: int, block_len: int, max_drafts: int,
+                       trace: Optional[List[ForwardRecord]] = None):
+        """SSD whose candidate list runs on into the next block (Section 3.2.2: positions of
+        block j+1 are selected only when block j has fewer remaining positions than the draft
+        length).  While the current block has more than max_drafts masked positions a forward
+        is the single-block chain of ``decode_block_ssd``.  Otherwise the nodes span the window
+        [current block | next block]: the candidates are ALL masked positions of the current
+        block by draft confidence, then the most confident drafts of the next block up to
+        max_drafts in total; a node whose current block is full predicts in the next block, so
+        nothing of block j+1 is accepted before block j is complete (Section 3.1).  The next
+        block keeps its accepted tokens and drafts when it becomes the current one.
+        Returns (tokens [gen_len], accept counts per forward, forwards that used a window)."""
+        mid = self.cfg.mask_id
+        cache = self.prefill(np.asarray(prompt))
+        ranges = block_ranges(gen_len, block_len)
+        fresh = lambda T: dict(ids=np.full(T, mid, dtype=np.int64), masked=np.ones(T, dtype=bool), dt=None, dc=None)
+        cur = fresh(ranges[0][1] - ranges[0][0])
+        out, counts, windows = [], [], 0
+        for j, (lo, hi) in enumerate(ranges):
+            T = hi - lo
+            nxt = fresh(ranges[j + 1][1] - ranges[j + 1][0]) if j + 1 < len(ranges) else None
+            while cur["masked"].any():
+                r = int(cur["masked"].sum())
+                window = cur["dt"] is not None and nxt is not None and r <= max_drafts
+                if not window:
+                    cand = [] if cur["dt"] is None else select_candidates(cur["dt"], cur["dc"], cur["masked"], max_drafts)
+                    node_ids, node_masked = build_chain(cur["ids"], cur["masked"], cand, mid)
+                    tok, conf, gap, _ = self.verify(node_ids, node_masked, cache)
+                    pred = node_predictions(tok, conf, node_masked)
+                else:
+                    windows += 1
+                    T2 = len(nxt["ids"])
+                    # every masked position of the current block, then the next block's (which keeps one to predict)
+                    cand = select_candidates(cur["dt"], cur["dc"], cur["masked"], r, keep_one=False)
+                    if nxt["dt"] is not None:
+                        more = select_candidates(nxt["dt"], nxt["dc"], nxt["masked"], max_drafts - r)
+                        cand = cand + [(T + p, t) for (p, t) in more]
+                    ids2 = np.concatenate([cur["ids"], nxt["ids"]])
+                    masked2 = np.concatenate([cur["masked"], nxt["masked"]])
+                    node_ids, node_masked = build_chain(ids2, masked2, cand, mid)
+                    tok, conf, gap = self.verify_window(node_ids, node_masked, T, cache)
+                    # a node predicts in the current block while that has a masked position, else in the next
+                    pred = []
+                    for i in range(node_ids.shape[0]):
+                        in_cur = node_masked[i, :T].any()
+                        scope = np.zeros(T + T2, dtype=bool)
+                        scope[:T] = in_cur
+                        scope[T:] = not in_cur
+                        q = best_masked_position(conf[i], node_masked[i] & scope)
+                        pred.append((q, int(tok[i, q])))
+                a = accept_length(pred, cand)
+                accepted = list(cand[:a]) + [pred[a]]
+                if trace is not None:
+                    ib = cur["ids"].copy() if not window else np.concatenate([cur["ids"], nxt["ids"]])
+                    mb = cur["masked"].copy() if not window else np.concatenate([cur["masked"], nxt["masked"]])
+                    trace.append(ForwardRecord(j, cache.length, ib, mb, None, None, list(cand), node_ids, node_masked,
+                                               tok, conf, gap, pred, len(accepted), a))
+                for (p, t) in accepted:
+                    blk, pp = (cur, p) if p < T else (nxt, p - T)
+                    blk["ids"][pp] = t
+                    blk["masked"][pp] = False
+                cur["dt"] = np.where(cur["masked"], tok[a][:T], 0).astype(np.int64)
+                cur["dc"] = np.where(cur["masked"], conf[a][:T], 0.0)
+                if window:
+                    nxt["dt"] = np.where(nxt["masked"], tok[a][T:], 0).astype(np.int64)
+                    nxt["dc"] = np.where(nxt["masked"], conf[a][T:], 0.0)
+                counts.append(len(accepted))
+            self.commit_block(cur["ids"], cache)
+            out.append(cur["ids"])
+            cur = nxt
+        return np.concatenate(out), counts, windows
 
     # ---- acceptance-rate limit of self-drafting (Section 5.1, Table 2) ---------------
     def acceptance_limit_block(self, block_len: int, cache: Cache, draft_len: int, k_max: int):

@@ -519,3 +519,140 @@ def test_acceptance_limit_on_the_model_keeps_stepwise_tokens():
     got, red = o.acceptance_limit(prompt, w.gen_len, w.block_len, 2, 4)
     assert np.array_equal(got, want)
     assert np.all(np.diff(red) >= 0) and np.all(red >= 0) and np.all(red <= 2.0 / 3.0 + 1e-12)
+
+
+# ---------------------------------------------------------------------------------------
+# candidates that run on into the next block (Section 3.2.2) under the block order of Section 3.1
+# ---------------------------------------------------------------------------------------
+class ScriptedWindowOracle(ScriptedOracle):
+    """Scripted model over a window of two blocks: ``rule(ids_row, masked_row)`` sees the rows it is given
+    (one block, or current + next block) and answers (tok, conf) for them.  prefill / commit do nothing."""
+
+    def verify_window(self, node_ids, node_masked, T, cache):
+        tok, conf, gap, _ = self.verify(node_ids, node_masked, cache)
+        return tok, conf, gap
+
+    def prefill(self, prompt):
+        return NoCache()
+
+    def commit_block(self, ids, cache):
+        self.committed = getattr(self, "committed", []) + [np.array(ids)]
+
+
+def _stepwise_order_two_level(rule_for_block, n_blocks, B):
+    """Stepwise (position, token) order over several blocks: block by block, highest confidence first."""
+    order = []
+    for j in range(n_blocks):
+        ids = np.full(B, 999)
+        masked = np.ones(B, dtype=bool)
+        while masked.any():
+            t, c = rule_for_block(j, ids, masked)
+            q = so.best_masked_position(c, masked)
+            order.append((j, q, int(t[q])))
+            ids[q] = t[q]
+            masked[q] = False
+    return order
+
+
+@pytest.mark.parametrize("w", [SMALL, SMALL_GQA], ids=lambda w: w.name)
+@pytest.mark.parametrize("max_drafts", [0, 1, 2, 3, 5, 64])
+def test_spill_equals_stepwise_small(w, max_drafts):
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    for gen_len in (w.gen_len, w.gen_len + 3):                     # whole blocks, and a ragged last block
+        a, _, _ = o.generate(prompt, gen_len, w.block_len, mode="stepwise")
+        b, counts, windows = o.generate_spill(prompt, gen_len, w.block_len, max_drafts)
+        assert np.array_equal(a, b)
+        assert sum(counts) == gen_len and all(1 <= c <= max_drafts + 1 for c in counts)
+        if max_drafts == 0:
+            assert windows == 0 and counts == [1] * gen_len
+
+
+def test_spill_never_accepts_into_the_next_block_before_the_current_one_is_full():
+    w = SMALL_GQA
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    trace = []
+    o.generate_spill(prompt, w.gen_len, w.block_len, 5, trace=trace)
+    T = w.block_len
+    crossed = 0
+    for rec in trace:
+        if len(rec.ids_before) == T:
+            continue                                                # single-block forward
+        a = rec.last_node
+        accepted = list(rec.cand[:a]) + [rec.pred[a]]
+        masked = rec.masked_before.copy()
+        for (p, _) in accepted:
+            if p >= T:
+                assert not masked[:T].any()                         # the current block was complete by then
+                crossed += 1
+            masked[p] = False
+        # candidates: the whole current block first, then the next block
+        cur_part = [p for (p, _) in rec.cand if p < T]
+        assert rec.cand[:len(cur_part)] == [c for c in rec.cand if c[0] < T]
+        assert len(cur_part) == int(rec.masked_before[:T].sum())
+    assert crossed > 0
+
+
+def test_spill_accepts_the_stepwise_continuation_across_the_boundary():
+    """Scripted model whose confidences drift with the context: every forward accepts exactly 1 + the longest
+    common prefix of its candidate list with the true stepwise continuation (which finishes the current
+    block before it enters the next), capped by the list."""
+    B, V, n_blocks, N = 6, 50, 4, 4
+    rng = np.random.default_rng(2)
+    toks = rng.integers(0, V - 1, (n_blocks, B))
+    base = rng.random((n_blocks, B))
+    drift = 0.08 * rng.random((n_blocks, B + 1, B))
+
+    def block_rule(j, ids, masked):
+        return toks[j].copy(), base[j] + drift[j, int(masked.sum())]
+
+    state = {"j": 0}
+
+    def rule(ids, masked):
+        if len(ids) == B:
+            return block_rule(state["j"], ids, masked)
+        t0, c0 = block_rule(state["j"], ids[:B], masked[:B])
+        t1, c1 = block_rule(state["j"] + 1, ids[B:], masked[B:])
+        return np.concatenate([t0, t1]), np.concatenate([c0, c1])
+
+    order = _stepwise_order_two_level(block_rule, n_blocks, B)
+
+    class Tracking(ScriptedWindowOracle):
+        def commit_block(self, ids, cache):
+            super().commit_block(ids, cache)
+            state["j"] += 1
+
+    o = Tracking(V, rule)
+    trace = []
+    got, counts, windows = o.generate_spill(np.zeros(1, int), n_blocks * B, B, N, trace=trace)
+    assert np.array_equal(got, toks.reshape(-1)) and windows > 0
+    done = 0
+    for rec in trace:
+        cont = [((jj - rec.block) * B + q, t) for (jj, q, t) in order[done:]]
+        lcp = 0
+        while lcp < len(rec.cand) and rec.cand[lcp] == cont[lcp]:
+            lcp += 1
+        assert rec.accepted == lcp + 1
+        done += rec.accepted
+    assert done == n_blocks * B
+    # with drafts that are always right a window forward accepts its whole list plus one, and the generation
+    # takes fewer forwards than block-by-block chains
+    fixed = ScriptedWindowOracle(V, lambda ids, masked: (np.resize(toks[0], len(ids)), np.resize(np.linspace(0.9, 0.1, B), len(ids))))
+    tr_f = []
+    _, counts_f, _ = fixed.generate_spill(np.zeros(1, int), n_blocks * B, B, N - 1, trace=tr_f)
+    assert counts_f[0] == 1 and sum(counts_f) == n_blocks * B
+    assert all(rec.accepted == len(rec.cand) + 1 for rec in tr_f)
+    plain = ScriptedOracle(V, lambda ids, masked: (toks[0].copy(), np.linspace(0.9, 0.1, B)))
+    n_plain = sum(len(plain.decode_block_ssd(B, NoCache(), N - 1)[1]) for _ in range(n_blocks))
+    assert len(counts_f) < n_plain
+
+
+def test_spill_needs_fewer_forwards_on_the_tiny_peaked_model():
+    w = wl.TINY.replace(name="tiny_peaked", lm_head_scale=8.0)
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    a, counts, _ = o.generate(prompt, w.gen_len, w.block_len, mode="ssd", max_drafts=3)
+    b, counts_spill, windows = o.generate_spill(prompt, w.gen_len, w.block_len, 3)
+    assert np.array_equal(a, b)
+    assert windows > 0 and len(counts_spill) < sum(len(c) for c in counts)
