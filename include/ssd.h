@@ -110,12 +110,21 @@ int ssd_set_block_state(ssd_ctx* ctx, const int32_t* ids, const uint8_t* masked,
                         const int32_t* draft_tok, const float* draft_conf);
 /* Read the state back; any pointer may be NULL.  draft arrays are zero where not masked. */
 int ssd_get_block_state(ssd_ctx* ctx, int32_t* ids, uint8_t* masked, int32_t* draft_tok, float* draft_conf);
+/* The same for the next block's half of the window (only for a block begun with option "cross_block" > 0):
+ * HOST arrays [batch, cross_block].  ssd_set_block_state resets this half to "all masked, no drafts". */
+int ssd_set_next_block_state(ssd_ctx* ctx, const int32_t* ids, const uint8_t* masked,
+                             const int32_t* draft_tok, const float* draft_conf);
+int ssd_get_next_block_state(ssd_ctx* ctx, int32_t* ids, uint8_t* masked, int32_t* draft_tok, float* draft_conf);
 /* One iteration of Algorithm 1's loop for every unfinished sequence: candidate selection with
  * draft length N = min(max_drafts, masked-1) (0 if there are no drafts), chain of N+1 nodes,
  * one batched forward, traversal, state and draft update.  `max_drafts` < 0 uses the config's;
  * 0 gives a stepwise step.  accepted HOST [batch] (0 for finished sequences), n_nodes HOST
  * [batch]; both may be NULL. */
 int ssd_block_step(ssd_ctx* ctx, int32_t max_drafts, int32_t* accepted, int32_t* n_nodes);
+/* Test hook: (token, confidence) of the first n_rows rows of the latest forward, in its row order
+ * [sequence slot][node][rows of the node] (a node's rows: a finished block riding in front, if any, the
+ * current block, the next block's half of a window, if any); -1 / 0 on rows nothing was asked of. */
+int ssd_read_forward_outputs(ssd_ctx* ctx, int32_t n_rows, int32_t* out_tok, float* out_conf);
 /* Commit the (fully unmasked) block: its K/V are appended to the prefix cache and
  * ssd_cache_length grows by the block.  The paper leaves open how a block's K/V reach the cache;
  * here it is one forward over the block's final tokens, and by default that forward is not run
@@ -250,6 +259,17 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically (in
  *        steps of 128) while a prefix would need more than 7 parts;
  *   "max_drafts" lower the draft-length cap below the capacity fixed at creation;
+ *   "cross_block" T2 > 0 = candidates may come from the next block (Section 3.2.2): the block after the next
+ *        one to be begun is T2 tokens long.  While a sequence's current block holds more masked positions
+ *        than the draft length a forward is unchanged; once it cannot fill the chain (r <= max_drafts) the
+ *        nodes of the forward span the window [current block | next block] (block-causal, like the whole
+ *        sequence), the candidates are all masked positions of the current block followed by the next
+ *        block's most confident drafts, and a node predicts in the next block only once its current block
+ *        is full, so nothing of block j+1 is accepted before block j is complete (Section 3.1).  What the
+ *        next block has accepted, and its drafts, are kept for its own ssd_block_begin / ssd_decode_block
+ *        (same block_tokens); set the option again before every block and to 0 before the last.  The tokens
+ *        are still those of stepwise decoding.  A finished block whose commit rides in front of such a
+ *        block's first forward makes every node a chain [finished block | node].  0 = off (default);
  *   "mix_order"  1 = the verification tree is the greedy chain plus the mix-order branches of
  *        Section 5.2 (Table 3): every chain node that has a grandchild gets one more child, its state
  *        with candidate i+2 in place of candidate i+1; when a node predicts that candidate (right

@@ -585,9 +585,15 @@ class Oracle:
                 a = accept_length(pred, cand)
                 accepted = list(cand[:a]) + [pred[a]]
                 if trace is not None:
-                    ib = cur["ids"].copy() if not window else np.concatenate([cur["ids"], nxt["ids"]])
-                    mb = cur["masked"].copy() if not window else np.concatenate([cur["masked"], nxt["masked"]])
-                    trace.append(ForwardRecord(j, cache.length, ib, mb, None, None, list(cand), node_ids, node_masked,
+                    # a window forward records [current | next]; a next block without drafts shows tokens -1
+                    ib, mb = cur["ids"].copy(), cur["masked"].copy()
+                    db = None if cur["dt"] is None else cur["dt"].copy()
+                    cb = None if cur["dc"] is None else cur["dc"].copy()
+                    if window:
+                        ib, mb = np.concatenate([ib, nxt["ids"]]), np.concatenate([mb, nxt["masked"]])
+                        db = np.concatenate([db, nxt["dt"] if nxt["dt"] is not None else np.full(T2, -1)])
+                        cb = np.concatenate([cb, nxt["dc"] if nxt["dc"] is not None else np.zeros(T2)])
+                    trace.append(ForwardRecord(j, cache.length, ib, mb, db, cb, list(cand), node_ids, node_masked,
                                                tok, conf, gap, pred, len(accepted), a))
                 for (p, t) in accepted:
                     blk, pp = (cur, p) if p < T else (nxt, p - T)

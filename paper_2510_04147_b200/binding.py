@@ -27,6 +27,7 @@ PROF_TOP = PROF_FAMILIES[:5]          # the last four break "gemm" down by proje
 
 EXPORTS = ["ssd_create", "ssd_destroy", "ssd_last_error", "ssd_load_weights", "ssd_prefill", "ssd_prefill_dev",
            "ssd_decode_block", "ssd_block_begin", "ssd_set_block_state", "ssd_get_block_state", "ssd_block_step",
+           "ssd_set_next_block_state", "ssd_get_next_block_state", "ssd_read_forward_outputs",
            "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_write_cache", "ssd_verify_layers",
            "ssd_verify_forward_topk", "ssd_probe_acceptance_limit", "ssd_cache_length", "ssd_rewind", "ssd_gemm_bf16",
            "ssd_gemm_bf16_noalloc",
@@ -72,6 +73,9 @@ def load_library() -> C.CDLL:
     lib.ssd_block_begin.argtypes = [vp, i32]
     lib.ssd_set_block_state.argtypes = [vp, vp, vp, vp, vp]
     lib.ssd_get_block_state.argtypes = [vp, vp, vp, vp, vp]
+    lib.ssd_set_next_block_state.argtypes = [vp, vp, vp, vp, vp]
+    lib.ssd_get_next_block_state.argtypes = [vp, vp, vp, vp, vp]
+    lib.ssd_read_forward_outputs.argtypes = [vp, i32, vp, vp]
     lib.ssd_block_step.argtypes = [vp, i32, vp, vp]
     lib.ssd_block_commit.argtypes = [vp]
     lib.ssd_verify_forward.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
@@ -203,6 +207,27 @@ class Ssd:
         self._check(self.lib.ssd_get_block_state(self._ctx, _np_ptr(ids), _np_ptr(masked), _np_ptr(dt), _np_ptr(dc)))
         return ids, masked, dt, dc
 
+    def set_next_block_state(self, ids, masked, draft_tok=None, draft_conf=None):
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        masked = np.ascontiguousarray(masked, dtype=np.uint8)
+        dt = None if draft_tok is None else np.ascontiguousarray(draft_tok, dtype=np.int32)
+        dc = None if draft_conf is None else np.ascontiguousarray(draft_conf, dtype=np.float32)
+        self._check(self.lib.ssd_set_next_block_state(self._ctx, _np_ptr(ids), _np_ptr(masked), _np_ptr(dt), _np_ptr(dc)))
+
+    def get_next_block_state(self, batch: int, next_tokens: int):
+        ids = np.zeros((batch, next_tokens), np.int32)
+        masked = np.zeros((batch, next_tokens), np.uint8)
+        dt = np.zeros((batch, next_tokens), np.int32)
+        dc = np.zeros((batch, next_tokens), np.float32)
+        self._check(self.lib.ssd_get_next_block_state(self._ctx, _np_ptr(ids), _np_ptr(masked), _np_ptr(dt), _np_ptr(dc)))
+        return ids, masked, dt, dc
+
+    def read_forward_outputs(self, n_rows: int):
+        tok = np.zeros(n_rows, np.int32)
+        conf = np.zeros(n_rows, np.float32)
+        self._check(self.lib.ssd_read_forward_outputs(self._ctx, n_rows, _np_ptr(tok), _np_ptr(conf)))
+        return tok, conf
+
     def block_step(self, max_drafts: int, batch: int):
         acc = np.zeros(batch, np.int32)
         nn = np.zeros(batch, np.int32)
@@ -309,16 +334,21 @@ class Ssd:
             self.load_weights(name, t.contiguous())
             del t
 
-    def generate(self, mode: int, gen_len: int, block_len: int, batch: int):
+    def generate(self, mode: int, gen_len: int, block_len: int, batch: int, cross_block: bool = False):
         """All blocks of one generation after prefill.  Returns (tokens [batch, gen_len], accept counts
-        per block, forwards per block)."""
+        per block, forwards per block).  ``cross_block``: candidates may run on into the next block (the
+        option is set to the next block's length before every block, to 0 before the last)."""
         toks, accs, nfs = [], [], []
         done = 0
         while done < gen_len:
             t = min(block_len, gen_len - done)
+            if cross_block:
+                self.set_option("cross_block", min(block_len, gen_len - done - t))
             tok, acc, nf = self.decode_block(mode, t, batch)
             toks.append(tok)
             accs.append(acc)
             nfs.append(nf)
             done += t
+        if cross_block:
+            self.set_option("cross_block", 0)
         return np.concatenate(toks, axis=1), accs, nfs

@@ -485,7 +485,8 @@ int launch_attention_verify(cudaStream_t st, const AttnArgs& a) {
   if (a.hd != 64 && a.hd != 128) return -2;
   if (!a.qkv_partial || !a.rope || a.kv_split < kKTile || (a.kv_split % kKTile)) return -1;
   if ((a.cache_k_out != nullptr) != (a.cache_v_out != nullptr)) return -1;
-  if (a.cache_k_out != nullptr && a.map.rows_per_seq != a.map.T) return -1;   // commit: one node per sequence
+  // a commit writes the K/V of one node per sequence, or of the rows before chain_T0 of the first node
+  if (a.cache_k_out != nullptr && a.map.rows_per_seq != a.map.T && a.map.chain_T0 <= 0) return -1;
   const int n_prefix = (a.S + a.kv_split - 1) / a.kv_split;
   const int n_parts = n_prefix + 1;
   if (n_parts > kAttnMaxClusterParts) return -2;

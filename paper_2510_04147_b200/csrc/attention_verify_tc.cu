@@ -583,7 +583,8 @@ int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a) {
   if (a.kv_split < kKeys || (a.kv_split % kKeys) != 0) return 1;
   if ((a.cache_k_out != nullptr) != (a.cache_v_out != nullptr)) return -1;
   const int rps = a.map.rows_per_seq, T = a.map.T;
-  if (a.cache_k_out != nullptr && rps != T) return -1;
+  // a commit writes the K/V of one node per sequence, or of the rows before chain_T0 of the first node
+  if (a.cache_k_out != nullptr && rps != T && a.map.chain_T0 <= 0) return -1;
   const int n_prefix = (a.S + a.kv_split - 1) / a.kv_split;
   const int n_parts = n_prefix + 1;
   if (n_parts > kAttnMaxClusterParts) return 1;

@@ -210,13 +210,15 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g);
 int gemm_tc_init();   // resolves the driver entry point for tensor-map encoding
 
 // ---------------------------------------------------------------- tree build / acceptance
-struct BlockState {       // device arrays, [max_batch][block_len] unless noted
+struct BlockState {       // device arrays, [max_batch][stride] unless noted; a row holds [current block | next block]
   int* ids;
   uint8_t* masked;
   int* draft_tok;
   float* draft_conf;
-  int* has_drafts;        // [max_batch]
-  int* remaining;         // [max_batch] r
+  int* has_drafts;        // [max_batch] bit 0: the current block has drafts, bit 1: the next block has
+  int* remaining;         // [max_batch] r of the current block
+  int* remaining_nxt;     // [max_batch] masked positions of the next block
+  int* window;            // [max_batch] 1: the sequence takes candidates from the next block in the current forward
   int* cand_pos;          // [max_batch][block_len]
   int* cand_tok;
   int* n_cand;            // [max_batch] N of the current forward
@@ -226,20 +228,20 @@ struct BlockState {       // device arrays, [max_batch][block_len] unless noted
   int* last_pos;          // [max_batch] position and token of the last token the latest step accepted
   int* last_tok;          //             (the last valid node's own prediction)
   int* seq_map;           // [max_batch] slot -> sequence of the current forward
-  int stride;             // block_len (row pitch of the arrays above)
+  int stride;             // 2 * block_len (row pitch of the arrays above)
 };
 // Nodes of the verification tree for N candidates: the greedy chain has N + 1; the mix-order tree adds
 // one branch for every chain node that has a grandchild (N - 1 of them): 2N nodes for N >= 1.
 __host__ __device__ inline int tree_nodes(int N, int mix_order) { return N + 1 + ((mix_order && N >= 2) ? N - 1 : 0); }
-// slot a (= rank among unfinished sequences): candidates, node rows [a][n_cap][T].  With prev_ids
-// (device [batch][prev_stride]) the rows of a slot are [prev_T tokens of the finished block, not
-// masked][n_cap][T]: the layout of the forward that also commits the previous block.
-void launch_tree_build(cudaStream_t st, BlockState s, int batch, int T, int max_drafts, int n_cap, int mask_id,
+// slot a (= rank among unfinished sequences): candidates, node rows [a][n_cap][prev_T + T + T2].  A node's rows
+// are: the prev_T tokens of a finished block (prev_ids, device [batch][prev_stride]; nothing asked of them) when
+// the forward also commits that block, then the T rows of the current block, then - in a forward whose window
+// includes it - the T2 rows of the next block.
+void launch_tree_build(cudaStream_t st, BlockState s, int batch, int T, int T2, int max_drafts, int n_cap, int mask_id,
                        int* node_ids, uint8_t* node_masked, const int* prev_ids, int prev_T, int prev_stride,
                        int mix_order);
-// per slot: per-node best masked position, chain walk, state/draft update; a slot's node rows start
-// `row_offset` rows into its `slot_rows` rows (0 and n_cap * T without a finished block in front)
-void launch_accept(cudaStream_t st, BlockState s, int n_slots, int T, int n_cap, const int* tok, const float* conf,
-                   const uint8_t* node_masked, int* nonfinite_flag, int slot_rows, int row_offset, int mix_order);
+// per slot: per-node best masked position, walk, state/draft update (same row layout)
+void launch_accept(cudaStream_t st, BlockState s, int n_slots, int T, int T2, int n_cap, const int* tok, const float* conf,
+                   const uint8_t* node_masked, int* nonfinite_flag, int prev_T, int mix_order);
 
 }  // namespace ssd

@@ -8,6 +8,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <algorithm>
 #include <string>
 #include <vector>
 
@@ -80,7 +81,15 @@ struct ssd_ctx {
   // A finished block whose K/V are not in the cache yet: its commit is folded into the next block's
   // first forward (or run on its own when something else needs the cache first).
   int pending_T = 0;
-  int* pending_ids = nullptr;    // [max_batch][block_len] tokens of that block
+  int* pending_ids = nullptr;    // [max_batch][stride] tokens of that block
+  // Candidates from the next block (Section 3.2.2): the block after the current one is next_T tokens long
+  // (option "cross_block", 0 = there is none / off); window_T2 is the value the block in progress was begun
+  // with; when a block is committed its neighbour's state (tokens accepted across the boundary, drafts) is
+  // carried over to the next ssd_block_begin.
+  int next_T = 0, window_T2 = 0;
+  bool carry = false;
+  int carry_T = 0;
+  std::vector<int> h_remaining_nxt;
   int* prompt_stage = nullptr;   // [max_batch][max_seq] device copy of a host prompt (ssd_prefill)
   int fuse_commit = 1;
   std::vector<int> h_remaining, h_has_drafts, h_nodes, h_max_accept;
@@ -206,12 +215,13 @@ __global__ void sum_splits_kernel(const float* partial, int splits, size_t strid
   out[i] = v;
 }
 
-__global__ void block_init_kernel(BlockState s, int batch, int max_batch, int T, int mask_id) {
+// Fresh state: the current block (T positions) and the next one (T2, may be 0) all masked, no drafts.
+__global__ void block_init_kernel(BlockState s, int batch, int max_batch, int T, int T2, int mask_id) {
   const int b = blockIdx.x;
   for (int t = threadIdx.x; t < s.stride; t += blockDim.x) {
     const size_t o = (size_t)b * s.stride + t;
     s.ids[o] = mask_id;
-    s.masked[o] = (b < batch && t < T) ? 1 : 0;
+    s.masked[o] = (b < batch && t < T + T2) ? 1 : 0;
     s.draft_tok[o] = 0;
     s.draft_conf[o] = 0.f;
     s.cand_pos[o] = 0;
@@ -221,6 +231,44 @@ __global__ void block_init_kernel(BlockState s, int batch, int max_batch, int T,
   if (threadIdx.x == 0) {
     s.has_drafts[b] = 0;
     s.remaining[b] = (b < batch) ? T : 0;
+    s.remaining_nxt[b] = (b < batch) ? T2 : 0;
+    s.window[b] = 0;
+    s.n_cand[b] = 0;
+    s.n_forwards[b] = 0;
+    s.last_accept[b] = 0;
+    s.seq_map[b] = b;
+  }
+}
+
+// The next block (old_T .. old_T + T positions of the row) becomes the current one, with whatever was
+// accepted into it and its drafts; behind it a fresh next block of T2 positions.
+__global__ void block_shift_kernel(BlockState s, int batch, int old_T, int T, int T2, int mask_id) {
+  __shared__ int ids[512];
+  __shared__ int dt[512];
+  __shared__ float dc[512];
+  __shared__ uint8_t mk[512];
+  const int b = blockIdx.x;
+  for (int t = threadIdx.x; t < T; t += blockDim.x) {
+    const size_t o = (size_t)b * s.stride + old_T + t;
+    ids[t] = s.ids[o]; mk[t] = s.masked[o]; dt[t] = s.draft_tok[o]; dc[t] = s.draft_conf[o];
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < s.stride; t += blockDim.x) {
+    const size_t o = (size_t)b * s.stride + t;
+    const bool keep = t < T;
+    s.ids[o] = keep ? ids[t] : mask_id;
+    s.masked[o] = keep ? mk[t] : ((b < batch && t < T + T2) ? 1 : 0);
+    s.draft_tok[o] = keep ? dt[t] : 0;
+    s.draft_conf[o] = keep ? dc[t] : 0.f;
+    s.cand_pos[o] = 0;
+    s.cand_tok[o] = 0;
+    s.accept_log[o] = 0;
+  }
+  if (threadIdx.x == 0) {
+    s.has_drafts[b] = (s.has_drafts[b] >> 1) & 1;
+    s.remaining[b] = s.remaining_nxt[b];
+    s.remaining_nxt[b] = (b < batch) ? T2 : 0;
+    s.window[b] = 0;
     s.n_cand[b] = 0;
     s.n_forwards[b] = 0;
     s.last_accept[b] = 0;
@@ -254,6 +302,7 @@ struct LayerRange {
   bool from_stream = false;
   bool lm_head = true;
   int topk = 0;                  // > 0: the LM head also ranks the `topk` most probable tokens of every wanted row
+  bool commit_chain = false;     // the rows before chain_T0 of every sequence's first node go to the K/V cache
 };
 
 // One forward over R rows.  FILL: K/V go to the cache at positions pos0.., attention over the cache
@@ -324,7 +373,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     } else {
       // rotary embedding, node-local K/V and the merge of the key parts happen inside the attention kernel
       a.qkv_partial = c->partial; a.qkv_splits = g.splits; a.qkv_split_stride = (size_t)R * c->nqkv; a.rope = c->rope;
-      if (commit_form || map.chain_T0 > 0) {
+      if (commit_form || (map.chain_T0 > 0 && range.commit_chain)) {
         a.cache_k_out = c->cacheK + (size_t)l * c->cache_layer_stride;
         a.cache_v_out = c->cacheV + (size_t)l * c->cache_layer_stride;
       }
@@ -405,7 +454,7 @@ int ensure_topk_buffers(ssd_ctx* c) {
   ALLOC(c, c->tile_topi, tiles * c->R_dec * kLmTopKMax);
   ALLOC(c, c->topk_tok, (size_t)c->R_dec * kLmTopKMax);
   ALLOC(c, c->topk_prob, (size_t)c->R_dec * kLmTopKMax);
-  ALLOC(c, c->draft_top, (size_t)c->cfg.max_batch * c->cfg.block_len * kLmTopKMax);
+  ALLOC(c, c->draft_top, (size_t)c->cfg.max_batch * c->bs.stride * kLmTopKMax);
   ALLOC(c, c->probe_counts, kLmTopKMax + 1);
   CUDA_TRY(c, cudaStreamSynchronize(c->st));
   return SSD_OK;
@@ -525,6 +574,7 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
   c->split_down = auto_split(gemm_tiles(c->d), c->ffn_pad);
   c->h_remaining.assign(k.max_batch, 0);
   c->h_has_drafts.assign(k.max_batch, 0);
+  c->h_remaining_nxt.assign(k.max_batch, 0);
   c->h_nodes.assign(k.max_batch, 0);
   c->h_max_accept.assign(k.max_batch, 0);
 
@@ -588,8 +638,8 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     ALLOC(c, c->node_masked, R);
     ALLOC(c, c->flags, 4);
     ALLOC(c, c->marks, kMaxMarks);
-    const size_t sb = (size_t)k.max_batch * k.block_len;
-    c->bs.stride = k.block_len;
+    const size_t sb = (size_t)k.max_batch * 2 * k.block_len;      // a row holds [current block | next block]
+    c->bs.stride = 2 * k.block_len;
     ALLOC(c, c->bs.ids, sb); ALLOC(c, c->bs.masked, sb); ALLOC(c, c->bs.draft_tok, sb); ALLOC(c, c->bs.draft_conf, sb);
     ALLOC(c, c->bs.cand_pos, sb); ALLOC(c, c->bs.cand_tok, sb); ALLOC(c, c->bs.accept_log, sb);
     ALLOC(c, c->pending_ids, sb);
@@ -597,7 +647,8 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     ALLOC(c, c->bs.has_drafts, k.max_batch); ALLOC(c, c->bs.remaining, k.max_batch); ALLOC(c, c->bs.n_cand, k.max_batch);
     ALLOC(c, c->bs.n_forwards, k.max_batch); ALLOC(c, c->bs.last_accept, k.max_batch); ALLOC(c, c->bs.seq_map, k.max_batch);
     ALLOC(c, c->bs.last_pos, k.max_batch); ALLOC(c, c->bs.last_tok, k.max_batch);
-    CUDA_TRY(c, cudaMallocHost(&c->h_pinned, (2 + 3 * (size_t)k.max_batch) * sizeof(int)));
+    ALLOC(c, c->bs.remaining_nxt, k.max_batch); ALLOC(c, c->bs.window, k.max_batch);
+    CUDA_TRY(c, cudaMallocHost(&c->h_pinned, (2 + 5 * (size_t)k.max_batch) * sizeof(int)));
     CUDA_TRY(c, cudaStreamSynchronize(c->st));
     return SSD_OK;
   };
@@ -692,6 +743,7 @@ int ssd_prefill_dev(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t
   c->cache_len = prompt_len;
   c->in_block = false;
   c->pending_T = 0;
+  c->carry = false;
   return SSD_OK;
 }
 
@@ -724,6 +776,7 @@ int ssd_rewind(ssd_ctx* c, int32_t length) {
   c->pending_T = 0;                     // a block cut off entirely is never committed
   c->cache_len = length;
   c->in_block = false;
+  c->carry = false;
   return SSD_OK;
 }
 
@@ -733,13 +786,29 @@ int ssd_block_begin(ssd_ctx* c, int32_t T) {
   if (T < 1 || T > c->cfg.block_len) return fail(c, SSD_ERR_INVALID_ARG, "block_tokens %d outside [1, %d]", T, c->cfg.block_len);
   if (c->cache_len + c->pending_T + T > c->cfg.max_seq)
     return fail(c, SSD_ERR_OVERFLOW, "cache %d + block %d exceeds max_seq %d", c->cache_len + c->pending_T, T, c->cfg.max_seq);
-  block_init_kernel<<<c->cfg.max_batch, 128, 0, c->st>>>(c->bs, c->batch, c->cfg.max_batch, T, c->cfg.mask_id);
+  // the block after this one takes part as the second half of the window while there is room for it
+  int T2 = c->next_T;
+  if (T2 > 0 && c->cache_len + c->pending_T + T + T2 > c->cfg.max_seq) T2 = 0;
+  if (c->carry && c->carry_T == T) {
+    // this block was the second half of the previous block's window: keep what it already holds
+    block_shift_kernel<<<c->cfg.max_batch, 128, 0, c->st>>>(c->bs, c->batch, c->block_tokens, T, T2, c->cfg.mask_id);
+    for (int b = 0; b < c->cfg.max_batch; ++b) {
+      c->h_remaining[b] = b < c->batch ? c->h_remaining_nxt[b] : 0;
+      c->h_has_drafts[b] = (c->h_has_drafts[b] >> 1) & 1;
+      c->h_remaining_nxt[b] = b < c->batch ? T2 : 0;
+    }
+  } else {
+    block_init_kernel<<<c->cfg.max_batch, 128, 0, c->st>>>(c->bs, c->batch, c->cfg.max_batch, T, T2, c->cfg.mask_id);
+    for (int b = 0; b < c->cfg.max_batch; ++b) {
+      c->h_remaining[b] = b < c->batch ? T : 0;
+      c->h_has_drafts[b] = 0;
+      c->h_remaining_nxt[b] = b < c->batch ? T2 : 0;
+    }
+  }
   c->launches += 1;
   CUDA_TRY(c, cudaGetLastError());
-  for (int b = 0; b < c->cfg.max_batch; ++b) {
-    c->h_remaining[b] = b < c->batch ? T : 0;
-    c->h_has_drafts[b] = 0;
-  }
+  c->carry = false;
+  c->window_T2 = T2;
   c->block_tokens = T;
   c->in_block = true;
   return SSD_OK;
@@ -754,6 +823,10 @@ int ssd_set_block_state(ssd_ctx* c, const int32_t* ids, const uint8_t* masked, c
     if (frc) return frc;
   }
   const int T = c->block_tokens, st = c->bs.stride;
+  // (the next block's half of the window starts afresh; ssd_set_next_block_state can fill it)
+  block_init_kernel<<<c->cfg.max_batch, 128, 0, c->st>>>(c->bs, c->batch, c->cfg.max_batch, T, c->window_T2, c->cfg.mask_id);
+  c->launches += 1;
+  for (int b = 0; b < c->batch; ++b) c->h_remaining_nxt[b] = c->window_T2;
   for (int b = 0; b < c->batch; ++b) {
     int r = 0;
     for (int t = 0; t < T; ++t) {
@@ -803,28 +876,42 @@ struct ProbeStep { int k_max; bool open_round; };
 
 int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nullptr) {
   const int T = c->block_tokens, B = c->batch;
-  int active = 0, n_cap = 1;
-  for (int b = 0; b < B; ++b) {
-    c->h_nodes[b] = 0;
-    c->h_max_accept[b] = 0;
-    if (c->h_remaining[b] <= 0) continue;
-    ++active;
-    const int N = c->h_has_drafts[b] ? (md < c->h_remaining[b] - 1 ? md : c->h_remaining[b] - 1) : 0;
-    c->h_nodes[b] = tree_nodes(N, c->mix_order);
-    c->h_max_accept[b] = N + 1;            // (a branch ends the walk at most N tokens in)
-    if (c->h_nodes[b] > n_cap) n_cap = c->h_nodes[b];
-  }
-  if (n_cap > c->n_max) return fail(c, SSD_ERR_OVERFLOW, "a tree of %d nodes exceeds the capacity of %d nodes fixed at creation", n_cap, c->n_max);
+  // chain length of sequence b; with `window` it may take candidates from the next block (Section 3.2.2)
+  auto drafts_of = [&](int b, bool window) -> int {
+    const int r = c->h_remaining[b];
+    if (!(c->h_has_drafts[b] & 1)) return 0;
+    if (window && r <= md) {
+      int more = 0;
+      if (c->h_has_drafts[b] & 2) more = std::max(0, std::min(md - r, c->h_remaining_nxt[b] - 1));
+      return r + more;
+    }
+    return md < r - 1 ? md : r - 1;
+  };
+  auto shape = [&](bool window, int* active_out) -> int {
+    int active = 0, n_cap = 1;
+    for (int b = 0; b < B; ++b) {
+      c->h_nodes[b] = 0;
+      c->h_max_accept[b] = 0;
+      if (c->h_remaining[b] <= 0) continue;
+      ++active;
+      const int N = drafts_of(b, window);
+      c->h_nodes[b] = tree_nodes(N, c->mix_order);
+      c->h_max_accept[b] = N + 1;            // (a branch ends the walk at most N tokens in)
+      if (c->h_nodes[b] > n_cap) n_cap = c->h_nodes[b];
+    }
+    *active_out = active;
+    return n_cap;
+  };
+  int active = 0;
+  int n_cap = shape(false, &active);
   *launched = active > 0;
   if (active == 0) return SSD_OK;
-  // A block waiting for its commit rides in front of the first forward of this block: per sequence
-  // one causal chain [finished block | this block, all MASK].  Only a fresh block qualifies (every
-  // sequence untouched, so one node each); otherwise the commit runs on its own first.
+  // A block waiting for its commit rides in front of this block's forward: every node is one causal chain
+  // [finished block | this block's node state], and the first node's finished-block rows write the K/V.  All
+  // sequences must take part (each has a block to commit); otherwise the commit runs on its own first.
   int Tp = 0;
   if (c->pending_T > 0) {
-    bool fresh = active == B && n_cap == 1;
-    for (int b = 0; b < B && fresh; ++b) fresh = c->h_remaining[b] == T && !c->h_has_drafts[b];
-    if (fresh && B * (c->pending_T + T) <= c->R_dec) {
+    if (active == B && active * n_cap * (c->pending_T + T) <= c->R_dec) {
       Tp = c->pending_T;
     } else {
       const int frc = flush_pending(c);
@@ -832,30 +919,47 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nu
       CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
     }
   }
-  const int slot_rows = Tp + n_cap * T;
+  // The window [this block | next block]: whenever a sequence can no longer fill its chain from this block.
+  int T2 = 0;
+  if (Tp == 0 && c->window_T2 > 0 && !c->mix_order && !probe) {
+    bool any = false;
+    for (int b = 0; b < B; ++b) any = any || (c->h_remaining[b] > 0 && (c->h_has_drafts[b] & 1) && c->h_remaining[b] <= md);
+    if (any) {
+      int act2 = 0;
+      const int cap2 = shape(true, &act2);
+      if (cap2 <= c->n_max && active * cap2 * (T + c->window_T2) <= c->R_dec) {
+        T2 = c->window_T2;
+        n_cap = cap2;
+      } else {
+        n_cap = shape(false, &act2);         // no room for the window: single-block chains
+      }
+    }
+  }
+  if (n_cap > c->n_max) return fail(c, SSD_ERR_OVERFLOW, "a tree of %d nodes exceeds the capacity of %d nodes fixed at creation", n_cap, c->n_max);
+  const int node_rows = Tp + T + T2;
+  const int slot_rows = n_cap * node_rows;
   const int R = active * slot_rows;
+  if (R > c->R_dec) return fail(c, SSD_ERR_OVERFLOW, "%d rows exceed the capacity %d set by max_batch/max_drafts/block_len", R, c->R_dec);
   {
     Scope sc(c, SSD_PROF_TREE, (double)R * 5);
-    launch_tree_build(c->st, c->bs, B, T, md, n_cap, c->cfg.mask_id, c->node_ids, c->node_masked,
+    launch_tree_build(c->st, c->bs, B, T, T2, md, n_cap, c->cfg.mask_id, c->node_ids, c->node_masked,
                       Tp > 0 ? c->pending_ids : nullptr, Tp, c->bs.stride, c->mix_order);
   }
-  RowMap map{n_cap * T, T, c->cache_len, 0, c->bs.seq_map};
-  if (Tp > 0) {                // one chain of Tp + T rows at positions cache_len ...
-    map.rows_per_seq = slot_rows;
-    map.T = slot_rows;
-    map.chain_T0 = Tp;
-  }
+  RowMap map{slot_rows, node_rows, c->cache_len, 0, c->bs.seq_map};
+  if (Tp > 0) map.chain_T0 = Tp;                // a node's rows: [finished block | this block]
+  else if (T2 > 0) map.chain_T0 = T;            //                [this block | next block]
   if (active <= 8) {           // the host mirrors `remaining`, so it knows the slot -> sequence map too
     for (int b = 0; b < B; ++b)
       if (c->h_remaining[b] > 0) map.inline_seq[map.n_inline++] = b;
   }
   LayerRange range;
   if (probe && probe->open_round) range.topk = probe->k_max;
+  range.commit_chain = Tp > 0;
   int rc = forward(c, FWD_VERIFY, c->node_ids, R, map, active, false, c->node_masked, range);
   if (rc) return rc;
   {
     Scope sc(c, SSD_PROF_TREE, (double)R * 9);
-    launch_accept(c->st, c->bs, active, T, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1, slot_rows, Tp, c->mix_order);
+    launch_accept(c->st, c->bs, active, T, T2, n_cap, c->tok, c->conf, c->node_masked, c->flags + 1, Tp, c->mix_order);
   }
   if (probe) {
     // the forward that opens a round is the draft: keep its top-k per block position; every later token of
@@ -871,7 +975,7 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nu
     c->pending_T = 0;
   }
   for (int b = 0; b < B; ++b)
-    if (c->h_nodes[b] > 0) c->h_has_drafts[b] = 1;
+    if (c->h_nodes[b] > 0) c->h_has_drafts[b] |= 1 | ((T2 > 0 && c->h_remaining[b] <= md && (c->h_has_drafts[b] & 1)) ? 2 : 0);
   return SSD_OK;
 }
 
@@ -884,11 +988,15 @@ int step_collect(ssd_ctx* c, int32_t* accepted, int32_t* n_nodes) {
   CUDA_TRY(c, cudaMemcpyAsync(hp + 2, c->bs.remaining, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   if (accepted) CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + mb, c->bs.last_accept, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   if (n_nodes) CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 2 * mb, c->bs.n_cand, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 3 * mb, c->bs.remaining_nxt, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 4 * mb, c->bs.has_drafts, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   CUDA_TRY(c, cudaStreamSynchronize(c->st));
   const int rc = check_flags_after_sync(c);
   if (rc) return rc;
   for (int b = 0; b < B; ++b) {
     c->h_remaining[b] = hp[2 + b];
+    c->h_remaining_nxt[b] = hp[2 + 3 * mb + b];
+    c->h_has_drafts[b] = hp[2 + 4 * mb + b];
     if (accepted) accepted[b] = hp[2 + mb + b];
     if (n_nodes) n_nodes[b] = c->h_nodes[b] > 0 ? tree_nodes(hp[2 + 2 * mb + b], c->mix_order) : 0;
   }
@@ -932,6 +1040,50 @@ int ssd_block_commit(ssd_ctx* c) {
     if (rc) return rc;
   }
   c->in_block = false;
+  // what the window already holds of the next block is kept for its ssd_block_begin
+  c->carry = c->window_T2 > 0;
+  c->carry_T = c->window_T2;
+  return SSD_OK;
+}
+
+int ssd_set_next_block_state(ssd_ctx* c, const int32_t* ids, const uint8_t* masked, const int32_t* draft_tok, const float* draft_conf) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
+  if (c->window_T2 <= 0) return fail(c, SSD_ERR_STATE, "the block in progress was begun without a next block (option cross_block)");
+  if (!ids || !masked || ((draft_tok == nullptr) != (draft_conf == nullptr))) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
+  const int T = c->block_tokens, T2 = c->window_T2, st = c->bs.stride;
+  for (int b = 0; b < c->batch; ++b) {
+    int r = 0;
+    for (int t = 0; t < T2; ++t) {
+      r += masked[b * T2 + t] ? 1 : 0;
+      if (!masked[b * T2 + t] && (ids[b * T2 + t] < 0 || ids[b * T2 + t] >= c->V)) return fail(c, SSD_ERR_INVALID_ARG, "token id outside the vocabulary");
+      if (draft_tok && masked[b * T2 + t] && (draft_tok[b * T2 + t] < 0 || draft_tok[b * T2 + t] >= c->V)) return fail(c, SSD_ERR_INVALID_ARG, "draft id outside the vocabulary");
+    }
+    c->h_remaining_nxt[b] = r;
+    c->h_has_drafts[b] = (c->h_has_drafts[b] & 1) | (draft_tok ? 2 : 0);
+  }
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->bs.ids + T, st * sizeof(int), ids, T2 * sizeof(int), T2 * sizeof(int), c->batch, cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->bs.masked + T, st, masked, T2, T2, c->batch, cudaMemcpyHostToDevice, c->st));
+  if (draft_tok) {
+    CUDA_TRY(c, cudaMemcpy2DAsync(c->bs.draft_tok + T, st * sizeof(int), draft_tok, T2 * sizeof(int), T2 * sizeof(int), c->batch, cudaMemcpyHostToDevice, c->st));
+    CUDA_TRY(c, cudaMemcpy2DAsync(c->bs.draft_conf + T, st * sizeof(float), draft_conf, T2 * sizeof(float), T2 * sizeof(float), c->batch, cudaMemcpyHostToDevice, c->st));
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(c->bs.remaining_nxt, c->h_remaining_nxt.data(), c->batch * sizeof(int), cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaMemcpyAsync(c->bs.has_drafts, c->h_has_drafts.data(), c->batch * sizeof(int), cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  return SSD_OK;
+}
+
+int ssd_get_next_block_state(ssd_ctx* c, int32_t* ids, uint8_t* masked, int32_t* draft_tok, float* draft_conf) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (!c->in_block) return fail(c, SSD_ERR_STATE, "no block in progress");
+  if (c->window_T2 <= 0) return fail(c, SSD_ERR_STATE, "the block in progress was begun without a next block (option cross_block)");
+  const int T = c->block_tokens, T2 = c->window_T2, st = c->bs.stride;
+  if (ids) CUDA_TRY(c, cudaMemcpy2DAsync(ids, T2 * sizeof(int), c->bs.ids + T, st * sizeof(int), T2 * sizeof(int), c->batch, cudaMemcpyDeviceToHost, c->st));
+  if (masked) CUDA_TRY(c, cudaMemcpy2DAsync(masked, T2, c->bs.masked + T, st, T2, c->batch, cudaMemcpyDeviceToHost, c->st));
+  if (draft_tok) CUDA_TRY(c, cudaMemcpy2DAsync(draft_tok, T2 * sizeof(int), c->bs.draft_tok + T, st * sizeof(int), T2 * sizeof(int), c->batch, cudaMemcpyDeviceToHost, c->st));
+  if (draft_conf) CUDA_TRY(c, cudaMemcpy2DAsync(draft_conf, T2 * sizeof(float), c->bs.draft_conf + T, st * sizeof(float), T2 * sizeof(float), c->batch, cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
   return SSD_OK;
 }
 
@@ -1144,6 +1296,15 @@ int ssd_probe_acceptance_limit(ssd_ctx* c, int32_t T, int32_t draft_len, int32_t
   return ssd_block_commit(c);
 }
 
+int ssd_read_forward_outputs(ssd_ctx* c, int32_t n_rows, int32_t* out_tok, float* out_conf) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (n_rows < 0 || n_rows > c->R_cap) return fail(c, SSD_ERR_INVALID_ARG, "row count outside [0, %d]", c->R_cap);
+  if (out_tok) CUDA_TRY(c, cudaMemcpyAsync(out_tok, c->tok, (size_t)n_rows * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  if (out_conf) CUDA_TRY(c, cudaMemcpyAsync(out_conf, c->conf, (size_t)n_rows * sizeof(float), cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(c, cudaStreamSynchronize(c->st));
+  return SSD_OK;
+}
+
 int ssd_gemm_bf16(ssd_ctx* c, const void* x_dev, const void* w_dev, float* out_dev, int32_t rows, int32_t n, int32_t k, int32_t split_k) {
   if (!c) return SSD_ERR_INVALID_ARG;
   if (!x_dev || !w_dev || !out_dev) return fail(c, SSD_ERR_INVALID_ARG, "null argument");
@@ -1243,6 +1404,11 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "max_drafts")) {
     if (value < 0 || value + 1 > c->n_max) return fail(c, SSD_ERR_INVALID_ARG, "max_drafts must be in [0, %d] (the capacity fixed at creation)", c->n_max - 1);
     c->cfg.max_drafts = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "cross_block")) {
+    if (value < 0 || value > c->cfg.block_len) return fail(c, SSD_ERR_INVALID_ARG, "cross_block is the length of the block after the next one to be begun: 0 (none) .. %d", c->cfg.block_len);
+    c->next_T = value;
     return SSD_OK;
   }
   if (!strcmp(key, "mix_order")) {

@@ -751,3 +751,170 @@ def test_acceptance_limit_probe_matches_a_recount_and_the_oracle(peaked_ssd, tin
     assert osteps == steps
     if np.array_equal(oids, tok_step[0]):
         assert np.all(np.abs(matched - omatched) <= 1)
+
+
+# ------------------------------------------------------------------------------------------
+# candidates from the next block (Section 3.2.2)
+# ------------------------------------------------------------------------------------------
+def _equal_up_to_a_near_tie(got, want, oracle, prompt, gen_len, w, rtol):
+    """`got` equals `want` (stepwise tokens), or first differs at a position whose stepwise decision the oracle
+    sees as a near-tie within the rounding tolerance (token gap or position margin); after such a position the
+    contexts differ and nothing more can be compared."""
+    diff = np.nonzero(got != want)[0]
+    if len(diff) == 0:
+        return True
+    first = int(diff[0])
+    trace = []
+    oracle.generate(prompt, gen_len, w.block_len, mode="stepwise", trace=trace)
+    for rec in trace:
+        q, _ = rec.pred[0]
+        pos = rec.block * w.block_len + q
+        cm = np.sort(np.where(rec.node_masked[0], rec.conf[0], -1.0))[::-1]
+        margin = cm[0] - cm[1] if len(cm) > 1 and cm[1] >= 0 else np.inf
+        near = (rec.gap[0, q] <= 2 * rtol * rec.conf[0, q]) or (margin <= 2 * rtol * cm[0])
+        if near and pos <= first:
+            return True                                   # a decision at or before the first difference was a near-tie
+        if pos == first:
+            return bool(near)
+    return False
+
+
+def test_cross_block_generation_is_lossless_and_saves_forwards(tiny_oracles):
+    """GPU SSD with candidates that run on into the next block decodes the stepwise tokens, with fewer
+    forwards than block-by-block chains.  (Plain SSD equals stepwise bit for bit.  Across a block boundary a
+    window node sees the finished block as rows of its own forward where the stepwise forward reads the same
+    K/V from the cache: the same values summed in another order, so a decision that is a near-tie within
+    rounding noise may fall the other way; anything else must agree.)"""
+    w = PEAKED
+    o64, _ = tiny_oracles[w.name]
+    rtol = CONF_RTOL * w.lm_head_scale
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    N = 3
+    ssd = _make_ssd(w, max_drafts=2 * N + 1)              # room for windows of two blocks
+    try:
+        ssd.set_option("max_drafts", N)
+        ssd.prefill(prompt)
+        tok_s, _, _ = ssd.generate(b.MODE_STEPWISE, w.gen_len, w.block_len, 1)
+        ssd.prefill(prompt)
+        tok_p, acc_p, nf_p = ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1)
+        ssd.prefill(prompt)
+        tok_x, acc_x, nf_x = ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1, cross_block=True)
+        assert ssd.cache_length() == w.prompt_len + w.gen_len
+        # ragged last block and a second batch entry
+        prompts2 = wl.make_prompts(w, batch=2).numpy()
+        ssd2 = _make_ssd(w, max_drafts=2 * N + 1, max_batch=2)
+        try:
+            ssd2.set_option("max_drafts", N)
+            ssd2.prefill(prompts2)
+            r_s, _, _ = ssd2.generate(b.MODE_STEPWISE, 40, w.block_len, 2)
+            ssd2.prefill(prompts2)
+            r_x, _, _ = ssd2.generate(b.MODE_SSD, 40, w.block_len, 2, cross_block=True)
+        finally:
+            ssd2.destroy()
+    finally:
+        ssd.destroy()
+    assert np.array_equal(tok_p, tok_s)
+    assert _equal_up_to_a_near_tie(tok_x[0], tok_s[0], o64, prompt[0], w.gen_len, w, rtol)
+    for i in range(2):
+        assert _equal_up_to_a_near_tie(r_x[i], r_s[i], o64, prompts2[i], 40, w, rtol)
+    f_plain, f_cross = sum(int(n[0]) for n in nf_p), sum(int(n[0]) for n in nf_x)
+    print(f"forwards: block by block {f_plain}, with candidates from the next block {f_cross}")
+    assert f_cross < f_plain
+    total = 0
+    for acc, nf in zip(acc_x, nf_x):
+        used = acc[0][:nf[0]]
+        assert np.all(used >= 1) and np.all(used <= N + 1)
+        total += used.sum()
+    assert total == w.gen_len                              # every token was accepted by exactly one forward
+
+
+def test_cross_block_window_steps_match_oracle(tiny_oracles):
+    """Window forwards of the oracle's run replayed on the GPU from the oracle's state of BOTH blocks.
+      numeric - the forward's confidences on every asked row of every window node against the oracle's;
+      integer - candidate list, per-node prediction scope (current block while it has a masked row, else the
+                next block), walk, new state and drafts of both blocks: bit-exact against the oracle's logic
+                applied to the GPU forward's own outputs, no exemption; and equal to the oracle's own accepted
+                count wherever the oracle's decisions have safe margins."""
+    w = PEAKED
+    _, ob = tiny_oracles[w.name]
+    prompt = wl.make_prompts(w).numpy()
+    N, T = 5, w.block_len
+    trace = []
+    tokens, _, windows = ob.generate_spill(prompt[0], w.gen_len, T, N, trace=trace)
+    assert windows > 0
+    rtol = CONF_RTOL * w.lm_head_scale
+    ssd = _make_ssd(w, max_drafts=2 * N + 1)
+    checked = crossed = strict = 0
+    try:
+        ssd.set_option("max_drafts", N)
+        ssd.set_option("fuse_commit", 0)
+        ssd.prefill(prompt)
+        cur_block = 0
+        for rec in trace:
+            if rec.block != cur_block:
+                ssd.set_option("cross_block", 0)
+                ssd.block_begin(T)
+                ssd.set_block_state(tokens[cur_block * T:(cur_block + 1) * T][None], np.zeros((1, T), np.uint8))
+                ssd.block_commit()
+                cur_block = rec.block
+            if len(rec.ids_before) == T:
+                continue                                          # single-block forwards are covered elsewhere
+            T2 = len(rec.ids_before) - T
+            W = T + T2
+            ssd.set_option("cross_block", T2)
+            ssd.block_begin(T)
+            dc32 = rec.draft_conf.astype(np.float32)
+            ssd.set_block_state(rec.ids_before[None, :T], rec.masked_before[None, :T].astype(np.uint8),
+                                rec.draft_tok[None, :T], dc32[None, :T])
+            nxt_has = rec.draft_tok[T:].max() >= 0
+            if nxt_has:
+                ssd.set_next_block_state(rec.ids_before[None, T:], rec.masked_before[None, T:].astype(np.uint8),
+                                         np.maximum(rec.draft_tok[None, T:], 0), dc32[None, T:])
+            else:
+                ssd.set_next_block_state(rec.ids_before[None, T:], rec.masked_before[None, T:].astype(np.uint8))
+            acc, nn = ssd.block_step(N, 1)
+            n = rec.node_ids.shape[0]
+            assert nn[0] == n
+            tok_g, conf_g = ssd.read_forward_outputs(n * W)
+            tok_g, conf_g = tok_g.reshape(n, W), conf_g.reshape(n, W)
+            m = rec.node_masked
+            # ---- numeric layer (inputs are the oracle's; float32 drafts may reorder exact-tie candidates only)
+            assert np.all(tok_g[~m] == -1)
+            assert np.allclose(conf_g[m], rec.conf[m], rtol=rtol, atol=1e-6)
+            # ---- integer layer on the GPU's own outputs
+            pred = []
+            for i in range(n):
+                scope = m[i].copy()
+                if m[i, :T].any():
+                    scope[T:] = False
+                else:
+                    scope[:T] = False
+                q = so.best_masked_position(conf_g[i], scope)
+                pred.append((q, int(tok_g[i, q])))
+            a = so.accept_length(pred, rec.cand)
+            accepted = list(rec.cand[:a]) + [pred[a]]
+            assert acc[0] == len(accepted)
+            want_ids, want_m = rec.ids_before.copy(), rec.masked_before.copy()
+            seen_next = False
+            for (p, t) in accepted:
+                if p >= T:
+                    assert not want_m[:T].any()                   # block order: the current block was full by then
+                    crossed += 1
+                want_ids[p], want_m[p] = t, False
+            ids0, m0, dt0, dc0 = ssd.get_block_state(1, T)
+            ids1, m1, dt1, dc1 = ssd.get_next_block_state(1, T2)
+            ids_g, m_g = np.concatenate([ids0[0], ids1[0]]), np.concatenate([m0[0], m1[0]]).astype(bool)
+            dt_g, dc_g = np.concatenate([dt0[0], dt1[0]]), np.concatenate([dc0[0], dc1[0]])
+            assert np.array_equal(m_g, want_m) and np.array_equal(ids_g[~want_m], want_ids[~want_m])
+            assert np.array_equal(dt_g[want_m], tok_g[a][want_m])
+            assert np.array_equal(dc_g[want_m].view(np.uint32), conf_g[a][want_m].view(np.uint32))
+            checked += 1
+            if pred == list(rec.pred):                             # same decisions as the oracle: same count
+                strict += 1
+                assert acc[0] == rec.accepted
+    finally:
+        ssd.destroy()
+    print(f"cross-block: {checked} window forwards replayed, {strict} with the oracle's own decisions, "
+          f"{crossed} tokens accepted across the boundary")
+    assert checked > 0 and crossed > 0
