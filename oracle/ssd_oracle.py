@@ -21,6 +21,9 @@ What is defined here, and from where:
 * candidates that run on into the next block when the current one cannot fill the chain
   (Section 3.2.2), under the block order of Section 3.1 -> ``Oracle.verify_window``,
   ``Oracle.generate_spill``;
+* the dual cache with a refresh interval of the paper's experimental set-up (Section 4.1) and
+  the chain cap that keeps SSD identical to stepwise decoding under it ->
+  ``Oracle.refresh_all``, ``Oracle.generate_dual_cache``;
 * the acceptance-rate limit of self-drafting, Section 5.1 / Table 2 (how many stepwise
   tokens lie within the draft forward's top-k candidates) -> ``token_topk``,
   ``Oracle.acceptance_limit``;
@@ -609,6 +612,67 @@ class Oracle:
             out.append(cur["ids"])
             cur = nxt
         return np.concatenate(out), counts, windows
+
+    # ---- dual cache with a refresh interval (Section 4.1, implementation details) ------
+    def refresh_all(self, tokens: np.ndarray) -> Cache:
+        """K/V of EVERY position of the sequence [prompt | generation, MASK where undecoded] from one
+        forward in which all positions see all positions (no block structure)."""
+        cache = Cache(self.cfg)
+        _, ks, vs = self.forward_rows(np.asarray(tokens), 0, cache, want_logits=False)
+        cache.append([k[0] for k in ks], [v[0] for v in vs])
+        return cache
+
+    def generate_dual_cache(self, prompt: np.ndarray, gen_len: int, block_len: int, refresh: int,
+                            max_drafts: int = 0, counts_out: Optional[list] = None):
+        """Decoding under the dual cache of the paper's set-up (Section 4.1): the K/V of all positions
+        OUTSIDE the current block - the prefix and the still masked suffix - are cached, a forward
+        computes the current block's rows against them, and the cache is refreshed (``refresh_all``)
+        at the start of every block and again whenever `refresh` tokens have been decoded since the
+        last refresh.  Between refreshes the cached K/V are stale: this is an approximation of
+        full-sequence decoding, so stepwise decoding is defined WITH the schedule.  max_drafts = 0 is
+        that stepwise decoding; with max_drafts > 0 the verification chain is additionally capped so
+        that a forward never accepts past the next refresh point (draft length <= refresh - decoded
+        since the last refresh - 1), which keeps the tokens those of stepwise decoding under the same
+        schedule.  Returns (tokens [gen_len], forwards, refreshes)."""
+        mid = self.cfg.mask_id
+        P = len(prompt)
+        x = np.concatenate([np.asarray(prompt, dtype=np.int64), np.full(gen_len, mid, dtype=np.int64)])
+        forwards = refreshes = 0
+        for (lo, hi) in block_ranges(gen_len, block_len):
+            S, T = P + lo, hi - lo
+            ids = np.full(T, mid, dtype=np.int64)
+            masked = np.ones(T, dtype=bool)
+            dt = dc = None
+            since = refresh                                     # a block starts with a refresh
+            while masked.any():
+                if since >= refresh:
+                    full = self.refresh_all(x)
+                    refreshes += 1
+                    since = 0
+                    outside = Cache(self.cfg)                   # everything but the current block's rows
+                    outside.k = [np.concatenate([k[:S], k[S + T:]], axis=0) for k in full.k]
+                    outside.v = [np.concatenate([v[:S], v[S + T:]], axis=0) for v in full.v]
+                cap = min(max_drafts, refresh - since - 1)
+                cand = [] if dt is None else select_candidates(dt, dc, masked, cap)
+                node_ids, node_masked = build_chain(ids, masked, cand, mid)
+                # (the cached keys carry their positions inside the rotated K, so they need not be a prefix)
+                logits, _, _ = self.forward_rows(node_ids, S, outside)
+                n, _, V = logits.shape
+                tok, conf = token_and_confidence(logits.reshape(n * T, V), mid)
+                tok, conf = tok.reshape(n, T), conf.reshape(n, T)
+                pred = node_predictions(tok, conf, node_masked)
+                a = accept_length(pred, cand)
+                for (p, t) in list(cand[:a]) + [pred[a]]:
+                    ids[p] = t
+                    masked[p] = False
+                x[S:S + T] = np.where(masked, mid, ids)
+                dt = np.where(masked, tok[a], 0).astype(np.int64)
+                dc = np.where(masked, conf[a], 0.0)
+                since += a + 1
+                forwards += 1
+                if counts_out is not None:
+                    counts_out.append(a + 1)
+        return x[P:], forwards, refreshes
 
     # ---- acceptance-rate limit of self-drafting (Section 5.1, Table 2) ---------------
     def acceptance_limit_block(self, block_len: int, cache: Cache, draft_len: int, k_max: int):

@@ -656,3 +656,84 @@ def test_spill_needs_fewer_forwards_on_the_tiny_peaked_model():
     b, counts_spill, windows = o.generate_spill(prompt, w.gen_len, w.block_len, 3)
     assert np.array_equal(a, b)
     assert windows > 0 and len(counts_spill) < sum(len(c) for c in counts)
+
+
+# ---------------------------------------------------------------------------------------
+# dual cache with a refresh interval (Section 4.1, implementation details)
+# ---------------------------------------------------------------------------------------
+def _uncached_full_attention_stepwise(o, prompt, gen_len, block_len):
+    """Textbook masked-diffusion stepwise decoding without any cache: every step runs the model over the WHOLE
+    sequence [prompt | generation with MASK], all positions seeing all positions, and unmasks the most
+    confident masked position of the current block."""
+    mid = o.cfg.mask_id
+    P = len(prompt)
+    x = np.concatenate([prompt, np.full(gen_len, mid)])
+    for (lo, hi) in so.block_ranges(gen_len, block_len):
+        masked = np.zeros(P + gen_len, dtype=bool)
+        masked[P + lo:P + hi] = True
+        while masked.any():
+            logits, _, _ = o.forward_rows(x[None], 0, so.Cache(o.cfg))
+            tok, conf = so.token_and_confidence(logits[0], mid)
+            q = so.best_masked_position(conf, masked)
+            x[q] = tok[q]
+            masked[q] = False
+    return x[P:]
+
+
+@pytest.mark.parametrize("w", [SMALL, SMALL_GQA], ids=lambda w: w.name)
+def test_dual_cache_refreshed_every_token_is_uncached_decoding(w):
+    """With a refresh before every forward nothing is ever stale: the dual cache is exact and reproduces
+    full-sequence decoding without a cache."""
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    want = _uncached_full_attention_stepwise(o, prompt, w.gen_len, w.block_len)
+    got, forwards, refreshes = o.generate_dual_cache(prompt, w.gen_len, w.block_len, refresh=1)
+    assert np.array_equal(got, want)
+    assert forwards == refreshes == w.gen_len
+
+
+@pytest.mark.parametrize("w", [SMALL, SMALL_GQA], ids=lambda w: w.name)
+@pytest.mark.parametrize("refresh", [2, 3, 4, 100])
+def test_ssd_under_the_dual_cache_equals_stepwise_under_the_same_schedule(w, refresh):
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    want, f0, r0 = o.generate_dual_cache(prompt, w.gen_len, w.block_len, refresh, max_drafts=0)
+    assert f0 == w.gen_len
+    n_blocks = -(-w.gen_len // w.block_len)
+    # a refresh at every block start and after every `refresh` tokens inside a block
+    assert r0 == sum(-(-(hi - lo) // refresh) for (lo, hi) in so.block_ranges(w.gen_len, w.block_len))
+    for N in (1, 2, 5):
+        counts = []
+        got, f, r = o.generate_dual_cache(prompt, w.gen_len, w.block_len, refresh, max_drafts=N, counts_out=counts)
+        assert np.array_equal(got, want)
+        assert r == r0 and f <= f0 and sum(counts) == w.gen_len
+        assert all(1 <= c <= min(N + 1, refresh) for c in counts)
+    if refresh == 100:
+        assert r0 == n_blocks
+
+
+def test_dual_cache_is_an_approximation_between_refreshes():
+    """Stale K/V change the model's outputs: with a long interval the confidences seen by a forward differ from
+    those of exact decoding, which is why stepwise decoding is defined together with its schedule."""
+    w = SMALL
+    o = make_oracle(w)
+    prompt = wl.make_prompts(w)[0].numpy()
+    mid = w.mask_id
+    x = np.concatenate([prompt, np.full(w.gen_len, mid)])
+    P, T = len(prompt), w.block_len
+    full = o.refresh_all(x)
+    x2 = x.copy()
+    x2[P] = 5                                             # one token decoded since the refresh
+    fresh = o.refresh_all(x2)
+    ids = x2[P:P + T]
+
+    def block_logits(cache):
+        outside = so.Cache(o.cfg)
+        outside.k = [np.concatenate([k[:P], k[P + T:]], axis=0) for k in cache.k]
+        outside.v = [np.concatenate([v[:P], v[P + T:]], axis=0) for v in cache.v]
+        return o.forward_rows(ids[None], P, outside)[0][0]
+
+    stale, exact = block_logits(full), block_logits(fresh)
+    whole, _, _ = o.forward_rows(x2[None], 0, so.Cache(o.cfg))
+    assert np.allclose(exact, whole[0][P:P + T], rtol=1e-9, atol=1e-12)      # fresh cache == no cache
+    assert np.abs(stale - exact).max() > 1e-6                                 # stale suffix K/V: not the same
