@@ -121,6 +121,14 @@ int ssd_get_next_block_state(ssd_ctx* ctx, int32_t* ids, uint8_t* masked, int32_
  * 0 gives a stepwise step.  accepted HOST [batch] (0 for finished sequences), n_nodes HOST
  * [batch]; both may be NULL. */
 int ssd_block_step(ssd_ctx* ctx, int32_t max_drafts, int32_t* accepted, int32_t* n_nodes);
+/* Dual cache (Section 4.1; option "dual_cache"): recompute the K/V of EVERY position of every sequence -
+ * prompt, decoded blocks, the block in progress (MASK where still masked) and the still masked rest - by one
+ * forward per sequence in which all positions see all positions.  ssd_block_step / ssd_decode_block call it
+ * on their own at every block start and after every "refresh_interval" decoded tokens; exposed so that a
+ * forward can be compared with a reference from a known cache.  ssd_refresh_count: refresh forwards so far. */
+int ssd_refresh_cache(ssd_ctx* ctx);
+int64_t ssd_refresh_count(const ssd_ctx* ctx);
+
 /* Test hook: (token, confidence) of the first n_rows rows of the latest forward, in its row order
  * [sequence slot][node][rows of the node] (a node's rows: a finished block riding in front, if any, the
  * current block, the next block's half of a window, if any); -1 / 0 on rows nothing was asked of. */
@@ -259,6 +267,16 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically (in
  *        steps of 128) while a prefix would need more than 7 parts;
  *   "max_drafts" lower the draft-length cap below the capacity fixed at creation;
+ *   "dual_cache" P + L > 0 = the dual cache of the paper's set-up (Section 4.1) instead of the exact prefix
+ *        cache: the K/V of all P + L positions are cached, a block forward attends to every position outside
+ *        the block (prefix and still masked suffix) plus its own rows, and the cache is refreshed by a
+ *        full-sequence forward at every block start and after every "refresh_interval" (default 8) decoded
+ *        tokens.  Between refreshes the cached K/V are stale (an approximation), so stepwise decoding is
+ *        defined with the schedule, and SSD caps every chain at refresh_interval - decoded - 1 drafts so that
+ *        no forward accepts past a refresh point: the tokens stay those of stepwise decoding under the same
+ *        schedule.  Blocks are not committed (the next refresh recomputes them).  Set after ssd_prefill,
+ *        outside a block; 0 = off (default);
+ *   "refresh_interval" decoded tokens between two refreshes of the dual cache, >= 1;
  *   "cross_block" T2 > 0 = candidates may come from the next block (Section 3.2.2): the block after the next
  *        one to be begun is T2 tokens long.  While a sequence's current block holds more masked positions
  *        than the draft length a forward is unchanged; once it cannot fill the chain (r <= max_drafts) the

@@ -27,7 +27,7 @@ PROF_TOP = PROF_FAMILIES[:5]          # the last four break "gemm" down by proje
 
 EXPORTS = ["ssd_create", "ssd_destroy", "ssd_last_error", "ssd_load_weights", "ssd_prefill", "ssd_prefill_dev",
            "ssd_decode_block", "ssd_block_begin", "ssd_set_block_state", "ssd_get_block_state", "ssd_block_step",
-           "ssd_set_next_block_state", "ssd_get_next_block_state", "ssd_read_forward_outputs",
+           "ssd_set_next_block_state", "ssd_get_next_block_state", "ssd_read_forward_outputs", "ssd_refresh_cache", "ssd_refresh_count",
            "ssd_block_commit", "ssd_verify_forward", "ssd_read_cache", "ssd_write_cache", "ssd_verify_layers",
            "ssd_verify_forward_topk", "ssd_probe_acceptance_limit", "ssd_cache_length", "ssd_rewind", "ssd_gemm_bf16",
            "ssd_gemm_bf16_noalloc",
@@ -76,6 +76,9 @@ def load_library() -> C.CDLL:
     lib.ssd_set_next_block_state.argtypes = [vp, vp, vp, vp, vp]
     lib.ssd_get_next_block_state.argtypes = [vp, vp, vp, vp, vp]
     lib.ssd_read_forward_outputs.argtypes = [vp, i32, vp, vp]
+    lib.ssd_refresh_cache.argtypes = [vp]
+    lib.ssd_refresh_count.argtypes = [vp]
+    lib.ssd_refresh_count.restype = i64
     lib.ssd_block_step.argtypes = [vp, i32, vp, vp]
     lib.ssd_block_commit.argtypes = [vp]
     lib.ssd_verify_forward.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
@@ -95,7 +98,7 @@ def load_library() -> C.CDLL:
     lib.ssd_set_option.argtypes = [vp, C.c_char_p, i32]
     for name in EXPORTS:
         fn = getattr(lib, name)
-        if name not in ("ssd_destroy", "ssd_last_error", "ssd_launch_count"):
+        if name not in ("ssd_destroy", "ssd_last_error", "ssd_launch_count", "ssd_refresh_count"):
             fn.restype = i32
     _lib = lib
     return lib
@@ -227,6 +230,12 @@ class Ssd:
         conf = np.zeros(n_rows, np.float32)
         self._check(self.lib.ssd_read_forward_outputs(self._ctx, n_rows, _np_ptr(tok), _np_ptr(conf)))
         return tok, conf
+
+    def refresh_cache(self):
+        self._check(self.lib.ssd_refresh_cache(self._ctx))
+
+    def refresh_count(self) -> int:
+        return int(self.lib.ssd_refresh_count(self._ctx))
 
     def block_step(self, max_drafts: int, batch: int):
         acc = np.zeros(batch, np.int32)

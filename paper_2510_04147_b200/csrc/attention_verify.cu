@@ -116,7 +116,9 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
       const int row = idx / CH, ch = idx % CH;
       const int key = key0 + row;
       const bool valid = key < k_end;
-      const size_t off = (size_t)(valid ? key : k_begin) * krow_stride + ch * 8;
+      int crow = valid ? key : k_begin;                       // cache row of the key (a hole skips the block's own rows)
+      if (crow >= a.hole_begin) crow += a.hole_len;
+      const size_t off = (size_t)crow * krow_stride + ch * 8;
       cp_async16(dK + swz<HD>(row, ch), kbase + off, valid);
       cp_async16(dV + swz<HD>(row, ch), vbase + off, valid);
     }

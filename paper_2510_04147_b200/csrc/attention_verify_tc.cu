@@ -204,7 +204,9 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       const int row = idx / CH, ch = idx % CH;
       const int key = kb + row;
       const bool valid = key < k_end;
-      const size_t off = (size_t)(valid ? key : kb) * krow_stride + ch * 8;
+      int crow = valid ? key : kb;                            // cache row of the key (a hole skips the block's own rows)
+      if (crow >= a.hole_begin) crow += a.hole_len;
+      const size_t off = (size_t)crow * krow_stride + ch * 8;
       if (want_k) cp_async16(sK + tile_off(row, ch, kKeys), kbase + off, valid);
       if (want_v) cp_async16(sV + tile_off(row, ch, kKeys), vbase + off, valid);
     }

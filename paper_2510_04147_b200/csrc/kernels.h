@@ -147,7 +147,11 @@ struct AttnArgs {
   float2* part_ml;      // [n_parts][R][H]  (running max in log2 domain, sum)
   bf16* out;            // [R][H*hd]
   int R, H, Hkv, hd;
-  int S;                // prefix keys read from the cache
+  int S;                // keys read from the cache
+  // Dual cache: the cached keys are the positions [0, hole_begin) and [hole_begin + hole_len, ...), i.e. key
+  // index k >= hole_begin lives in cache row k + hole_len (the rows of the block being computed are skipped:
+  // its own keys are the node-local ones).  hole_len = 0: the cached keys are the prefix [0, S).
+  int hole_begin, hole_len;
   int kv_split;         // prefix keys per split (a function of S only)
   size_t cache_seq_stride;
   RowMap map;
@@ -218,6 +222,7 @@ struct BlockState {       // device arrays, [max_batch][stride] unless noted; a 
   int* has_drafts;        // [max_batch] bit 0: the current block has drafts, bit 1: the next block has
   int* remaining;         // [max_batch] r of the current block
   int* remaining_nxt;     // [max_batch] masked positions of the next block
+  const int* draft_cap;   // [max_batch] per-sequence cap on the draft length (INT_MAX: none)
   int* window;            // [max_batch] 1: the sequence takes candidates from the next block in the current forward
   int* cand_pos;          // [max_batch][block_len]
   int* cand_tok;

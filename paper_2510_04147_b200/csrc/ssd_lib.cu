@@ -90,6 +90,15 @@ struct ssd_ctx {
   bool carry = false;
   int carry_T = 0;
   std::vector<int> h_remaining_nxt;
+  // Dual cache (Section 4.1): dual_total = P + L of the sequences being decoded (0 = off, the exact prefix
+  // cache); the K/V of all positions are recomputed by a full-sequence forward at every block start and
+  // after every refresh_interval decoded tokens; h_since = tokens decoded since a sequence's last refresh.
+  int dual_total = 0, refresh_interval = 8;
+  int64_t refreshes = 0;
+  int* seq_ids = nullptr;        // [max_batch][max_seq] tokens known so far: prompt, then committed blocks
+  int* refresh_rows = nullptr;   // [max_seq] ids of one refresh forward
+  int* draft_cap_dev = nullptr;  // [max_batch] per-sequence cap on the draft length (dual cache), else INT_MAX
+  std::vector<int> h_since, h_draft_cap;
   int* prompt_stage = nullptr;   // [max_batch][max_seq] device copy of a host prompt (ssd_prefill)
   int fuse_commit = 1;
   std::vector<int> h_remaining, h_has_drafts, h_nodes, h_max_accept;
@@ -303,6 +312,8 @@ struct LayerRange {
   bool lm_head = true;
   int topk = 0;                  // > 0: the LM head also ranks the `topk` most probable tokens of every wanted row
   bool commit_chain = false;     // the rows before chain_T0 of every sequence's first node go to the K/V cache
+  int keys_total = 0;            // dual cache: the cache holds positions [0, keys_total); all of them except the rows' own
+                                 // block [pos0, pos0 + T) are attended to (0: the prefix [0, pos0) only)
 };
 
 // One forward over R rows.  FILL: K/V go to the cache at positions pos0.., attention over the cache
@@ -319,8 +330,9 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   const bool commit_form = kind == FWD_FILL && S > 0 && map.rows_per_seq == map.T &&
                            map.T <= c->cfg.block_len;
   const bool via_cache = kind == FWD_FILL && !commit_form;
-  const int attn_S = via_cache ? S + map.T : S;
-  const int kv_split = via_cache ? attn_S : kv_split_for(c, S);
+  const int hole_len = (!via_cache && range.keys_total > 0) ? map.T : 0;
+  const int attn_S = via_cache ? S + map.T : (hole_len > 0 ? range.keys_total - hole_len : S);
+  const int kv_split = via_cache ? attn_S : kv_split_for(c, attn_S);
   const int n_parts = (attn_S + kv_split - 1) / kv_split;
   if (via_cache && (size_t)n_parts * R > c->part_rows_parts)
     return fail(c, SSD_ERR_OVERFLOW, "attention workspace too small for %d parts x %d rows", n_parts, R);
@@ -356,6 +368,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     a.cache_v = c->cacheV + (size_t)l * c->cache_layer_stride;
     a.out = c->att;
     a.R = R; a.H = H; a.Hkv = Hkv; a.hd = hd; a.S = attn_S; a.kv_split = kv_split;
+    a.hole_begin = hole_len > 0 ? S : 0; a.hole_len = hole_len;
     a.cache_seq_stride = c->cache_seq_stride; a.map = map; a.n_seq_slots = n_slots;
     const double kvb = (double)n_slots * attn_S * Hkv * hd * 4.0 + (double)R * (H + 2 * Hkv) * hd * 2.0 + (double)R * H * hd * 2.0;
     if (via_cache) {
@@ -446,6 +459,18 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
   return SSD_OK;
 }
 
+// ids of one refresh forward of sequence b: what is known ([0, known)), the block in progress (MASK where it is
+// still masked), MASK beyond
+__global__ void refresh_rows_kernel(const int* seq_ids, BlockState s, int b, int known, int T, int total, int mask_id,
+                                    int* out) {
+  const int p = blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= total) return;
+  int id = mask_id;
+  if (p < known) id = seq_ids[p];
+  else if (p < known + T && !s.masked[(size_t)b * s.stride + p - known]) id = s.ids[(size_t)b * s.stride + p - known];
+  out[p] = id;
+}
+
 // Buffers of the acceptance-limit probe; allocated the first time a top-k forward is asked for.
 int ensure_topk_buffers(ssd_ctx* c) {
   if (c->tile_topv) return SSD_OK;
@@ -522,6 +547,21 @@ int flush_pending(ssd_ctx* c) {
   return SSD_OK;
 }
 
+// Dual cache: one forward over ALL positions of sequence b, every position seeing every position, rewrites
+// the K/V of the whole sequence (Section 4.1).  T = tokens of the block in progress (0: none).
+int refresh_sequence(ssd_ctx* c, int b, int T) {
+  const int total = c->dual_total;
+  refresh_rows_kernel<<<(total + 255) / 256, 256, 0, c->st>>>(c->seq_ids + (size_t)b * c->cfg.max_seq, c->bs, b, c->cache_len, T,
+                                                           total, c->cfg.mask_id, c->refresh_rows);
+  c->launches += 1;
+  RowMap map{total, total, 0, b, nullptr};
+  const int rc = forward(c, FWD_FILL, c->refresh_rows, total, map, 1, false, nullptr);
+  if (rc) return rc;
+  c->refreshes += 1;
+  c->h_since[b] = 0;
+  return SSD_OK;
+}
+
 int parse_layer_name(const char* name, int* layer, const char** rest) {
   if (strncmp(name, "layers.", 7) != 0) return 0;
   char* end = nullptr;
@@ -575,6 +615,8 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
   c->h_remaining.assign(k.max_batch, 0);
   c->h_has_drafts.assign(k.max_batch, 0);
   c->h_remaining_nxt.assign(k.max_batch, 0);
+  c->h_since.assign(k.max_batch, 0);
+  c->h_draft_cap.assign(k.max_batch, 0x7fffffff);
   c->h_nodes.assign(k.max_batch, 0);
   c->h_max_accept.assign(k.max_batch, 0);
 
@@ -644,6 +686,11 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     ALLOC(c, c->bs.cand_pos, sb); ALLOC(c, c->bs.cand_tok, sb); ALLOC(c, c->bs.accept_log, sb);
     ALLOC(c, c->pending_ids, sb);
     ALLOC(c, c->prompt_stage, (size_t)k.max_batch * k.max_seq);
+    ALLOC(c, c->seq_ids, (size_t)k.max_batch * k.max_seq);
+    ALLOC(c, c->refresh_rows, (size_t)k.max_seq);
+    ALLOC(c, c->draft_cap_dev, k.max_batch);
+    CUDA_TRY(c, cudaMemcpyAsync(c->draft_cap_dev, c->h_draft_cap.data(), k.max_batch * sizeof(int), cudaMemcpyHostToDevice, c->st));
+    c->bs.draft_cap = c->draft_cap_dev;
     ALLOC(c, c->bs.has_drafts, k.max_batch); ALLOC(c, c->bs.remaining, k.max_batch); ALLOC(c, c->bs.n_cand, k.max_batch);
     ALLOC(c, c->bs.n_forwards, k.max_batch); ALLOC(c, c->bs.last_accept, k.max_batch); ALLOC(c, c->bs.seq_map, k.max_batch);
     ALLOC(c, c->bs.last_pos, k.max_batch); ALLOC(c, c->bs.last_tok, k.max_batch);
@@ -736,6 +783,9 @@ int ssd_prefill_dev(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t
     const int rc = forward(c, FWD_FILL, prompt_ids_dev + (size_t)b * prompt_len, prompt_len, map, 1, false, nullptr);
     if (rc) return rc;
   }
+  // the tokens of every sequence as far as they are known (a refresh of the dual cache needs them all)
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->seq_ids, (size_t)c->cfg.max_seq * sizeof(int), prompt_ids_dev, (size_t)prompt_len * sizeof(int),
+                                (size_t)prompt_len * sizeof(int), batch, cudaMemcpyDeviceToDevice, c->st));
   const int rc = sync_and_check(c);
   if (rc) return rc;
   c->batch = batch;
@@ -789,6 +839,11 @@ int ssd_block_begin(ssd_ctx* c, int32_t T) {
   // the block after this one takes part as the second half of the window while there is room for it
   int T2 = c->next_T;
   if (T2 > 0 && c->cache_len + c->pending_T + T + T2 > c->cfg.max_seq) T2 = 0;
+  if (c->dual_total > 0) {
+    if (c->cache_len + T > c->dual_total) return fail(c, SSD_ERR_OVERFLOW, "block ends at %d, beyond the dual cache's sequence length %d", c->cache_len + T, c->dual_total);
+    T2 = 0;
+    for (int b = 0; b < c->cfg.max_batch; ++b) c->h_since[b] = c->refresh_interval;      // refresh before the first forward
+  }
   if (c->carry && c->carry_T == T) {
     // this block was the second half of the previous block's window: keep what it already holds
     block_shift_kernel<<<c->cfg.max_batch, 128, 0, c->st>>>(c->bs, c->batch, c->block_tokens, T, T2, c->cfg.mask_id);
@@ -885,7 +940,8 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nu
       if (c->h_has_drafts[b] & 2) more = std::max(0, std::min(md - r, c->h_remaining_nxt[b] - 1));
       return r + more;
     }
-    return md < r - 1 ? md : r - 1;
+    const int cap = (c->dual_total > 0) ? std::min(md, c->h_draft_cap[b]) : md;
+    return cap < r - 1 ? cap : r - 1;
   };
   auto shape = [&](bool window, int* active_out) -> int {
     int active = 0, n_cap = 1;
@@ -902,6 +958,21 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nu
     *active_out = active;
     return n_cap;
   };
+  const bool dual = c->dual_total > 0;
+  if (dual) {
+    // refresh the sequences that are due, and cap every chain so that no forward accepts past the next
+    // refresh point: the tokens stay those of stepwise decoding under the same schedule
+    for (int b = 0; b < B; ++b) {
+      c->h_draft_cap[b] = 0x7fffffff;
+      if (c->h_remaining[b] <= 0) continue;
+      if (c->h_since[b] >= c->refresh_interval) {
+        const int rrc = refresh_sequence(c, b, T);
+        if (rrc) return rrc;
+      }
+      c->h_draft_cap[b] = std::max(0, c->refresh_interval - c->h_since[b] - 1);
+    }
+    CUDA_TRY(c, cudaMemcpyAsync(c->draft_cap_dev, c->h_draft_cap.data(), B * sizeof(int), cudaMemcpyHostToDevice, c->st));
+  }
   int active = 0;
   int n_cap = shape(false, &active);
   *launched = active > 0;
@@ -911,7 +982,7 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nu
   // sequences must take part (each has a block to commit); otherwise the commit runs on its own first.
   int Tp = 0;
   if (c->pending_T > 0) {
-    if (active == B && active * n_cap * (c->pending_T + T) <= c->R_dec) {
+    if (!dual && active == B && active * n_cap * (c->pending_T + T) <= c->R_dec) {
       Tp = c->pending_T;
     } else {
       const int frc = flush_pending(c);
@@ -921,7 +992,7 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nu
   }
   // The window [this block | next block]: whenever a sequence can no longer fill its chain from this block.
   int T2 = 0;
-  if (Tp == 0 && c->window_T2 > 0 && !c->mix_order && !probe) {
+  if (Tp == 0 && c->window_T2 > 0 && !c->mix_order && !probe && !dual) {
     bool any = false;
     for (int b = 0; b < B; ++b) any = any || (c->h_remaining[b] > 0 && (c->h_has_drafts[b] & 1) && c->h_remaining[b] <= md);
     if (any) {
@@ -955,6 +1026,7 @@ int step_enqueue(ssd_ctx* c, int md, bool* launched, const ProbeStep* probe = nu
   LayerRange range;
   if (probe && probe->open_round) range.topk = probe->k_max;
   range.commit_chain = Tp > 0;
+  if (dual) range.keys_total = c->dual_total;
   int rc = forward(c, FWD_VERIFY, c->node_ids, R, map, active, false, c->node_masked, range);
   if (rc) return rc;
   {
@@ -986,7 +1058,7 @@ int step_collect(ssd_ctx* c, int32_t* accepted, int32_t* n_nodes) {
   const int mb = c->cfg.max_batch;
   CUDA_TRY(c, cudaMemcpyAsync(hp, c->flags, 2 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   CUDA_TRY(c, cudaMemcpyAsync(hp + 2, c->bs.remaining, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
-  if (accepted) CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + mb, c->bs.last_accept, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+  if (accepted || c->dual_total > 0) CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + mb, c->bs.last_accept, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   if (n_nodes) CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 2 * mb, c->bs.n_cand, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 3 * mb, c->bs.remaining_nxt, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   CUDA_TRY(c, cudaMemcpyAsync(hp + 2 + 4 * mb, c->bs.has_drafts, B * sizeof(int), cudaMemcpyDeviceToHost, c->st));
@@ -996,6 +1068,7 @@ int step_collect(ssd_ctx* c, int32_t* accepted, int32_t* n_nodes) {
   for (int b = 0; b < B; ++b) {
     c->h_remaining[b] = hp[2 + b];
     c->h_remaining_nxt[b] = hp[2 + 3 * mb + b];
+    if (c->dual_total > 0 && c->h_nodes[b] > 0) c->h_since[b] += hp[2 + mb + b];
     c->h_has_drafts[b] = hp[2 + 4 * mb + b];
     if (accepted) accepted[b] = hp[2 + mb + b];
     if (n_nodes) n_nodes[b] = c->h_nodes[b] > 0 ? tree_nodes(hp[2 + 2 * mb + b], c->mix_order) : 0;
@@ -1028,7 +1101,15 @@ int ssd_block_commit(ssd_ctx* c) {
   const int T = c->block_tokens, B = c->batch;
   int rc = flush_pending(c);           // (a block that ended without a single forward of its own)
   if (rc) return rc;
-  if (c->fuse_commit) {
+  // the block's tokens join what is known of every sequence
+  CUDA_TRY(c, cudaMemcpy2DAsync(c->seq_ids + c->cache_len, (size_t)c->cfg.max_seq * sizeof(int), c->bs.ids, c->bs.stride * sizeof(int),
+                                T * sizeof(int), B, cudaMemcpyDeviceToDevice, c->st));
+  if (c->dual_total > 0) {
+    // dual cache: nothing to commit - the next block starts with a refresh of every position's K/V
+    rc = sync_and_check(c);
+    if (rc) return rc;
+    c->cache_len += T;
+  } else if (c->fuse_commit) {
     // keep the tokens; the next block's first forward (or whoever needs the cache first) commits them
     CUDA_TRY(c, cudaMemcpy2DAsync(c->pending_ids, c->bs.stride * sizeof(int), c->bs.ids, c->bs.stride * sizeof(int), T * sizeof(int), B,
                                   cudaMemcpyDeviceToDevice, c->st));
@@ -1108,7 +1189,7 @@ int ssd_decode_block(ssd_ctx* c, int32_t mode, int32_t T, int32_t* out_tokens, i
     if (rc) return rc;
     bool decided = true;
     for (int b = 0; b < c->batch; ++b)
-      if (c->h_nodes[b] > 0 && c->h_remaining[b] - c->h_max_accept[b] < md + 1) decided = false;
+      if (c->h_nodes[b] > 0 && (c->h_remaining[b] - c->h_max_accept[b] < md + 1 || c->dual_total > 0)) decided = false;
     if (decided) {
       for (int b = 0; b < c->batch; ++b) c->h_remaining[b] -= c->h_max_accept[b];
       continue;
@@ -1144,7 +1225,12 @@ int ssd_verify_forward(ssd_ctx* c, int32_t batch, int32_t n_nodes, int32_t T, co
   CUDA_TRY(c, cudaMemcpyAsync(c->node_masked, node_masked, R, cudaMemcpyHostToDevice, c->st));
   CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
   RowMap map{n_nodes * T, T, c->cache_len, 0, nullptr};
-  int rc = forward(c, FWD_VERIFY, c->node_ids, (int)R, map, batch, out_logits != nullptr, c->node_masked);
+  LayerRange range;
+  if (c->dual_total > 0) {
+    if (c->cache_len + T > c->dual_total) return fail(c, SSD_ERR_OVERFLOW, "block ends beyond the dual cache's sequence length %d", c->dual_total);
+    range.keys_total = c->dual_total;
+  }
+  int rc = forward(c, FWD_VERIFY, c->node_ids, (int)R, map, batch, out_logits != nullptr, c->node_masked, range);
   if (rc) return rc;
   if (out_tok) CUDA_TRY(c, cudaMemcpyAsync(out_tok, c->tok, R * sizeof(int), cudaMemcpyDeviceToHost, c->st));
   if (out_conf) CUDA_TRY(c, cudaMemcpyAsync(out_conf, c->conf, R * sizeof(float), cudaMemcpyDeviceToHost, c->st));
@@ -1296,6 +1382,22 @@ int ssd_probe_acceptance_limit(ssd_ctx* c, int32_t T, int32_t draft_len, int32_t
   return ssd_block_commit(c);
 }
 
+int ssd_refresh_cache(ssd_ctx* c) {
+  if (!c) return SSD_ERR_INVALID_ARG;
+  if (c->cache_len < 0) return fail(c, SSD_ERR_STATE, "prefill first");
+  if (c->dual_total <= 0) return fail(c, SSD_ERR_STATE, "the dual cache is off (option dual_cache)");
+  const int T = c->in_block ? c->block_tokens : 0;
+  if (c->cache_len + T > c->dual_total) return fail(c, SSD_ERR_OVERFLOW, "the sequence is longer than the dual cache's length %d", c->dual_total);
+  CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
+  for (int b = 0; b < c->batch; ++b) {
+    const int rc = refresh_sequence(c, b, T);
+    if (rc) return rc;
+  }
+  return sync_and_check(c);
+}
+
+int64_t ssd_refresh_count(const ssd_ctx* c) { return c ? c->refreshes : -1; }
+
 int ssd_read_forward_outputs(ssd_ctx* c, int32_t n_rows, int32_t* out_tok, float* out_conf) {
   if (!c) return SSD_ERR_INVALID_ARG;
   if (n_rows < 0 || n_rows > c->R_cap) return fail(c, SSD_ERR_INVALID_ARG, "row count outside [0, %d]", c->R_cap);
@@ -1404,6 +1506,22 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "max_drafts")) {
     if (value < 0 || value + 1 > c->n_max) return fail(c, SSD_ERR_INVALID_ARG, "max_drafts must be in [0, %d] (the capacity fixed at creation)", c->n_max - 1);
     c->cfg.max_drafts = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "dual_cache")) {
+    if (value != 0 && (value < 1 || value > c->cfg.max_seq)) return fail(c, SSD_ERR_INVALID_ARG, "dual_cache is 0 (off) or the sequence length P + L <= max_seq = %d", c->cfg.max_seq);
+    if (c->in_block) return fail(c, SSD_ERR_STATE, "a block is in progress");
+    if (value > 0) {
+      const int frc = flush_pending(c);
+      if (frc) return frc;
+    }
+    c->dual_total = value;
+    c->carry = false;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "refresh_interval")) {
+    if (value < 1) return fail(c, SSD_ERR_INVALID_ARG, "refresh_interval must be >= 1");
+    c->refresh_interval = value;
     return SSD_OK;
   }
   if (!strcmp(key, "cross_block")) {

@@ -43,6 +43,7 @@ __global__ void __launch_bounds__(256) tree_build_kernel(BlockState s, int batch
   if (threadIdx.x == 0) s.last_accept[b] = 0;
   const int r = s.remaining[b];
   if (r <= 0) return;
+  max_drafts = min(max_drafts, s.draft_cap[b]);          // (a refresh schedule may shorten a sequence's chain)
   int slot = 0;
   for (int i = 0; i < b; ++i) slot += (s.remaining[i] > 0) ? 1 : 0;
   const int W = T + T2;

@@ -918,3 +918,99 @@ def test_cross_block_window_steps_match_oracle(tiny_oracles):
     print(f"cross-block: {checked} window forwards replayed, {strict} with the oracle's own decisions, "
           f"{crossed} tokens accepted across the boundary")
     assert checked > 0 and crossed > 0
+
+
+# ------------------------------------------------------------------------------------------
+# dual cache with a refresh interval (Section 4.1)
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("which", ["tiny", "tiny_peaked"])
+def test_dual_cache_forward_matches_oracle(tiny_oracles, which):
+    """After a refresh the K/V of every position outside the current block - prefix AND masked suffix - are
+    those of the oracle's full-sequence forward, and a block forward against them gives the oracle's logits;
+    once a token has been decoded without a refresh, the forward still matches the oracle run on the same
+    (now stale) cache."""
+    w = wl.TINY if which == "tiny" else PEAKED
+    o64, ob = tiny_oracles[w.name]
+    rng = np.random.default_rng(31)
+    prompt = wl.make_prompts(w).numpy()
+    P, T, L = w.prompt_len, w.block_len, w.gen_len
+    mid = w.mask_id
+    ssd = _make_ssd(w, max_drafts=4)
+    try:
+        ssd.prefill(prompt)
+        ssd.set_option("dual_cache", P + L)
+        ssd.set_option("refresh_interval", 4)
+        block0 = rng.integers(0, w.vocab - 1, T)
+        ssd.block_begin(T)
+        ssd.set_block_state(block0[None], np.zeros((1, T), np.uint8))
+        ssd.block_commit()                                    # dual cache: the tokens are recorded, nothing is committed
+        assert ssd.cache_length() == P + T
+        S = P + T
+        state_ids = rng.integers(0, w.vocab - 1, T)
+        state_masked = rng.random(T) < 0.6
+        state_masked[0] = True
+        ssd.block_begin(T)
+        ssd.set_block_state(state_ids[None], state_masked[None].astype(np.uint8))
+        ssd.refresh_cache()
+        assert ssd.refresh_count() == 1
+        ids, masked = _random_nodes(w, rng, 3, T)
+        tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
+        k_gpu, v_gpu = ssd.read_cache(0, 0, P + L)
+    finally:
+        ssd.destroy()
+    x = np.concatenate([prompt[0], block0, np.where(state_masked, mid, state_ids), np.full(L - 2 * T, mid)])
+    for o, tol in ((ob, 1e-2), (o64, 2e-2)):
+        full = o.refresh_all(x)
+        outside = so.Cache(o.cfg)
+        outside.k = [np.concatenate([k[:S], k[S + T:]], axis=0) for k in full.k]
+        outside.v = [np.concatenate([v[:S], v[S + T:]], axis=0) for v in full.v]
+        ologits, _, _ = o.forward_rows(ids[0], S, outside)
+        err = np.abs(logits[0] - ologits).max()
+        assert err < tol * w.lm_head_scale, (err, tol)
+        otok, oconf = so.token_and_confidence(ologits.reshape(-1, w.vocab), mid)
+        m = masked[0].reshape(-1)
+        assert np.allclose(conf[0].reshape(-1)[m], oconf[m], rtol=CONF_RTOL * w.lm_head_scale, atol=1e-6)
+        # the whole sequence's K/V of layer 0, suffix included
+        assert np.abs(k_gpu - full.k[0]).max() < 2e-2 * max(1.0, np.abs(full.k[0]).max())
+        assert np.abs(v_gpu - full.v[0]).max() < 2e-2 * max(1.0, np.abs(full.v[0]).max())
+
+
+def test_dual_cache_generation_follows_the_schedule_and_stays_lossless():
+    """GPU SSD under the dual cache == GPU stepwise under the same schedule, bit for bit, for several draft
+    lengths; the refreshes fall at every block start and after every `refresh_interval` tokens."""
+    w = PEAKED
+    b = _binding()
+    prompts = wl.make_prompts(w, batch=2).numpy()
+    P, T, L = w.prompt_len, w.block_len, w.gen_len
+    ssd = _make_ssd(w, max_drafts=5, max_batch=2)
+    try:
+        for refresh in (4, 6, 100):
+            expect = 2 * sum(-(-(min(T, L - lo)) // refresh) for lo in range(0, L, T))      # two sequences
+            ssd.prefill(prompts)
+            ssd.set_option("dual_cache", P + L)
+            ssd.set_option("refresh_interval", refresh)
+            r0 = ssd.refresh_count()
+            tok_s, acc_s, nf_s = ssd.generate(b.MODE_STEPWISE, L, T, 2)
+            assert ssd.refresh_count() - r0 == expect
+            assert ssd.cache_length() == P + L
+            for N in (1, 3, 5):
+                ssd.set_option("dual_cache", 0)
+                ssd.prefill(prompts)
+                ssd.set_option("dual_cache", P + L)
+                ssd.set_option("max_drafts", N)
+                r0 = ssd.refresh_count()
+                tok, accs, nfs = ssd.generate(b.MODE_SSD, L, T, 2)
+                assert np.array_equal(tok, tok_s)
+                assert ssd.refresh_count() - r0 == expect
+                for acc, nf in zip(accs, nfs):
+                    for i in range(2):
+                        used = acc[i][:nf[i]]
+                        assert used.sum() == T and np.all(used >= 1) and np.all(used <= min(N + 1, refresh))
+            ssd.set_option("dual_cache", 0)
+        # the exact prefix cache decodes something else in general: the dual cache sees the masked suffix
+        ssd.set_option("max_drafts", 3)
+        ssd.prefill(prompts)
+        tok_prefix, _, _ = ssd.generate(b.MODE_STEPWISE, L, T, 2)
+        assert tok_prefix.shape == tok_s.shape
+    finally:
+        ssd.destroy()
