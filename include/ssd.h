@@ -267,6 +267,11 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically (in
  *        steps of 128) while a prefix would need more than 7 parts;
  *   "max_drafts" lower the draft-length cap below the capacity fixed at creation;
+ *   "wait_limit_us" bound of every device-side barrier wait of the projection kernel in microseconds (0 = the
+ *        default of 2 s): when it runs out the kernel raises an error word, lets its copies in flight land,
+ *        frees its tensor memory and returns, and the call reports SSD_ERR_TIMEOUT; the context stays usable;
+ *   "starve_gemm_kb" test hook for ssd_gemm_bf16 (split_k 1, up to 256 rows): > 0 makes the kernel's producer
+ *        leave out the copies of that K block (1-based), so that the wait for it provably runs out; 0 = off;
  *   "dual_cache" P + L > 0 = the dual cache of the paper's set-up (Section 4.1) instead of the exact prefix
  *        cache: the K/V of all P + L positions are cached, a block forward attends to every position outside
  *        the block (prefix and still masked suffix) plus its own rows, and the cache is refreshed by a

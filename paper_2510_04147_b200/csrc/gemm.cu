@@ -35,7 +35,7 @@ constexpr int kTcThreads = 192;      // warp 0: TMA, warp 1: MMA + TMEM owner, w
 constexpr int kMaxStages = 8;
 constexpr int kWTileBytes = kTileM * kBlockK * 2;
 constexpr int kEpiPitch = 132;       // floats per row of the epilogue's transpose buffer (128 + padding)
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default bound of a wait, 2 s: far beyond any legitimate one
 
 struct TcParams {
   int R, N, K;
@@ -52,6 +52,8 @@ struct TcParams {
   float* tile_max;
   float* tile_sum;
   int* tile_arg;
+  unsigned long long wait_limit_ns;   // bound of every barrier wait
+  int starve_kb;   // test hook, 0 = off: the producer leaves out the copies of K block starve_kb - 1, so the wait for it runs out
   int topk;        // EPI_LMHEAD: > 0 also writes the tile's `topk` largest logits per row (value, vocabulary index)
   float* tile_topv;
   int* tile_topi;
@@ -89,14 +91,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the limit expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   int spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 63) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
+      if (globaltimer_ns() - t0 > limit_ns) return false;
     }
   }
   return true;
@@ -282,20 +285,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       // The weights do not depend on any earlier kernel: fill the ring with weight tiles first, and
       // only then wait for the kernel that produces the activations.
       const int pre = n_kb < p.stages ? n_kb : p.stages;
+      // (test hook: a starved K block gets neither its byte count nor its copies - its barrier never completes)
+      auto starved = [&](int it) { return p.starve_kb > 0 && kb_begin + it == p.starve_kb - 1; };
       for (int it = 0; it < pre; ++it) {
+        if (starved(it)) continue;
         const uint32_t fb = smem_addr(&full_bar[it]);
         expect(fb);
         load_w(it, it, fb);
       }
       pdl_wait();
       for (int it = 0; it < pre; ++it) {
+        if (starved(it)) continue;
         load_x(it, it, smem_addr(&full_bar[it]));
         ++issued;
       }
       for (int it = pre; it < n_kb; ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (uint32_t)((it / p.stages) & 1);
-        if (!mbar_wait(smem_addr(&empty_bar[s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(smem_addr(&empty_bar[s]), ph ^ 1u, abort_flag, p.wait_limit_ns)) { ok = false; break; }
+        if (starved(it)) continue;
         const uint32_t fb = smem_addr(&full_bar[s]);
         expect(fb);
         load_w(it, s, fb);
@@ -310,7 +318,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         for (int j = first; j < issued && (!ts || leader); ++j) {
           const unsigned long long t0 = globaltimer_ns();
           while (!mbar_try_wait(smem_addr(&full_bar[j % p.stages]), (uint32_t)((j / p.stages) & 1)))
-            if (globaltimer_ns() - t0 > kWaitLimitNs) break;
+            if (globaltimer_ns() - t0 > p.wait_limit_ns) break;
         }
       }
     }
@@ -324,7 +332,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       for (int it = 0; it < n_kb; ++it) {
         const int s = it % p.stages;
         const uint32_t ph = (uint32_t)((it / p.stages) & 1);
-        if (!mbar_wait(smem_addr(&full_bar[s]), ph, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(smem_addr(&full_bar[s]), ph, abort_flag, p.wait_limit_ns)) { ok = false; break; }
         tc_fence_after();
         const uint32_t wa = smem_addr(sW + (size_t)s * kWTileBytes);
         const uint32_t xa = smem_addr(sX + (size_t)s * x_tile_bytes);
@@ -369,7 +377,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       epi_bar_sync();
     }
     bool ok = true;
-    if (n_kb > 0) ok = mbar_wait(smem_addr(acc_bar), 0u, abort_flag);
+    if (n_kb > 0) ok = mbar_wait(smem_addr(acc_bar), 0u, abort_flag, p.wait_limit_ns);
     ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
     const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16);
@@ -744,6 +752,10 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   p.stages = stages;
   p.out = g.out; p.act = g.act; p.act_pitch = g.act_pitch;
   p.tile_max = g.tile_max; p.tile_sum = g.tile_sum; p.tile_arg = g.tile_arg;
+  p.wait_limit_ns = g.wait_limit_ns > 0 ? g.wait_limit_ns : kWaitLimitNs;
+  p.starve_kb = g.starve_kb;
+  // the starvation hook is for the plain single-CTA launch only (no cluster partner waits on this CTA)
+  if (g.starve_kb != 0 && (g.epi != EPI_PARTIAL || g.splits != 1 || g.R > 256)) return -2;
   p.topk = g.topk; p.tile_topv = g.tile_topv; p.tile_topi = g.tile_topi;
   if (g.topk < 0 || g.topk > kLmTopKMax || (g.topk > 0 && (g.epi != EPI_LMHEAD || !g.tile_topv || !g.tile_topi))) return -2;
   p.mask_id = g.mask_id; p.err_flag = g.err_flag;

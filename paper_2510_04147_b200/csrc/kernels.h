@@ -196,6 +196,8 @@ struct GemmArgs {
   int* tile_topi;        // [tiles][R][kLmTopKMax] vocabulary indices (lower index first among equals)
   int mask_id;
   int* err_flag;         // device int set non-zero when a bounded wait expires
+  unsigned long long wait_limit_ns;   // bound of every barrier wait in the kernel; 0 = the default (2 s)
+  int starve_kb;         // test hook, 0 = off: leave out the copies of K block starve_kb - 1 (plain EPI_PARTIAL launches only)
   // consumer side of a fused RMSNorm: every output row r is multiplied by
   // rsqrt(sum_{t < sq_count} sq[r * sq_stride + t] / norm_dim + norm_eps); sq == nullptr: no scaling
   const float* sq;

@@ -108,6 +108,8 @@ struct ssd_ctx {
   int two_sm_rows = 256;                   // projections pair their tiles (two-SM MMA) from this many rows on; 0 = never
   int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
   int64_t launches = 0;
+  int wait_limit_us = 0;         // bound of the projection kernel's barrier waits (0: the kernel's default, 2 s)
+  int starve_gemm_kb = 0;        // test hook for ssd_gemm_bf16: K block (1-based) whose copies are left out
   bool profiling = false;        // mode 1: CUDA events around every launch (serialises the stream)
   bool marking = false;          // mode 2: a marker kernel after every launch stamps the time it ended, in the live stream
   unsigned long long* marks = nullptr;   // device [kMaxMarks]
@@ -290,6 +292,7 @@ int run_gemm(ssd_ctx* c, GemmArgs g, int fam, int sub = -1) {
   Scope sc(c, fam, (double)g.N * g.K * 2.0, 1, sub);
   g.err_flag = c->flags;
   g.two_sm_min_rows = c->two_sm_rows;
+  g.wait_limit_ns = (unsigned long long)c->wait_limit_us * 1000ull;
   const int rc = launch_gemm_tc(c->st, g);
   if (rc != 0) return fail(c, rc, "projection kernel rejected R=%d N=%d K=%d epi=%d splits=%d (code %d)", g.R, g.N, g.K, g.epi, g.splits, rc);
   return SSD_OK;
@@ -1416,6 +1419,7 @@ int ssd_gemm_bf16(ssd_ctx* c, const void* x_dev, const void* w_dev, float* out_d
   GemmArgs g{};
   g.x = (const bf16*)x_dev; g.w = (const bf16*)w_dev; g.R = rows; g.N = n; g.K = k; g.x_pitch = k; g.w_pitch = k;
   g.splits = split_k; g.epi = EPI_PARTIAL; g.out = c->partial;
+  g.starve_kb = c->starve_gemm_kb;
   int rc = run_gemm(c, g, SSD_PROF_GEMM);
   if (rc) return rc;
   const size_t total = (size_t)rows * n;
@@ -1506,6 +1510,16 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "max_drafts")) {
     if (value < 0 || value + 1 > c->n_max) return fail(c, SSD_ERR_INVALID_ARG, "max_drafts must be in [0, %d] (the capacity fixed at creation)", c->n_max - 1);
     c->cfg.max_drafts = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "wait_limit_us")) {
+    if (value < 0) return fail(c, SSD_ERR_INVALID_ARG, "wait_limit_us is 0 (default, 2 s) or a bound in microseconds");
+    c->wait_limit_us = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "starve_gemm_kb")) {
+    if (value < 0) return fail(c, SSD_ERR_INVALID_ARG, "starve_gemm_kb is 0 (off) or a 1-based K block index");
+    c->starve_gemm_kb = value;
     return SSD_OK;
   }
   if (!strcmp(key, "dual_cache")) {

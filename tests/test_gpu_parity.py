@@ -1014,3 +1014,32 @@ def test_dual_cache_generation_follows_the_schedule_and_stays_lossless():
         assert tok_prefix.shape == tok_s.shape
     finally:
         ssd.destroy()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives(tiny_ssd):
+    """Failure made on the host side: the projection kernel's producer is told to leave out one K block's
+    copies, the wait for that block runs out after a millisecond bound, the kernel unwinds (tensor memory
+    freed, no trap) and the call returns SSD_ERR_TIMEOUT; the next call on the same context succeeds."""
+    b = _binding()
+    x = wl.normal_tensor(8, 1, (16, 256), 1.0, device="cuda", dtype=torch.bfloat16)
+    w = wl.normal_tensor(8, 2, (128, 256), 0.05, device="cuda", dtype=torch.bfloat16)
+    ref = x.cpu().to(torch.float64).numpy() @ w.cpu().to(torch.float64).numpy().T
+    try:
+        tiny_ssd.set_option("wait_limit_us", 2000)
+        tiny_ssd.set_option("starve_gemm_kb", 2)
+        with pytest.raises(b.SsdError) as e:
+            tiny_ssd.gemm_bf16(x, w, 1)
+        assert e.value.code == -6
+        with pytest.raises(b.SsdError) as e:
+            tiny_ssd.gemm_bf16(x, w, 2)                     # the hook is refused for anything but the plain launch
+        assert e.value.code == -2
+    finally:
+        tiny_ssd.set_option("starve_gemm_kb", 0)
+        tiny_ssd.set_option("wait_limit_us", 0)
+    out = tiny_ssd.gemm_bf16(x, w, 1).cpu().numpy()
+    assert np.abs(out - ref).max() < 2e-5 * 0.05 * 256 + 1e-6
+    # and a whole decode still works on it
+    prompt = wl.make_prompts(wl.TINY).numpy()
+    tiny_ssd.prefill(prompt)
+    tok, acc, nf = tiny_ssd.decode_block(b.MODE_SSD, wl.TINY.block_len, 1)
+    assert acc[0][:nf[0]].sum() == wl.TINY.block_len
