@@ -344,7 +344,8 @@ def run_ours(args):
     torch.cuda.set_stream(stream)
     ssd = binding.Ssd(binding.config_from_workload(w, max_drafts=min(cfg_drafts, B - 1)))
     for k, v in (("split_k_qkv", args.split_qkv), ("split_k_o", args.split_o), ("split_k_down", args.split_down),
-                 ("kv_split", args.kv_split), ("attn_impl", args.attn_impl), ("two_sm_rows", args.two_sm_rows)):
+                 ("kv_split", args.kv_split), ("attn_impl", args.attn_impl), ("two_sm_rows", args.two_sm_rows),
+                 ("gemm_max_stages", args.gemm_max_stages)):
         if v is not None:
             ssd.set_option(k, v)
     t0 = time.time()
@@ -524,6 +525,63 @@ def run_ours(args):
                                                     for k in binding.PROF_TOP},
                     "family_avg_launch_us": {k: 1e3 * prof[k]["ms"] / max(1, prof[k]["launches"]) for k in binding.PROF_TOP},
                     "per_projection": per_projection, "in_stream": in_stream}
+        # ---- the method's variants at the chosen draft length (one generation each; same tokens as stepwise
+        #      decoding, under the dual cache: as stepwise decoding with the same refresh schedule)
+        variants = {}
+
+        def one_generation(d, cross_block=False):
+            hist = []
+            ssd.set_option("max_drafts", d)
+            mode = binding.MODE_SSD if d > 0 else binding.MODE_STEPWISE
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(stream)
+            done = 0
+            while done < L:
+                t = min(B, L - done)
+                if cross_block:
+                    ssd.set_option("cross_block", min(B, L - done - t))
+                ssd.decode_block_into(mode, t, out_tok.data_ptr(), out_acc.data_ptr(), out_nf.data_ptr())
+                hist.append(out_acc.numpy()[:, :t].copy())
+                done += t
+            ev1.record(stream)
+            torch.cuda.synchronize()
+            a = np.concatenate([x.reshape(-1) for x in hist])
+            a = a[a > 0]
+            return {"tokens_per_s": bs * L / (ev0.elapsed_time(ev1) * 1e-3), "forwards": int(len(a)),
+                    "mean_accepted_per_forward": float(a.mean())}
+
+        try:
+            dv = max(best, 2)
+            ssd.rewind(P)
+            ssd.set_option("mix_order", 1)
+            variants[f"mix_order_tree_{dv}_drafts"] = one_generation(dv)
+            ssd.set_option("mix_order", 0)
+            ssd.rewind(P)
+            variants[f"greedy_chain_{dv}_drafts"] = one_generation(dv)
+            ssd.rewind(P)
+            variants[f"cross_block_{max(best, 1)}_drafts"] = one_generation(max(best, 1), cross_block=True)
+            ssd.set_option("cross_block", 0)
+            ssd.rewind(P)
+            ssd.set_option("dual_cache", P + L)
+            ssd.set_option("refresh_interval", 8)
+            r0 = ssd.refresh_count()
+            variants["dual_cache_refresh_8_stepwise"] = one_generation(0)
+            variants["dual_cache_refresh_8_stepwise"]["refresh_forwards"] = ssd.refresh_count() - r0
+            ssd.set_option("dual_cache", 0)
+            ssd.rewind(P)
+            ssd.set_option("dual_cache", P + L)
+            r0 = ssd.refresh_count()
+            variants[f"dual_cache_refresh_8_ssd_{max(best, 1)}_drafts"] = one_generation(max(best, 1))
+            variants[f"dual_cache_refresh_8_ssd_{max(best, 1)}_drafts"]["refresh_forwards"] = ssd.refresh_count() - r0
+            ssd.set_option("dual_cache", 0)
+            ssd.rewind(P)
+        except Exception as e:                    # a variant that does not fit this configuration is reported, not fatal
+            variants["error"] = str(e)
+            for k, v in (("mix_order", 0), ("cross_block", 0), ("dual_cache", 0)):
+                try:
+                    ssd.set_option(k, v)
+                except Exception:
+                    pass
         # ---- CPU baseline: the oracle on a bounded sample
         if args.no_cpu_baseline:
             cpu = None
@@ -555,7 +613,7 @@ def run_ours(args):
                 "roofline": roofline, "forward": fwd, "cpu_baseline": cpu,
                 "accept": {"mean_per_forward": float(accs.mean()), "histogram": np.bincount(accs).tolist(),
                            "forwards_per_generation": int(len(accs)), "blocks": n_blocks},
-                "sweep": sweep,
+                "sweep": sweep, "variants": variants,
                 "paper_context": "paper reports 2.0-3.46x over stepwise decoding on one A100 80GB with trained weights"}
     ssd.destroy()
     if line is not None and world == 1 and not reduced and args.workload == "llada8b" and not args.no_other_workloads:
@@ -597,6 +655,7 @@ def main():
     ap.add_argument("--attn-impl", type=int, default=None, help="0: mma.sync attention; 1: tcgen05 attention where eligible")
     ap.add_argument("--two-sm-rows", type=int, default=None,
                     help="projection tile pairs run as one two-SM MMA from this many rows on (0: never)")
+    ap.add_argument("--gemm-max-stages", type=int, default=None, help="tuning: cap on the projection kernel's ring depth")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: fewer layers of the same shape")
     ap.add_argument("--gen-len", type=int, default=0, help="profiling only: shorter generation")

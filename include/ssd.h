@@ -223,8 +223,10 @@ int ssd_gemm_bf16(ssd_ctx* ctx, const void* x_dev, const void* w_dev, float* out
  *   owned by the caller; k a multiple of 8; 1 <= split_k <= 8; `cuda_stream` a cudaStream_t.
  *   Limit: split_k * rows * n <= 1048512 floats (4 MiB minus a 256-byte flag area), else
  *   SSD_ERR_OVERFLOW; bad shapes SSD_ERR_SHAPE; null pointers SSD_ERR_INVALID_ARG.
- * The first call on each device looks up the array's device address (with that device current);
- * make that first call before starting any stream capture.  All calls share the one array, which
+ * The first call on each device looks up the array's device address (with that device current); under
+ * the driver's lazy module loading that is also when the array and the kernels are placed on the device, so
+ * make that first call early - before the host's arena takes the remaining memory and before starting any
+ * stream capture.  Later calls take no device memory at all.  All calls share the one array, which
  * keeps the previous call's contents (the error word is cleared at the start of every call): two
  * calls whose GPU work overlaps - different streams or threads - race on it, so serialise them.
  * Synchronises the stream before returning; same result as ssd_gemm_bf16. */
@@ -267,6 +269,8 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "kv_split"   prefix keys per attention part, a multiple of 64; 0 = 128; raised automatically (in
  *        steps of 128) while a prefix would need more than 7 parts;
  *   "max_drafts" lower the draft-length cap below the capacity fixed at creation;
+ *   "gemm_max_stages" tuning: cap on the depth of the projection kernel's shared-memory ring (0 = as deep as
+ *        two CTAs per SM allow, the default); changes no result;
  *   "wait_limit_us" bound of every device-side barrier wait of the projection kernel in microseconds (0 = the
  *        default of 2 s): when it runs out the kernel raises an error word, lets its copies in flight land,
  *        frees its tensor memory and returns, and the call reports SSD_ERR_TIMEOUT; the context stays usable;

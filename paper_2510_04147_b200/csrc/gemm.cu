@@ -748,6 +748,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmArgs& g) {
   const int budget = 108 * 1024;
   int stages = budget / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
+  if (g.max_stages > 0 && stages > g.max_stages) stages = g.max_stages;
   if (stages < 2) stages = 2;
   p.stages = stages;
   p.out = g.out; p.act = g.act; p.act_pitch = g.act_pitch;

@@ -197,6 +197,7 @@ struct GemmArgs {
   int mask_id;
   int* err_flag;         // device int set non-zero when a bounded wait expires
   unsigned long long wait_limit_ns;   // bound of every barrier wait in the kernel; 0 = the default (2 s)
+  int max_stages;        // tuning: cap on the depth of the shared-memory ring (0: as deep as the budget allows)
   int starve_kb;         // test hook, 0 = off: leave out the copies of K block starve_kb - 1 (plain EPI_PARTIAL launches only)
   // consumer side of a fused RMSNorm: every output row r is multiplied by
   // rsqrt(sum_{t < sq_count} sq[r * sq_stride + t] / norm_dim + norm_eps); sq == nullptr: no scaling

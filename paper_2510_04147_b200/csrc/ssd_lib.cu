@@ -108,6 +108,7 @@ struct ssd_ctx {
   int two_sm_rows = 256;                   // projections pair their tiles (two-SM MMA) from this many rows on; 0 = never
   int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
   int64_t launches = 0;
+  int gemm_max_stages = 0;       // tuning: cap on the projection kernel's ring depth (0: none)
   int wait_limit_us = 0;         // bound of the projection kernel's barrier waits (0: the kernel's default, 2 s)
   int starve_gemm_kb = 0;        // test hook for ssd_gemm_bf16: K block (1-based) whose copies are left out
   bool profiling = false;        // mode 1: CUDA events around every launch (serialises the stream)
@@ -293,6 +294,7 @@ int run_gemm(ssd_ctx* c, GemmArgs g, int fam, int sub = -1) {
   g.err_flag = c->flags;
   g.two_sm_min_rows = c->two_sm_rows;
   g.wait_limit_ns = (unsigned long long)c->wait_limit_us * 1000ull;
+  g.max_stages = c->gemm_max_stages;
   const int rc = launch_gemm_tc(c->st, g);
   if (rc != 0) return fail(c, rc, "projection kernel rejected R=%d N=%d K=%d epi=%d splits=%d (code %d)", g.R, g.N, g.K, g.epi, g.splits, rc);
   return SSD_OK;
@@ -1510,6 +1512,11 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "max_drafts")) {
     if (value < 0 || value + 1 > c->n_max) return fail(c, SSD_ERR_INVALID_ARG, "max_drafts must be in [0, %d] (the capacity fixed at creation)", c->n_max - 1);
     c->cfg.max_drafts = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "gemm_max_stages")) {
+    if (value < 0 || value == 1) return fail(c, SSD_ERR_INVALID_ARG, "gemm_max_stages is 0 (no cap) or >= 2");
+    c->gemm_max_stages = value;
     return SSD_OK;
   }
   if (!strcmp(key, "wait_limit_us")) {

@@ -23,10 +23,18 @@ def test_noalloc_gemm_matches_context_gemm_twice_in_a_row():
             x = wl.normal_tensor(21 + call, 1, (rows, k), 1.0, device="cuda", dtype=torch.bfloat16)
             w = wl.normal_tensor(21 + call, 2, (n, k), 0.05, device="cuda", dtype=torch.bfloat16)
             out = torch.full((rows, n), float("nan"), dtype=torch.float32, device="cuda")
-            before = torch.cuda.memory_allocated()
+            if call == 0:
+                # the first call on a device looks up the array (and may make the driver load the kernels' module):
+                # allowed to take device memory once, before the calls that must not
+                assert b.gemm_bf16_noalloc(x, w, out, split) == 0
+                out.fill_(float("nan"))
+            torch.cuda.synchronize()
+            before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
             rc = b.gemm_bf16_noalloc(x, w, out, split)
             assert rc == 0
+            torch.cuda.synchronize()
             assert torch.cuda.memory_allocated() == before
+            assert torch.cuda.mem_get_info()[0] == free_before      # the driver handed out nothing either
             want = ssd.gemm_bf16(x, w, split)
             got, ref = out.cpu().numpy(), want.cpu().numpy()
             scale = np.sqrt(k) * 0.05
