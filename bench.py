@@ -531,7 +531,7 @@ def run_ours(args):
         variants = {}
 
         def one_generation(d, cross_block=False):
-            hist = []
+            hist, toks = [], []
             ssd.set_option("max_drafts", d)
             mode = binding.MODE_SSD if d > 0 else binding.MODE_STEPWISE
             ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -543,16 +543,24 @@ def run_ours(args):
                     ssd.set_option("cross_block", min(B, L - done - t))
                 ssd.decode_block_into(mode, t, out_tok.data_ptr(), out_acc.data_ptr(), out_nf.data_ptr())
                 hist.append(out_acc.numpy()[:, :t].copy())
+                toks.append(out_tok.numpy()[:, :t].copy())
                 done += t
             ev1.record(stream)
             torch.cuda.synchronize()
             a = np.concatenate([x.reshape(-1) for x in hist])
             a = a[a > 0]
             return {"tokens_per_s": bs * L / (ev0.elapsed_time(ev1) * 1e-3), "forwards": int(len(a)),
-                    "mean_accepted_per_forward": float(a.mean())}
+                    "mean_accepted_per_forward": float(a.mean()), "_tokens": np.concatenate(toks, axis=1)}
+
+        def same_tokens(res, ref):
+            """Share of the generation (from its start) that equals the reference decoding, token for token."""
+            neq = np.nonzero(res["_tokens"].reshape(-1) != ref["_tokens"].reshape(-1))[0]
+            return 1.0 if len(neq) == 0 else float(neq[0]) / res["_tokens"].size
 
         try:
             dv = max(best, 2)
+            ssd.rewind(P)
+            ref_step = one_generation(0)
             ssd.rewind(P)
             ssd.set_option("mix_order", 1)
             variants[f"mix_order_tree_{dv}_drafts"] = one_generation(dv)
@@ -576,6 +584,13 @@ def run_ours(args):
             variants[f"dual_cache_refresh_8_ssd_{max(best, 1)}_drafts"]["refresh_forwards"] = ssd.refresh_count() - r0
             ssd.set_option("dual_cache", 0)
             ssd.rewind(P)
+            # losslessness on the device: the share of the generation that equals stepwise decoding from its start
+            # (1.0 = all of it; candidates from the next block may part ways at a near-tie, see the design notes)
+            for k, v in variants.items():
+                ref = variants["dual_cache_refresh_8_stepwise"] if k.startswith("dual_cache") else ref_step
+                v["leading_share_equal_to_stepwise"] = same_tokens(v, ref)
+            for v in variants.values():
+                v.pop("_tokens", None)
         except Exception as e:                    # a variant that does not fit this configuration is reported, not fatal
             variants["error"] = str(e)
             for k, v in (("mix_order", 0), ("cross_block", 0), ("dual_cache", 0)):

@@ -376,3 +376,175 @@ def test_both_attention_forms_agree_at_full_width():
     assert np.sqrt((diff ** 2).mean()) < 2 * rms_bound
     m = masked[0]
     assert np.allclose(out[0][1][0][m], out[1][1][0][m], rtol=np.exp(4.0 * max_bound) - 1.0, atol=1e-6)
+
+
+# ------------------------------------------------------------------------------------------
+# the variants of the method at full width (tcgen05 attention: chains of two blocks, several nodes in a
+# forward that commits, a hole in the cached key range)
+# ------------------------------------------------------------------------------------------
+PEAKED_WIDTH = WIDTH_CASES["llada_width_peaked"][0]
+
+
+def _stepwise_trace_is_near_tie_before(o, prompt, gen_len, w, first, e_max):
+    """Does the oracle's stepwise run hold, at or before generation position `first`, a decision that logit errors
+    up to e_max could flip (top-1/top-2 token gap, or the margin between the two most confident positions)?"""
+    trace = []
+    o.generate(prompt, gen_len, w.block_len, mode="stepwise", trace=trace)
+    ratio = 1.0 - np.exp(-2.0 * e_max)
+    for rec in trace:
+        q, _ = rec.pred[0]
+        cm = np.sort(np.where(rec.node_masked[0], rec.conf[0], -1.0))[::-1]
+        margin = cm[0] - cm[1] if len(cm) > 1 and cm[1] >= 0 else np.inf
+        if rec.gap[0, q] <= ratio * rec.conf[0, q] or margin <= ratio * cm[0]:
+            return True
+        if rec.block * w.block_len + q == first:
+            return False
+    return False
+
+
+def test_full_width_mix_order_and_cross_block_generations():
+    """At the LLaDA width (tcgen05 attention, 32-token blocks): mix-order SSD == stepwise bit for bit; SSD with
+    candidates from the next block (window nodes of 64 rows, commits riding in front of multi-node forwards)
+    decodes the stepwise tokens up to the first decision that is a near-tie within the bf16 noise bound."""
+    w = PEAKED_WIDTH
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    N = 3
+    ssd = _make(w, max_drafts=2 * N + 1)
+    try:
+        ssd.set_option("max_drafts", N)
+        ssd.prefill(prompt)
+        tok_s, _, _ = ssd.generate(b.MODE_STEPWISE, w.gen_len, w.block_len, 1)
+        ssd.set_option("mix_order", 1)
+        ssd.prefill(prompt)
+        tok_m, _, nf_m = ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1)
+        ssd.set_option("mix_order", 0)
+        ssd.prefill(prompt)
+        tok_p, _, nf_p = ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1)
+        ssd.prefill(prompt)
+        tok_x, acc_x, nf_x = ssd.generate(b.MODE_SSD, w.gen_len, w.block_len, 1, cross_block=True)
+        assert ssd.cache_length() == w.prompt_len + w.gen_len
+    finally:
+        ssd.destroy()
+    assert np.array_equal(tok_m, tok_s) and np.array_equal(tok_p, tok_s)
+    assert sum(int(n[0]) for n in nf_m) <= sum(int(n[0]) for n in nf_p)
+    assert sum(int(a[0][:n[0]].sum()) for a, n in zip(acc_x, nf_x)) == w.gen_len
+    diff = np.nonzero(tok_x[0] != tok_s[0])[0]
+    if len(diff):
+        res = {}
+        for mode in (None, "bf16"):
+            o = make_oracle(w, as_bf16=True, operand_rounding=mode)
+            cache = o.prefill(prompt[0])
+            res[mode] = o.verify(np.full((1, w.block_len), w.mask_id), np.ones((1, w.block_len), bool), cache)[3]
+        _, e_max = _noise_bounds(res[None], res["bf16"])
+        assert _stepwise_trace_is_near_tie_before(make_oracle(w, as_bf16=True), prompt[0], w.gen_len, w, int(diff[0]), e_max)
+    print(f"full width: forwards chain {sum(int(n[0]) for n in nf_p)}, mix-order {sum(int(n[0]) for n in nf_m)}, "
+          f"cross-block {sum(int(n[0]) for n in nf_x)}; cross-block tokens differing from stepwise: {len(diff)}")
+
+
+def test_full_width_window_forward_matches_oracle():
+    """One window forward [current block | next block] at the LLaDA width, state of both blocks given: the
+    confidences of every asked row of every node against the oracle's block-causal window, and the walk / new
+    state bit-exact against the oracle's logic applied to the GPU forward's own outputs."""
+    from oracle import ssd_oracle as so
+    w = PEAKED_WIDTH
+    rng = np.random.default_rng(17)
+    prompt = wl.make_prompts(w).numpy()
+    T, N, mid = w.block_len, 3, w.mask_id
+    W2 = 2 * T
+    # current block: two positions left; next block: untouched but with drafts (as after an earlier window forward)
+    ids = rng.integers(0, w.vocab - 1, W2)
+    masked = np.zeros(W2, bool)
+    masked[[5, 20]] = True
+    masked[T:] = True
+    dt = rng.integers(0, w.vocab - 1, W2)
+    dc = rng.random(W2).astype(np.float32)
+    ssd = _make(w, max_drafts=2 * N + 1)
+    try:
+        ssd.set_option("max_drafts", N)
+        ssd.prefill(prompt)
+        ssd.set_option("cross_block", T)
+        ssd.block_begin(T)
+        ssd.set_block_state(ids[None, :T], masked[None, :T].astype(np.uint8), dt[None, :T], dc[None, :T])
+        ssd.set_next_block_state(ids[None, T:], masked[None, T:].astype(np.uint8), dt[None, T:], dc[None, T:])
+        acc, nn = ssd.block_step(N, 1)
+        n = int(nn[0])
+        tok_g, conf_g = ssd.read_forward_outputs(n * W2)
+        tok_g, conf_g = tok_g.reshape(n, W2), conf_g.reshape(n, W2)
+        ids0, m0, _, dc0 = ssd.get_block_state(1, T)
+        ids1, m1, _, dc1 = ssd.get_next_block_state(1, T)
+    finally:
+        ssd.destroy()
+    cand = so.select_candidates(dt[:T], dc[:T], masked[:T], 2, keep_one=False)
+    cand += [(T + p, t) for (p, t) in so.select_candidates(dt[T:], dc[T:], masked[T:], N - 2)]
+    assert n == len(cand) + 1 == N + 1
+    node_ids, node_masked = so.build_chain(ids, masked, cand, mid)
+    res = {}
+    for mode in (None, "bf16"):
+        o = make_oracle(w, as_bf16=True, operand_rounding=mode)
+        res[mode] = o.verify_window(node_ids, node_masked, T, o.prefill(prompt[0]))
+    oconf, rconf = res[None][1], res["bf16"][1]
+    m = node_masked
+    # confidences: no further from the fp64 oracle than NOISE_MAX times the bf16-operand oracle's own distance
+    bound = NOISE_MAX * np.abs(rconf[m] / oconf[m] - 1.0).max()
+    assert np.abs(conf_g[m] / oconf[m] - 1.0).max() < max(bound, 1e-3), (np.abs(conf_g[m] / oconf[m] - 1.0).max(), bound)
+    assert np.all(tok_g[~m] == -1)
+    pred = []
+    for i in range(n):
+        scope = m[i].copy()
+        if m[i, :T].any():
+            scope[T:] = False
+        else:
+            scope[:T] = False
+        q = so.best_masked_position(conf_g[i], scope)
+        pred.append((q, int(tok_g[i, q])))
+    a = so.accept_length(pred, cand)
+    assert acc[0] == a + 1
+    want_ids, want_m = ids.copy(), masked.copy()
+    for (p, t) in list(cand[:a]) + [pred[a]]:
+        want_ids[p], want_m[p] = t, False
+    ids_g, m_g = np.concatenate([ids0[0], ids1[0]]), np.concatenate([m0[0], m1[0]]).astype(bool)
+    assert np.array_equal(m_g, want_m) and np.array_equal(ids_g[~want_m], want_ids[~want_m])
+    dc_g = np.concatenate([dc0[0], dc1[0]])
+    assert np.array_equal(dc_g[want_m].view(np.uint32), conf_g[a][want_m].view(np.uint32))
+
+
+@pytest.mark.parametrize("case", ["llada_width", "dream_width"])
+def test_full_width_dual_cache_forward_matches_oracle(case):
+    """The dual cache at full width (the tcgen05 attention reads the cached keys around a hole at the current
+    block): logits of a block forward after a refresh against the oracle's refresh_all + forward."""
+    from oracle import ssd_oracle as so
+    w, n_nodes = WIDTH_CASES[case]
+    rng = np.random.default_rng(23)
+    prompt = wl.make_prompts(w).numpy()
+    P, T, L, mid = w.prompt_len, w.block_len, w.gen_len, w.mask_id
+    block0 = rng.integers(0, w.vocab - 1, T)
+    ssd = _make(w, max_drafts=n_nodes)
+    try:
+        ssd.prefill(prompt)
+        ssd.set_option("dual_cache", P + L)
+        ssd.block_begin(T)
+        ssd.refresh_cache()
+        ids, masked = _nodes(w, rng, n_nodes, T)
+        tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)      # first block: suffix of T masked rows
+        ssd.set_block_state(block0[None], np.zeros((1, T), np.uint8))
+        ssd.block_commit()
+        ssd.block_begin(T)
+        ssd.refresh_cache()
+        tok2, conf2, logits2 = ssd.verify_forward(ids, masked, want_logits=True)   # last block: no suffix left
+    finally:
+        ssd.destroy()
+    x1 = np.concatenate([prompt[0], np.full(L, mid)])
+    x2 = np.concatenate([prompt[0], block0, np.full(L - T, mid)])
+    for x, S, got in ((x1, P, logits), (x2, P + T, logits2)):
+        ol = {}
+        for mode in (None, "bf16"):
+            o = make_oracle(w, as_bf16=True, operand_rounding=mode)
+            full = o.refresh_all(x)
+            outside = so.Cache(o.cfg)
+            outside.k = [np.concatenate([k[:S], k[S + T:]], axis=0) for k in full.k]
+            outside.v = [np.concatenate([v[:S], v[S + T:]], axis=0) for v in full.v]
+            ol[mode] = o.forward_rows(ids[0], S, outside)[0]
+        rms_bound, max_bound = _noise_bounds(ol[None], ol["bf16"])
+        err = got[0] - ol[None]
+        assert np.sqrt((err ** 2).mean()) < rms_bound and np.abs(err).max() < max_bound, (S, np.abs(err).max(), max_bound)
