@@ -592,6 +592,9 @@ def run_ours(args):
             for v in variants.values():
                 v.pop("_tokens", None)
         except Exception as e:                    # a variant that does not fit this configuration is reported, not fatal
+            for v in variants.values():
+                if isinstance(v, dict):
+                    v.pop("_tokens", None)
             variants["error"] = str(e)
             for k, v in (("mix_order", 0), ("cross_block", 0), ("dual_cache", 0)):
                 try:
