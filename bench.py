@@ -131,6 +131,9 @@ def _oracle_threads():
         return os.cpu_count() or 1
 
 
+_HEAD_WEIGHTS = {}      # the LM-head tensors of a workload, drawn once per process (4 GB in fp64 at the 8B shapes)
+
+
 def oracle_forward_times(w, layers, prefix_len, node_counts, device="cpu", with_head=True):
     """Times the oracle (as it stands) on verification forwards of `w`: for every layer index in `layers`
     the layer's tensors are drawn (outside the clock, one layer in memory at a time) and ``Oracle.layer`` is
@@ -166,7 +169,10 @@ def oracle_forward_times(w, layers, prefix_len, node_counts, device="cpu", with_
             t_layers[n] += time.perf_counter() - t0
         del o
     if with_head:
-        o = so.Oracle(cfg, draw(["norm_final", "lm_head"]))
+        if w.name not in _HEAD_WEIGHTS:
+            _HEAD_WEIGHTS.clear()
+            _HEAD_WEIGHTS[w.name] = draw(["norm_final", "lm_head"])
+        o = so.Oracle(cfg, _HEAD_WEIGHTS[w.name])
         for n in node_counts:
             h = rng.standard_normal((n * B, w.d_model))
             t0 = time.perf_counter()
