@@ -591,7 +591,8 @@ def run_ours(args):
             ssd.set_option("dual_cache", 0)
             ssd.rewind(P)
             # losslessness on the device: the share of the generation that equals stepwise decoding from its start
-            # (1.0 = all of it; candidates from the next block may part ways at a near-tie, see the design notes)
+            # (1.0 = all of it; with candidates from the next block a decision that is a near-tie within rounding noise
+            # may fall the other way at a block boundary, after which the two decodings are not comparable)
             for k, v in variants.items():
                 ref = variants["dual_cache_refresh_8_stepwise"] if k.startswith("dual_cache") else ref_step
                 v["leading_share_equal_to_stepwise"] = same_tokens(v, ref)

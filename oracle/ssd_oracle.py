@@ -30,7 +30,7 @@ What is defined here, and from where:
 * the mix-order tree of Section 5.2 (the chain plus one out-of-order branch per chain node
   that has a grandchild, 2N nodes) -> ``build_mix_order_tree``, ``accept_walk_mix_order``.
 
-Readings where the paper is silent (each also listed in the design notes):
+Readings where the paper is silent:
 the forward of a block attends to the cached prefix plus the block itself; a
 finished block enters the cache through one more forward over its final
 tokens; confidence is the maximum softmax probability with the mask token

@@ -5,8 +5,8 @@
 Runs the CPU oracle (and nothing else) on one root forward after a short prefill, once unrounded, once
 with every contraction's operands rounded to bfloat16, and once per rounding source alone, all modes
 through one pass over the weights.  Prints, per mode, the rms and the maximum of the logit difference
-from the unrounded run, and the same for the confidences.  The numbers quoted in the design notes'
-error budget come from this script; the GPU tests measure the same two totals on their own inputs.
+from the unrounded run, and the same for the confidences.  This is the per-source
+error budget of bf16 operands; the GPU tests measure the same two totals (all sources, none) on their own inputs.
 """
 from __future__ import annotations
 
