@@ -234,7 +234,9 @@ def run_reference(args):
             "warmup": args.warmup, "ms_per_step": sum(step_ms) / len(step_ms),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "prompt_len": w.prompt_len, "gen_len": w.gen_len, "block_len": w.block_len,
-                       "batch_per_gpu": w.batch, "decoding": "stepwise (oracle)", "step": f"{ls} layers + LM head of one forward",
+                       "batch_per_gpu": w.batch, "max_drafts": 0, "nodes_per_forward": 1,
+                       "l2_policy": "inputs larger than L2 (one layer's weights are 1.7 GB in fp64)", "replicas": 1,
+                       "decoding": "stepwise (oracle)", "step": f"{ls} layers + LM head of one forward",
                        "seconds_per_full_forward": t_fwd},
             "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
