@@ -1043,3 +1043,38 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(tiny_ssd):
     tiny_ssd.prefill(prompt)
     tok, acc, nf = tiny_ssd.decode_block(b.MODE_SSD, wl.TINY.block_len, 1)
     assert acc[0][:nf[0]].sum() == wl.TINY.block_len
+
+
+def test_variants_treat_every_sequence_of_a_batch_as_if_alone(peaked_ssd):
+    """Mix-order trees and the acceptance-limit probe on a batch of three: every sequence decodes exactly what
+    it decodes alone (tokens, accept counts, matched counts)."""
+    w = PEAKED
+    b = _binding()
+    prompts = wl.make_prompts(w, batch=3).numpy()
+    T = w.block_len
+    try:
+        peaked_ssd.set_option("max_drafts", 4)
+        peaked_ssd.set_option("mix_order", 1)
+        peaked_ssd.prefill(prompts)
+        tok_b, acc_b, nf_b = peaked_ssd.generate(b.MODE_SSD, 2 * T, T, 3)
+        for s in range(3):
+            peaked_ssd.prefill(prompts[s:s + 1])
+            tok_s, acc_s, nf_s = peaked_ssd.generate(b.MODE_SSD, 2 * T, T, 1)
+            assert np.array_equal(tok_s[0], tok_b[s])
+            for j in range(len(acc_s)):
+                assert np.array_equal(acc_s[j][0], acc_b[j][s]) and nf_s[j][0] == nf_b[j][s]
+        peaked_ssd.set_option("mix_order", 0)
+        peaked_ssd.prefill(prompts)
+        tok_p, matched_b, steps_b = peaked_ssd.probe_acceptance_limit(T, 3, 4, 3)
+        assert steps_b == 3 * T
+        total = np.zeros(4, np.int64)
+        for s in range(3):
+            peaked_ssd.prefill(prompts[s:s + 1])
+            tok_1, matched_1, steps_1 = peaked_ssd.probe_acceptance_limit(T, 3, 4, 1)
+            assert np.array_equal(tok_1[0], tok_p[s]) and steps_1 == T
+            total += matched_1
+        assert np.array_equal(total, matched_b)
+    finally:
+        peaked_ssd.set_option("mix_order", 0)
+        peaked_ssd.set_option("max_drafts", w.block_len - 1)
+        peaked_ssd.prefill(prompts[:1])
