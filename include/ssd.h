@@ -309,7 +309,7 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *        mma.sync form;
  *   "two_sm_rows" the QKV, gate/up and LM-head projections run pairs of weight tiles as ONE tcgen05.mma
  *        with cta_group::2 (two CTAs of a cluster, M = 256, each SM holding half of the activation tile)
- *        from this many padded rows per launch on; 0 = never; default 256, where it pays.  The results
+ *        from this many padded rows per launch on; 0 = never; default 128, where it starts to pay.  The results
  *        are bit-identical either way;
  *   "fuse_commit" 1 = a block's commit is folded into the next block's first forward (default); 0 = a
  *        commit forward of its own inside ssd_block_commit;

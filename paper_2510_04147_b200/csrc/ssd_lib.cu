@@ -105,7 +105,7 @@ struct ssd_ctx {
   int mix_order = 0;             // 1: the verification tree gets the out-of-order branches of Section 5.2
 
   int split_qkv = 1, split_o = 1, split_down = 1, kv_split_opt = 0;
-  int two_sm_rows = 256;                   // projections pair their tiles (two-SM MMA) from this many rows on; 0 = never
+  int two_sm_rows = 128;                   // projections pair their tiles (two-SM MMA) from this many rows on; 0 = never
   int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
   int64_t launches = 0;
   int gemm_max_stages = 0;       // tuning: cap on the projection kernel's ring depth (0: none)

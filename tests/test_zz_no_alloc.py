@@ -5,6 +5,8 @@ all calls share one fixed scratch array that still holds the previous call's par
 
 Collected last on purpose: a run that stops at the first failure has then run every other test.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -28,13 +30,20 @@ def test_noalloc_gemm_matches_context_gemm_twice_in_a_row():
                 # allowed to take device memory once, before the calls that must not
                 assert b.gemm_bf16_noalloc(x, w, out, split) == 0
                 out.fill_(float("nan"))
+            # (tensors of earlier tests that only a collection frees must not be freed in the middle of the comparison)
+            gc.collect()
             torch.cuda.synchronize()
-            before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
-            rc = b.gemm_bf16_noalloc(x, w, out, split)
+            gc.disable()
+            try:
+                before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+                rc = b.gemm_bf16_noalloc(x, w, out, split)
+                torch.cuda.synchronize()
+                after, free_after = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+            finally:
+                gc.enable()
             assert rc == 0
-            torch.cuda.synchronize()
-            assert torch.cuda.memory_allocated() == before
-            assert torch.cuda.mem_get_info()[0] == free_before      # the driver handed out nothing either
+            assert after == before
+            assert free_after == free_before      # the driver handed out nothing either
             want = ssd.gemm_bf16(x, w, split)
             got, ref = out.cpu().numpy(), want.cpu().numpy()
             scale = np.sqrt(k) * 0.05
