@@ -79,7 +79,9 @@ int ssd_load_weights(ssd_ctx* ctx, const char* tensor_name, const void* dev_ptr,
 
 /* Eq. 1 initial state: forward of the prompts (each prompt attends to itself only) that fills
  * the prefix K/V cache.  `prompt_ids` HOST [batch, prompt_len], ids in [0, vocab), no mask id
- * required.  Resets the decode position to prompt_len.  1 <= batch <= max_batch. */
+ * required.  Resets the decode position to prompt_len.  1 <= batch <= max_batch.  The prompts of a batch
+ * share forwards of up to 4096 rows (one stream of the weights for all of them); every sequence's cache is
+ * bit for bit what prefilling it alone gives. */
 int ssd_prefill(ssd_ctx* ctx, int32_t batch, int32_t prompt_len, const int32_t* prompt_ids);
 /* Same with `prompt_ids` in DEVICE memory (no host->device copy of inputs). */
 int ssd_prefill_dev(ssd_ctx* ctx, int32_t batch, int32_t prompt_len, const int32_t* prompt_ids_dev);

@@ -160,6 +160,8 @@ int dev_alloc(ssd_ctx* c, T** p, size_t n, bool zero = true) {
 
 constexpr int kMaxSplit = 16;
 
+constexpr int kPrefillRows = 4096;      // rows of one prefill forward when a batch's prompts are prefilled together
+
 // Split-K factor that fills the machine: two CTAs per SM on 148 SMs, at least four K blocks each.
 // A function of the matrix shape alone, so a row's summation order never depends on the row count.
 int auto_split(int tiles, int k) {
@@ -614,6 +616,9 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
   // first step of the next one
   c->R_dec = k.max_batch * (c->n_max > 2 ? c->n_max : 2) * k.block_len;
   c->R_cap = c->R_dec > k.max_seq ? c->R_dec : k.max_seq;
+  // room to prefill several sequences of a batch in one forward (one stream of the weights for all of them)
+  const long long group_rows = std::min<long long>((long long)k.max_batch * k.max_seq, kPrefillRows);
+  if (group_rows > c->R_cap) c->R_cap = (int)group_rows;
   c->split_qkv = auto_split(gemm_tiles(c->nqkv), c->d);
   c->split_o = auto_split(gemm_tiles(c->d), c->qdim);
   c->split_down = auto_split(gemm_tiles(c->d), c->ffn_pad);
@@ -783,9 +788,12 @@ int ssd_prefill_dev(ssd_ctx* c, int32_t batch, int32_t prompt_len, const int32_t
   if (prompt_len < 1 || prompt_len > c->cfg.max_seq) return fail(c, SSD_ERR_OVERFLOW, "prompt_len %d outside [1, %d]", prompt_len, c->cfg.max_seq);
   if (!all_loaded(c)) return fail(c, SSD_ERR_STATE, "not every weight tensor has been loaded");
   CUDA_TRY(c, cudaMemsetAsync(c->flags, 0, 4 * sizeof(int), c->st));
-  for (int b = 0; b < batch; ++b) {
+  // as many sequences per forward as the row capacity holds: their rows share one stream of the weights
+  const int group = std::max(1, c->R_cap / prompt_len);
+  for (int b = 0; b < batch; b += group) {
+    const int n = std::min(group, batch - b);
     RowMap map{prompt_len, prompt_len, 0, b, nullptr};
-    const int rc = forward(c, FWD_FILL, prompt_ids_dev + (size_t)b * prompt_len, prompt_len, map, 1, false, nullptr);
+    const int rc = forward(c, FWD_FILL, prompt_ids_dev + (size_t)b * prompt_len, n * prompt_len, map, n, false, nullptr);
     if (rc) return rc;
   }
   // the tokens of every sequence as far as they are known (a refresh of the dual cache needs them all)

@@ -125,6 +125,20 @@ def test_prefill_cache_matches_oracle(tiny_ssd, tiny_oracles):
             assert (np.abs(k - cache.k[l]) <= 4e-3).mean() > 0.99
 
 
+def test_prompts_prefilled_together_fill_the_cache_as_each_alone(peaked_ssd):
+    """The prompts of a batch share one prefill forward (one stream of the weights); a row's arithmetic does not
+    depend on what shares the forward with it, so every sequence's cache is, bit for bit, what prefilling it alone gives."""
+    w = PEAKED
+    prompts = wl.make_prompts(w, batch=3).numpy()
+    peaked_ssd.prefill(prompts)
+    together = [[peaked_ssd.read_cache(l, s, w.prompt_len) for l in range(w.n_layers)] for s in range(3)]
+    for s in range(3):
+        peaked_ssd.prefill(prompts[s:s + 1])
+        for l in range(w.n_layers):
+            k, v = peaked_ssd.read_cache(l, 0, w.prompt_len)
+            assert np.array_equal(k, together[s][l][0]) and np.array_equal(v, together[s][l][1])
+
+
 def _random_nodes(w, rng, n_nodes, T):
     ids = rng.integers(0, w.vocab - 1, (1, n_nodes, T))
     masked = rng.random((1, n_nodes, T)) < 0.6
