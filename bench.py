@@ -490,6 +490,13 @@ def run_ours(args):
             t_tc = fl / (peaks["bf16_tflops_sustained"] * 1e12)
             fwd[label] = {"nodes": max(nodes), "rows": rows, "ms": tmed, "algorithmic_gb": (wb + kvb) / 1e9,
                           "hbm_frac": t_hbm / (tmed * 1e-3), "frac_of_max_hbm_tensor": max(t_hbm, t_tc) / (tmed * 1e-3)}
+        # what a chain is worth when every draft is accepted (Table 2's upper bound: n tokens per forward of n
+        # nodes): n x (one-node forward time) / (n-node forward time).  The acceptance of a random-init model
+        # is far lower; this bounds what the forward's row dependence leaves of the method's speed-up.
+        t1 = fwd["stepwise_1_node"]["ms"]
+        for label, f in fwd.items():
+            if label.startswith("ssd_"):
+                f["speedup_over_stepwise_if_every_draft_accepted"] = f["nodes"] * t1 / f["ms"]
         # ---- dominant kernel: the projection GEMM family, CUDA events around every launch
         ssd.set_option("max_drafts", best)
         ssd.rewind(P)
