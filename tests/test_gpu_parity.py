@@ -481,6 +481,50 @@ def test_ragged_last_block(tiny_ssd):
     assert tiny_ssd.cache_length() == w.prompt_len + 40
 
 
+def test_blocks_of_one_and_two_tokens(peaked_ssd):
+    """B = 1: no draft can exist, every forward is a stepwise step; B = 2: at most one draft (N = min(max_drafts, r - 1))."""
+    w = PEAKED
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()
+    for block in (1, 2):
+        peaked_ssd.prefill(prompt)
+        want, _, nf0 = peaked_ssd.generate(b.MODE_STEPWISE, 6, block, 1)
+        peaked_ssd.prefill(prompt)
+        got, accs, nf = peaked_ssd.generate(b.MODE_SSD, 6, block, 1)
+        assert np.array_equal(got, want) and w.mask_id not in got
+        assert all(int(a.sum()) == block for a in accs)
+        if block == 1:
+            assert all(int(n[0]) == 1 for n in nf)
+        else:
+            assert all(1 <= int(n[0]) <= 2 for n in nf)
+        assert peaked_ssd.cache_length() == w.prompt_len + 6
+
+
+def test_prompt_of_one_token(tiny_ssd, tiny_oracles):
+    """The shortest prefix: one cached key.  Cache and root predictions against the oracle, SSD == stepwise."""
+    w = wl.TINY
+    _, ob = tiny_oracles[w.name]
+    b = _binding()
+    prompt = wl.make_prompts(w).numpy()[:, :1]
+    tiny_ssd.prefill(prompt)
+    assert tiny_ssd.cache_length() == 1
+    cache = ob.prefill(prompt[0])
+    for l in range(w.n_layers):
+        k, v = tiny_ssd.read_cache(l, 0, 1)
+        assert np.abs(k - cache.k[l]).max() < 2e-2 * max(1.0, np.abs(cache.k[l]).max())
+        assert np.abs(v - cache.v[l]).max() < 2e-2 * max(1.0, np.abs(cache.v[l]).max())
+    ids = np.full((1, 1, w.block_len), w.mask_id)
+    masked = np.ones((1, 1, w.block_len), dtype=bool)
+    tok, conf, logits = tiny_ssd.verify_forward(ids, masked, want_logits=True)
+    otok, oconf, ogap, ologits = ob.verify(ids[0], masked[0], cache)
+    assert np.abs(logits[0] - ologits).max() < 1e-2
+    assert np.allclose(conf[0], oconf, rtol=CONF_RTOL, atol=1e-6)
+    want, _, _ = tiny_ssd.generate(b.MODE_STEPWISE, 2 * w.block_len, w.block_len, 1)
+    tiny_ssd.prefill(prompt)
+    got, _, _ = tiny_ssd.generate(b.MODE_SSD, 2 * w.block_len, w.block_len, 1)
+    assert np.array_equal(got, want)
+
+
 # ------------------------------------------------------------------------------------------
 # error paths (host-side checks; nothing here faults a GPU)
 # ------------------------------------------------------------------------------------------
