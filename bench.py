@@ -354,7 +354,7 @@ def run_ours(args):
     ssd = binding.Ssd(binding.config_from_workload(w, max_drafts=min(cfg_drafts, B - 1)))
     for k, v in (("split_k_qkv", args.split_qkv), ("split_k_o", args.split_o), ("split_k_down", args.split_down),
                  ("kv_split", args.kv_split), ("attn_impl", args.attn_impl), ("two_sm_rows", args.two_sm_rows),
-                 ("gemm_max_stages", args.gemm_max_stages)):
+                 ("gemm_max_stages", args.gemm_max_stages), ("attn_pipe_keys", args.attn_pipe_keys)):
         if v is not None:
             ssd.set_option(k, v)
     t0 = time.time()
@@ -691,6 +691,8 @@ def main():
     ap.add_argument("--two-sm-rows", type=int, default=None,
                     help="projection tile pairs run as one two-SM MMA from this many rows on (0: never)")
     ap.add_argument("--gemm-max-stages", type=int, default=None, help="tuning: cap on the projection kernel's ring depth")
+    ap.add_argument("--attn-pipe-keys", type=int, default=None,
+                    help="tuning: prefixes of at least this many keys take the pipelined attention form (0: never)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: fewer layers of the same shape")
     ap.add_argument("--gen-len", type=int, default=0, help="profiling only: shorter generation")

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libssd_b200.so")
-SOURCES = ["elementwise.cu", "attention.cu", "attention_verify.cu", "attention_verify_tc.cu", "gemm.cu", "tree.cu", "ssd_lib.cu", "noalloc.cu"]
+SOURCES = ["elementwise.cu", "attention.cu", "attention_verify.cu", "attention_verify_tc.cu", "attention_verify_pipe.cu", "gemm.cu", "tree.cu", "ssd_lib.cu", "noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

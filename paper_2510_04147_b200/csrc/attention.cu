@@ -57,8 +57,9 @@ __global__ void __launch_bounds__(kAttnThreads) attn_split_kernel(AttnArgs a, in
   const bf16* vbase;
   size_t krow_stride = (size_t)a.Hkv * HD;
   if (!local) {
-    kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * HD;
-    vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * HD;
+    kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride;
+    vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride;
+    krow_stride = a.kv_pos_stride;
   } else {
     kbase = a.local_k + ((size_t)slot * rps * a.Hkv + kvh) * HD;
     vbase = a.local_v + ((size_t)slot * rps * a.Hkv + kvh) * HD;

@@ -106,9 +106,9 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
   // ---- prefix K/V: asynchronous copies from the cache, 128 keys per step
   auto load_prefix = [&](int pair, int buf) {
     const int seq = seq_of_slot(a.map, slot);
-    const bf16* kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * HD;
-    const bf16* vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * HD;
-    const size_t krow_stride = (size_t)a.Hkv * HD;
+    const bf16* kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride;
+    const bf16* vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride;
+    const size_t krow_stride = a.kv_pos_stride;
     const int key0 = k_begin + pair * kPairKeys;
     bf16* dK = sKV + (size_t)buf * kBufElems;
     bf16* dV = dK + kPairKeys * HD;
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(QT * 4, MINB) attn_verify_kernel(AttnArgs a, i
   const bool commit_kv = a.cache_k_out != nullptr && (h % (a.H / a.Hkv)) == 0;
   const int commit_rows = a.map.chain_T0 > 0 ? a.map.chain_T0 : rps;   // sequence-local rows whose K/V are cached
   auto cache_row = [&](int lr) -> size_t {
-    return (size_t)seq_of_slot(a.map, slot) * a.cache_seq_stride + ((size_t)(a.map.pos0 + lr) * a.Hkv + kvh) * HD;
+    return (size_t)seq_of_slot(a.map, slot) * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride + (size_t)(a.map.pos0 + lr) * a.kv_pos_stride;
   };
   // ---- one chunk (8 rotation pairs) of one row of a head of the fused projection: sum over the
   //      splits in split order (four splits' loads in flight at a time), rotary embedding, bf16

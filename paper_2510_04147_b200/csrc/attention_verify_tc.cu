@@ -197,9 +197,9 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   auto load_prefix = [&](int tile, bool want_k = true, bool want_v = true) {
     const int seq = seq_of_slot(a.map, slot);
     const int kb = k_begin + tile * kKeys;
-    const bf16* kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * kHD;
-    const bf16* vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * kHD;
-    const size_t krow_stride = (size_t)a.Hkv * kHD;
+    const bf16* kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride;
+    const bf16* vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride;
+    const size_t krow_stride = a.kv_pos_stride;
     for (int idx = tid; idx < kKeys * CH; idx += kTcAttnThreads) {
       const int row = idx / CH, ch = idx % CH;
       const int key = kb + row;
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
   const bool commit_kv = a.cache_k_out != nullptr && (h % (a.H / a.Hkv)) == 0;
   const int commit_rows = a.map.chain_T0 > 0 ? a.map.chain_T0 : rps;   // sequence-local rows whose K/V are cached
   auto cache_row = [&](int lr) -> size_t {
-    return (size_t)seq_of_slot(a.map, slot) * a.cache_seq_stride + ((size_t)(a.map.pos0 + lr) * a.Hkv + kvh) * kHD;
+    return (size_t)seq_of_slot(a.map, slot) * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride + (size_t)(a.map.pos0 + lr) * a.kv_pos_stride;
   };
   // The cache is not written by any kernel of this forward, so its tiles may be requested before the
   // dependency wait - unless the slot -> sequence map is only known on the device.

@@ -107,7 +107,8 @@ __global__ void __launch_bounds__(kRopeHeadsPerBlock * 32) qkv_rope_kernel(const
                                                                             size_t split_stride, int H, int Hkv, int hd,
                                                                             const float2* rope_table, RowMap map,
                                                                             bf16* q, bf16* k_dst, bf16* v_dst,
-                                                                            int kv_to_cache, size_t cache_seq_stride) {
+                                                                            int kv_to_cache, size_t cache_seq_stride,
+                                                                            size_t kv_pos_stride, size_t kv_head_stride) {
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.x;
@@ -121,10 +122,12 @@ __global__ void __launch_bounds__(kRopeHeadsPerBlock * 32) qkv_rope_kernel(const
   const int pos = map.pos0 + t;
   const int seq = map.seq_map ? map.seq_map[slot] : map.seq_base + slot;
   const float* prow = partial + (size_t)r * nqkv + (size_t)head * hd;
-  const size_t kv_row = kv_to_cache ? ((size_t)seq * cache_seq_stride + (size_t)pos * Hkv * hd) : (size_t)r * Hkv * hd;
+  // destination of KV head j of this row: the cache, or a plain [row][Hkv][hd] buffer
+  const size_t kv_row = kv_to_cache ? ((size_t)seq * cache_seq_stride + (size_t)pos * kv_pos_stride) : (size_t)r * Hkv * hd;
+  const size_t kv_head = kv_to_cache ? kv_head_stride : (size_t)hd;
   if (head < H + Hkv) {
     const float2* rt = rope_table + (size_t)pos * half;
-    bf16* dst = head < H ? q + ((size_t)r * H + head) * hd : k_dst + kv_row + (size_t)(head - H) * hd;
+    bf16* dst = head < H ? q + ((size_t)r * H + head) * hd : k_dst + kv_row + (size_t)(head - H) * kv_head;
     for (int i = lane; i < half; i += 32) {
       float x1 = 0.f, x2 = 0.f;
       for (int s = 0; s < splits; ++s) {
@@ -136,7 +139,7 @@ __global__ void __launch_bounds__(kRopeHeadsPerBlock * 32) qkv_rope_kernel(const
       dst[i + half] = __float2bfloat16_rn(x2 * cs.x + x1 * cs.y);
     }
   } else {
-    bf16* dst = v_dst + kv_row + (size_t)(head - H - Hkv) * hd;
+    bf16* dst = v_dst + kv_row + (size_t)(head - H - Hkv) * kv_head;
     for (int e = lane; e < hd; e += 32) {
       float x = 0.f;
       for (int s = 0; s < splits; ++s) x += prow[s * split_stride + e];
@@ -364,11 +367,11 @@ void launch_stream_prep(cudaStream_t st, const float* h, const float* gain, bf16
 
 void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H, int Hkv,
                      int hd, const float2* rope_table, RowMap map, bf16* q, bf16* k_dst, bf16* v_dst, int kv_to_cache,
-                     size_t cache_seq_stride) {
+                     size_t cache_seq_stride, size_t kv_pos_stride, size_t kv_head_stride) {
   const int heads = H + 2 * Hkv;
   dim3 grid(R, (heads + kRopeHeadsPerBlock - 1) / kRopeHeadsPerBlock);
   launch_pdl(qkv_rope_kernel, grid, dim3(kRopeHeadsPerBlock * 32), 0, st, partial, splits, split_stride, H, Hkv, hd,
-             rope_table, map, q, k_dst, v_dst, kv_to_cache, cache_seq_stride);
+             rope_table, map, q, k_dst, v_dst, kv_to_cache, cache_seq_stride, kv_pos_stride, kv_head_stride);
 }
 
 void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, int V, int mask_id,

@@ -112,7 +112,7 @@ void launch_stream_prep(cudaStream_t st, const float* h, const float* gain, bf16
 // kv_to_cache: k/v rows go to cache[(seq*max_seq + pos)*Hkv*hd] else to local [r][Hkv][hd].
 void launch_qkv_rope(cudaStream_t st, const float* partial, int splits, size_t split_stride, int R, int H,
                      int Hkv, int hd, const float2* rope_table, RowMap map, bf16* q, bf16* k_dst, bf16* v_dst,
-                     int kv_to_cache, size_t cache_seq_stride);
+                     int kv_to_cache, size_t cache_seq_stride, size_t kv_pos_stride, size_t kv_head_stride);
 // per row: argmax / max-softmax-probability over the vocabulary with mask_id excluded
 void launch_lm_stats_from_logits(cudaStream_t st, const float* logits, int R, int V, int mask_id,
                                  const uint8_t* row_wanted, int* tok, float* conf);
@@ -154,6 +154,8 @@ struct AttnArgs {
   int hole_begin, hole_len;
   int kv_split;         // prefix keys per split (a function of S only)
   size_t cache_seq_stride;
+  size_t kv_pos_stride, kv_head_stride;   // element (sequence, position, kv head) of the cache lies at
+                                          // seq * cache_seq_stride + head * kv_head_stride + pos * kv_pos_stride
   RowMap map;
   int n_seq_slots;
 };
@@ -166,6 +168,10 @@ int launch_attention_verify(cudaStream_t st, const AttnArgs& a);
 // node-local keys that fit one 128-key tile; needs a.err_flag.  Returns 0 (launched), 1 (shape not
 // covered: use launch_attention_verify) or a negative ssd error code.
 int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a);
+// The same for long prefixes: one CTA per (query tile, head, sequence) with all key tiles in one software pipeline
+// (no cluster, no merge).  Head dimension 128, node width dividing 128, any prefix length; needs a.err_flag.
+// Same return codes.
+int launch_attention_verify_pipe(cudaStream_t st, const AttnArgs& a);
 constexpr int kAttnMaxClusterParts = 8;
 
 // ---------------------------------------------------------------- projections

@@ -41,6 +41,9 @@ struct ssd_ctx {
 
   bf16 *cacheK = nullptr, *cacheV = nullptr;
   size_t cache_seq_stride = 0, cache_layer_stride = 0;
+  // The cache is head-major, [layer][sequence][kv head][position][hd]: the keys of one head - what an attention CTA
+  // streams - are contiguous, a 128-key tile is one 32 KB run instead of 128 runs of 256 bytes a whole row apart.
+  size_t kv_pos_stride = 0, kv_head_stride = 0;
   float2* rope = nullptr;
 
   int n_max = 1;         // nodes per sequence the buffers can hold
@@ -109,6 +112,7 @@ struct ssd_ctx {
   int attn_impl = 1;                       // 1: tcgen05 attention where the shape allows; 0: mma.sync form only
   int64_t launches = 0;
   int gemm_max_stages = 0;       // tuning: cap on the projection kernel's ring depth (0: none)
+  int attn_pipe_keys = 2048;     // prefixes of at least this many keys take the pipelined attention form (0: never)
   int wait_limit_us = 0;         // bound of the projection kernel's barrier waits (0: the kernel's default, 2 s)
   int starve_gemm_kb = 0;        // test hook for ssd_gemm_bf16: K block (1-based) whose copies are left out
   bool profiling = false;        // mode 1: CUDA events around every launch (serialises the stream)
@@ -376,7 +380,8 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     a.out = c->att;
     a.R = R; a.H = H; a.Hkv = Hkv; a.hd = hd; a.S = attn_S; a.kv_split = kv_split;
     a.hole_begin = hole_len > 0 ? S : 0; a.hole_len = hole_len;
-    a.cache_seq_stride = c->cache_seq_stride; a.map = map; a.n_seq_slots = n_slots;
+    a.cache_seq_stride = c->cache_seq_stride; a.kv_pos_stride = c->kv_pos_stride; a.kv_head_stride = c->kv_head_stride;
+    a.map = map; a.n_seq_slots = n_slots;
     const double kvb = (double)n_slots * attn_S * Hkv * hd * 4.0 + (double)R * (H + 2 * Hkv) * hd * 2.0 + (double)R * H * hd * 2.0;
     if (via_cache) {
       // the rotary pass writes K/V into the cache; attention then reads the cache, which holds the rows themselves
@@ -384,7 +389,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
         Scope sc(c, SSD_PROF_ELEMWISE, (double)R * c->nqkv * (4.0 * g.splits + 2.0));
         launch_qkv_rope(c->st, c->partial, g.splits, (size_t)R * c->nqkv, R, H, Hkv, hd, c->rope, map, c->q,
                         c->cacheK + (size_t)l * c->cache_layer_stride, c->cacheV + (size_t)l * c->cache_layer_stride, 1,
-                        c->cache_seq_stride);
+                        c->cache_seq_stride, c->kv_pos_stride, c->kv_head_stride);
       }
       if (l == nl - 1) break;   // only this layer's K/V were still needed
       a.q = c->q; a.part_o = c->part_o; a.part_ml = c->part_ml;
@@ -400,7 +405,9 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
       Scope sc(c, SSD_PROF_ATTN, kvb, 1);
       a.err_flag = c->flags;
       int arc = 1;
-      if (c->attn_impl == 1) arc = launch_attention_verify_tc(c->st, a);   // 1: shape not covered by the tcgen05 form
+      // a function of the prefix length alone: long prefixes walk their key tiles in one pipelined CTA per head
+      if (c->attn_impl == 1 && c->attn_pipe_keys > 0 && attn_S >= c->attn_pipe_keys) arc = launch_attention_verify_pipe(c->st, a);
+      if (arc == 1 && c->attn_impl == 1) arc = launch_attention_verify_tc(c->st, a);   // 1: shape not covered by the tcgen05 form
       if (arc == 1) arc = launch_attention_verify(c->st, a);
       if (arc != 0) return fail(c, arc, "verification attention rejected S=%d kv_split=%d (code %d)", attn_S, kv_split, arc);
       if (commit_form && l == nl - 1) break;   // the last layer's K/V are in the cache; nothing reads its output
@@ -646,6 +653,8 @@ int ssd_create(const ssd_config* cfg, void* cuda_stream, ssd_ctx** out) {
     ALLOC(c, c->lm_head, tiled_elems(c->V, d));
     ALLOC(c, c->g_final, d);
     c->cache_seq_stride = (size_t)k.max_seq * c->kvdim;
+    c->kv_pos_stride = (size_t)c->hd;
+    c->kv_head_stride = (size_t)k.max_seq * c->hd;
     c->cache_layer_stride = c->cache_seq_stride * k.max_batch;
     ALLOC(c, c->cacheK, c->cache_layer_stride * k.n_layers);
     ALLOC(c, c->cacheV, c->cache_layer_stride * k.n_layers);
@@ -1265,7 +1274,11 @@ int ssd_read_cache(ssd_ctx* c, int32_t layer, int32_t seq, int32_t length, float
     float* dst = which ? out_v : out_k;
     if (!dst) continue;
     const bf16* src = (which ? c->cacheV : c->cacheK) + (size_t)layer * c->cache_layer_stride + (size_t)seq * c->cache_seq_stride;
-    CUDA_TRY(c, cudaMemcpyAsync(tmp.data(), src, n * sizeof(bf16), cudaMemcpyDeviceToHost, c->st));
+    // the interface's layout is [position][kv head][hd]: one strided copy per head of the head-major cache
+    for (int j = 0; j < c->Hkv && length > 0; ++j)
+      CUDA_TRY(c, cudaMemcpy2DAsync(tmp.data() + (size_t)j * c->hd, (size_t)c->kvdim * sizeof(bf16), src + (size_t)j * c->kv_head_stride,
+                                    c->kv_pos_stride * sizeof(bf16), (size_t)c->hd * sizeof(bf16), (size_t)length,
+                                    cudaMemcpyDeviceToHost, c->st));
     CUDA_TRY(c, cudaStreamSynchronize(c->st));
     for (size_t i = 0; i < n; ++i) dst[i] = __bfloat162float(tmp[i]);
   }
@@ -1288,7 +1301,10 @@ int ssd_write_cache(ssd_ctx* c, int32_t layer, int32_t seq, int32_t length, cons
     const float* src = which ? v : k;
     bf16* dst = (which ? c->cacheV : c->cacheK) + (size_t)layer * c->cache_layer_stride + (size_t)seq * c->cache_seq_stride;
     for (size_t i = 0; i < n; ++i) tmp[i] = __float2bfloat16_rn(src[i]);
-    CUDA_TRY(c, cudaMemcpyAsync(dst, tmp.data(), n * sizeof(bf16), cudaMemcpyHostToDevice, c->st));
+    for (int j = 0; j < c->Hkv && length > 0; ++j)
+      CUDA_TRY(c, cudaMemcpy2DAsync(dst + (size_t)j * c->kv_head_stride, c->kv_pos_stride * sizeof(bf16), tmp.data() + (size_t)j * c->hd,
+                                    (size_t)c->kvdim * sizeof(bf16), (size_t)c->hd * sizeof(bf16), (size_t)length,
+                                    cudaMemcpyHostToDevice, c->st));
     CUDA_TRY(c, cudaStreamSynchronize(c->st));
   }
   return SSD_OK;
@@ -1530,6 +1546,11 @@ int ssd_set_option(ssd_ctx* c, const char* key, int32_t value) {
   if (!strcmp(key, "wait_limit_us")) {
     if (value < 0) return fail(c, SSD_ERR_INVALID_ARG, "wait_limit_us is 0 (default, 2 s) or a bound in microseconds");
     c->wait_limit_us = value;
+    return SSD_OK;
+  }
+  if (!strcmp(key, "attn_pipe_keys")) {
+    if (value < 0) return fail(c, SSD_ERR_INVALID_ARG, "attn_pipe_keys is 0 (never) or a prefix length in keys");
+    c->attn_pipe_keys = value;
     return SSD_OK;
   }
   if (!strcmp(key, "starve_gemm_kb")) {

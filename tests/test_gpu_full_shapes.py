@@ -56,11 +56,26 @@ def _binding():
     return binding
 
 
-def _make(w, max_drafts, max_batch=None, max_seq=None):
+def _make(w, max_drafts, max_batch=None, max_seq=None, attn_form="by_prefix_length"):
+    """attn_form "pipelined": the attention form of long prefixes (one CTA per head walks all key tiles) is taken
+    whatever the prefix length, so that the small cases here cover it; otherwise the prefix length decides."""
     b = _binding()
     ssd = b.Ssd(b.config_from_workload(w, max_drafts=max_drafts, max_batch=max_batch, max_seq=max_seq))
+    if attn_form == "pipelined":
+        ssd.set_option("attn_pipe_keys", 1)
     ssd.load_workload_weights(w)
     return ssd
+
+
+ATTN_FORMS = ["by_prefix_length", "pipelined"]
+_ORACLE_RESULTS = {}
+
+
+def _oracle_once(key, compute):
+    """The oracle's result for inputs that do not depend on the GPU, computed once for all attention forms of a test."""
+    if key not in _ORACLE_RESULTS:
+        _ORACLE_RESULTS[key] = compute()
+    return _ORACLE_RESULTS[key]
 
 
 def _nodes(w, rng, n_nodes, T, batch=1):
@@ -91,16 +106,20 @@ def test_full_width_forward_matches_oracle(case):
     rng = np.random.default_rng(11)
     T = w.block_len
     prompt = wl.make_prompts(w).numpy()
+    blk = rng.integers(0, w.vocab - 1, (1, T))
+    ids, masked = _nodes(w, rng, n_nodes, T)
+    gpu = {}
     ssd = _make(w, max_drafts=n_nodes)
     try:
-        ssd.prefill(prompt)
-        blk = rng.integers(0, w.vocab - 1, (1, T))
-        ssd.block_begin(T)
-        ssd.set_block_state(blk, np.zeros((1, T), np.uint8))
-        ssd.block_commit()                                   # prefix = prompt + one committed block
-        ids, masked = _nodes(w, rng, n_nodes, T)
-        tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
-        tok2, conf2, _ = ssd.verify_forward(ids, masked)     # fused LM-head statistics
+        for form in ATTN_FORMS:                              # the cluster-of-parts attention and the pipelined one
+            ssd.set_option("attn_pipe_keys", 1 if form == "pipelined" else 2048)
+            ssd.prefill(prompt)
+            ssd.block_begin(T)
+            ssd.set_block_state(blk, np.zeros((1, T), np.uint8))
+            ssd.block_commit()                               # prefix = prompt + one committed block
+            tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
+            tok2, conf2, _ = ssd.verify_forward(ids, masked) # fused LM-head statistics
+            gpu[form] = (tok, conf, logits, tok2, conf2)
     finally:
         ssd.destroy()
     res = {}
@@ -111,11 +130,19 @@ def test_full_width_forward_matches_oracle(case):
         res[mode] = o.verify(ids[0], masked[0], cache)
     otok, oconf, ogap, ologits = res[None]
     rms_bound, max_bound = _noise_bounds(ologits, res["bf16"][3])
-    err = logits[0] - ologits
-    rms, mx = float(np.sqrt((err ** 2).mean())), float(np.abs(err).max())
     m = masked[0]
     sure = m & _sure_tokens(ogap, oconf, max_bound)
-    print(f"{case}: logit std {ologits.std():.3f}; CUDA vs fp64 oracle rms {rms:.4f} max {mx:.4f}; bf16-operand oracle "
+    for form in ATTN_FORMS:
+        tok, conf, logits, tok2, conf2 = gpu[form]
+        _check_forward_against_oracle(case, form, w, m, sure, logits, tok, conf, tok2, conf2, otok, oconf, ologits, rms_bound,
+                                      max_bound)
+
+
+def _check_forward_against_oracle(case, form, w, m, sure, logits, tok, conf, tok2, conf2, otok, oconf, ologits, rms_bound,
+                                  max_bound):
+    err = logits[0] - ologits
+    rms, mx = float(np.sqrt((err ** 2).mean())), float(np.abs(err).max())
+    print(f"{case} ({form}): logit std {ologits.std():.3f}; CUDA vs fp64 oracle rms {rms:.4f} max {mx:.4f}; bf16-operand oracle "
           f"vs fp64 oracle rms {rms_bound / NOISE_RMS:.4f} max {max_bound / NOISE_MAX:.4f}; stated {STATED_TOL} "
           f"{'met' if mx < STATED_TOL else 'not attainable with bf16 operands at this logit scale'}; "
           f"sure rows {int(sure.sum())} of {int(m.sum())}")
@@ -346,8 +373,8 @@ def test_two_sm_projections_change_no_bit_of_a_forward(case, n_nodes):
 
 
 def test_both_attention_forms_agree_at_full_width():
-    """The tcgen05 attention (default where the shape allows) and the mma.sync form compute the same
-    forward up to the rounding of a different summation order."""
+    """The two tcgen05 attention forms (cluster of key parts; one pipelined CTA per head) and the mma.sync form
+    compute the same forward up to the rounding of a different summation order."""
     w, n_nodes = WIDTH_CASES["llada_width"]
     rng = np.random.default_rng(3)
     T = w.block_len
@@ -356,8 +383,9 @@ def test_both_attention_forms_agree_at_full_width():
     out = {}
     ssd = _make(w, max_drafts=n_nodes)
     try:
-        for impl in (0, 1):
-            ssd.set_option("attn_impl", impl)
+        for impl, pipe_keys in ((0, 0), (1, 0), (2, 1)):
+            ssd.set_option("attn_impl", min(impl, 1))
+            ssd.set_option("attn_pipe_keys", pipe_keys)
             ssd.prefill(prompt)
             tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
             out[impl] = (tok, conf, logits)
@@ -371,11 +399,38 @@ def test_both_attention_forms_agree_at_full_width():
         o = make_oracle(w, as_bf16=True, operand_rounding=mode)
         ol[mode] = o.verify(ids[0], masked[0], o.prefill(prm))[3]
     rms_bound, max_bound = _noise_bounds(ol[None], ol["bf16"])
-    diff = out[0][2][0] - out[1][2][0]
-    assert np.abs(diff).max() < 2 * max_bound, (np.abs(diff).max(), max_bound)
-    assert np.sqrt((diff ** 2).mean()) < 2 * rms_bound
     m = masked[0]
-    assert np.allclose(out[0][1][0][m], out[1][1][0][m], rtol=np.exp(4.0 * max_bound) - 1.0, atol=1e-6)
+    for x, y in ((0, 1), (1, 2)):
+        diff = out[x][2][0] - out[y][2][0]
+        assert np.abs(diff).max() > 0                        # (really two forms: some bit differs)
+        assert np.abs(diff).max() < 2 * max_bound, (np.abs(diff).max(), max_bound)
+        assert np.sqrt((diff ** 2).mean()) < 2 * rms_bound
+        assert np.allclose(out[x][1][0][m], out[y][1][0][m], rtol=np.exp(4.0 * max_bound) - 1.0, atol=1e-6)
+
+
+def test_pipelined_attention_treats_a_node_as_if_alone():
+    """The attention form of long prefixes: a node's (token, confidence) bits do not depend on how many nodes share
+    the forward (query tiles of 32, 64 or 128 rows, one or two tiles per head) nor on other sequences of the batch."""
+    w, _ = WIDTH_CASES["llada_width"]
+    w = w.replace(name="llada_width_pipe", batch=2)
+    rng = np.random.default_rng(29)
+    T = w.block_len
+    prompts = wl.make_prompts(w).numpy()
+    ids, masked = _nodes(w, rng, 5, T, batch=2)
+    ssd = _make(w, max_drafts=5, max_batch=2, attn_form="pipelined")
+    try:
+        ssd.prefill(prompts)
+        tok, conf, _ = ssd.verify_forward(ids, masked)                          # 2 sequences x 5 nodes: 128-row tiles, two per head
+        ssd.prefill(prompts[1:2])
+        tok5, conf5, _ = ssd.verify_forward(ids[1:2], masked[1:2])              # the second sequence alone
+        tok2, conf2, _ = ssd.verify_forward(ids[1:2, 1:3], masked[1:2, 1:3])    # two of its nodes: one 64-row tile
+        tok1, conf1, _ = ssd.verify_forward(ids[1:2, 4:5], masked[1:2, 4:5])    # one node: a 32-row tile
+    finally:
+        ssd.destroy()
+    bits = lambda x: np.ascontiguousarray(x).view(np.uint32)
+    assert np.array_equal(tok5[0], tok[1]) and np.array_equal(bits(conf5[0]), bits(conf[1]))
+    assert np.array_equal(tok2[0], tok[1, 1:3]) and np.array_equal(bits(conf2[0]), bits(conf[1, 1:3]))
+    assert np.array_equal(tok1[0], tok[1, 4:5]) and np.array_equal(bits(conf1[0]), bits(conf[1, 4:5]))
 
 
 # ------------------------------------------------------------------------------------------
@@ -402,7 +457,8 @@ def _stepwise_trace_is_near_tie_before(o, prompt, gen_len, w, first, e_max):
     return False
 
 
-def test_full_width_mix_order_and_cross_block_generations():
+@pytest.mark.parametrize("attn_form", ATTN_FORMS)
+def test_full_width_mix_order_and_cross_block_generations(attn_form):
     """At the LLaDA width (tcgen05 attention, 32-token blocks): mix-order SSD == stepwise bit for bit; SSD with
     candidates from the next block (window nodes of 64 rows, commits riding in front of multi-node forwards)
     decodes the stepwise tokens up to the first decision that is a near-tie within the bf16 noise bound."""
@@ -410,7 +466,7 @@ def test_full_width_mix_order_and_cross_block_generations():
     b = _binding()
     prompt = wl.make_prompts(w).numpy()
     N = 3
-    ssd = _make(w, max_drafts=2 * N + 1)
+    ssd = _make(w, max_drafts=2 * N + 1, attn_form=attn_form)
     try:
         ssd.set_option("max_drafts", N)
         ssd.prefill(prompt)
@@ -442,7 +498,8 @@ def test_full_width_mix_order_and_cross_block_generations():
           f"cross-block {sum(int(n[0]) for n in nf_x)}; cross-block tokens differing from stepwise: {len(diff)}")
 
 
-def test_full_width_window_forward_matches_oracle():
+@pytest.mark.parametrize("attn_form", ATTN_FORMS)
+def test_full_width_window_forward_matches_oracle(attn_form):
     """One window forward [current block | next block] at the LLaDA width, state of both blocks given: the
     confidences of every asked row of every node against the oracle's block-causal window, and the walk / new
     state bit-exact against the oracle's logic applied to the GPU forward's own outputs."""
@@ -459,7 +516,7 @@ def test_full_width_window_forward_matches_oracle():
     masked[T:] = True
     dt = rng.integers(0, w.vocab - 1, W2)
     dc = rng.random(W2).astype(np.float32)
-    ssd = _make(w, max_drafts=2 * N + 1)
+    ssd = _make(w, max_drafts=2 * N + 1, attn_form=attn_form)
     try:
         ssd.set_option("max_drafts", N)
         ssd.prefill(prompt)
@@ -479,10 +536,13 @@ def test_full_width_window_forward_matches_oracle():
     cand += [(T + p, t) for (p, t) in so.select_candidates(dt[T:], dc[T:], masked[T:], N - 2)]
     assert n == len(cand) + 1 == N + 1
     node_ids, node_masked = so.build_chain(ids, masked, cand, mid)
-    res = {}
-    for mode in (None, "bf16"):
-        o = make_oracle(w, as_bf16=True, operand_rounding=mode)
-        res[mode] = o.verify_window(node_ids, node_masked, T, o.prefill(prompt[0]))
+    def windows():
+        res = {}
+        for mode in (None, "bf16"):
+            o = make_oracle(w, as_bf16=True, operand_rounding=mode)
+            res[mode] = o.verify_window(node_ids, node_masked, T, o.prefill(prompt[0]))
+        return res
+    res = _oracle_once("window", windows)
     oconf, rconf = res[None][1], res["bf16"][1]
     m = node_masked
     # confidences: no further from the fp64 oracle than NOISE_MAX times the bf16-operand oracle's own distance
@@ -509,8 +569,9 @@ def test_full_width_window_forward_matches_oracle():
     assert np.array_equal(dc_g[want_m].view(np.uint32), conf_g[a][want_m].view(np.uint32))
 
 
+@pytest.mark.parametrize("attn_form", ATTN_FORMS)
 @pytest.mark.parametrize("case", ["llada_width", "dream_width"])
-def test_full_width_dual_cache_forward_matches_oracle(case):
+def test_full_width_dual_cache_forward_matches_oracle(case, attn_form):
     """The dual cache at full width (the tcgen05 attention reads the cached keys around a hole at the current
     block): logits of a block forward after a refresh against the oracle's refresh_all + forward."""
     from oracle import ssd_oracle as so
@@ -519,7 +580,7 @@ def test_full_width_dual_cache_forward_matches_oracle(case):
     prompt = wl.make_prompts(w).numpy()
     P, T, L, mid = w.prompt_len, w.block_len, w.gen_len, w.mask_id
     block0 = rng.integers(0, w.vocab - 1, T)
-    ssd = _make(w, max_drafts=n_nodes)
+    ssd = _make(w, max_drafts=n_nodes, attn_form=attn_form)
     try:
         ssd.prefill(prompt)
         ssd.set_option("dual_cache", P + L)
@@ -537,14 +598,17 @@ def test_full_width_dual_cache_forward_matches_oracle(case):
     x1 = np.concatenate([prompt[0], np.full(L, mid)])
     x2 = np.concatenate([prompt[0], block0, np.full(L - T, mid)])
     for x, S, got in ((x1, P, logits), (x2, P + T, logits2)):
-        ol = {}
-        for mode in (None, "bf16"):
-            o = make_oracle(w, as_bf16=True, operand_rounding=mode)
-            full = o.refresh_all(x)
-            outside = so.Cache(o.cfg)
-            outside.k = [np.concatenate([k[:S], k[S + T:]], axis=0) for k in full.k]
-            outside.v = [np.concatenate([v[:S], v[S + T:]], axis=0) for v in full.v]
-            ol[mode] = o.forward_rows(ids[0], S, outside)[0]
+        def block_forward():
+            ol = {}
+            for mode in (None, "bf16"):
+                o = make_oracle(w, as_bf16=True, operand_rounding=mode)
+                full = o.refresh_all(x)
+                outside = so.Cache(o.cfg)
+                outside.k = [np.concatenate([k[:S], k[S + T:]], axis=0) for k in full.k]
+                outside.v = [np.concatenate([v[:S], v[S + T:]], axis=0) for v in full.v]
+                ol[mode] = o.forward_rows(ids[0], S, outside)[0]
+            return ol
+        ol = _oracle_once(("dual_cache", case, S), block_forward)
         rms_bound, max_bound = _noise_bounds(ol[None], ol["bf16"])
         err = got[0] - ol[None]
         assert np.sqrt((err ** 2).mean()) < rms_bound and np.abs(err).max() < max_bound, (S, np.abs(err).max(), max_bound)
