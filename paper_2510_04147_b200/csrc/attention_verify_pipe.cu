@@ -8,10 +8,12 @@
 // partials of the fused q|k|v projection (summed in split order, rotary embedding, bf16) and writes the cache
 // rows of a commit.  Every cached K/V tile is read once per (query tile, head) and serves all nodes.
 //
-// Pipeline (three K and two V stages in shared memory, two S accumulators and one O accumulator in tensor
-// memory): while the threads run the softmax of tile u - row maximum, running (max, sum), P written over the K
-// tile - the tensor core already computes S = Q K^T of tile u+1, and the copies of K of tile u+2 and V of tile
-// u+1 are in flight; O += P V of tile u is issued when P is complete and finishes under the next tile's
+// Pipeline (two K stages, one P tile and two V stages in shared memory, two S accumulators and one O accumulator
+// in tensor memory): while the threads run the softmax of tile u - row maximum, running (max, sum), P written to
+// its tile - the tensor core already computes S = Q K^T of tile u+1.  K of tile u+2 is requested as soon as S of
+// tile u is complete (its stage is free then), V of tile u+1 as soon as O += P V of tile u-1 is: both a whole
+// iteration before they are needed.  O += P V of tile u is issued when P is complete and finishes under the next
+// tile's
 // softmax.  O is rescaled in tensor memory when a row's maximum grows.  A query row is one TMEM lane shared by
 // two threads (warps w and w+4), each owning half of the lane's columns; a tile of 32 or 64 rows is replicated
 // to 128 lanes so that more threads share a row.  The order of the tiles and of every sum is fixed by the shapes
@@ -28,10 +30,11 @@ using namespace attn;
 
 constexpr int kHD = 128;
 constexpr int kKeys = 128;                  // keys per tile
-constexpr int kPipeThreads = 256;
+constexpr int kPipeThreads = 256;           // softmax threads: two per TMEM lane
+constexpr int kPipeBlock = kPipeThreads + 32;   // + one warp that issues the MMAs
 constexpr int kHalfBytes = kKeys * 128;     // one 64-column half of a 128-row tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // a [128][128] bf16 tile
-constexpr int kStagesK = 3, kStagesV = 2;
+constexpr int kStagesK = 2, kStagesV = 2;      // + one P tile
 constexpr unsigned long long kPipeWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ unsigned long long gtimer_ns() {
@@ -51,17 +54,32 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// bounded: false when the limit expired
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// bounded: false when the limit expired or another thread of the CTA gave up (`abort` set)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
   unsigned long long t0 = 0;
   for (uint32_t spins = 1;; ++spins) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((spins & 255u) == 0) {
+      if (*abort) return false;
       const unsigned long long now = gtimer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kPipeWaitLimitNs) return false;
+      else if (now - t0 > kPipeWaitLimitNs) { *abort = 1; return false; }
     }
   }
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// barrier 1 of the softmax threads (the MMA warp does not take part); returns the AND of `v` over them
+__device__ __forceinline__ bool softmax_barrier_and(bool v) {
+  uint32_t r;
+  asm volatile(
+      "{\n.reg .pred p, q;\n"
+      "setp.ne.b32 q, %1, 0;\n"
+      "bar.red.and.pred p, 1, 256, q;\n"
+      "selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(r) : "r"((uint32_t)(v ? 1 : 0)) : "memory");
+  return r != 0;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -126,22 +144,32 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) 
       : "memory");
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
+// 2^x on the special-function unit (the one form used everywhere in this kernel, so that a key's probability has the
+// same bits on every code path)
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 // byte offset of 16-byte chunk `ch` (0..15 over 128 columns) of row `row` in a [half][128 rows][64] tile
 __device__ __forceinline__ uint32_t tile_off(int row, int ch) {
   return (uint32_t)((ch >> 3) * kHalfBytes + row * 128 + (((ch & 7) ^ (row & 7)) << 4));
 }
 
 template <int QT>
-__global__ void __launch_bounds__(kPipeThreads, 1) attn_verify_pipe_kernel(AttnArgs a, float scale_log2) {
+__global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArgs a, float scale_log2) {
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;                                   // [2][128][64] bf16
-  uint8_t* sKs = sQ + kTileBytes;                       // kStagesK K tiles; P overwrites K once S is complete
-  uint8_t* sVs = sKs + kStagesK * kTileBytes;           // kStagesV V tiles
-  float* sMax = reinterpret_cast<float*>(sVs + kStagesV * kTileBytes);      // [2 halves x 4 copies][128 rows]
-  float* sSum = sMax + 8 * 128;                                             // [8 chunks of 16 keys][128 rows]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sSum + 8 * 128);             // [0], [1] S ready (two buffers), [2] O ready
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3);
+  uint8_t* sKs = sQ + kTileBytes;                       // kStagesK K tiles: a stage is free as soon as its S = Q K^T is complete
+  uint8_t* sP = sKs + kStagesK * kTileBytes;            // P of the tile in work (bf16, the A operand of O += P V)
+  uint8_t* sVs = sP + kTileBytes;                       // kStagesV V tiles
+  float* sMax = reinterpret_cast<float*>(sVs + kStagesV * kTileBytes);      // 2 x [2 halves x 4 copies][128 rows] (tiles alternate)
+  float* sSum = sMax + 2 * 8 * 128;                                         // 2 x [8 chunks of 16 keys][128 rows]
+  // [0], [1] S ready (two accumulators), [2] O += P V complete, [3], [4] K stage landed, [5] P written and V landed
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sSum + 2 * 8 * 128);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   constexpr int CH = kHD / 8;                            // 16-byte chunks per row
 
   pdl_launch_dependents();
@@ -165,6 +193,10 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_verify_pipe_kernel(AttnA
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
     mbar_init(smem_u32(&bars[2]), 1);
+    mbar_init(smem_u32(&bars[3]), kPipeThreads);
+    mbar_init(smem_u32(&bars[4]), kPipeThreads);
+    mbar_init(smem_u32(&bars[5]), kPipeThreads);
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -173,23 +205,41 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_verify_pipe_kernel(AttnA
   }
 
   // ---- copies into a stage: cached K/V (zero rows past the end), or the node-local rows of the projection
+  // A thread copies the same 16-byte column chunk of the rows ld_row0, ld_row0 + 16, ...: the swizzle term of its
+  // shared-memory address and its byte offset inside a cache row are constants, so a copy costs a few instructions.
+  const bool softmax_thread = tid < kPipeThreads;        // warps 0-7; warp 8 issues the MMAs
+  const int ld_ch = tid % CH, ld_row0 = tid / CH;
+  const uint32_t ld_soff = tile_off(ld_row0, ld_ch);      // + 16 * 128 bytes per step (16 rows: the same swizzle phase)
   auto load_cached = [&](int u, bool want_k, bool want_v) {
-    uint8_t* dK = sKs + (size_t)(u % kStagesK) * kTileBytes;
-    uint8_t* dV = sVs + (size_t)(u % kStagesV) * kTileBytes;
+    const uint32_t dK = smem_u32(sKs + (size_t)(u % kStagesK) * kTileBytes) + ld_soff;
+    const uint32_t dV = smem_u32(sVs + (size_t)(u % kStagesV) * kTileBytes) + ld_soff;
     const int seq = seq_of_slot(a.map, slot);
     const int kb = (u - 1) * kKeys;
-    const bf16* kbase = a.cache_k + (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride;
-    const bf16* vbase = a.cache_v + (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride;
-    const size_t krow_stride = a.kv_pos_stride;
-    for (int idx = tid; idx < kKeys * CH; idx += kPipeThreads) {
-      const int row = idx / CH, ch = idx % CH;
-      const int key = kb + row;
+    const size_t base = (size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride + ld_ch * 8;
+    const bf16* kbase = a.cache_k + base;
+    const bf16* vbase = a.cache_v + base;
+    if (kb + kKeys <= a.S && (a.hole_len == 0 || kb + kKeys <= a.hole_begin)) {
+      // a whole tile of consecutive cache rows: 16 rows further per step
+      const size_t off0 = (size_t)(kb + ld_row0) * a.kv_pos_stride, step = (size_t)(kPipeThreads / CH) * a.kv_pos_stride;
+#pragma unroll
+      for (int it = 0; it < kKeys * CH / kPipeThreads; ++it) {
+        const uint32_t so = (uint32_t)it * (kPipeThreads / CH) * 128u;
+        if (want_k) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dK + so), "l"(kbase + off0 + it * step));
+        if (want_v) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dV + so), "l"(vbase + off0 + it * step));
+      }
+      return;
+    }
+#pragma unroll
+    for (int it = 0; it < kKeys * CH / kPipeThreads; ++it) {
+      const int key = kb + ld_row0 + it * (kPipeThreads / CH);
       const bool valid = key < a.S;
       int crow = valid ? key : kb;                            // cache row of the key (a hole skips the block's own rows)
       if (crow >= a.hole_begin) crow += a.hole_len;
-      const size_t off = (size_t)crow * krow_stride + ch * 8;
-      if (want_k) cp_async16(dK + tile_off(row, ch), kbase + off, valid);
-      if (want_v) cp_async16(dV + tile_off(row, ch), vbase + off, valid);
+      const size_t off = (size_t)crow * a.kv_pos_stride;
+      const int sz = valid ? 16 : 0;                          // 0: the chunk is filled with zeros
+      const uint32_t so = (uint32_t)it * (kPipeThreads / CH) * 128u;
+      if (want_k) asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dK + so), "l"(kbase + off), "r"(sz));
+      if (want_v) asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dV + so), "l"(vbase + off), "r"(sz));
     }
   };
   const bool commit_kv = a.cache_k_out != nullptr && (h % (a.H / a.Hkv)) == 0;
@@ -197,16 +247,16 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_verify_pipe_kernel(AttnA
   // The cache is not written below the rows' own positions by any kernel of this forward, so its first tile may be
   // requested before the dependency wait - unless the slot -> sequence map is only known on the device.
   const bool early = a.map.n_inline > 0 || a.map.seq_map == nullptr;
-  if (early && n_tiles > 1) load_cached(1, true, false);
+  if (softmax_thread && early && n_tiles > 1) load_cached(1, true, false);
   pdl_wait();                              // the QKV projection's partials are complete from here on
-  if (!early && n_tiles > 1) load_cached(1, true, false);
+  if (softmax_thread && !early && n_tiles > 1) load_cached(1, true, false);
   cp_async_commit();
 
   // ---- prologue: the query tile and the node-local K/V from the fp32 split-K partials of the fused q|k|v
   //      projection.  A work item = one 16-byte chunk of a row (with its rotation partner for Q and K): the
   //      partials are summed in split order, q and k rotated, everything rounded to bf16.  Rows past the end are
   //      zero (a masked key's V row must be finite: 0 * NaN would poison O).  Two items per thread in flight.
-  {
+  if (softmax_thread) {
     constexpr int HALF = kHD / 2, CPR = HALF / 8;
     uint8_t* dK = sKs, *dV = sVs;                        // tile 0 lives in the stages 0
     const uint4 zero = make_uint4(0, 0, 0, 0);
@@ -325,178 +375,245 @@ __global__ void __launch_bounds__(kPipeThreads, 1) attn_verify_pipe_kernel(AttnA
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_O = tmem_base + 256;
-  // f32 accumulate, bf16 operands, N = 128, M = 128; bit 16: B is MN-major (V as stored, [key][hd])
-  const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-  auto issue_s = [&](int u) {                            // S[u & 1] = Q . K(u)^T: eight k16 steps over the head dimension
-    const uint32_t kbase = smem_u32(sKs + (size_t)(u % kStagesK) * kTileBytes);
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const uint32_t qa = smem_u32(sQ) + (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
-      const uint32_t ka = kbase + (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
-      tc_mma_bf16(tmem_base + (uint32_t)(u & 1) * 128u, make_desc(qa, 16, 1024), make_desc(ka, 16, 1024), idesc, (uint32_t)(k != 0));
-    }
-    tc_commit(smem_u32(&bars[u & 1]));
-  };
-  if (tid == 0) issue_s(0);
-
-  // ---- softmax, log2 domain.  TMEM lane lt = copy `cw` of query row `row`; a copy covers the keys
-  //      [cw * QT, +QT) of a tile and the lane's two threads (hw = 0, 1) half of those each, in 16-key
-  //      chunks.  A tile's row sum is ALWAYS formed from its eight 16-key chunks as
-  //      (((c0 + c1) + (c2 + c3)) + (c4 + c5)) + (c6 + c7), each chunk summed in key order, whatever QT is.
-  constexpr int REP = 128 / QT;
-  constexpr int KPT = QT / 2;                           // keys of a tile per thread
-  constexpr int NCH = KPT / 16;                         // 16-key chunks per thread
-  const int lt = tid & 127, hw = tid >> 7;
-  const int cw = lt / QT, row = lt % QT;
-  const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;   // warps w and w + 4 read TMEM lanes 32 (w & 3) ...
-  const int col0 = cw * QT + hw * KPT;                  // first column (key of a tile) of this thread
-  const int lr = lr0 + row;
-  const bool row_live = lr < rps;
-  // node-local keys this row may see, as key indices of tile 0 (key j = sequence row lk_begin + j)
-  int loc_lo = (lr / T) * T - lk_begin, loc_hi = loc_lo + T;
-  if (a.map.chain_T0 > 0 && lr % T < a.map.chain_T0) loc_hi = loc_lo + a.map.chain_T0;   // finished block: not the next block
-  loc_hi = min(loc_hi, lk_rows);
-  float m_row = -INFINITY, l_row = 0.f;                 // running maximum and sum over the tiles so far
+  const uint32_t bar_s0 = smem_u32(&bars[0]), bar_o = smem_u32(&bars[2]), bar_k0 = smem_u32(&bars[3]), bar_p = smem_u32(&bars[5]);
   bool ok = true;
-#pragma unroll 1
-  for (int u = 0; u < n_tiles; ++u) {
-    uint8_t* sK = sKs + (size_t)(u % kStagesK) * kTileBytes;
-    uint8_t* sV = sVs + (size_t)(u % kStagesV) * kTileBytes;
-    // ---- the next tile's S runs under this tile's softmax (its K was requested one iteration ago, with this tile's V)
-    if (u + 1 < n_tiles) {
-      cp_async_wait<0>();
-      asm volatile("fence.proxy.async;" ::: "memory");
-      tc_fence_before();
-      __syncthreads();
-      if (tid == 0) { tc_fence_after(); issue_s(u + 1); }
-    }
-    ok = mbar_wait(smem_u32(&bars[u & 1]), (uint32_t)((u >> 1) & 1));
-    tc_fence_after();
-    ok = __syncthreads_and(ok ? 1 : 0) != 0;              // one decision for the CTA (barriers follow)
-    if (!ok) break;
-    const uint32_t tmem_S = tmem_base + (uint32_t)(u & 1) * 128u;
-    const int key_lo = u == 0 ? loc_lo : 0;
-    const int key_hi = u == 0 ? loc_hi : min(kKeys, a.S - (u - 1) * kKeys);
 
-    // this thread's scores of the tile: one round trip to tensor memory, kept in registers for both passes
-    uint32_t sv[KPT];
+  if (!softmax_thread) {
+    // ================================================================== MMA warp
+    // Per tile u: S(u+1) = Q K(u+1)^T as soon as the softmax threads report K(u+1) landed (they do so when they
+    // enter tile u, i.e. after they have read S(u-1), whose accumulator S(u+1) overwrites), then O += P(u) V(u) as
+    // soon as they report P(u) written and V(u) landed.  The tensor core runs the MMAs in issue order.
+    if ((tid & 31) == 0) {
+      // f32 accumulate, bf16 operands, N = 128, M = 128; bit 16: B is MN-major (V as stored, [key][hd])
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+      const uint32_t idesc_pv = idesc | (1u << 16);
+      auto issue_s = [&](int u) {                        // S[u & 1] = Q . K(u)^T: eight k16 steps over the head dimension
+        const uint32_t kbase = smem_u32(sKs + (size_t)(u % kStagesK) * kTileBytes);
 #pragma unroll
-    for (int ch = 0; ch < NCH; ++ch) tmem_ld16_issue(tmem_S + lane_addr + col0 + ch * 16, &sv[ch * 16]);
-    tmem_ld_wait();
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t qa = smem_u32(sQ) + (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
+          const uint32_t ka = kbase + (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
+          tc_mma_bf16(tmem_base + (uint32_t)(u & 1) * 128u, make_desc(qa, 16, 1024), make_desc(ka, 16, 1024), idesc, (uint32_t)(k != 0));
+        }
+        tc_commit(bar_s0 + 8u * (uint32_t)(u & 1));
+      };
+      issue_s(0);
+#pragma unroll 1
+      for (int u = 0; u < n_tiles && ok; ++u) {
+        if (u + 1 < n_tiles) {
+          ok = mbar_wait(bar_k0 + 8u * (uint32_t)((u + 1) & 1), (uint32_t)((u >> 1) & 1), abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_s(u + 1);
+        }
+        ok = mbar_wait(bar_p, (uint32_t)(u & 1), abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        // O (+)= P . V: eight k16 steps over the keys.  P is K-major (keys contiguous); V is used as stored,
+        // [key][hd] = MN-major: 8-key groups 1024 B apart, the two 64-column halves 16 KB apart.
+        const uint32_t vbase = smem_u32(sVs + (size_t)(u % kStagesV) * kTileBytes);
 #pragma unroll
-    for (int ch = 0; ch < NCH; ++ch) keep16(&sv[ch * 16]);
-    float m_loc = -INFINITY;
-#pragma unroll
-    for (int j = 0; j < KPT; ++j)
-      if (col0 + j >= key_lo && col0 + j < key_hi) m_loc = fmaxf(m_loc, __uint_as_float(sv[j]) * scale_log2);
-    sMax[(hw * 4 + cw) * 128 + row] = m_loc;
-    __syncthreads();
-    float m_tile = -INFINITY;
-#pragma unroll
-    for (int k = 0; k < REP; ++k) m_tile = fmaxf(m_tile, fmaxf(sMax[k * 128 + row], sMax[(4 + k) * 128 + row]));
-    const float m_new = fmaxf(m_row, m_tile);
-    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-    const float corr = exp2f(m_row - m_use);              // 0 while no visible key has been met
-    if (u > 0) {
-      // O += P V of the previous tile is complete: its K stage is free for K of tile u + 2, its V stage for V of
-      // tile u + 1, and the output so far may be rescaled
-      ok = mbar_wait(smem_u32(&bars[2]), (uint32_t)((u - 1) & 1));
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t pa = smem_u32(sP) + (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
+          const uint32_t va = vbase + (uint32_t)(2 * k * 1024);
+          tc_mma_bf16(tmem_O, make_desc(pa, 16, 1024), make_desc(va, kHalfBytes, 1024), idesc_pv, (uint32_t)((u | k) != 0));
+        }
+        tc_commit(bar_o);
+      }
+      if (!ok) atomicExch(a.err_flag, 6);
+    }
+  } else {
+    // ================================================================== softmax threads (log2 domain)
+    // TMEM lane lt = copy `cw` of query row `row`; a copy covers the keys [cw * QT, +QT) of a tile and the lane's
+    // two threads (hw = 0, 1) half of those each, in 16-key chunks.  A tile's row sum is ALWAYS formed from its
+    // eight 16-key chunks as (((c0 + c1) + (c2 + c3)) + (c4 + c5)) + (c6 + c7), each chunk summed in key order,
+    // whatever QT is.  The threads meet once per tile (exchange of the row maxima); everything else is handed
+    // over through mbarriers, so that no thread waits for the MMA issue.
+    constexpr int REP = 128 / QT;
+    constexpr int KPT = QT / 2;                           // keys of a tile per thread
+    constexpr int NCH = KPT / 16;                         // 16-key chunks per thread
+    // A thread takes its keys in passes of at most 32 (its scores then fit in registers): one pass for tiles of 32
+    // or 64 rows, whose scores stay in registers from the maximum to the exponentials; two for 128 rows, read again.
+    constexpr int HK = KPT < 32 ? KPT : 32, NP = KPT / HK, NCP = HK / 16;
+    const int lt = tid & 127, hw = tid >> 7;
+    const int cw = lt / QT, row = lt % QT;
+    const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;   // warps w and w + 4 read TMEM lanes 32 (w & 3) ...
+    const int col0 = cw * QT + hw * KPT;                  // first column (key of a tile) of this thread
+    const int lr = lr0 + row;
+    const bool row_live = lr < rps;
+    // node-local keys this row may see, as key indices of tile 0 (key j = sequence row lk_begin + j)
+    int loc_lo = (lr / T) * T - lk_begin, loc_hi = loc_lo + T;
+    if (a.map.chain_T0 > 0 && lr % T < a.map.chain_T0) loc_hi = loc_lo + a.map.chain_T0;   // finished block: not the next block
+    loc_hi = min(loc_hi, lk_rows);
+    float m_row = -INFINITY, l_row = 0.f;                 // running maximum; running sum up to the tile before the last one met
+    bool broke = false;                                   // the loop ended at the meeting point, for all threads alike
+    float corr_prev = 1.f;                                // rescale factor of the tile whose sum is still to be added
+    auto tile_sum = [&](int u) -> float {                 // the row's sum over tile u, from the eight chunk sums
+      const float* q = sSum + (u & 1) * 8 * 128 + row;
+      return (((q[0 * 128] + q[1 * 128]) + (q[2 * 128] + q[3 * 128])) + (q[4 * 128] + q[5 * 128])) + (q[6 * 128] + q[7 * 128]);
+    };
+#pragma unroll 1
+    for (int u = 0; u < n_tiles; ++u) {
+      // ---- K of the next tile (requested a whole iteration ago) has landed for this thread: tell the MMA warp.
+      //      Copy groups are committed in the order K(u+1), V(u), K(u+2), V(u+1), ...
+      if (u + 1 < n_tiles) {
+        cp_async_wait<1>();                                 // everything but V(u), which has until O += P V
+        asm volatile("fence.proxy.async;" ::: "memory");
+        tc_fence_before();                                  // (this thread's reads of S(u-1) are complete)
+        mbar_arrive(bar_k0 + 8u * (uint32_t)((u + 1) & 1));
+      }
+      ok = mbar_wait(bar_s0 + 8u * (uint32_t)(u & 1), (uint32_t)((u >> 1) & 1), abort_flag);
       tc_fence_after();
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;        // the tensor-memory accesses below are warp-wide
+      // S of tile u is complete: its K stage takes K of tile u + 2
+      if (ok && u + 2 < n_tiles) load_cached(u + 2, true, false);
+      cp_async_commit();
+      const uint32_t tmem_S = tmem_base + (uint32_t)(u & 1) * 128u;
+      const int key_lo = u == 0 ? loc_lo : 0;
+      const int key_hi = u == 0 ? loc_hi : min(kKeys, a.S - (u - 1) * kKeys);
+      const bool all_vis = key_lo <= col0 && key_hi >= col0 + KPT;   // every key of this thread's columns is visible
+      // this thread's scores of the tile, a pass at a time: one round trip to tensor memory per pass
+      uint32_t sv[HK];
+      auto load_scores = [&](int pass) {
+#pragma unroll
+        for (int ch = 0; ch < NCP; ++ch) tmem_ld16_issue(tmem_S + lane_addr + col0 + pass * HK + ch * 16, &sv[ch * 16]);
+        tmem_ld_wait();
+#pragma unroll
+        for (int ch = 0; ch < NCP; ++ch) keep16(&sv[ch * 16]);
+      };
+      float m_loc = -INFINITY;
+      if (ok) {
+#pragma unroll
+        for (int pass = 0; pass < NP; ++pass) {
+          load_scores(pass);
+          if (all_vis) {                                    // (scale > 0: the maximum of the products is the product of the maximum)
+            float m = __uint_as_float(sv[0]);
+#pragma unroll
+            for (int j = 1; j < HK; ++j) m = fmaxf(m, __uint_as_float(sv[j]));
+            m_loc = fmaxf(m_loc, __fmul_rn(m, scale_log2));
+          } else {
+#pragma unroll
+            for (int j = 0; j < HK; ++j) {
+              const int key = col0 + pass * HK + j;
+              if (key >= key_lo && key < key_hi) m_loc = fmaxf(m_loc, __fmul_rn(__uint_as_float(sv[j]), scale_log2));
+            }
+          }
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < HK; ++j) sv[j] = 0u;
+      }
+      float* sMaxU = sMax + (u & 1) * 8 * 128;
+      sMaxU[(hw * 4 + cw) * 128 + row] = m_loc;
+      ok = softmax_barrier_and(ok);                         // the one meeting of a tile; also one decision for all
+      if (!ok) { broke = true; break; }
+      if (u > 0) {                                          // (every chunk sum of the previous tile is visible now)
+        l_row = l_row * corr_prev + tile_sum(u - 1);
+      }
+      float m_tile = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < REP; ++k) m_tile = fmaxf(m_tile, fmaxf(sMaxU[k * 128 + row], sMaxU[(4 + k) * 128 + row]));
+      const float m_new = fmaxf(m_row, m_tile);
+      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+      const float corr = ex2(m_row - m_use);                // 0 while no visible key has been met
+      if (u > 0) {
+        // O += P V of the previous tile is complete: the P tile may be rewritten, its V stage takes V of tile u + 1,
+        // and the output so far may be rescaled
+        ok = mbar_wait(bar_o, (uint32_t)((u - 1) & 1), abort_flag);
+        tc_fence_after();
+        ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+      }
+      if (ok && u + 1 < n_tiles) load_cached(u + 1, false, true);
+      cp_async_commit();
+      // the output so far was accumulated against the old maximum: rescale this thread's columns of its lane - unless
+      // no row of the warp moved its maximum (a factor of exactly 1 changes nothing)
+      if (ok && u > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+        for (int pass = 0; pass < NP; ++pass) {
+          uint32_t ov[HK];
+#pragma unroll
+          for (int ch = 0; ch < NCP; ++ch) tmem_ld16_issue(tmem_O + lane_addr + col0 + pass * HK + ch * 16, &ov[ch * 16]);
+          tmem_ld_wait();
+#pragma unroll
+          for (int ch = 0; ch < NCP; ++ch) keep16(&ov[ch * 16]);
+#pragma unroll
+          for (int ch = 0; ch < NCP; ++ch) {
+            float v[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ov[ch * 16 + j]) * corr;
+            tmem_st16(tmem_O + lane_addr + col0 + pass * HK + ch * 16, v);
+          }
+        }
+      }
+      float* sSumU = sSum + (u & 1) * 8 * 128;
+#pragma unroll
+      for (int ch = 0; ch < NCH; ++ch) {
+        if (NP > 1 && ch % NCP == 0 && ok) load_scores(ch / NCP);     // (one pass: the scores are still in registers)
+        const int c0 = col0 + ch * 16;
+        uint32_t packed[8];
+        float csum = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; j += 2) {
+          const int key = c0 + j;
+          const float s0 = __uint_as_float(sv[(ch % NCP) * 16 + j]), s1 = __uint_as_float(sv[(ch % NCP) * 16 + j + 1]);
+          // (the same arithmetic whether or not the visibility test is needed)
+          float p0 = ex2(__fmaf_rn(s0, scale_log2, -m_use)), p1 = ex2(__fmaf_rn(s1, scale_log2, -m_use));
+          if (!all_vis) {
+            p0 = (key >= key_lo && key < key_hi) ? p0 : 0.f;
+            p1 = (key + 1 >= key_lo && key + 1 < key_hi) ? p1 : 0.f;
+          }
+          csum += p0;
+          csum += p1;
+          packed[j >> 1] = pack_bf16(p0, p1);
+        }
+        sSumU[(c0 >> 4) * 128 + row] = csum;              // chunk index = c0 / 16
+        // P, in every copy of the row
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const uint4 val = row_live ? make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3])
+                                     : make_uint4(0, 0, 0, 0);
+#pragma unroll
+          for (int k = 0; k < REP; ++k)
+            *reinterpret_cast<uint4*>(sP + tile_off(k * QT + row, (c0 >> 3) + q)) = val;
+        }
+      }
+      // ---- this thread's part of P is written, its part of V(u) has landed, its rescale of O is complete: the MMA
+      //      warp issues O += P V once every softmax thread has said so
+      cp_async_wait<2>();                                   // V of this tile (two younger groups may still be in flight)
+      asm volatile("fence.proxy.async;" ::: "memory");      // P and V are read by the tensor core
+      tc_fence_before();
+      mbar_arrive(bar_p);
+      corr_prev = corr;
+      m_row = m_new;
     }
-    if (ok && u + 2 < n_tiles) load_cached(u + 2, true, false);
-    if (ok && u + 1 < n_tiles) load_cached(u + 1, false, true);
-    cp_async_commit();
-    // the output so far was accumulated against the old maximum: rescale this thread's columns of its lane - unless
-    // no row of the warp moved its maximum (a factor of exactly 1 changes nothing)
-    if (ok && u > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
-      uint32_t ov[KPT];
-#pragma unroll
-      for (int ch = 0; ch < NCH; ++ch) tmem_ld16_issue(tmem_O + lane_addr + col0 + ch * 16, &ov[ch * 16]);
-      tmem_ld_wait();
-#pragma unroll
-      for (int ch = 0; ch < NCH; ++ch) keep16(&ov[ch * 16]);
+    cp_async_wait<0>();                                     // nothing of this thread's copies is left in flight
+    if (!broke) ok = softmax_barrier_and(ok);               // the last tile's chunk sums are visible
+    if (ok) {
+      l_row = l_row * corr_prev + tile_sum(n_tiles - 1);
+      ok = mbar_wait(bar_o, (uint32_t)((n_tiles - 1) & 1), abort_flag);
+      tc_fence_after();
+    }
+    ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+    if (ok) {
+      // every copy of a row holds the same O row: a thread normalises and stores the columns it owns, [col0, +KPT)
+      const float inv = 1.f / l_row;
+      bf16* dst = a.out + ((grow0 + row) * a.H + h) * kHD + col0;
 #pragma unroll
       for (int ch = 0; ch < NCH; ++ch) {
         float v[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(ov[ch * 16 + j]) * corr;
-        tmem_st16(tmem_O + lane_addr + col0 + ch * 16, v);
+        tmem_ld16(tmem_O + lane_addr + col0 + ch * 16, v);
+        if (!row_live) continue;
+        uint4 lo = make_uint4(pack_bf16(v[0] * inv, v[1] * inv), pack_bf16(v[2] * inv, v[3] * inv),
+                              pack_bf16(v[4] * inv, v[5] * inv), pack_bf16(v[6] * inv, v[7] * inv));
+        uint4 hi = make_uint4(pack_bf16(v[8] * inv, v[9] * inv), pack_bf16(v[10] * inv, v[11] * inv),
+                              pack_bf16(v[12] * inv, v[13] * inv), pack_bf16(v[14] * inv, v[15] * inv));
+        *reinterpret_cast<uint4*>(dst + ch * 16) = lo;
+        *reinterpret_cast<uint4*>(dst + ch * 16 + 8) = hi;
       }
-    }
-#pragma unroll
-    for (int ch = 0; ch < NCH; ++ch) {
-      const int c0 = col0 + ch * 16;
-      uint32_t packed[8];
-      float csum = 0.f;
-#pragma unroll
-      for (int j = 0; j < 16; j += 2) {
-        const int key = c0 + j;
-        const float s0 = __uint_as_float(sv[ch * 16 + j]), s1 = __uint_as_float(sv[ch * 16 + j + 1]);
-        const float p0 = (key >= key_lo && key < key_hi) ? exp2f(s0 * scale_log2 - m_use) : 0.f;
-        const float p1 = (key + 1 >= key_lo && key + 1 < key_hi) ? exp2f(s1 * scale_log2 - m_use) : 0.f;
-        csum += p0;
-        csum += p1;
-        packed[j >> 1] = pack_bf16(p0, p1);
-      }
-      sSum[(c0 >> 4) * 128 + row] = csum;               // chunk index = c0 / 16
-      // P overwrites K, in every copy of the row
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        const uint4 val = row_live ? make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3])
-                                   : make_uint4(0, 0, 0, 0);
-#pragma unroll
-        for (int k = 0; k < REP; ++k)
-          *reinterpret_cast<uint4*>(sK + tile_off(k * QT + row, (c0 >> 3) + q)) = val;
-      }
-    }
-    if (u + 1 >= n_tiles) cp_async_wait<0>();             // the last tile's V (no later S waited for it)
-    asm volatile("fence.proxy.async;" ::: "memory");      // P is read by the tensor core
-    tc_fence_before();
-    ok = __syncthreads_and(ok ? 1 : 0) != 0;
-    if (!ok) break;
-    if (tid == 0) {
-      tc_fence_after();
-      // ---- O (+)= P . V: eight k16 steps over the keys.  P is K-major (keys contiguous); V is used as
-      //      stored, [key][hd] = MN-major: 8-key groups 1024 B apart, the two 64-column halves 16 KB apart.
-      const uint32_t idesc_pv = idesc | (1u << 16);
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const uint32_t pa = smem_u32(sK) + (uint32_t)((k >> 2) * kHalfBytes + (k & 3) * 32);
-        const uint32_t va = smem_u32(sV) + (uint32_t)(2 * k * 1024);
-        tc_mma_bf16(tmem_O, make_desc(pa, 16, 1024), make_desc(va, kHalfBytes, 1024), idesc_pv, (uint32_t)((u | k) != 0));
-      }
-      tc_commit(smem_u32(&bars[2]));
-    }
-    const float l_tile = (((sSum[0 * 128 + row] + sSum[1 * 128 + row]) + (sSum[2 * 128 + row] + sSum[3 * 128 + row])) +
-                          (sSum[4 * 128 + row] + sSum[5 * 128 + row])) + (sSum[6 * 128 + row] + sSum[7 * 128 + row]);
-    l_row = l_row * corr + l_tile;
-    m_row = m_new;
-  }
-  cp_async_wait<0>();                                     // nothing of this CTA's copies is left in flight
-  if (ok) {
-    ok = mbar_wait(smem_u32(&bars[2]), (uint32_t)((n_tiles - 1) & 1));
-    tc_fence_after();
-  }
-  ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
-  if (ok) {
-    // every copy of a row holds the same O row: a thread normalises and stores the columns it owns, [col0, +KPT)
-    const float inv = 1.f / l_row;
-    bf16* dst = a.out + ((grow0 + row) * a.H + h) * kHD + col0;
-#pragma unroll
-    for (int ch = 0; ch < NCH; ++ch) {
-      float v[16];
-      tmem_ld16(tmem_O + lane_addr + col0 + ch * 16, v);
-      if (!row_live) continue;
-      uint4 lo = make_uint4(pack_bf16(v[0] * inv, v[1] * inv), pack_bf16(v[2] * inv, v[3] * inv),
-                            pack_bf16(v[4] * inv, v[5] * inv), pack_bf16(v[6] * inv, v[7] * inv));
-      uint4 hi = make_uint4(pack_bf16(v[8] * inv, v[9] * inv), pack_bf16(v[10] * inv, v[11] * inv),
-                            pack_bf16(v[12] * inv, v[13] * inv), pack_bf16(v[14] * inv, v[15] * inv));
-      *reinterpret_cast<uint4*>(dst + ch * 16) = lo;
-      *reinterpret_cast<uint4*>(dst + ch * 16 + 8) = hi;
+    } else if ((tid & 31) == 0) {
+      atomicExch(a.err_flag, 6);
     }
   }
-  if (!ok && tid == 0) atomicExch(a.err_flag, 6);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {
@@ -517,7 +634,7 @@ int launch_attention_verify_pipe(cudaStream_t st, const AttnArgs& a) {
   const int qt_rows = rps <= 32 ? 32 : (rps <= 64 ? 64 : 128);
   const int q_tiles = (rps + qt_rows - 1) / qt_rows;
   const float scale_log2 = (1.0f / sqrtf((float)a.hd)) * 1.4426950408889634f;
-  const size_t smem = (size_t)kTileBytes * (1 + kStagesK + kStagesV) + 8192 + 64 + 1024;   // Q, K and V stages, softmax exchange
+  const size_t smem = (size_t)kTileBytes * (2 + kStagesK + kStagesV) + 16384 + 64 + 1024;   // Q, P, K and V stages, softmax exchange
   static bool attr_set[kMaxDevices] = {};        // the shared-memory opt-in is per device
   const int dev = device_slot();
   if (dev < 0) return -4;
@@ -529,7 +646,7 @@ int launch_attention_verify_pipe(cudaStream_t st, const AttnArgs& a) {
     attr_set[dev] = true;
   }
   dim3 grid(a.H, a.n_seq_slots * q_tiles);
-  dim3 block(kPipeThreads);
+  dim3 block(kPipeBlock);
   cudaError_t e;
   if (qt_rows == 32) e = launch_pdl(attn_verify_pipe_kernel<32>, grid, block, smem, st, a, scale_log2);
   else if (qt_rows == 64) e = launch_pdl(attn_verify_pipe_kernel<64>, grid, block, smem, st, a, scale_log2);
