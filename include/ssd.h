@@ -309,6 +309,9 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "attn_impl"  1 = attention of the verification forward on tcgen05 where the shape allows (head
  *        dimension 128, parts of whole 128-key tiles, block length dividing 128), the default; 0 = always the
  *        mma.sync form;
+ *   "attn_pipe_keys" with attn_impl 1: prefixes of at least this many cached keys take the pipelined tcgen05
+ *        form (one CTA per head walks all key tiles) instead of the cluster of key parts; a function of the
+ *        prefix length alone.  Default 2048; 0 = never;
  *   "two_sm_rows" the QKV, gate/up and LM-head projections run pairs of weight tiles as ONE tcgen05.mma
  *        with cta_group::2 (two CTAs of a cluster, M = 256, each SM holding half of the activation tile)
  *        from this many padded rows per launch on; 0 = never; default 128, where it starts to pay.  The results
