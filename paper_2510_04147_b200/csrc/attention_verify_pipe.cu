@@ -21,6 +21,7 @@
 #include "attn_common.cuh"
 
 #include <cuda.h>
+#include <string.h>
 
 namespace ssd {
 
@@ -31,7 +32,7 @@ using namespace attn;
 constexpr int kHD = 128;
 constexpr int kKeys = 128;                  // keys per tile
 constexpr int kPipeThreads = 256;           // softmax threads: two per TMEM lane
-constexpr int kPipeBlock = kPipeThreads + 32;   // + one warp that issues the MMAs
+constexpr int kPipeBlock = kPipeThreads + 64;   // + one warp that issues the MMAs + one that asks for the bulk tile copies
 constexpr int kHalfBytes = kKeys * 128;     // one 64-column half of a 128-row tile
 constexpr int kTileBytes = 2 * kHalfBytes;  // a [128][128] bf16 tile
 constexpr int kStagesK = 2, kStagesV = 2;      // + one P tile
@@ -66,6 +67,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       else if (now - t0 > kPipeWaitLimitNs) { *abort = 1; return false; }
     }
   }
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// one box of a 2-D tensor map into shared memory; its bytes count on the mbarrier
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -157,7 +167,9 @@ __device__ __forceinline__ uint32_t tile_off(int row, int ch) {
 }
 
 template <int QT>
-__global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArgs a, float scale_log2) {
+__global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                                               const __grid_constant__ CUtensorMap tmV, AttnArgs a,
+                                                                               float scale_log2, int use_tma) {
   extern __shared__ uint8_t smem_dyn[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;                                   // [2][128][64] bf16
@@ -168,7 +180,8 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
   float* sSum = sMax + 2 * 8 * 128;                                         // 2 x [8 chunks of 16 keys][128 rows]
   // [0], [1] S ready (two accumulators), [2] O += P V complete, [3], [4] K stage landed, [5] P written and V landed
   uint64_t* bars = reinterpret_cast<uint64_t*>(sSum + 2 * 8 * 128);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 6);
+  // ... [6], [7] V stage landed (bulk copies only)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   constexpr int CH = kHD / 8;                            // 16-byte chunks per row
 
@@ -193,9 +206,11 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
     mbar_init(smem_u32(&bars[2]), 1);
-    mbar_init(smem_u32(&bars[3]), kPipeThreads);
-    mbar_init(smem_u32(&bars[4]), kPipeThreads);
+    mbar_init(smem_u32(&bars[3]), kPipeThreads + 1);        // every softmax thread (it has read S of the tile whose accumulator
+    mbar_init(smem_u32(&bars[4]), kPipeThreads + 1);        // is reused; its own copies have landed) + the copy thread
     mbar_init(smem_u32(&bars[5]), kPipeThreads);
+    mbar_init(smem_u32(&bars[6]), 1);
+    mbar_init(smem_u32(&bars[7]), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -203,11 +218,15 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  __syncthreads();                          // the barriers exist before the copy thread uses them
 
   // ---- copies into a stage: cached K/V (zero rows past the end), or the node-local rows of the projection
   // A thread copies the same 16-byte column chunk of the rows ld_row0, ld_row0 + 16, ...: the swizzle term of its
   // shared-memory address and its byte offset inside a cache row are constants, so a copy costs a few instructions.
-  const bool softmax_thread = tid < kPipeThreads;        // warps 0-7; warp 8 issues the MMAs
+  const bool softmax_thread = tid < kPipeThreads;        // warps 0-7; warp 8 issues the MMAs, warp 9 asks for the bulk copies
+  // Whole tiles of cached keys are copied by the tensor-map engine (one thread asks, the bytes count on an mbarrier);
+  // a last, partial tile is copied by the softmax threads, which fill the rows past the end with zeros.
+  auto bulk = [&](int u) { return use_tma != 0 && u >= 1 && u * kKeys <= a.S; };
   const int ld_ch = tid % CH, ld_row0 = tid / CH;
   const uint32_t ld_soff = tile_off(ld_row0, ld_ch);      // + 16 * 128 bytes per step (16 rows: the same swizzle phase)
   auto load_cached = [&](int u, bool want_k, bool want_v) {
@@ -247,9 +266,24 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
   // The cache is not written below the rows' own positions by any kernel of this forward, so its first tile may be
   // requested before the dependency wait - unless the slot -> sequence map is only known on the device.
   const bool early = a.map.n_inline > 0 || a.map.seq_map == nullptr;
-  if (softmax_thread && early && n_tiles > 1) load_cached(1, true, false);
+  if (softmax_thread && early && n_tiles > 1 && !bulk(1)) load_cached(1, true, false);
+  auto ask_tile1 = [&]() {                 // copy warp, lanes 0 (K) and 1 (V): both stages 1 are free from the start
+    const int lane = tid & 31;
+    if (warp != kPipeThreads / 32 + 1 || lane >= 2 || n_tiles < 2) return;
+    const uint32_t kb_ = smem_u32(&bars[3]) + 8u, vb_ = smem_u32(&bars[6]) + 8u;
+    if (!bulk(1)) { if (lane == 0) mbar_arrive(kb_); return; }
+    const int seq = seq_of_slot(a.map, slot);
+    const int r0 = (int)(((size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride) / kHD);
+    const uint32_t dst = smem_u32((lane == 0 ? sKs : sVs) + kTileBytes);
+    const uint32_t bar = lane == 0 ? kb_ : vb_;
+    mbar_arrive_expect_tx(bar, (uint32_t)kTileBytes);
+    tma_load_2d(dst, lane == 0 ? &tmK : &tmV, bar, 0, r0);
+    tma_load_2d(dst + kHalfBytes, lane == 0 ? &tmK : &tmV, bar, 64, r0);
+  };
+  if (early) ask_tile1();
   pdl_wait();                              // the QKV projection's partials are complete from here on
-  if (softmax_thread && !early && n_tiles > 1) load_cached(1, true, false);
+  if (!early) ask_tile1();
+  if (softmax_thread && !early && n_tiles > 1 && !bulk(1)) load_cached(1, true, false);
   cp_async_commit();
 
   // ---- prologue: the query tile and the node-local K/V from the fp32 split-K partials of the fused q|k|v
@@ -376,9 +410,10 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_O = tmem_base + 256;
   const uint32_t bar_s0 = smem_u32(&bars[0]), bar_o = smem_u32(&bars[2]), bar_k0 = smem_u32(&bars[3]), bar_p = smem_u32(&bars[5]);
+  const uint32_t bar_v0 = smem_u32(&bars[6]);
   bool ok = true;
 
-  if (!softmax_thread) {
+  if (warp == kPipeThreads / 32) {
     // ================================================================== MMA warp
     // Per tile u: S(u+1) = Q K(u+1)^T as soon as the softmax threads report K(u+1) landed (they do so when they
     // enter tile u, i.e. after they have read S(u-1), whose accumulator S(u+1) overwrites), then O += P(u) V(u) as
@@ -407,6 +442,7 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
           issue_s(u + 1);
         }
         ok = mbar_wait(bar_p, (uint32_t)(u & 1), abort_flag);
+        if (ok && bulk(u)) ok = mbar_wait(bar_v0 + 8u * (uint32_t)(u & 1), (uint32_t)(((u - 1) >> 1) & 1), abort_flag);
         if (!ok) break;
         tc_fence_after();
         // O (+)= P . V: eight k16 steps over the keys.  P is K-major (keys contiguous); V is used as stored,
@@ -419,6 +455,41 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
           tc_mma_bf16(tmem_O, make_desc(pa, 16, 1024), make_desc(va, kHalfBytes, 1024), idesc_pv, (uint32_t)((u | k) != 0));
         }
         tc_commit(bar_o);
+      }
+      if (!ok) atomicExch(a.err_flag, 6);
+    }
+  } else if (!softmax_thread) {
+    // ================================================================== copy warp (bulk tiles)
+    // Lane 0 asks for K of tile t once S of tile t-2 is complete (its stage is free then), lane 1 for V of tile t once
+    // O += P V of tile t-2 is.  A tile the softmax threads copy themselves only gets lane 0's arrival on its K barrier.
+    const int lane = tid & 31;
+    if (lane < 2 && n_tiles > 1) {
+      const int seq = seq_of_slot(a.map, slot);
+      const int row_base = (int)(((size_t)seq * a.cache_seq_stride + (size_t)kvh * a.kv_head_stride) / kHD);   // row of key 0 in the [rows][128] view
+#pragma unroll 1
+      for (int t = 2; t < n_tiles && ok; ++t) {          // (tile 1 was asked for before the prologue)
+        const int r0 = row_base + (t - 1) * kKeys;
+        if (lane == 0) {
+          if (t >= 2) ok = mbar_wait(bar_s0 + 8u * (uint32_t)(t & 1), (uint32_t)(((t - 2) >> 1) & 1), abort_flag);
+          if (!ok) break;
+          const uint32_t kb_ = bar_k0 + 8u * (uint32_t)(t & 1);
+          if (bulk(t)) {
+            const uint32_t dst = smem_u32(sKs + (size_t)(t % kStagesK) * kTileBytes);
+            mbar_arrive_expect_tx(kb_, (uint32_t)kTileBytes);
+            tma_load_2d(dst, &tmK, kb_, 0, r0);
+            tma_load_2d(dst + kHalfBytes, &tmK, kb_, 64, r0);
+          } else {
+            mbar_arrive(kb_);
+          }
+        } else if (bulk(t)) {
+          if (t >= 2) ok = mbar_wait(bar_o, (uint32_t)((t - 2) & 1), abort_flag);
+          if (!ok) break;
+          const uint32_t vb_ = bar_v0 + 8u * (uint32_t)(t & 1);
+          const uint32_t dst = smem_u32(sVs + (size_t)(t % kStagesV) * kTileBytes);
+          mbar_arrive_expect_tx(vb_, (uint32_t)kTileBytes);
+          tma_load_2d(dst, &tmV, vb_, 0, r0);
+          tma_load_2d(dst + kHalfBytes, &tmV, vb_, 64, r0);
+        }
       }
       if (!ok) atomicExch(a.err_flag, 6);
     }
@@ -457,8 +528,10 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
       // ---- K of the next tile (requested a whole iteration ago) has landed for this thread: tell the MMA warp.
       //      Copy groups are committed in the order K(u+1), V(u), K(u+2), V(u+1), ...
       if (u + 1 < n_tiles) {
-        cp_async_wait<1>();                                 // everything but V(u), which has until O += P V
-        asm volatile("fence.proxy.async;" ::: "memory");
+        if (!bulk(u + 1)) {                                 // (a tile this thread helped to copy)
+          cp_async_wait<1>();                               // everything but V(u), which has until O += P V
+          asm volatile("fence.proxy.async;" ::: "memory");
+        }
         tc_fence_before();                                  // (this thread's reads of S(u-1) are complete)
         mbar_arrive(bar_k0 + 8u * (uint32_t)((u + 1) & 1));
       }
@@ -466,7 +539,7 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
       tc_fence_after();
       ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;        // the tensor-memory accesses below are warp-wide
       // S of tile u is complete: its K stage takes K of tile u + 2
-      if (ok && u + 2 < n_tiles) load_cached(u + 2, true, false);
+      if (ok && u + 2 < n_tiles && !bulk(u + 2)) load_cached(u + 2, true, false);
       cp_async_commit();
       const uint32_t tmem_S = tmem_base + (uint32_t)(u & 1) * 128u;
       const int key_lo = u == 0 ? loc_lo : 0;
@@ -523,7 +596,7 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(AttnArg
         tc_fence_after();
         ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
       }
-      if (ok && u + 1 < n_tiles) load_cached(u + 1, false, true);
+      if (ok && u + 1 < n_tiles && !bulk(u + 1)) load_cached(u + 1, false, true);
       cp_async_commit();
       // the output so far was accumulated against the old maximum: rescale this thread's columns of its lane - unless
       // no row of the warp moved its maximum (a factor of exactly 1 changes nothing)
@@ -634,7 +707,7 @@ int launch_attention_verify_pipe(cudaStream_t st, const AttnArgs& a) {
   const int qt_rows = rps <= 32 ? 32 : (rps <= 64 ? 64 : 128);
   const int q_tiles = (rps + qt_rows - 1) / qt_rows;
   const float scale_log2 = (1.0f / sqrtf((float)a.hd)) * 1.4426950408889634f;
-  const size_t smem = (size_t)kTileBytes * (2 + kStagesK + kStagesV) + 16384 + 64 + 1024;   // Q, P, K and V stages, softmax exchange
+  const size_t smem = (size_t)kTileBytes * (2 + kStagesK + kStagesV) + 16384 + 128 + 1024;   // Q, P, K and V stages, softmax exchange
   static bool attr_set[kMaxDevices] = {};        // the shared-memory opt-in is per device
   const int dev = device_slot();
   if (dev < 0) return -4;
@@ -645,12 +718,25 @@ int launch_attention_verify_pipe(cudaStream_t st, const AttnArgs& a) {
       return -4;
     attr_set[dev] = true;
   }
+  // Whole tiles of cached keys go through the tensor-map engine when a head's keys are contiguous rows of the cache
+  // viewed as [rows][128] (head-major layout, no hole in the key range); otherwise every tile is copied by the threads.
+  alignas(64) CUtensorMap tmK, tmV;
+  memset(&tmK, 0, sizeof(tmK));
+  memset(&tmV, 0, sizeof(tmV));
+  int use_tma = 0;
+  if (a.cache_rows > 0 && a.kv_pos_stride == (size_t)kHD && a.hole_len == 0 && (a.cache_seq_stride % kHD) == 0 &&
+      (a.kv_head_stride % kHD) == 0 && a.cache_rows < (size_t)0x7fffffff) {
+    if (encode_tmap_bf16_2d(&tmK, a.cache_k, a.cache_rows, kHD, kHD, kKeys) != 0 ||
+        encode_tmap_bf16_2d(&tmV, a.cache_v, a.cache_rows, kHD, kHD, kKeys) != 0)
+      return -4;
+    use_tma = 1;
+  }
   dim3 grid(a.H, a.n_seq_slots * q_tiles);
   dim3 block(kPipeBlock);
   cudaError_t e;
-  if (qt_rows == 32) e = launch_pdl(attn_verify_pipe_kernel<32>, grid, block, smem, st, a, scale_log2);
-  else if (qt_rows == 64) e = launch_pdl(attn_verify_pipe_kernel<64>, grid, block, smem, st, a, scale_log2);
-  else e = launch_pdl(attn_verify_pipe_kernel<128>, grid, block, smem, st, a, scale_log2);
+  if (qt_rows == 32) e = launch_pdl(attn_verify_pipe_kernel<32>, grid, block, smem, st, tmK, tmV, a, scale_log2, use_tma);
+  else if (qt_rows == 64) e = launch_pdl(attn_verify_pipe_kernel<64>, grid, block, smem, st, tmK, tmV, a, scale_log2, use_tma);
+  else e = launch_pdl(attn_verify_pipe_kernel<128>, grid, block, smem, st, tmK, tmV, a, scale_log2, use_tma);
   return e == cudaSuccess ? 0 : -4;
 }
 

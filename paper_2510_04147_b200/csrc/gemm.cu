@@ -709,6 +709,13 @@ bool make_tmap(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, ui
 
 }  // namespace
 
+// (for other kernels of the library that copy bf16 tiles with the tensor-map engine: boxes of 64 columns x box_rows rows,
+// 128-byte swizzle)
+int encode_tmap_bf16_2d(void* map_out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems, uint32_t box_rows) {
+  if (!g_encode && gemm_tc_init() != 0) return -4;
+  return make_tmap(reinterpret_cast<CUtensorMap*>(map_out), base, rows, cols, pitch_elems, box_rows) ? 0 : -4;
+}
+
 int gemm_tc_init() {
   if (g_encode) return 0;
   void* fn = nullptr;

@@ -154,6 +154,7 @@ struct AttnArgs {
   int hole_begin, hole_len;
   int kv_split;         // prefix keys per split (a function of S only)
   size_t cache_seq_stride;
+  size_t cache_rows;                      // rows of hd elements in one layer's K (or V) cache: max_batch * Hkv * max_seq; 0: unknown
   size_t kv_pos_stride, kv_head_stride;   // element (sequence, position, kv head) of the cache lies at
                                           // seq * cache_seq_stride + head * kv_head_stride + pos * kv_pos_stride
   RowMap map;
@@ -221,6 +222,9 @@ int gemm_tiles(int N);
 // tensor-core path (TMA + tcgen05). Returns 0 or a negative ssd error code.
 int launch_gemm_tc(cudaStream_t st, const GemmArgs& g);
 int gemm_tc_init();   // resolves the driver entry point for tensor-map encoding
+// Tensor map (a CUtensorMap, 128 bytes, 64-byte aligned) over a row-major bf16 matrix [rows][cols] with `pitch_elems`
+// elements between rows: boxes of 64 columns x box_rows rows, 128-byte swizzle.  Returns 0 or a negative ssd error code.
+int encode_tmap_bf16_2d(void* map_out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems, uint32_t box_rows);
 
 // ---------------------------------------------------------------- tree build / acceptance
 struct BlockState {       // device arrays, [max_batch][stride] unless noted; a row holds [current block | next block]

@@ -380,6 +380,7 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
     a.out = c->att;
     a.R = R; a.H = H; a.Hkv = Hkv; a.hd = hd; a.S = attn_S; a.kv_split = kv_split;
     a.hole_begin = hole_len > 0 ? S : 0; a.hole_len = hole_len;
+    a.cache_rows = c->cache_layer_stride / (size_t)hd;
     a.cache_seq_stride = c->cache_seq_stride; a.kv_pos_stride = c->kv_pos_stride; a.kv_head_stride = c->kv_head_stride;
     a.map = map; a.n_seq_slots = n_slots;
     const double kvb = (double)n_slots * attn_S * Hkv * hd * 4.0 + (double)R * (H + 2 * Hkv) * hd * 2.0 + (double)R * H * hd * 2.0;
