@@ -63,6 +63,7 @@ def _make(w, max_drafts, max_batch=None, max_seq=None, attn_form="by_prefix_leng
     ssd = b.Ssd(b.config_from_workload(w, max_drafts=max_drafts, max_batch=max_batch, max_seq=max_seq))
     if attn_form == "pipelined":
         ssd.set_option("attn_pipe_keys", 1)
+        ssd.set_option("attn_pipe_ctas", 1)
     ssd.load_workload_weights(w)
     return ssd
 
@@ -111,8 +112,9 @@ def test_full_width_forward_matches_oracle(case):
     gpu = {}
     ssd = _make(w, max_drafts=n_nodes)
     try:
+        ssd.set_option("attn_pipe_ctas", 1)
         for form in ATTN_FORMS:                              # the cluster-of-parts attention and the pipelined one
-            ssd.set_option("attn_pipe_keys", 1 if form == "pipelined" else 2048)
+            ssd.set_option("attn_pipe_keys", 1 if form == "pipelined" else 1 << 30)
             ssd.prefill(prompt)
             ssd.block_begin(T)
             ssd.set_block_state(blk, np.zeros((1, T), np.uint8))
@@ -383,6 +385,7 @@ def test_both_attention_forms_agree_at_full_width():
     out = {}
     ssd = _make(w, max_drafts=n_nodes)
     try:
+        ssd.set_option("attn_pipe_ctas", 1)
         for impl, pipe_keys in ((0, 0), (1, 0), (2, 1)):
             ssd.set_option("attn_impl", min(impl, 1))
             ssd.set_option("attn_pipe_keys", pipe_keys)
