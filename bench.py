@@ -195,6 +195,8 @@ def pick_workload(args):
         over["gen_len"] = args.gen_len
     if args.prompt_len:
         over["prompt_len"] = args.prompt_len
+    if args.batch:
+        over["batch"] = args.batch
     return (w.replace(**over), True) if over else (w, False)
 
 
@@ -354,7 +356,8 @@ def run_ours(args):
     ssd = binding.Ssd(binding.config_from_workload(w, max_drafts=min(cfg_drafts, B - 1)))
     for k, v in (("split_k_qkv", args.split_qkv), ("split_k_o", args.split_o), ("split_k_down", args.split_down),
                  ("kv_split", args.kv_split), ("attn_impl", args.attn_impl), ("two_sm_rows", args.two_sm_rows),
-                 ("gemm_max_stages", args.gemm_max_stages), ("attn_pipe_keys", args.attn_pipe_keys)):
+                 ("gemm_max_stages", args.gemm_max_stages), ("attn_pipe_keys", args.attn_pipe_keys),
+                 ("attn_pipe_ctas", args.attn_pipe_ctas)):
         if v is not None:
             ssd.set_option(k, v)
     t0 = time.time()
@@ -693,10 +696,13 @@ def main():
     ap.add_argument("--gemm-max-stages", type=int, default=None, help="tuning: cap on the projection kernel's ring depth")
     ap.add_argument("--attn-pipe-keys", type=int, default=None,
                     help="tuning: prefixes of at least this many keys take the pipelined attention form (0: never)")
+    ap.add_argument("--attn-pipe-ctas", type=int, default=None,
+                    help="tuning: ... when the batch gives it at least this many (head, sequence) CTAs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="profiling only: fewer layers of the same shape")
     ap.add_argument("--gen-len", type=int, default=0, help="profiling only: shorter generation")
     ap.add_argument("--prompt-len", type=int, default=0, help="profiling only: another prompt length")
+    ap.add_argument("--batch", type=int, default=0, help="profiling only: another batch size")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -309,12 +309,12 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *   "attn_impl"  1 = attention of the verification forward on tcgen05 where the shape allows (head
  *        dimension 128, parts of whole 128-key tiles, block length dividing 128), the default; 0 = always the
  *        mma.sync form;
- *   "attn_pipe_keys" with attn_impl 1: prefixes of at least this many cached keys take the pipelined tcgen05
- *        form (one CTA per head and sequence walks all key tiles) instead of the cluster of key parts, provided the
- *        prefilled batch gives it at least "attn_pipe_ctas" (default 96) such CTAs: batch * heads.  A single long
- *        sequence is faster with its key parts side by side.  Default 2048; 0 = never.  The two forms sum in
- *        different orders, so for prefixes this long a sequence's bits depend on the prefilled batch SIZE (never on
- *        the other sequences' contents, on the node count, or on which sequences are still unfinished);
+ *   "attn_pipe_ctas", "attn_pipe_keys" with attn_impl 1: a prefilled batch that gives at least attn_pipe_ctas
+ *        (default 96) pairs (head, sequence) - batch * heads - takes the pipelined tcgen05 form, one CTA per pair
+ *        walking all key tiles, instead of the cluster of key parts; one or two sequences are faster with their
+ *        key parts side by side.  attn_pipe_keys (default 1; 0 = never) is the shortest prefix that may take it.
+ *        The two forms sum in different orders, so a sequence's bits depend on the prefilled batch SIZE - never
+ *        on the other sequences' contents, on the node count, or on which sequences are still unfinished;
  *   "two_sm_rows" the QKV, gate/up and LM-head projections run pairs of weight tiles as ONE tcgen05.mma
  *        with cta_group::2 (two CTAs of a cluster, M = 256, each SM holding half of the activation tile)
  *        from this many padded rows per launch on; 0 = never; default 128, where it starts to pay.  The results

@@ -56,19 +56,17 @@ def _binding():
     return binding
 
 
-def _make(w, max_drafts, max_batch=None, max_seq=None, attn_form="by_prefix_length"):
-    """attn_form "pipelined": the attention form of long prefixes (one CTA per head walks all key tiles) is taken
-    whatever the prefix length, so that the small cases here cover it; otherwise the prefix length decides."""
+def _make(w, max_drafts, max_batch=None, max_seq=None, attn_form="cluster_of_parts"):
+    """attn_form "pipelined": the attention form of larger batches (one CTA per head and sequence walks all key tiles)
+    is taken whatever the batch size, so that the small cases here cover it; otherwise the cluster-of-parts form."""
     b = _binding()
     ssd = b.Ssd(b.config_from_workload(w, max_drafts=max_drafts, max_batch=max_batch, max_seq=max_seq))
-    if attn_form == "pipelined":
-        ssd.set_option("attn_pipe_keys", 1)
-        ssd.set_option("attn_pipe_ctas", 1)
+    ssd.set_option("attn_pipe_ctas", 1 if attn_form == "pipelined" else 1 << 20)
     ssd.load_workload_weights(w)
     return ssd
 
 
-ATTN_FORMS = ["by_prefix_length", "pipelined"]
+ATTN_FORMS = ["cluster_of_parts", "pipelined"]
 _ORACLE_RESULTS = {}
 
 
@@ -112,9 +110,8 @@ def test_full_width_forward_matches_oracle(case):
     gpu = {}
     ssd = _make(w, max_drafts=n_nodes)
     try:
-        ssd.set_option("attn_pipe_ctas", 1)
         for form in ATTN_FORMS:                              # the cluster-of-parts attention and the pipelined one
-            ssd.set_option("attn_pipe_keys", 1 if form == "pipelined" else 1 << 30)
+            ssd.set_option("attn_pipe_ctas", 1 if form == "pipelined" else 1 << 20)
             ssd.prefill(prompt)
             ssd.block_begin(T)
             ssd.set_block_state(blk, np.zeros((1, T), np.uint8))
@@ -278,13 +275,18 @@ def test_full_size_row_invariance(llada_full):
     assert np.all(np.isfinite(live)) and live.min() > 1.0 / w.vocab and live.max() < 1.0
 
 
-def test_batched_full_width_sequences_equal_single_runs():
-    """Config 3's launch shape (several sequences in one forward, own tree each) at full width."""
+@pytest.mark.parametrize("attn_form", ["cluster_of_parts", "pipelined"])
+def test_batched_full_width_sequences_equal_single_runs(attn_form):
+    """Config 3's launch shape (several sequences in one forward, own tree each) at full width.  The batch size
+    chooses between the two tcgen05 attention forms (three sequences x 32 heads take the pipelined one, a single
+    sequence the cluster of key parts), which sum in different orders; with the form held fixed, every sequence of a
+    batch decodes bit for bit as it does alone."""
     w = wl.LLADA_8B_BATCH.replace(name="llada_batch_width", n_layers=2, vocab=4096, prompt_len=96, gen_len=32, batch=3)
     b = _binding()
     prompts = wl.make_prompts(w).numpy()
     ssd = _make(w, max_drafts=3, max_batch=3)
     try:
+        ssd.set_option("attn_pipe_ctas", 1 if attn_form == "pipelined" else 1 << 20)
         ssd.prefill(prompts)
         tok_b, acc_b, nf_b = ssd.decode_block(b.MODE_SSD, w.block_len, 3)
         singles = []
@@ -385,10 +387,9 @@ def test_both_attention_forms_agree_at_full_width():
     out = {}
     ssd = _make(w, max_drafts=n_nodes)
     try:
-        ssd.set_option("attn_pipe_ctas", 1)
-        for impl, pipe_keys in ((0, 0), (1, 0), (2, 1)):
+        for impl, pipe_ctas in ((0, 1 << 20), (1, 1 << 20), (2, 1)):
             ssd.set_option("attn_impl", min(impl, 1))
-            ssd.set_option("attn_pipe_keys", pipe_keys)
+            ssd.set_option("attn_pipe_ctas", pipe_ctas)
             ssd.prefill(prompt)
             tok, conf, logits = ssd.verify_forward(ids, masked, want_logits=True)
             out[impl] = (tok, conf, logits)
