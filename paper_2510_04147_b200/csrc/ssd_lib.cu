@@ -411,7 +411,9 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
       // (a batch of three or more sequences at 32 heads); one or two sequences are faster with their key parts side by side.  A function of the prefix
       // length and of the PREFILLED batch size (not of the rows or of the sequences still unfinished), so stepwise and
       // SSD forwards of one generation always take the same form.
-      if (c->attn_impl == 1 && c->attn_pipe_keys > 0 && attn_S >= c->attn_pipe_keys && c->batch * H >= c->attn_pipe_ctas)
+      // (Two thirds of that many CTAs are enough while the prefix is short: two sequences below 1024 cached keys.)
+      const int pipe_ctas = attn_S < 1024 ? (2 * c->attn_pipe_ctas + 2) / 3 : c->attn_pipe_ctas;
+      if (c->attn_impl == 1 && c->attn_pipe_keys > 0 && attn_S >= c->attn_pipe_keys && c->batch * H >= pipe_ctas)
         arc = launch_attention_verify_pipe(c->st, a);
       if (arc == 1 && c->attn_impl == 1) arc = launch_attention_verify_tc(c->st, a);   // 1: shape not covered by the tcgen05 form
       if (arc == 1) arc = launch_attention_verify(c->st, a);
