@@ -1,6 +1,7 @@
 // Shared-prefix bidirectional attention of the verification forward (Eq. 5) on the tcgen05 tensor cores for
-// LONG prefixes: one CTA per (query tile, head, sequence) walks all key tiles of the head in one software
-// pipeline.  (Short prefixes take the cluster form, which runs the key parts side by side.)
+// BATCHES: one CTA per (query tile, head, sequence) walks all key tiles of the head in one software pipeline.  It
+// wins once there are about as many such CTAs as SMs; one sequence takes the cluster form, which runs the key parts
+// of a head side by side.
 //
 // A query tile is up to 128 rows of one sequence (nodes side by side); its keys are the node-local keys (tile
 // 0, visibility per row: the row's own node, block-causal inside a chain of two blocks) followed by the cached

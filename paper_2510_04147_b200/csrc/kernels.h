@@ -169,7 +169,7 @@ int launch_attention_verify(cudaStream_t st, const AttnArgs& a);
 // node-local keys that fit one 128-key tile; needs a.err_flag.  Returns 0 (launched), 1 (shape not
 // covered: use launch_attention_verify) or a negative ssd error code.
 int launch_attention_verify_tc(cudaStream_t st, const AttnArgs& a);
-// The same for long prefixes: one CTA per (query tile, head, sequence) with all key tiles in one software pipeline
+// The same for batches of sequences: one CTA per (query tile, head, sequence) with all key tiles in one software pipeline
 // (no cluster, no merge).  Head dimension 128, node width dividing 128, any prefix length; needs a.err_flag.
 // Same return codes.
 int launch_attention_verify_pipe(cudaStream_t st, const AttnArgs& a);
