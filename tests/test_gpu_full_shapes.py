@@ -88,6 +88,9 @@ WIDTH_CASES = {
     # name: (workload at full width / 2 layers / small vocabulary, nodes in the checked forward)
     "llada_width": (wl.LLADA_8B.replace(name="llada_width", n_layers=2, vocab=4096, prompt_len=160, gen_len=64), 3),
     "dream_width": (wl.DREAM_7B.replace(name="dream_width", n_layers=2, vocab=4096, prompt_len=200, gen_len=64), 2),
+    # prefix of whole 128-key tiles only (224 + one committed block = 256 keys): no partial tile at the end
+    "llada_width_whole_tiles": (wl.LLADA_8B.replace(name="llada_width_whole_tiles", n_layers=1, vocab=2048, prompt_len=224,
+                                                    gen_len=64), 2),
     # long prefix, 64-token blocks: several 128-key steps per attention part, double-buffered K/V
     "long_width": (wl.LLADA_8B_LONG.replace(name="long_width", n_layers=1, vocab=2048, prompt_len=1100, gen_len=128,
                                             batch=1), 2),
