@@ -404,7 +404,7 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(const _
     }
   }
   cp_async_wait<0>();
-  asm volatile("fence.proxy.async;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -531,7 +531,7 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(const _
       if (u + 1 < n_tiles) {
         if (!bulk(u + 1)) {                                 // (a tile this thread helped to copy)
           cp_async_wait<1>();                               // everything but V(u), which has until O += P V
-          asm volatile("fence.proxy.async;" ::: "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         tc_fence_before();                                  // (this thread's reads of S(u-1) are complete)
         mbar_arrive(bar_k0 + 8u * (uint32_t)((u + 1) & 1));
@@ -654,7 +654,7 @@ __global__ void __launch_bounds__(kPipeBlock, 1) attn_verify_pipe_kernel(const _
       // ---- this thread's part of P is written, its part of V(u) has landed, its rescale of O is complete: the MMA
       //      warp issues O += P V once every softmax thread has said so
       cp_async_wait<2>();                                   // V of this tile (two younger groups may still be in flight)
-      asm volatile("fence.proxy.async;" ::: "memory");      // P and V are read by the tensor core
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // P and V are read by the tensor core
       tc_fence_before();
       mbar_arrive(bar_p);
       corr_prev = corr;

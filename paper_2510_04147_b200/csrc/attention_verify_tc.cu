@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       finish(A, x1, x2);
     }
     if (!waited) cluster_wait();
-    asm volatile("fence.proxy.async;" ::: "memory");      // these stores are read by the tensor core
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // these stores are read by the tensor core
     cluster_sync_all();
   }
   // The MMA always works on 128 query rows (= 128 TMEM lanes, one per thread).  A tile of QT < 128
@@ -357,7 +357,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
     }
   }
   cp_async_wait<0>();
-  asm volatile("fence.proxy.async;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -400,7 +400,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       load_prefix(t, false, true);
       cp_async_commit();
       cp_async_wait<1>();
-      asm volatile("fence.proxy.async;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
@@ -481,7 +481,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       }
     }
     cp_async_wait<0>();                                   // V of a later tile
-    asm volatile("fence.proxy.async;" ::: "memory");      // P (and V) are read by the tensor core
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // P (and V) are read by the tensor core
     tc_fence_before();
     __syncthreads();
     if (tid == 0) {
