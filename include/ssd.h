@@ -310,10 +310,9 @@ int ssd_profile_read(ssd_ctx* ctx, int64_t* launches, double* milliseconds, doub
  *        dimension 128, parts of whole 128-key tiles, block length dividing 128), the default; 0 = always the
  *        mma.sync form;
  *   "attn_pipe_ctas", "attn_pipe_keys" with attn_impl 1: a prefilled batch that gives at least attn_pipe_ctas
- *        (default 96) pairs (head, sequence) - batch * heads - takes the pipelined tcgen05 form, one CTA per pair
- *        walking all key tiles, instead of the cluster of key parts; one or two sequences are faster with their
- *        key parts side by side (below 1024 cached keys two thirds of attn_pipe_ctas are enough: two sequences at
- *        32 heads).  attn_pipe_keys (default 1; 0 = never) is the shortest prefix that may take it.
+ *        (default 64) pairs (head, sequence) - batch * heads - takes the pipelined tcgen05 form, one CTA per pair
+ *        walking all key tiles, instead of the cluster of key parts; one sequence is faster with its key parts
+ *        side by side.  attn_pipe_keys (default 1; 0 = never) is the shortest prefix that may take it.
  *        The two forms sum in different orders, so a sequence's bits depend on the prefilled batch SIZE - never
  *        on the other sequences' contents, on the node count, or on which sequences are still unfinished;
  *   "two_sm_rows" the QKV, gate/up and LM-head projections run pairs of weight tiles as ONE tcgen05.mma

@@ -113,7 +113,7 @@ struct ssd_ctx {
   int64_t launches = 0;
   int gemm_max_stages = 0;       // tuning: cap on the projection kernel's ring depth (0: none)
   int attn_pipe_keys = 1;        // prefixes of at least this many keys take the pipelined attention form (0: never) ...
-  int attn_pipe_ctas = 96;       // ... when the prefilled batch gives it at least this many (head, sequence) CTAs
+  int attn_pipe_ctas = 64;       // ... when the prefilled batch gives it at least this many (head, sequence) CTAs
   int wait_limit_us = 0;         // bound of the projection kernel's barrier waits (0: the kernel's default, 2 s)
   int starve_gemm_kb = 0;        // test hook for ssd_gemm_bf16: K block (1-based) whose copies are left out
   bool profiling = false;        // mode 1: CUDA events around every launch (serialises the stream)
@@ -408,12 +408,10 @@ int forward(ssd_ctx* c, int kind, const int* ids_dev, int R, RowMap map, int n_s
       a.err_flag = c->flags;
       int arc = 1;
       // One pipelined CTA per (head, sequence) walks all key tiles - when there are enough of those to fill the machine
-      // (a batch of three or more sequences at 32 heads); one or two sequences are faster with their key parts side by side.  A function of the prefix
+      // (a batch of two or more sequences at 32 heads); one sequence is faster with its key parts side by side.  A function of the prefix
       // length and of the PREFILLED batch size (not of the rows or of the sequences still unfinished), so stepwise and
       // SSD forwards of one generation always take the same form.
-      // (Two thirds of that many CTAs are enough while the prefix is short: two sequences below 1024 cached keys.)
-      const int pipe_ctas = attn_S < 1024 ? (2 * c->attn_pipe_ctas + 2) / 3 : c->attn_pipe_ctas;
-      if (c->attn_impl == 1 && c->attn_pipe_keys > 0 && attn_S >= c->attn_pipe_keys && c->batch * H >= pipe_ctas)
+      if (c->attn_impl == 1 && c->attn_pipe_keys > 0 && attn_S >= c->attn_pipe_keys && c->batch * H >= c->attn_pipe_ctas)
         arc = launch_attention_verify_pipe(c->st, a);
       if (arc == 1 && c->attn_impl == 1) arc = launch_attention_verify_tc(c->st, a);   // 1: shape not covered by the tcgen05 form
       if (arc == 1) arc = launch_attention_verify(c->st, a);
