@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(kTcAttnThreads, 2) attn_verify_tc_kernel(AttnA
       finish(A, x1, x2);
     }
     if (!waited) cluster_wait();
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // these stores are read by the tensor core
+    asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");  // these stores (into other CTAs too) are read by the tensor core
     cluster_sync_all();
   }
   // The MMA always works on 128 query rows (= 128 TMEM lanes, one per thread).  A tile of QT < 128
