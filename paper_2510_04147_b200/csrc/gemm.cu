@@ -465,38 +465,68 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       // EPI_LMHEAD: lane = vocabulary entry; reduce over the 128 lanes per row (= column)
       const int n = tile * kTileM + lrow;
       const bool live = (n < p.N) && (n != p.mask_id);
-      float* s_max = scratch;                       // [4][256]
-      float* s_sum = scratch + 4 * 256;
-      int* s_arg = reinterpret_cast<int*>(scratch + 8 * 256);
-      for (int c0 = 0; c0 < p.npad; c0 += 32) {
-        float v[32];
-        tmem_ld32(taddr + c0, v);
-        if (p.sq != nullptr) {
+      {
+        // Statistics.  32 rows at a time are transposed through shared memory (dead entries as -inf); four threads
+        // then share a row: each scans a quarter of the tile's 128 entries in index order - maximum with the lowest
+        // index among equals, sum of exp(x - its maximum) - and the quarters are merged (0 + 1) + (2 + 3).  The order
+        // depends on the tile alone.
+        const int rr = et >> 2, qf = (et & 3) * 32;
+        for (int c0 = 0; c0 < p.npad; c0 += 32) {
+          float v[32];
+          tmem_ld32(taddr + c0, v);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] *= s_inv[c0 + j];
-        }
-        float my_m = -INFINITY, my_s = 0.f;
-        int my_a = 0x7fffffff;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float x = live ? v[j] : -INFINITY;
-          float m = x;
-          int a = n;
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const float om = __shfl_xor_sync(0xffffffffu, m, o);
-            const int oa = __shfl_xor_sync(0xffffffffu, a, o);
-            if (om > m || (om == m && oa < a)) { m = om; a = oa; }
+          for (int j = 0; j < 32; ++j) {
+            const float x = p.sq != nullptr ? v[j] * s_inv[c0 + j] : v[j];
+            scratch[j * kEpiPitch + lrow] = live ? x : -INFINITY;
           }
-          float e = (m == -INFINITY) ? 0.f : expf(x - m);
+          epi_bar_sync();
+          float m = -INFINITY, sum = 0.f;
+          int arg = 0x7fffffff;
+          {
+            float x[32];
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
-          if (lane == j) { my_m = m; my_s = e; my_a = a; }
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const float4 t4 = *reinterpret_cast<const float4*>(scratch + rr * kEpiPitch + qf + q4 * 4);
+              x[q4 * 4] = t4.x; x[q4 * 4 + 1] = t4.y; x[q4 * 4 + 2] = t4.z; x[q4 * 4 + 3] = t4.w;
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (x[j] > m) { m = x[j]; arg = tile * kTileM + qf + j; }
+            if (m != -INFINITY) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) sum += expf(x[j] - m);          // (exp(-inf) = 0 for dead entries)
+            }
+          }
+#pragma unroll
+          for (int o = 1; o <= 2; o <<= 1) {                               // quarters: (0 + 1), (2 + 3), then the pairs
+            const float om = __shfl_xor_sync(0xffffffffu, m, o);
+            const float os = __shfl_xor_sync(0xffffffffu, sum, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+            // the same value from both partners: the lower quarter's (maximum, index) wins a tie
+            const bool lower = (et & o) == 0;
+            const float m_lo = lower ? m : om, s_lo = lower ? sum : os, m_hi = lower ? om : m, s_hi = lower ? os : sum;
+            const int a_lo = lower ? arg : oa, a_hi = lower ? oa : arg;
+            const float M = fmaxf(m_lo, m_hi);
+            float S = 0.f;
+            if (m_lo != -INFINITY) S += s_lo * expf(m_lo - M);
+            if (m_hi != -INFINITY) S += s_hi * expf(m_hi - M);
+            arg = (m_hi > m_lo) ? a_hi : a_lo;
+            m = M;
+            sum = S;
+          }
+          if ((et & 3) == 0 && c0 + rr < rows_here) {
+            const size_t o = (size_t)tile * p.R + row0 + c0 + rr;
+            p.tile_max[o] = m;
+            p.tile_sum[o] = sum;
+            p.tile_arg[o] = arg;
+          }
+          epi_bar_sync();
         }
-        s_max[quad * 256 + c0 + lane] = my_m;
-        s_sum[quad * 256 + c0 + lane] = my_s;
-        s_arg[quad * 256 + c0 + lane] = my_a;
-        if (p.topk > 0) {
+      }
+      if (p.topk > 0) {
+        // The tile's largest logits on top of the statistics above (the acceptance-limit probe)
+      for (int c0 = 0; c0 < p.npad; c0 += 32) {
+        {
           // The tile's `topk` largest logits of every row of the chunk (value descending, lower index first):
           // per warp by repeated warp-wide argmax with the winner struck out, then the four warps' sorted
           // lists are merged by one thread per row.
@@ -555,25 +585,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           epi_bar_sync();
         }
       }
-      epi_bar_sync();
-      for (int c = (warp - 2) * 32 + lane; c < rows_here; c += 128) {
-        float M = -INFINITY;
-        int A = 0x7fffffff;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float m = s_max[q * 256 + c];
-          if (m > M) { M = m; A = s_arg[q * 256 + c]; }
-        }
-        float S = 0.f;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float m = s_max[q * 256 + c];
-          if (m != -INFINITY) S += s_sum[q * 256 + c] * expf(m - M);
-        }
-        const size_t o = (size_t)tile * p.R + row0 + c;
-        p.tile_max[o] = M;
-        p.tile_sum[o] = S;
-        p.tile_arg[o] = A;
       }
     }
   }
