@@ -31,7 +31,7 @@ METRIC = "decode tokens/s at batch 1 (LLaDA-8B-shaped) and % HBM roofline per ve
 # profiles/gemm_tc_kernel_and_attn_verify_tc_llada8b_4layers_counters.md (mean over the four projections of a
 # LLaDA-8B-shaped layer).
 # Valid only for the kernel source it was taken from: reported as null once gemm.cu has changed.
-GEMM_TRAFFIC = {"workload": "llada8b", "bytes_per_launch": 112.9e6, "gemm_cu_sha256_16": "e49a986261cb2295"}
+GEMM_TRAFFIC = {"workload": "llada8b", "bytes_per_launch": 113.1e6, "gemm_cu_sha256_16": "a35294ed124f87be"}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
